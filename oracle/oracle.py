@@ -1,0 +1,168 @@
+"""ctypes front end of the CPU oracle (dssd_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this module.
+
+The arithmetic lives in dssd_oracle.c; this file compiles it with gcc, passes
+numpy arrays through and, when asked, runs disjoint slices of the batch on
+several host threads (sequences are independent, so this changes no result).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dssd_oracle.c")
+_LIB = os.path.join(_HERE, "libdssd_oracle.so")
+
+F32 = 0
+BF16 = 1
+
+FLAG_BAD_TOKEN = 1
+FLAG_NONFINITE = 2
+RS_FLAG_BONUS = 1
+RS_FLAG_FALLBACK = 2
+RS_FLAG_INVALID = 4
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (plain C, strict IEEE semantics: no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-ffp-contract=off",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c = ctypes
+        lib.dssd_oracle_edge_verify.restype = c.c_int
+        lib.dssd_oracle_edge_verify.argtypes = [
+            c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+            c.c_int, c.c_int, c.c_int,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.dssd_oracle_device_resample.restype = c.c_int
+        lib.dssd_oracle_device_resample.argtypes = [
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _chunks(B: int, threads: int):
+    threads = max(1, min(threads, B))
+    edges = np.linspace(0, B, threads + 1).astype(int)
+    return [(int(edges[i]), int(edges[i + 1])) for i in range(threads) if edges[i + 1] > edges[i]]
+
+
+def edge_verify(target_logits: np.ndarray, draft_tokens: np.ndarray, draft_q_tok: np.ndarray,
+                uniforms: np.ndarray, temperature: float, want_p_row64: bool = False,
+                threads: int = 1) -> Dict[str, np.ndarray]:
+    """Edge half of the round.  target_logits: [B, gamma+1, V] float32, or uint16 = bf16 bits."""
+    lib = _load()
+    tl = np.ascontiguousarray(target_logits)
+    assert tl.ndim == 3 and tl.dtype in (np.float32, np.uint16)
+    dtype = BF16 if tl.dtype == np.uint16 else F32
+    B, g1, V = tl.shape
+    gamma = g1 - 1
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(B, gamma)
+    qt = np.ascontiguousarray(draft_q_tok, dtype=np.float32).reshape(B, gamma)
+    u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, gamma)
+    out = {
+        "accept_len": np.zeros(B, np.int32),
+        "p_row": np.zeros((B, V), np.float32),
+        "p_row64": np.zeros((B, V), np.float64) if want_p_row64 else None,
+        "p_tok": np.zeros((B, gamma), np.float64),
+        "lse": np.zeros((B, gamma + 1), np.float64),
+        "flags": np.zeros(B, np.uint32),
+        "margin_acc": np.zeros(B, np.float64),
+    }
+
+    def run(rng):
+        b0, b1 = rng
+        rc = lib.dssd_oracle_edge_verify(
+            _ptr(tl[b0:b1]), dtype, V, _ptr(tok[b0:b1]), _ptr(qt[b0:b1]), _ptr(u[b0:b1]),
+            ctypes.c_float(temperature), b1 - b0, gamma, V,
+            _ptr(out["accept_len"][b0:b1]), _ptr(out["p_row"][b0:b1]),
+            _ptr(out["p_row64"][b0:b1]) if want_p_row64 else None,
+            _ptr(out["p_tok"][b0:b1]), _ptr(out["lse"][b0:b1]), _ptr(out["flags"][b0:b1]),
+            _ptr(out["margin_acc"][b0:b1]))
+        if rc != 0:
+            raise ValueError("dssd_oracle_edge_verify: invalid arguments")
+
+    parts = _chunks(B, threads)
+    if len(parts) == 1:
+        run(parts[0])
+    else:
+        with ThreadPoolExecutor(len(parts)) as ex:
+            list(ex.map(run, parts))
+    return out
+
+
+def device_resample(p_row: np.ndarray, draft_q: Optional[np.ndarray], accept_len: np.ndarray,
+                    uniforms_rs: np.ndarray, gamma: int, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Device half of the round.  p_row: [B, V] float32; draft_q: [B, gamma, V] float32."""
+    lib = _load()
+    p = np.ascontiguousarray(p_row, dtype=np.float32)
+    B, V = p.shape
+    if gamma > 0:
+        q = np.ascontiguousarray(draft_q, dtype=np.float32).reshape(B, gamma, V)
+    else:
+        q = np.zeros((B, 0, V), np.float32)
+    n = np.ascontiguousarray(accept_len, dtype=np.int32).reshape(B)
+    u = np.ascontiguousarray(uniforms_rs, dtype=np.float32).reshape(B)
+    out = {
+        "token": np.zeros(B, np.int32),
+        "flags": np.zeros(B, np.uint32),
+        "margin_cdf": np.zeros(B, np.float64),
+        "Z": np.zeros(B, np.float64),
+    }
+
+    def run(rng):
+        b0, b1 = rng
+        rc = lib.dssd_oracle_device_resample(
+            _ptr(p[b0:b1]), _ptr(q[b0:b1]) if gamma > 0 else None, _ptr(n[b0:b1]), _ptr(u[b0:b1]),
+            b1 - b0, gamma, V, _ptr(out["token"][b0:b1]), _ptr(out["flags"][b0:b1]),
+            _ptr(out["margin_cdf"][b0:b1]), _ptr(out["Z"][b0:b1]))
+        if rc != 0:
+            raise ValueError("dssd_oracle_device_resample: invalid arguments")
+
+    parts = _chunks(B, threads)
+    if len(parts) == 1:
+        run(parts[0])
+    else:
+        with ThreadPoolExecutor(len(parts)) as ex:
+            list(ex.map(run, parts))
+    return out
+
+
+def verify_round(inputs: Dict[str, np.ndarray], temperature: float, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Both halves on one generated batch: the device half consumes the float32 row
+    that the edge half emitted, as it would after the downlink."""
+    ev = edge_verify(inputs["target_logits"], inputs["draft_tokens"], inputs["draft_q_tok"],
+                     inputs["uniforms"], temperature, threads=threads)
+    gamma = inputs["target_logits"].shape[1] - 1
+    rs = device_resample(ev["p_row"], inputs["draft_q"], ev["accept_len"], inputs["uniforms_rs"],
+                         gamma, threads=threads)
+    out = dict(ev)
+    out["token"] = rs["token"]
+    out["rs_flags"] = rs["flags"]
+    out["margin_cdf"] = rs["margin_cdf"]
+    out["Z"] = rs["Z"]
+    return out
