@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the split speculative verification round on B200.
+
+One step = one pass of the whole verification round (dssd_edge_verify, then
+dssd_device_resample) over one batch of synthetic inputs that are already resident in HBM.
+The metric is verified rows per second, rows = B * (gamma + 1).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl ours|reference]
+
+With N > 1 (launched through torch.distributed.run) every rank verifies its own batch of the
+same shape (sequences are independent: no data-path collective); time is the maximum over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import dssd_inputs as di  # noqa: E402
+
+METRIC = "verified_rows_per_s"
+UNIT = "rows/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
+# bytes per launch), valid only for the kernel source whose hash is recorded with it.
+NCU_TRAFFIC = {}
+
+
+def _kernel_hash() -> str:
+    h = hashlib.sha256()
+    for f in ("edge_verify.cu", "edge_verify.h", "dssd_device.cuh"):
+        with open(os.path.join(ROOT, "paper_2507_12000_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def edge_algorithmic_bytes(w: di.Workload) -> int:
+    """Bytes dssd_edge_verify must move: every logit once, plus the float32 row it emits."""
+    return w.B * w.V * ((w.gamma + 1) * w.logit_bytes + 4)
+
+
+def resample_algorithmic_bytes(w: di.Workload, n_bonus: int) -> int:
+    """p row for every sequence, q row for the rejected ones, one token each."""
+    return w.V * 4 * (2 * w.B - n_bonus) + 4 * w.B
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the benchmark runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.samples = []  # (t, sm_mhz, reasons bitmask, power_w)
+        self.stop_flag = False
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:  # NVML missing: report no clocks rather than fail the run
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                power = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                self.samples.append((time.perf_counter(), mhz, int(reasons), power))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        scope = "timed region"
+        if not inside:
+            inside, scope = self.samples, "warm-up and timed region (timed region shorter than one sample)"
+        names = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in names.items() if mask & b], "samples": len(inside),
+                "power_w_max": max(s[3] for s in inside), "scope": scope}
+
+
+def _torch_inputs(d, device=None, pin=False):
+    import torch
+
+    out = {}
+    for k, v in d.items():
+        t = torch.from_numpy(v.view(np.int16)).view(torch.bfloat16) if v.dtype == np.uint16 else torch.from_numpy(v)
+        if device is not None:
+            t = t.to(device)
+        elif pin:
+            t = t.pin_memory()
+        out[k] = t
+    return out
+
+
+def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, repeats: int = 1):
+    """rows/s of the CPU oracle (both halves) on the first n_seq sequences."""
+    from oracle import oracle as O
+
+    sub = {k: v[:n_seq] for k, v in d.items()}
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.verify_round(sub, w.temperature, threads=threads)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return n_seq * (w.gamma + 1) / best, best
+
+
+def run_reference(args, w: di.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as O
+
+    O.build()
+    cores = os.cpu_count() or 1
+    n_seq = min(w.B, args.ref_sequences)
+    d = di.generate(w, 0, n_seq, threads=cores)
+    for _ in range(args.warmup):
+        O.verify_round(d, w.temperature, threads=cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.verify_round(d, w.temperature, threads=cores)
+    dt = time.perf_counter() - t0
+    value = args.steps * n_seq * (w.gamma + 1) / dt
+    sample = f"first {n_seq} of {w.B} sequences of {w.name} per step, both halves, float64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def _config(w: di.Workload, args):
+    return {"workload": f"{w.name}: B={w.B} gamma={w.gamma} V={w.V} {w.dtype} T={w.temperature} "
+                        f"sigma_d={w.sigma_d} (per GPU)",
+            "B": w.B, "gamma": w.gamma, "V": w.V, "logits_dtype": w.dtype, "temperature": w.temperature,
+            "l2": "inputs larger than L2, no flush" if w.rows * w.V * w.logit_bytes > 200e6 else
+                  "inputs rotate through copies larger than L2",
+            "parallelism": f"batch-sharded x{args.gpus}, no collective"}
+
+
+def run_ours(args, w: di.Workload):
+    import torch
+    import torch.distributed as dist
+
+    from oracle import oracle as O
+
+    O.build()  # before the first CUDA call
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cores = os.cpu_count() or 1
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2507_12000_b200 import binding as B
+
+    # every rank draws its own batch (weak scaling): same shape, different seed
+    wr = di.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    d = di.generate(wr, threads=max(1, cores // max(1, min(world, 8))))
+    logit_bytes = d["target_logits"].nbytes
+    # inputs smaller than L2 rotate through enough copies to exceed it
+    copies = 1 if logit_bytes > 200e6 else int(min(64, 300e6 // max(logit_bytes, 1) + 1))
+    sets = [_torch_inputs(d, dev) for _ in range(copies)]
+    gamma, Bn, V = w.gamma, w.B, w.V
+    ws_e = torch.empty(B.dssd_edge_verify_workspace_bytes(Bn, gamma, V), dtype=torch.uint8, device=dev)
+    ws_r = torch.empty(B.dssd_device_resample_workspace_bytes(Bn, gamma, V), dtype=torch.uint8, device=dev)
+    ev_out = None
+    rs_out = None
+
+    def step(i):
+        nonlocal ev_out, rs_out
+        g = sets[i % copies]
+        ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                    w.temperature, out=ev_out, workspace=ws_e)
+        rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
+                                        gamma, out=rs_out, workspace=ws_r)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.perf_counter()
+    for i in range(K):
+        g = sets[i % copies]
+        ev[i][0].record()
+        ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                    w.temperature, out=ev_out, workspace=ws_e)
+        ev[i][1].record()
+        rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
+                                        gamma, out=rs_out, workspace=ws_r)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    t_host1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
+    edge_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    rs_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    sampler.stop_flag = True
+    sampler.join(timeout=1.0)
+    clocks = sampler.summary(t_host0, t_host1)
+    n_gpu = ev_out["accept_len"].cpu().numpy()
+    n_bonus = int((n_gpu == gamma).sum())
+
+    # ---- end to end through the host-buffer entry point: copies inside the timed region ----
+    host = _torch_inputs(d, pin=True)
+    arena = torch.empty(B.dssd_round_host_arena_bytes(Bn, gamma, V, B.DSSD_BF16 if w.dtype == "bf16" else B.DSSD_F32),
+                        dtype=torch.uint8, device=dev)
+    h_out = None
+    e2e_steps = max(3, min(K, args.e2e_steps))
+    for _ in range(2):
+        h_out = B.dssd_round_host(host, w.temperature, arena, out=h_out)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        h_out = B.dssd_round_host(host, w.temperature, arena, out=h_out)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(host[k].numel() * host[k].element_size() for k in
+              ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs"))
+    d2h = 4 * Bn * 4
+    assert (h_out["accept_len"].numpy() == n_gpu).all()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    rows = w.rows
+    ms_per_step = total_ms / K
+    value = world * rows / (ms_per_step * 1e-3)
+    peak, peak_kind = _peaks()
+    edge_avg_ms = sum(edge_ms) / K
+    edge_bytes = edge_algorithmic_bytes(w)
+    achieved = edge_bytes / (edge_avg_ms * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC.get(w.name)
+    if traffic is not None and traffic.get("kernel_hash") != _kernel_hash():
+        traffic = None
+    rs_avg_ms = sum(rs_ms) / K
+    rs_bytes = resample_algorithmic_bytes(w, n_bonus)
+
+    # ---- CPU baseline: the oracle as it stands, on this machine's host cores, rank 0, N = 1 ----
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_seq = min(Bn, args.ref_sequences)
+        rate, secs = oracle_rate(w, d, n_seq, cores)
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {n_seq} of {Bn} sequences of {w.name}, both halves, one pass of {secs:.2f} s wall "
+                         f"on {cores} threads"}
+        ref = O.verify_round({k: v[:n_seq] for k, v in d.items()}, w.temperature, threads=cores)
+        near = ref["margin_acc"] < 1e-6
+        parity = {"sequences_checked": n_seq,
+                  "accept_len_mismatch": int(((n_gpu[:n_seq] != ref["accept_len"]) & ~near).sum()),
+                  "near_boundary_accept": int(near.sum()),
+                  "token_mismatch": int((rs_out["token"].cpu().numpy()[:n_seq] != ref["token"]).sum()),
+                  "accept_rate": float(ref["accept_len"].mean() / max(gamma, 1))}
+    else:
+        parity = None
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": _config(w, args),
+        "roofline": {"bound": "hbm", "kernel": "edge_verify_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": edge_bytes, "avg_launch_ms": edge_avg_ms,
+                     "min_launch_ms": min(edge_ms),
+                     "traffic": None if traffic is None else traffic["bytes"]},
+        "resample": {"avg_launch_ms": rs_avg_ms, "algorithmic_bytes_per_launch": rs_bytes,
+                     "achieved_gbs": rs_bytes / (rs_avg_ms * 1e-3) / 1e9,
+                     "frac": rs_bytes / (rs_avg_ms * 1e-3) / 1e9 / peak},
+        "edge_rows_per_s": world * rows / (edge_avg_ms * 1e-3),
+        "cpu_baseline": cpu,
+        "parity": parity,
+        "e2e": {"value": world * rows / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 2 * K,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--ref-sequences", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = di.get_workload(args.workload)
+    if args.steps is None:
+        args.steps = 3 if args.impl == "reference" else 2000
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,175 @@
+/*
+ * dssd.h - C ABI of the split speculative verification library for NVIDIA B200 (sm_100a).
+ *
+ * One verification round of Distributed Split Speculative Decoding (DSSD, Algorithm 2 of the
+ * paper) for B independent sequences:
+ *
+ *   dssd_edge_verify      the edge (base-station) half: "Verification Process" and the
+ *                         payload of "Downlink Transmission" (Section 3, Algorithm 2);
+ *   dssd_device_resample  the device half: "Resample" (Section 3, Algorithm 2), plus the
+ *                         bonus draw x_{gamma+1} ~ P_{gamma+1} that Algorithm 2 performs when
+ *                         every draft token was accepted;
+ *   dssd_round_host       both halves on host buffers, with the copies to and from the GPU.
+ *
+ * Notation follows the paper: gamma draft tokens x_1..x_gamma with draft probabilities
+ * q_i(x_i), target distributions P_1..P_{gamma+1} over a vocabulary of V entries, uniforms
+ * r_i.  Indices here are 0-based: accept_len n = j - 1, where j is the paper's 1-based position
+ * of the first rejected token (j = gamma + 1, n = gamma, when all drafts were accepted).
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - The caller owns every buffer.  The library allocates no memory, keeps no state between
+ *     calls, enqueues its work on the given CUDA stream and returns without synchronising.
+ *   - Buffers need only their natural alignment; 16-byte aligned rows take the fast path.
+ *   - A status other than DSSD_OK means nothing was enqueued (except DSSD_ERR_CUDA, after
+ *     which the outputs are undefined).  Data-dependent anomalies never fault or trap: they
+ *     are reported per sequence in the flags outputs.
+ *   - Calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef DSSD_H
+#define DSSD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DSSD_OK = 0,
+    DSSD_ERR_INVALID_ARG = 1, /* NULL required pointer, B < 1, gamma < 0, V < 1, T <= 0 or not finite, row_stride < V */
+    DSSD_ERR_UNSUPPORTED = 2, /* a size beyond DSSD_MAX_* or an unknown dtype */
+    DSSD_ERR_WORKSPACE = 3,   /* workspace NULL, misaligned (256 bytes) or too small */
+    DSSD_ERR_CUDA = 4         /* a CUDA call failed; see dssd_last_cuda_error() */
+} dssd_status;
+
+typedef enum {
+    DSSD_F32 = 0, /* IEEE binary32 logits  */
+    DSSD_BF16 = 1 /* bfloat16 logits       */
+} dssd_dtype;
+
+#define DSSD_MAX_V (1 << 30)
+#define DSSD_MAX_ROWS 0x7fffffff /* B * (gamma + 1) */
+
+/* flags written by dssd_edge_verify, one word per sequence */
+#define DSSD_EDGE_FLAG_BAD_TOKEN 1u /* some x_i outside [0, V): that position is rejected        */
+#define DSSD_EDGE_FLAG_NONFINITE 2u /* some row of the sequence has no finite log-sum-exp (NaN,  \
+                                       +inf, or all -inf): that position is rejected, its row is NaN */
+#define DSSD_EDGE_FLAG_TIMEOUT 4u   /* internal wait ran out; p_row of this sequence was not written */
+
+/* flags written by dssd_device_resample, one word per sequence */
+#define DSSD_RS_FLAG_BONUS 1u    /* n == gamma: token drawn from P_{gamma+1}                       */
+#define DSSD_RS_FLAG_FALLBACK 2u /* residual mass sum max(0, p - q) <= 0: token drawn from p instead */
+#define DSSD_RS_FLAG_INVALID 4u  /* no positive mass at all, or n outside [0, gamma]: token = -1    */
+
+/* Human-readable name of a status (static storage, never NULL). */
+const char *dssd_status_string(int status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int dssd_version(void);
+
+/* CUDA error code (cudaError_t as int) behind the calling thread's last DSSD_ERR_CUDA, else 0. */
+int dssd_last_cuda_error(void);
+
+/*
+ * Bytes of scratch that dssd_edge_verify needs for these sizes (0 if the sizes are invalid).
+ * Depends on the sizes only, not on the GPU.
+ */
+size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V);
+
+/*
+ * Edge half of one round (Algorithm 2, "Verification Process" at the edge and the payload of
+ * "Downlink Transmission"; Section 3).
+ *
+ * For every sequence b and position i = 0..gamma the target distribution is
+ *   P_i(v) = softmax(l_{b,i,v} / T)                      (temperature: Section 4)
+ * computed through the row's log-sum-exp.  Draft token x_i is accepted iff
+ *   u_i < min(1, p_i(x_i) / q_i(x_i))
+ * (Algorithm 2 prints the ratio upside down; this direction is the one consistent with the
+ * residual max(0, P - Q) of the "Resample" step).  n is the first position that fails, or gamma.
+ * The single row P_n(.) - the rejected position's target distribution, or the bonus position's
+ * when n == gamma - is written in float32: it is the downlink payload of Section 3.1
+ * (b_prob = 32).  Unlike the paper, the row is also written when n == gamma, so that
+ * dssd_device_resample can draw the bonus token; a caller that wants the paper's byte saving
+ * simply does not transmit it.
+ *
+ * Comparison details: the test is evaluated in float64 from a float64 log-sum-exp; u == 1 never
+ * accepts; q <= 0 accepts iff p > 0; a NaN q or an out-of-range token rejects.
+ *
+ * target_logits  [B, gamma+1, V] of `dtype`, unit stride along V, `row_stride` elements between
+ *                consecutive rows (>= V); row (b, i) starts at element (b*(gamma+1)+i)*row_stride
+ * draft_tokens   [B, gamma] int32      x_i          (may be NULL iff gamma == 0)
+ * draft_q_tok    [B, gamma] float32    q_i(x_i)     (may be NULL iff gamma == 0)
+ * uniforms       [B, gamma] float32    u_i in [0,1) (may be NULL iff gamma == 0)
+ * temperature    T > 0, finite
+ * accept_len     [B] int32     out: n in [0, gamma]
+ * p_row          [B, V] float32 out: P_n(.)
+ * p_tok          [B, gamma] float32   out, optional (NULL ok): p_i(x_i)
+ * lse            [B, gamma+1] float32 out, optional (NULL ok): ln sum_v exp(l_v / T)
+ * flags          [B] uint32    out, optional (NULL ok): DSSD_EDGE_FLAG_*
+ * workspace      >= dssd_edge_verify_workspace_bytes(B, gamma, V) bytes, 256-byte aligned;
+ *                contents need not be initialised and are garbage afterwards
+ * cuda_stream    cudaStream_t (NULL = the legacy default stream)
+ */
+dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                             const int32_t *draft_tokens, const float *draft_q_tok,
+                             const float *uniforms, float temperature, int B, int gamma, int V,
+                             int32_t *accept_len, float *p_row, float *p_tok, float *lse,
+                             uint32_t *flags, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream);
+
+/* Bytes of scratch that dssd_device_resample needs (0 if the sizes are invalid). */
+size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V);
+
+/*
+ * Device half of one round (Algorithm 2, "Resample"; Section 3 "Verification Process (on
+ * Device)"), and the bonus draw of Algorithm 2's "Sample x_{gamma+1} ~ P_{gamma+1}".
+ *
+ * For a rejected sequence (n < gamma):  r_v = max(0, p_v - q_{n,v}),  Z = sum_v r_v,
+ *   token = min{k : sum_{v<=k} r_v > u' * Z}      (inverse CDF in index order, float64 sums);
+ * for n == gamma the same draw with r = p.  If rounding leaves no such k the last index with
+ * r_v > 0 is returned.  If Z <= 0 (p == q) the draw falls back to r = p and sets
+ * DSSD_RS_FLAG_FALLBACK.
+ *
+ * p_row       [B, V] float32        the row produced by dssd_edge_verify (the downlink payload)
+ * draft_q     [B, gamma, V] float32 the device's own Q_i(.); only row n of each sequence is read
+ *                                   (may be NULL iff gamma == 0)
+ * accept_len  [B] int32             n
+ * uniforms    [B] float32           u' in [0,1)
+ * token       [B] int32   out
+ * flags       [B] uint32  out, optional (NULL ok): DSSD_RS_FLAG_*
+ * workspace   >= dssd_device_resample_workspace_bytes(B, gamma, V) bytes, 256-byte aligned
+ */
+dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
+                                 const int32_t *accept_len, const float *uniforms, int B,
+                                 int gamma, int V, int32_t *token, uint32_t *flags,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Bytes of device memory that dssd_round_host needs as its arena (0 if the sizes are invalid). */
+size_t dssd_round_host_arena_bytes(int B, int gamma, int V, dssd_dtype dtype);
+
+/*
+ * Both halves of Algorithm 2's verification on HOST buffers: copies the inputs to the GPU,
+ * runs dssd_edge_verify and dssd_device_resample, and copies the results back, all enqueued on
+ * `cuda_stream`.  The host buffers must stay valid until the stream has finished; use pinned
+ * memory for the copies to be asynchronous.
+ *
+ * host inputs:  target_logits [B, gamma+1, V] contiguous, draft_tokens, draft_q_tok, uniforms
+ *               [B, gamma], draft_q [B, gamma, V], uniforms_rs [B]
+ * host outputs: accept_len [B], token [B], edge_flags [B] (NULL ok), rs_flags [B] (NULL ok),
+ *               p_row [B, V] (NULL ok: the row then stays on the GPU)
+ * device_arena  device memory, >= dssd_round_host_arena_bytes(...) bytes, 256-byte aligned
+ */
+dssd_status dssd_round_host(const void *target_logits, dssd_dtype dtype,
+                            const int32_t *draft_tokens, const float *draft_q_tok,
+                            const float *uniforms, const float *draft_q, const float *uniforms_rs,
+                            float temperature, int B, int gamma, int V, int32_t *accept_len,
+                            int32_t *token, uint32_t *edge_flags, uint32_t *rs_flags,
+                            float *p_row, void *device_arena, size_t arena_bytes,
+                            void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSSD_H */

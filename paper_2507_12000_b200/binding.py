@@ -1,0 +1,194 @@
+"""Thin Python binding of libdssd.so (see include/dssd.h for the contract of every call).
+
+Only argument marshalling happens here: torch tensors supply device memory and the CUDA
+stream; every step of the verification round runs inside the library's kernels.  There is no
+CPU path: if the library cannot be loaded the import fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdssd.so")
+
+DSSD_OK = 0
+DSSD_ERR_INVALID_ARG = 1
+DSSD_ERR_UNSUPPORTED = 2
+DSSD_ERR_WORKSPACE = 3
+DSSD_ERR_CUDA = 4
+DSSD_F32 = 0
+DSSD_BF16 = 1
+
+EDGE_FLAG_BAD_TOKEN = 1
+EDGE_FLAG_NONFINITE = 2
+EDGE_FLAG_TIMEOUT = 4
+RS_FLAG_BONUS = 1
+RS_FLAG_FALLBACK = 2
+RS_FLAG_INVALID = 4
+
+
+class DssdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = lib.dssd_status_string(status).decode()
+        extra = f" (cudaError {lib.dssd_last_cuda_error()})" if status == DSSD_ERR_CUDA else ""
+        super().__init__(f"{where}: {name}{extra}")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2507_12000_b200.build` "
+            "(needs nvcc); this package has no CPU fallback")
+    c = ctypes
+    L = c.CDLL(LIB_PATH)
+    L.dssd_status_string.restype = c.c_char_p
+    L.dssd_status_string.argtypes = [c.c_int]
+    L.dssd_version.restype = c.c_int
+    L.dssd_last_cuda_error.restype = c.c_int
+    for f in (L.dssd_edge_verify_workspace_bytes, L.dssd_device_resample_workspace_bytes):
+        f.restype = c.c_size_t
+        f.argtypes = [c.c_int, c.c_int, c.c_int]
+    L.dssd_round_host_arena_bytes.restype = c.c_size_t
+    L.dssd_round_host_arena_bytes.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int]
+    L.dssd_edge_verify.restype = c.c_int
+    L.dssd_edge_verify.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_device_resample.restype = c.c_int
+    L.dssd_device_resample.argtypes = [
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_round_host.restype = c.c_int
+    L.dssd_round_host.argtypes = [
+        c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_size_t, c.c_void_p]
+    return L
+
+
+lib = _load()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None or t.numel() == 0 else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return DSSD_BF16
+    if t.dtype == torch.float32:
+        return DSSD_F32
+    raise TypeError(f"target_logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def dssd_edge_verify_workspace_bytes(B: int, gamma: int, V: int) -> int:
+    return int(lib.dssd_edge_verify_workspace_bytes(B, gamma, V))
+
+
+def dssd_device_resample_workspace_bytes(B: int, gamma: int, V: int) -> int:
+    return int(lib.dssd_device_resample_workspace_bytes(B, gamma, V))
+
+
+def dssd_round_host_arena_bytes(B: int, gamma: int, V: int, dtype: int) -> int:
+    return int(lib.dssd_round_host_arena_bytes(B, gamma, V, dtype))
+
+
+def dssd_edge_verify(target_logits: torch.Tensor, draft_tokens: torch.Tensor, draft_q_tok: torch.Tensor,
+                     uniforms: torch.Tensor, temperature: float, *, out: Optional[Dict[str, torch.Tensor]] = None,
+                     want_p_tok: bool = True, want_lse: bool = True, workspace: Optional[torch.Tensor] = None,
+                     stream=None) -> Dict[str, torch.Tensor]:
+    """Edge half of one round.  target_logits: CUDA tensor [B, gamma+1, V], float32 or bfloat16,
+    unit stride along V and a common stride between rows.  Returns accept_len, p_row, flags and,
+    if asked, p_tok and lse.  Pass `out` (a previous result) and `workspace` to allocate nothing."""
+    assert target_logits.is_cuda and target_logits.dim() == 3
+    B, g1, V = target_logits.shape
+    gamma = g1 - 1
+    assert target_logits.stride(2) == 1 or V == 1
+    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
+    if B > 1 and target_logits.stride(0) != g1 * row_stride:
+        raise ValueError("rows of target_logits must be equally spaced")
+    dev = target_logits.device
+    if out is None:
+        out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_row": torch.empty(B, V, dtype=torch.float32, device=dev),
+            "flags": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_tok": torch.empty(B, gamma, dtype=torch.float32, device=dev) if want_p_tok else None,
+            "lse": torch.empty(B, g1, dtype=torch.float32, device=dev) if want_lse else None,
+        }
+    need = dssd_edge_verify_workspace_bytes(B, gamma, V)
+    if workspace is None:
+        workspace = _workspace(need, dev)
+    st = lib.dssd_edge_verify(
+        target_logits.data_ptr(), _dtype_code(target_logits), row_stride,
+        _ptr(draft_tokens), _ptr(draft_q_tok), _ptr(uniforms), ctypes.c_float(temperature), B, gamma, V,
+        out["accept_len"].data_ptr(), out["p_row"].data_ptr(), _ptr(out.get("p_tok")), _ptr(out.get("lse")),
+        _ptr(out.get("flags")), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_verify")
+    return out
+
+
+def dssd_device_resample(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], accept_len: torch.Tensor,
+                         uniforms_rs: torch.Tensor, gamma: int, *, out: Optional[Dict[str, torch.Tensor]] = None,
+                         workspace: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """Device half of one round.  p_row [B, V] float32, draft_q [B, gamma, V] float32 (contiguous)."""
+    assert p_row.is_cuda and p_row.dim() == 2 and p_row.is_contiguous() and p_row.dtype == torch.float32
+    B, V = p_row.shape
+    if gamma > 0:
+        assert draft_q.is_contiguous() and draft_q.dtype == torch.float32 and draft_q.numel() == B * gamma * V
+    dev = p_row.device
+    if out is None:
+        out = {"token": torch.empty(B, dtype=torch.int32, device=dev),
+               "flags": torch.empty(B, dtype=torch.int32, device=dev)}
+    need = dssd_device_resample_workspace_bytes(B, gamma, V)
+    if workspace is None:
+        workspace = _workspace(need, dev)
+    st = lib.dssd_device_resample(
+        p_row.data_ptr(), _ptr(draft_q) if gamma > 0 else None, accept_len.data_ptr(), uniforms_rs.data_ptr(),
+        B, gamma, V, out["token"].data_ptr(), _ptr(out.get("flags")), workspace.data_ptr(), workspace.numel(),
+        _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_device_resample")
+    return out
+
+
+def dssd_round_host(host: Dict[str, torch.Tensor], temperature: float, arena: torch.Tensor, *,
+                    out: Optional[Dict[str, torch.Tensor]] = None, want_p_row: bool = False,
+                    stream=None) -> Dict[str, torch.Tensor]:
+    """Both halves on HOST tensors (pinned for asynchronous copies); `arena` is CUDA scratch of
+    dssd_round_host_arena_bytes(...) bytes.  Results land in host tensors once the stream is done."""
+    tl = host["target_logits"]
+    assert not tl.is_cuda and tl.is_contiguous() and tl.dim() == 3
+    B, g1, V = tl.shape
+    gamma = g1 - 1
+    if out is None:
+        pin = torch.cuda.is_available()
+        out = {k: torch.empty(B, dtype=torch.int32, pin_memory=pin)
+               for k in ("accept_len", "token", "edge_flags", "rs_flags")}
+        out["p_row"] = torch.empty(B, V, dtype=torch.float32, pin_memory=pin) if want_p_row else None
+    st = lib.dssd_round_host(
+        tl.data_ptr(), _dtype_code(tl), _ptr(host.get("draft_tokens")), _ptr(host.get("draft_q_tok")),
+        _ptr(host.get("uniforms")), _ptr(host.get("draft_q")), host["uniforms_rs"].data_ptr(),
+        ctypes.c_float(temperature), B, gamma, V, out["accept_len"].data_ptr(), out["token"].data_ptr(),
+        _ptr(out.get("edge_flags")), _ptr(out.get("rs_flags")), _ptr(out.get("p_row")),
+        arena.data_ptr(), arena.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_round_host")
+    return out

@@ -1,0 +1,228 @@
+// C ABI of the library: argument checks, workspace carving, launches.  See include/dssd.h.
+#include <cuda_runtime.h>
+#include <math.h>
+
+#include "device_resample.h"
+#include "dssd.h"
+#include "edge_verify.h"
+
+namespace {
+
+thread_local int t_last_cuda_error = 0;
+
+dssd_status cuda_fail(cudaError_t e)
+{
+    t_last_cuda_error = (int)e;
+    return DSSD_ERR_CUDA;
+}
+
+// 0 = fine, else the status to return
+dssd_status check_sizes(int B, int gamma, int V)
+{
+    if (B < 1 || gamma < 0 || V < 1) return DSSD_ERR_INVALID_ARG;
+    if (V > DSSD_MAX_V) return DSSD_ERR_UNSUPPORTED;
+    if ((long long)B * ((long long)gamma + 1) > (long long)DSSD_MAX_ROWS) return DSSD_ERR_UNSUPPORTED;
+    return DSSD_OK;
+}
+
+int max_lse_slices(int V)
+{
+    const int smallest_slice = dssd::kEdgeLseSliceBytes / 4;
+    return (V + smallest_slice - 1) / smallest_slice;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+
+extern "C" {
+
+const char *dssd_status_string(int status)
+{
+    switch (status) {
+        case DSSD_OK: return "DSSD_OK";
+        case DSSD_ERR_INVALID_ARG: return "DSSD_ERR_INVALID_ARG";
+        case DSSD_ERR_UNSUPPORTED: return "DSSD_ERR_UNSUPPORTED";
+        case DSSD_ERR_WORKSPACE: return "DSSD_ERR_WORKSPACE";
+        case DSSD_ERR_CUDA: return "DSSD_ERR_CUDA";
+        default: return "DSSD_ERR_UNKNOWN";
+    }
+}
+
+int dssd_version(void) { return 100; }
+
+int dssd_last_cuda_error(void) { return t_last_cuda_error; }
+
+size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    return dssd::edge_workspace_layout(B, gamma, V, max_lse_slices(V), nullptr, nullptr);
+}
+
+dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                             const int32_t *draft_tokens, const float *draft_q_tok,
+                             const float *uniforms, float temperature, int B, int gamma, int V,
+                             int32_t *accept_len, float *p_row, float *p_tok, float *lse,
+                             uint32_t *flags, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !accept_len || !p_row) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(target_logits) % esz) || (reinterpret_cast<uintptr_t>(p_row) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_edge_verify_workspace_bytes(B, gamma, V))
+        return DSSD_ERR_WORKSPACE;
+
+    dssd::EdgeParams P{};
+    P.logits = target_logits;
+    P.row_stride = row_stride;
+    P.draft_tokens = draft_tokens;
+    P.draft_q_tok = draft_q_tok;
+    P.uniforms = uniforms;
+    P.temperature = temperature;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V;
+    P.accept_len = accept_len;
+    P.p_row = p_row;
+    P.p_tok = p_tok;
+    P.lse = lse;
+    P.flags = flags;
+    cudaError_t e = dssd::edge_verify_launch(P, (int)dtype, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    return dssd::resample_workspace_layout(B, V, nullptr, nullptr);
+}
+
+dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
+                                 const int32_t *accept_len, const float *uniforms, int B,
+                                 int gamma, int V, int32_t *token, uint32_t *flags,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (!p_row || !accept_len || !uniforms || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft_q) return DSSD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(p_row) % 4) || (reinterpret_cast<uintptr_t>(draft_q) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_device_resample_workspace_bytes(B, gamma, V))
+        return DSSD_ERR_WORKSPACE;
+
+    dssd::ResampleParams P{};
+    P.p_row = p_row;
+    P.draft_q = draft_q;
+    P.accept_len = accept_len;
+    P.uniforms = uniforms;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V;
+    P.token = token;
+    P.flags = flags;
+    cudaError_t e = dssd::resample_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+size_t dssd_round_host_arena_bytes(int B, int gamma, int V, dssd_dtype dtype)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return 0;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    const size_t Bz = (size_t)B, g = (size_t)gamma, Vz = (size_t)V;
+    size_t n = 0;
+    n += align256(Bz * (g + 1) * Vz * esz);  // target_logits
+    n += align256(Bz * g * Vz * 4);          // draft_q
+    n += 3 * align256(Bz * g * 4);           // draft_tokens, draft_q_tok, uniforms
+    n += align256(Bz * 4);                   // uniforms_rs
+    n += align256(Bz * Vz * 4);              // p_row
+    n += 4 * align256(Bz * 4);               // accept_len, token, edge flags, resample flags
+    n += align256(dssd_edge_verify_workspace_bytes(B, gamma, V));
+    n += align256(dssd_device_resample_workspace_bytes(B, gamma, V));
+    return n;
+}
+
+dssd_status dssd_round_host(const void *target_logits, dssd_dtype dtype,
+                            const int32_t *draft_tokens, const float *draft_q_tok,
+                            const float *uniforms, const float *draft_q, const float *uniforms_rs,
+                            float temperature, int B, int gamma, int V, int32_t *accept_len,
+                            int32_t *token, uint32_t *edge_flags, uint32_t *rs_flags,
+                            float *p_row, void *device_arena, size_t arena_bytes,
+                            void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !uniforms_rs || !accept_len || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms || !draft_q)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255u) ||
+        arena_bytes < dssd_round_host_arena_bytes(B, gamma, V, dtype))
+        return DSSD_ERR_WORKSPACE;
+
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    const size_t Bz = (size_t)B, g = (size_t)gamma, Vz = (size_t)V;
+    char *cur = static_cast<char *>(device_arena);
+    auto take = [&](size_t bytes) {
+        char *p = cur;
+        cur += align256(bytes);
+        return p;
+    };
+    void *d_logits = take(Bz * (g + 1) * Vz * esz);
+    float *d_q = reinterpret_cast<float *>(take(Bz * g * Vz * 4));
+    int32_t *d_tok_in = reinterpret_cast<int32_t *>(take(Bz * g * 4));
+    float *d_qtok = reinterpret_cast<float *>(take(Bz * g * 4));
+    float *d_u = reinterpret_cast<float *>(take(Bz * g * 4));
+    float *d_urs = reinterpret_cast<float *>(take(Bz * 4));
+    float *d_prow = reinterpret_cast<float *>(take(Bz * Vz * 4));
+    int32_t *d_n = reinterpret_cast<int32_t *>(take(Bz * 4));
+    int32_t *d_token = reinterpret_cast<int32_t *>(take(Bz * 4));
+    uint32_t *d_ef = reinterpret_cast<uint32_t *>(take(Bz * 4));
+    uint32_t *d_rf = reinterpret_cast<uint32_t *>(take(Bz * 4));
+    const size_t ws_e = dssd_edge_verify_workspace_bytes(B, gamma, V);
+    const size_t ws_r = dssd_device_resample_workspace_bytes(B, gamma, V);
+    void *d_ws_e = take(ws_e);
+    void *d_ws_r = take(ws_r);
+
+    cudaError_t e;
+#define DSSD_TRY(call) \
+    if ((e = (call)) != cudaSuccess) return cuda_fail(e)
+    DSSD_TRY(cudaMemcpyAsync(d_logits, target_logits, Bz * (g + 1) * Vz * esz, cudaMemcpyHostToDevice, s));
+    if (gamma > 0) {
+        DSSD_TRY(cudaMemcpyAsync(d_tok_in, draft_tokens, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_qtok, draft_q_tok, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_u, uniforms, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_q, draft_q, Bz * g * Vz * 4, cudaMemcpyHostToDevice, s));
+    }
+    DSSD_TRY(cudaMemcpyAsync(d_urs, uniforms_rs, Bz * 4, cudaMemcpyHostToDevice, s));
+    st = dssd_edge_verify(d_logits, dtype, (int64_t)V, gamma ? d_tok_in : nullptr, gamma ? d_qtok : nullptr,
+                          gamma ? d_u : nullptr, temperature, B, gamma, V, d_n, d_prow, nullptr, nullptr,
+                          d_ef, d_ws_e, ws_e, cuda_stream);
+    if (st != DSSD_OK) return st;
+    st = dssd_device_resample(d_prow, gamma ? d_q : nullptr, d_n, d_urs, B, gamma, V, d_token, d_rf, d_ws_r,
+                              ws_r, cuda_stream);
+    if (st != DSSD_OK) return st;
+    DSSD_TRY(cudaMemcpyAsync(accept_len, d_n, Bz * 4, cudaMemcpyDeviceToHost, s));
+    DSSD_TRY(cudaMemcpyAsync(token, d_token, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (edge_flags) DSSD_TRY(cudaMemcpyAsync(edge_flags, d_ef, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (rs_flags) DSSD_TRY(cudaMemcpyAsync(rs_flags, d_rf, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (p_row) DSSD_TRY(cudaMemcpyAsync(p_row, d_prow, Bz * Vz * 4, cudaMemcpyDeviceToHost, s));
+#undef DSSD_TRY
+    return DSSD_OK;
+}
+
+}  // extern "C"

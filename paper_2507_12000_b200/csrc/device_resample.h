@@ -1,0 +1,33 @@
+// Host-side interface of the resample kernel (internal to the library).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace dssd {
+
+constexpr int kResampleChunk = 8192;  // vocabulary entries per ticket
+
+struct ResampleParams {
+    const float *p_row;
+    const float *draft_q;
+    const int32_t *accept_len;
+    const float *uniforms;
+    int B, gamma, V;
+    int32_t *token;
+    uint32_t *flags;
+    int n_chunks;
+    unsigned long long total_tickets;
+    // scratch
+    unsigned long long *ticket;
+    unsigned *seq_cnt;   // [B]
+    double *chunk_sum;   // [B, n_chunks]
+    size_t zero_bytes;
+};
+
+size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base);
+
+cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream);
+
+}  // namespace dssd

@@ -1,0 +1,120 @@
+// Device-side helpers shared by the verification kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dssd.h"
+
+namespace dssd {
+
+constexpr int kThreads = 256;           // threads per CTA in every kernel
+constexpr int kWarps = kThreads / 32;
+#define DSSD_NEG_INF (__int_as_float(0xff800000))
+
+// ---- memory ------------------------------------------------------------------------------
+
+// 16-byte streaming load of data that no one writes during the kernel; does not allocate in L1.
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 16-byte streaming store (evict-first): output that this kernel never reads back.
+__device__ __forceinline__ void st_stream16(void *p, float a, float b, float c, float d)
+{
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_release(unsigned *p, unsigned v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// ---- arithmetic --------------------------------------------------------------------------
+
+// 2^x on the special-function unit (max relative error about 2^-22; -inf -> 0, NaN -> NaN).
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <int DT>
+struct Elem;
+template <>
+struct Elem<DSSD_F32> {
+    static constexpr int kBytes = 4;
+    static constexpr int kVec = 4;   // elements per 16-byte vector
+    __device__ static __forceinline__ float load(const void *row, int64_t i)
+    {
+        return __ldg(reinterpret_cast<const float *>(row) + i);
+    }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+};
+template <>
+struct Elem<DSSD_BF16> {
+    static constexpr int kBytes = 2;
+    static constexpr int kVec = 8;
+    __device__ static __forceinline__ float load(const void *row, int64_t i)
+    {
+        uint32_t h = __ldg(reinterpret_cast<const unsigned short *>(row) + i);
+        return __uint_as_float(h << 16);
+    }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
+    {
+        f[0] = bf16_lo(v.x);
+        f[1] = bf16_hi(v.x);
+        f[2] = bf16_lo(v.y);
+        f[3] = bf16_hi(v.y);
+        f[4] = bf16_lo(v.z);
+        f[5] = bf16_hi(v.z);
+        f[6] = bf16_lo(v.w);
+        f[7] = bf16_hi(v.w);
+    }
+};
+
+__device__ __forceinline__ double warp_sum(double x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ float warp_max(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+}  // namespace dssd

@@ -1,0 +1,107 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, sizes its workspaces, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2507_12000_b200 import build
+
+    build.build()
+    from paper_2507_12000_b200 import binding
+
+    return binding
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "dssd.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(dssd_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported(B):
+    names = _declared()
+    assert "dssd_edge_verify" in names and "dssd_device_resample" in names and "dssd_round_host" in names
+    for n in names:
+        assert hasattr(B.lib, n), n
+
+
+def test_version_and_status_strings(B):
+    assert B.lib.dssd_version() >= 100
+    assert B.lib.dssd_status_string(0) == b"DSSD_OK"
+    assert B.lib.dssd_status_string(3) == b"DSSD_ERR_WORKSPACE"
+    assert B.lib.dssd_status_string(99) == b"DSSD_ERR_UNKNOWN"
+
+
+def test_workspace_sizes(B):
+    assert B.dssd_edge_verify_workspace_bytes(0, 4, 100) == 0
+    assert B.dssd_edge_verify_workspace_bytes(1, -1, 100) == 0
+    assert B.dssd_edge_verify_workspace_bytes(1, 4, 0) == 0
+    a = B.dssd_edge_verify_workspace_bytes(1, 4, 1024)
+    b = B.dssd_edge_verify_workspace_bytes(256, 4, 151936)
+    c = B.dssd_edge_verify_workspace_bytes(1024, 16, 50272)
+    assert 0 < a < b < c < 64 << 20 and a % 256 == 0
+    r = B.dssd_device_resample_workspace_bytes(256, 4, 151936)
+    assert 0 < r < 4 << 20
+    assert B.dssd_round_host_arena_bytes(8, 4, 32000, B.DSSD_BF16) > 8 * 5 * 32000 * 2 + 8 * 4 * 32000 * 4
+    assert B.dssd_round_host_arena_bytes(8, 4, 32000, 7) == 0
+
+
+def test_bad_arguments_are_rejected_before_any_launch(B):
+    L = B.lib
+    buf = (ctypes.c_char * 4096)()
+    p = ctypes.addressof(buf)
+    p = (p + 255) & ~255  # any non-NULL, aligned address: it is never dereferenced on these paths
+    f = ctypes.c_float
+    ok_ws = 1 << 30
+
+    def ev(logits=p, dtype=0, stride=16, tok=p, qt=p, u=p, T=1.0, Bn=1, g=2, V=16, n=p, prow=p, ws=p, wsb=ok_ws):
+        return L.dssd_edge_verify(logits, dtype, stride, tok, qt, u, f(T), Bn, g, V, n, prow, None, None, None,
+                                  ws, wsb, None)
+
+    assert ev(logits=None) == B.DSSD_ERR_INVALID_ARG
+    assert ev(n=None) == B.DSSD_ERR_INVALID_ARG
+    assert ev(prow=None) == B.DSSD_ERR_INVALID_ARG
+    assert ev(tok=None) == B.DSSD_ERR_INVALID_ARG
+    assert ev(Bn=0) == B.DSSD_ERR_INVALID_ARG
+    assert ev(g=-1) == B.DSSD_ERR_INVALID_ARG
+    assert ev(V=0) == B.DSSD_ERR_INVALID_ARG
+    assert ev(T=0.0) == B.DSSD_ERR_INVALID_ARG
+    assert ev(T=-1.0) == B.DSSD_ERR_INVALID_ARG
+    assert ev(T=float("inf")) == B.DSSD_ERR_INVALID_ARG
+    assert ev(T=float("nan")) == B.DSSD_ERR_INVALID_ARG
+    assert ev(stride=15) == B.DSSD_ERR_INVALID_ARG
+    assert ev(dtype=5) == B.DSSD_ERR_UNSUPPORTED
+    assert ev(V=(1 << 30) + 1, stride=(1 << 30) + 1) == B.DSSD_ERR_UNSUPPORTED
+    assert ev(Bn=1 << 30, g=3) == B.DSSD_ERR_UNSUPPORTED
+    assert ev(ws=None) == B.DSSD_ERR_WORKSPACE
+    assert ev(ws=p + 8) == B.DSSD_ERR_WORKSPACE
+    assert ev(wsb=16) == B.DSSD_ERR_WORKSPACE
+
+    def rs(prow=p, q=p, n=p, u=p, Bn=1, g=2, V=16, tok=p, ws=p, wsb=ok_ws):
+        return L.dssd_device_resample(prow, q, n, u, Bn, g, V, tok, None, ws, wsb, None)
+
+    assert rs(prow=None) == B.DSSD_ERR_INVALID_ARG
+    assert rs(q=None) == B.DSSD_ERR_INVALID_ARG
+    assert rs(tok=None) == B.DSSD_ERR_INVALID_ARG
+    assert rs(Bn=-3) == B.DSSD_ERR_INVALID_ARG
+    assert rs(wsb=8) == B.DSSD_ERR_WORKSPACE
+    assert rs(ws=None) == B.DSSD_ERR_WORKSPACE
+
+    assert L.dssd_round_host(None, 0, p, p, p, p, p, f(1.0), 1, 2, 16, p, p, None, None, None, p, ok_ws, None) \
+        == B.DSSD_ERR_INVALID_ARG
+    assert L.dssd_round_host(p, 0, p, p, p, p, p, f(1.0), 1, 2, 16, p, p, None, None, None, p, 64, None) \
+        == B.DSSD_ERR_WORKSPACE
+    assert L.dssd_last_cuda_error() == 0
+
+
+def test_missing_library_fails_loudly(B, monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(ImportError, match="no CPU fallback"):
+        B._load()
