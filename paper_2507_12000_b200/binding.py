@@ -13,7 +13,8 @@ from typing import Dict, Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libdssd.so")
+# DSSD_LIBRARY overrides the in-tree library (e.g. a build with other tuning constants)
+LIB_PATH = os.environ.get("DSSD_LIBRARY") or os.path.join(_PKG, "libdssd.so")
 
 DSSD_OK = 0
 DSSD_ERR_INVALID_ARG = 1

@@ -25,12 +25,6 @@ dssd_status check_sizes(int B, int gamma, int V)
     return DSSD_OK;
 }
 
-int max_lse_slices(int V)
-{
-    const int smallest_slice = dssd::kEdgeLseSliceBytes / 4;
-    return (V + smallest_slice - 1) / smallest_slice;
-}
-
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 }  // namespace
@@ -56,7 +50,7 @@ int dssd_last_cuda_error(void) { return t_last_cuda_error; }
 size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V)
 {
     if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
-    return dssd::edge_workspace_layout(B, gamma, V, max_lse_slices(V), nullptr, nullptr);
+    return dssd::edge_workspace_layout(B, gamma, dssd::edge_max_runs_per_row(V), nullptr, nullptr);
 }
 
 dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,

@@ -1,22 +1,24 @@
 // Edge half of the verification round as one persistent streaming kernel.
 //
-// The work is an ordered list of tickets that WARPS draw from a global counter.  Group g of the list:
-//   LSE(g, i, k)       stream slice k of target row (g, i): max and sum of exp -> 8-byte partial
-//   EMIT(g - lag, k)   first-rejection scan over the sequence's acceptance bits (warp ballot), then
-//                      slice k of row n streamed again and p_row = exp(l/T - lse) written
-// A warp draws one ticket ahead and requests the first half of its next LSE slice before it works on
-// the second half of the current one, so loads are always in flight.  Each LSE ticket bumps its row's
-// arrival counter; the warp that brings the last slice of a row folds the row's partials (float64
-// log-sum-exp) and evaluates the acceptance test for that position, at once and without waiting.
-// Drawing is self-balancing: a warp that was held up simply draws fewer tickets, so the tickets
-// below the counter complete within a short window, EMIT tickets (which trail their sequence by
-// `lag` groups) normally find every row folded, and row n is read the second time from L2.
-// An EMIT ticket whose rows are not all folded yet is parked and retried after each later ticket;
-// only when a second one would have to be parked, or the list is exhausted, does a warp wait
-// (bounded, with a timeout flag) - for rows whose LSE tickets were drawn by running warps.
-// A warp works alone: no shared memory, no CTA barrier.  Results travel through 8-byte slots that
-// the host pre-filled with all ones and that carry their own validity, so no fence is needed:
-// a consumer that sees the fill pattern knows the store has not landed yet.
+// Every warp is an independent worker with a private ring of shared-memory stages.  Logits
+// travel global -> shared memory as bulk asynchronous copies (TMA, untiled) that the warp's
+// lane 0 issues up to kEdgeStages slices ahead; a stage's arrival is signalled on an mbarrier.
+// Work comes as tickets drawn from global counters:
+//   LSE(row, run)    a run of consecutive slices of one target row: online maximum and sum of
+//                    2^(l * c1 - ref2) in float32 -> one 8-byte partial (ref2, sum).  ref2 is an
+//                    integer, so partials combine by exact power-of-two scaling.
+//   EMIT(slot, run)  a run of slices of row n of a sequence taken from the `ready` queue: the row
+//                    is streamed again (from L2) and p_row = 2^(l * c1 - ref2) / S is written.
+// The warp that brings a row's last partial folds the row (float64 log-sum-exp, acceptance test
+// of that position); the warp that folds a sequence's last row runs the first-rejection scan
+// (ballot + find-first-set) and pushes the sequence to `ready`.  EMIT tickets are claimed, by
+// compare-and-swap, only for sequences already pushed, and are preferred over LSE tickets, so the
+// second read of row n follows the first closely and hits L2.
+// Nothing on this path waits on a fence: results travel through 8-byte slots that the host
+// pre-filled with all ones and that carry their own validity; a consumer that sees the fill
+// pattern polls (bounded) for a store that a running warp has already issued.  A warp only ever
+// waits for work held by running warps, and never while its own ring holds unprocessed slices,
+// so the kernel needs no co-residency guarantee.
 #include "edge_verify.h"
 
 #include <math.h>
@@ -27,22 +29,22 @@ namespace dssd {
 
 namespace {
 
+#ifndef DSSD_EDGE_WAR
+#define DSSD_EDGE_WAR 1
+#endif
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kVPL = kEdgeVecPerLane;
+constexpr int kS = kEdgeSliceBytes;
 constexpr unsigned kBitAccept = 1u, kBitBadToken = 2u, kBitNonFinite = 4u, kBitTimeout = 8u;
 
-enum Kind : int { kEnd = 0, kSkip = 1, kLseFast = 2, kLseSlow = 3, kEmit = 4 };
-
-struct Ticket {
-    int kind;
-    int slice;
-    long long index;  // LSE: row; EMIT: sequence
-};
-
-__device__ __forceinline__ float ref_of(float m) { return m == DSSD_NEG_INF ? 0.f : m; }
+enum Kind : int { kEnd = 0, kIdle = 1, kLse = 2, kEmit = 3 };
 
 // counters start at all ones (the workspace fill pattern): logical value = raw + 1
 __device__ __forceinline__ unsigned logical(unsigned raw) { return raw + 1u; }
+__device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
+
+__device__ __forceinline__ unsigned long long shfl0(unsigned long long v) { return __shfl_sync(kFull, v, 0); }
+__device__ __forceinline__ int shfl0(int v) { return __shfl_sync(kFull, v, 0); }
+__device__ __forceinline__ float shfl0(float v) { return __shfl_sync(kFull, v, 0); }
 
 template <int DT>
 __device__ __forceinline__ const char *row_ptr(const EdgeParams &P, long long row)
@@ -50,237 +52,196 @@ __device__ __forceinline__ const char *row_ptr(const EdgeParams &P, long long ro
     return static_cast<const char *>(P.logits) + (size_t)row * (size_t)P.row_stride * Elem<DT>::kBytes;
 }
 
-template <int DT>
-__device__ __forceinline__ Ticket decode(const EdgeParams &P, unsigned t)
-{
-    Ticket k{kEnd, 0, 0};
-    if (t >= P.total_tickets) return k;
-    k.kind = kSkip;
-    const unsigned g = t / P.tickets_per_group;
-    const int idx = (int)(t - g * P.tickets_per_group);
-    if (idx < P.lse_tickets) {
-        if ((int)g >= P.B) return k;
-        const int pos = idx / P.n_lse_slices;
-        k.slice = idx - pos * P.n_lse_slices;
-        k.index = (long long)g * (P.gamma + 1) + pos;
-        const int e0 = k.slice * P.lse_slice;
-        const uintptr_t a = reinterpret_cast<uintptr_t>(row_ptr<DT>(P, k.index)) + (size_t)e0 * Elem<DT>::kBytes;
-        k.kind = (e0 + P.lse_slice <= P.V && (a & 15u) == 0) ? kLseFast : kLseSlow;
-        return k;
-    }
-    const long long b = (long long)g - P.lag;
-    if (b < 0 || b >= P.B) return k;
-    k.kind = kEmit;
-    k.index = b;
-    k.slice = idx - P.lse_tickets;
-    return k;
-}
+// One slice of work, identical in every lane of the warp.
+struct Slice {
+    int kind;
+    int k;          // slice index within the row
+    int first_last; // bit0: first slice of its ticket, bit1: last
+    int run;        // ticket index within the row (LSE: partial slot)
+    long long row;  // LSE: the row; EMIT: row n of the sequence
+    long long b;    // EMIT: the sequence, -1 when nothing may be written
+    float ref2, invS;  // EMIT
+};
 
-// one half (kVPL 16-byte vectors per lane) of a full, aligned LSE slice
-template <int DT>
-__device__ __forceinline__ void load_half(const EdgeParams &P, const Ticket &k, int half, uint4 (&v)[kVPL])
-{
-    const int lane = threadIdx.x & 31;
-    const uint4 *p = reinterpret_cast<const uint4 *>(row_ptr<DT>(P, k.index) + (size_t)k.slice * kEdgeLseSliceBytes) +
-                     half * (32 * kVPL) + lane;
-#pragma unroll
-    for (int u = 0; u < kVPL; ++u) v[u] = ld_stream16(p + u * 32);
-}
+// Where the warp is in its current ticket, and what lane 0 has fetched ahead.  Values fetched
+// ahead are kept raw (as loaded) and converted where they are used, so that nothing depends on
+// a load or atomic until its round trip is over.
+struct Cursor {
+    int kind;
+    int k, k_begin, k_end, run;
+    long long row, b;
+    float ref2, invS;
+    unsigned long long lse_raw;   // lane 0: atomic result holding the LSE ticket in hand
+    unsigned long long head_raw;  // lane 0: last value loaded from emit_head
+    unsigned tail_raw;            // lane 0: last value loaded from ready_tail
+    unsigned long long parked;    // lane 0: EMIT ticket claimed ahead of its sequence, or kNoTicket
+};
+constexpr unsigned long long kNoTicket = ~0ull;
 
-struct Online {  // per-lane running max m and sum of 2^((z - ref(m)) * c1)
-    float m, s0, s1;
+// Geometry of slice k of a row: an optional scalar head (up to the first 16-byte boundary, slice
+// 0 only), a 16-byte aligned body that one bulk copy brings in, a scalar tail (< 16 bytes).
+struct Geo {
+    const char *rowp;
+    const char *src;  // body start
+    uint32_t bulk;    // body bytes, a multiple of 16
+    int e0;           // element index of the body's first element
+    int head;         // scalar elements [0, head)
+    int tail;         // scalar elements [e0 + bulk / size, +tail)
 };
 
 template <int DT>
-__device__ __forceinline__ void accum_half(Online &o, const uint4 (&v)[kVPL], float c1)
+__device__ __forceinline__ Geo slice_geo(const EdgeParams &P, long long row, int k)
 {
     using E = Elem<DT>;
-    float m = o.m;
-#pragma unroll
-    for (int u = 0; u < kVPL; ++u) {
-        float f[E::kVec];
-        E::unpack(v[u], f);
-#pragma unroll
-        for (int j = 0; j < E::kVec; ++j) m = fmaxf(m, f[j]);
-    }
-    if (m > o.m) {
-        const float f = (o.m == DSSD_NEG_INF) ? 0.f : ex2((o.m - m) * c1);
+    Geo g;
+    g.rowp = row_ptr<DT>(P, row);
+    const long long rowbytes = (long long)P.V * E::kBytes;
+    long long h = (long long)((16u - (unsigned)(reinterpret_cast<uintptr_t>(g.rowp) & 15u)) & 15u);
+    if (h > rowbytes) h = rowbytes;
+    const long long off = (long long)k * kS;
+    long long len = rowbytes - h - off;
+    len = len < 0 ? 0 : (len > kS ? kS : len);
+    g.bulk = (uint32_t)len & ~15u;
+    g.src = g.rowp + h + off;
+    g.e0 = (int)((h + off) / E::kBytes);
+    g.head = k == 0 ? (int)(h / E::kBytes) : 0;
+    g.tail = (int)((len - g.bulk) / E::kBytes);
+    return g;
+}
+
+// ---- per-lane online log-sum-exp state ---------------------------------------------------
+
+struct Online {
+    float m;    // running maximum of the raw logits (-inf: nothing seen)
+    float ref;  // rint(m * c1), or 0 while m == -inf: terms are 2^(l * c1 - ref) <= 2^0.5
+    float s0, s1, s2, s3;
+};
+
+__device__ __forceinline__ void online_reset(Online &o)
+{
+    o.m = DSSD_NEG_INF;
+    o.ref = 0.f;
+    o.s0 = o.s1 = o.s2 = o.s3 = 0.f;
+}
+
+__device__ __forceinline__ void online_raise(Online &o, float bm, float c1)
+{
+    if (bm > o.m) {
+        const float nref = rintf(bm * c1);
+        const float f = (o.m == DSSD_NEG_INF) ? 0.f : ex2(o.ref - nref);  // an exact power of two
         o.s0 *= f;
         o.s1 *= f;
-        o.m = m;
-    }
-    const float ref = ref_of(o.m);
-#pragma unroll
-    for (int u = 0; u < kVPL; ++u) {
-        float f[E::kVec];
-        E::unpack(v[u], f);
-#pragma unroll
-        for (int j = 0; j < E::kVec; j += 2) {
-            o.s0 += ex2((f[j] - ref) * c1);
-            o.s1 += ex2((f[j + 1] - ref) * c1);
-        }
+        o.s2 *= f;
+        o.s3 *= f;
+        o.m = bm;
+        o.ref = nref;
     }
 }
 
-// lane-local (m, s) -> warp-wide (M, S), one 8-byte store
-__device__ __forceinline__ void publish_partial(const EdgeParams &P, const Ticket &k, float m, float s)
+__device__ __forceinline__ void online_add(Online &o, float z, float c1)
 {
-    const float M = warp_max(m);
-    s *= (m == DSSD_NEG_INF) ? 0.f : ex2((m - ref_of(M)) * P.c1);
-    s = warp_sum(s);
-    if ((threadIdx.x & 31) == 0)
-        st_relaxed_u64(&P.part[(size_t)k.index * P.n_lse_slices + k.slice],
-                       (unsigned long long)__float_as_uint(M) | ((unsigned long long)__float_as_uint(s) << 32));
+    online_raise(o, z, c1);
+    o.s0 += ex2(fmaf(z, c1, -o.ref));
 }
 
-// LSE ticket, ragged or unaligned slice: scalar head, vector body, scalar tail, online max
 template <int DT>
-__device__ __noinline__ void lse_slow(const EdgeParams &P, const Ticket &k)
+__device__ __forceinline__ void accum_block(Online &o, const uint4 (&v)[4], float c1);
+
+template <>
+__device__ __forceinline__ void accum_block<DSSD_BF16>(Online &o, const uint4 (&v)[4], float c1)
+{
+    uint32_t mx = max_bf16x2(max_bf16x2(v[0].x, v[0].y), max_bf16x2(v[0].z, v[0].w));
+#pragma unroll
+    for (int u = 1; u < 4; ++u)
+        mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(v[u].x, v[u].y), max_bf16x2(v[u].z, v[u].w)));
+    online_raise(o, fmaxf(bf16_lo(mx), bf16_hi(mx)), c1);
+    const float nref = -o.ref;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        o.s0 += ex2(fmaf(bf16_lo(v[u].x), c1, nref));
+        o.s1 += ex2(fmaf(bf16_hi(v[u].x), c1, nref));
+        o.s2 += ex2(fmaf(bf16_lo(v[u].y), c1, nref));
+        o.s3 += ex2(fmaf(bf16_hi(v[u].y), c1, nref));
+        o.s0 += ex2(fmaf(bf16_lo(v[u].z), c1, nref));
+        o.s1 += ex2(fmaf(bf16_hi(v[u].z), c1, nref));
+        o.s2 += ex2(fmaf(bf16_lo(v[u].w), c1, nref));
+        o.s3 += ex2(fmaf(bf16_hi(v[u].w), c1, nref));
+    }
+}
+
+template <>
+__device__ __forceinline__ void accum_block<DSSD_F32>(Online &o, const uint4 (&v)[4], float c1)
+{
+    float bm = DSSD_NEG_INF;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        bm = fmaxf(bm, fmaxf(fmaxf(__uint_as_float(v[u].x), __uint_as_float(v[u].y)),
+                             fmaxf(__uint_as_float(v[u].z), __uint_as_float(v[u].w))));
+    online_raise(o, bm, c1);
+    const float nref = -o.ref;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        o.s0 += ex2(fmaf(__uint_as_float(v[u].x), c1, nref));
+        o.s1 += ex2(fmaf(__uint_as_float(v[u].y), c1, nref));
+        o.s2 += ex2(fmaf(__uint_as_float(v[u].z), c1, nref));
+        o.s3 += ex2(fmaf(__uint_as_float(v[u].w), c1, nref));
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ uint4 neg_inf_vec()
+{
+    return DT == DSSD_BF16 ? make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u)
+                           : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+}
+
+// One slice of an LSE ticket: the stage's vectors, then the scalar head and tail from global.
+template <int DT>
+__device__ __forceinline__ void lse_consume(const EdgeParams &P, const Geo &g, uint32_t stage, Online &o)
 {
     using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
     const float c1 = P.c1;
-    const char *rowp = row_ptr<DT>(P, k.index);
-    const int e0 = k.slice * P.lse_slice, e1 = min(P.V, e0 + P.lse_slice);
-    const uintptr_t a0 = reinterpret_cast<uintptr_t>(rowp) + (size_t)e0 * E::kBytes;
-    int head = (int)(((16u - (unsigned)(a0 & 15u)) & 15u) / E::kBytes);
-    head = min(head, e1 - e0);
-    const int nvec = (e1 - e0 - head) / E::kVec;
-    const int tail0 = e0 + head + nvec * E::kVec;
-    const uint4 *body = reinterpret_cast<const uint4 *>(rowp + (size_t)(e0 + head) * E::kBytes);
-    float m = DSSD_NEG_INF, s = 0.f;
-    auto add = [&](float z) {
-        if (z > m) {
-            s *= (m == DSSD_NEG_INF) ? 0.f : ex2((m - z) * c1);
-            m = z;
-        }
-        s += ex2((z - ref_of(m)) * c1);
-    };
-    for (int i = lane; i < nvec; i += 32) {
-        float f[E::kVec];
-        E::unpack(ld_stream16(body + i), f);
+    const int nvec = (int)(g.bulk >> 4);
+    const uint32_t base = stage + (uint32_t)lane * 16u;
+    int i = lane;
+    for (; i + 96 < nvec; i += 128) {
+        uint4 v[4];
 #pragma unroll
-        for (int j = 0; j < E::kVec; ++j) add(f[j]);
+        for (int u = 0; u < 4; ++u) v[u] = lds16(base + (uint32_t)(i - lane + 32 * u) * 16u);
+        accum_block<DT>(o, v, c1);
     }
-    if (lane < head) add(E::load(rowp, e0 + lane));
-    if (lane < e1 - tail0) add(E::load(rowp, tail0 + lane));
-    publish_partial(P, k, m, s);
+    if (i < nvec) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            v[u] = (i + 32 * u < nvec) ? lds16(base + (uint32_t)(i - lane + 32 * u) * 16u) : neg_inf_vec<DT>();
+        accum_block<DT>(o, v, c1);
+    }
+    if (lane < g.head) online_add(o, E::load(g.rowp, lane), c1);
+    if (lane < g.tail) online_add(o, E::load(g.rowp, (int64_t)g.e0 + (int64_t)(g.bulk / E::kBytes) + lane), c1);
 }
 
-// Run by the warp that brought a row's last slice: the partials of the row -> log-sum-exp
-// (float64), acceptance test, RowInfo.
-template <int DT>
-__device__ __noinline__ void fold_row(const EdgeParams &P, long long row)
+// lane-local state -> the ticket's partial (ref2, sum), one 8-byte store
+__device__ __forceinline__ void publish_partial(const EdgeParams &P, long long row, int run, const Online &o)
 {
-    using E = Elem<DT>;
-    const int lane = threadIdx.x & 31;
-    const double T = (double)P.temperature;
-    const unsigned long long *part = reinterpret_cast<const unsigned long long *>(P.part) + (size_t)row * P.n_lse_slices;
-    const long long b = row / (P.gamma + 1);
-    const int pos = (int)(row - b * (P.gamma + 1));
-    // lane 0 starts on the drafted token early: its loads overlap the partials'
-    int x = -1;
-    float zx = 0.f, qx = 0.f, ux = 0.f;
-    if (lane == 0 && pos < P.gamma) {
-        const size_t di = (size_t)b * P.gamma + pos;
-        x = P.draft_tokens[di];
-        qx = P.draft_q_tok[di];
-        ux = P.uniforms[di];
-        if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
+    const bool empty = (o.m == DSSD_NEG_INF);
+    const float R = warp_max(empty ? DSSD_NEG_INF : o.ref);
+    float s = (o.s0 + o.s1) + (o.s2 + o.s3);
+    s = empty ? 0.f : s * ex2(o.ref - R);  // exact scaling
+    s = warp_sum(s);
+    if ((threadIdx.x & 31) == 0) {
+        const float Rp = (R == DSSD_NEG_INF) ? 0.f : R;
+        st_relaxed_u64(&P.part[(size_t)row * P.n_lse_runs + run],
+                       (unsigned long long)__float_as_uint(Rp) | ((unsigned long long)__float_as_uint(s) << 32));
     }
-    // The arrival counter says every slice has been counted; a partial whose store has not landed
-    // yet still shows the fill pattern and is polled for.
-    float Mr = DSSD_NEG_INF;
-    double S = 0.0;
-    bool bad = false, timeout = false;
-    auto fetch = [&](int k) {
-        unsigned long long w = ld_relaxed_u64(part + k);
-        for (unsigned it = 0; (unsigned)w == kFull && it < P.spin_limit; ++it) {
-            __nanosleep(32);
-            w = ld_relaxed_u64(part + k);
-        }
-        if ((unsigned)w == kFull) timeout = true;
-        return w;
-    };
-    constexpr int kKeep = 4;  // partials per lane kept in registers: rows of up to 128 slices in one pass
-    if (P.n_lse_slices <= 32 * kKeep) {
-        unsigned long long w[kKeep];
-#pragma unroll
-        for (int j = 0; j < kKeep; ++j) w[j] = (lane + 32 * j < P.n_lse_slices) ? ld_relaxed_u64(part + lane + 32 * j) : 0ull;
-#pragma unroll
-        for (int j = 0; j < kKeep; ++j)
-            if (lane + 32 * j < P.n_lse_slices) {
-                if ((unsigned)w[j] == kFull) w[j] = fetch(lane + 32 * j);
-                if ((unsigned)w[j] != kFull) Mr = fmaxf(Mr, __uint_as_float((unsigned)w[j]));
-            }
-        timeout = __any_sync(kFull, timeout);
-        Mr = warp_max(Mr);
-#pragma unroll
-        for (int j = 0; j < kKeep; ++j)
-            if (lane + 32 * j < P.n_lse_slices && !timeout) {
-                const float pm = __uint_as_float((unsigned)w[j]), ps = __uint_as_float((unsigned)(w[j] >> 32));
-                if (ps != ps) bad = true;
-                if (pm != DSSD_NEG_INF) S += (double)ps * exp(((double)pm - (double)Mr) / T);
-            }
-    } else {
-        for (int k = lane; k < P.n_lse_slices; k += 32) {
-            const unsigned long long w = fetch(k);
-            if ((unsigned)w != kFull) Mr = fmaxf(Mr, __uint_as_float((unsigned)w));
-        }
-        timeout = __any_sync(kFull, timeout);
-        Mr = warp_max(Mr);
-        if (!timeout) {
-            for (int k = lane; k < P.n_lse_slices; k += 32) {
-                const unsigned long long w = ld_relaxed_u64(part + k);
-                const float pm = __uint_as_float((unsigned)w), ps = __uint_as_float((unsigned)(w >> 32));
-                if (ps != ps) bad = true;
-                if (pm != DSSD_NEG_INF) S += (double)ps * exp(((double)pm - (double)Mr) / T);
-            }
-        }
-    }
-    S = warp_sum(S);
-    bad = __any_sync(kFull, bad);
-    if (lane != 0) return;
-    double lse = (double)Mr / T + log(S);
-    const bool finite = !timeout && !bad && (lse == lse) && (fabs(lse) < INFINITY);
-    if (!finite) lse = NAN;
-    unsigned bits = (finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u);
-    if (timeout) *P.error = 1u;
-    if (P.lse) P.lse[row] = (float)lse;
-    if (pos < P.gamma) {
-        double p = NAN;
-        bool accept = false;
-        if (x < 0 || x >= P.V) {
-            bits |= kBitBadToken;
-        } else {
-            // u < min(1, p(x)/q(x)), evaluated in float64
-            p = exp((double)zx / T - lse);
-            const double q = (double)qx;
-            const double u = (double)ux;
-            double ratio;
-            if (q != q) ratio = NAN;
-            else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
-            else ratio = p / q;
-            accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
-        }
-        if (P.p_tok) P.p_tok[(size_t)b * P.gamma + pos] = (float)p;
-        bits |= accept ? kBitAccept : 0u;
-    }
-    const float invS = finite ? (float)(1.0 / S) : NAN;
-    unsigned long long *ri = reinterpret_cast<unsigned long long *>(P.row_info + row);
-    st_relaxed_u64(ri, (unsigned long long)__float_as_uint(Mr) | ((unsigned long long)__float_as_uint(invS) << 32));
-    st_relaxed_u64(ri + 1, (unsigned long long)bits);
 }
 
-// EMIT ticket: first-rejection scan, then one slice of p_row[b, :].
-// With `wait` false it returns false, having done nothing, if some row of the sequence is not
-// folded yet; with `wait` true it polls (bounded) for those rows.
-template <int DT>
-__device__ __noinline__ bool emit_slice(const EdgeParams &P, long long b, int slice, bool wait)
+// Run by the warp that folded the last row of sequence b: first-rejection scan over the
+// acceptance bits (one row per lane, ballot + find-first-set), then the push to `ready`.
+__device__ __noinline__ void finish_sequence(const EdgeParams &P, long long b)
 {
-    using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    // one row per lane: its acceptance bits and its (M, 1/S); ballot + find-first-set gives n
     int n = P.gamma;
     unsigned fl = 0;
     unsigned long long w0n = 0;
@@ -293,18 +254,15 @@ __device__ __noinline__ bool emit_slice(const EdgeParams &P, long long b, int sl
             const unsigned long long *ri = reinterpret_cast<const unsigned long long *>(P.row_info + b * (P.gamma + 1) + i);
             w0 = ld_relaxed_u64(ri);
             bits = (unsigned)ld_relaxed_u64(ri + 1);
-            if (wait) {
-                for (unsigned it = 0; (bits == kFull || (unsigned)w0 == kFull) && it < P.spin_limit; ++it) {
-                    __nanosleep(100);
-                    w0 = ld_relaxed_u64(ri);
-                    bits = (unsigned)ld_relaxed_u64(ri + 1);
-                }
+            for (unsigned it = 0; (bits == kFull || (unsigned)w0 == kFull) && it < P.spin_limit; ++it) {
+                __nanosleep(64);
+                w0 = ld_relaxed_u64(ri);
+                bits = (unsigned)ld_relaxed_u64(ri + 1);
             }
-            if (bits == kFull || (unsigned)w0 == kFull) { timeout = true; bits = kBitTimeout; }
-        }
-        if (__any_sync(kFull, timeout)) {
-            if (!wait) return false;
-            timeout = true;
+            if (bits == kFull || (unsigned)w0 == kFull) {
+                timeout = true;
+                bits = kBitTimeout;
+            }
         }
         const unsigned rej = __ballot_sync(kFull, i < P.gamma && !(bits & kBitAccept));
         if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
@@ -313,115 +271,397 @@ __device__ __noinline__ bool emit_slice(const EdgeParams &P, long long b, int sl
               (__ballot_sync(kFull, bits & kBitTimeout) ? DSSD_EDGE_FLAG_TIMEOUT : 0u);
         if (n >= base && n < base + 32) w0n = __shfl_sync(kFull, w0, n - base);
     }
-    if (slice == 0 && lane == 0) {
+    timeout = __any_sync(kFull, timeout);
+    if (lane == 0) {
         P.accept_len[b] = timeout ? -1 : n;
         if (P.flags) P.flags[b] = fl;
         if (timeout) *P.error = 1u;
+        const unsigned slot = logical(atomicAdd(P.ready_tail, 1u));
+        unsigned long long *rs = reinterpret_cast<unsigned long long *>(P.ready + slot);
+        st_relaxed_u64(rs, (unsigned long long)(unsigned)b | ((unsigned long long)(unsigned)(timeout ? -1 : n) << 32));
+        st_relaxed_u64(rs + 1, timeout ? 0ull : w0n);
     }
-    if (timeout) return true;
-    const long long row = b * (P.gamma + 1) + n;
-    const float M = ref_of(__uint_as_float((unsigned)w0n)), invS = __uint_as_float((unsigned)(w0n >> 32));
-    const float c1 = P.c1;
-    const char *rowp = row_ptr<DT>(P, row);
-    float *outp = P.p_row + (size_t)b * P.V;
-    const int e0 = slice * P.emit_slice, e1 = min(P.V, e0 + P.emit_slice);
-    const bool aligned = (((reinterpret_cast<uintptr_t>(rowp) + (size_t)e0 * E::kBytes) |
-                           reinterpret_cast<uintptr_t>(outp + e0)) & 15u) == 0;
-    int done = e0;
-    if (aligned) {
-        const int nvec = (e1 - e0) / E::kVec;
-        const uint4 *body = reinterpret_cast<const uint4 *>(rowp + (size_t)e0 * E::kBytes);
-        constexpr int kU = 4;
-        int i = lane;
-        for (; i + (kU - 1) * 32 < nvec; i += kU * 32) {
-            uint4 v[kU];
-#pragma unroll
-            for (int u = 0; u < kU; ++u) v[u] = ld_stream16(body + i + u * 32);
-#pragma unroll
-            for (int u = 0; u < kU; ++u) {
-                float f[E::kVec];
-                E::unpack(v[u], f);
-#pragma unroll
-                for (int j = 0; j < E::kVec; ++j) f[j] = ex2((f[j] - M) * c1) * invS;
-                float *o = outp + e0 + (size_t)(i + u * 32) * E::kVec;
-#pragma unroll
-                for (int j = 0; j < E::kVec; j += 4) st_stream16(o + j, f[j], f[j + 1], f[j + 2], f[j + 3]);
+}
+
+// Run by the warp that brought a row's last partial: partials -> log-sum-exp (float64),
+// acceptance test of the position, RowInfo; then the sequence's arrival count.
+template <int DT>
+__device__ __noinline__ void fold_row(const EdgeParams &P, long long row)
+{
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    const double c1 = (double)P.c1;
+    const unsigned long long *part = P.part + (size_t)row * P.n_lse_runs;
+    const long long b = row / (P.gamma + 1);
+    const int pos = (int)(row - b * (P.gamma + 1));
+    // lane 0 starts on the drafted token early: its loads overlap the partials'
+    int x = -1;
+    float zx = 0.f, qx = 0.f, ux = 0.f;
+    if (lane == 0 && pos < P.gamma) {
+        const size_t di = (size_t)b * P.gamma + pos;
+        x = P.draft_tokens[di];
+        qx = P.draft_q_tok[di];
+        ux = P.uniforms[di];
+        if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
+    }
+    // The arrival counter says every ticket of the row has been counted; a partial whose store
+    // has not landed yet still shows the fill pattern and is polled for.
+    float Rr = DSSD_NEG_INF;
+    bool bad = false, timeout = false;
+    for (int k = lane; k < P.n_lse_runs; k += 32) {
+        unsigned long long w = ld_relaxed_u64(part + k);
+        for (unsigned it = 0; (unsigned)w == kFull && it < P.spin_limit; ++it) {
+            __nanosleep(32);
+            w = ld_relaxed_u64(part + k);
+        }
+        if ((unsigned)w == kFull) {
+            timeout = true;
+        } else {
+            const float ps = __uint_as_float((unsigned)(w >> 32));
+            if (ps != ps) bad = true;
+            if (ps > 0.f) Rr = fmaxf(Rr, __uint_as_float((unsigned)w));
+        }
+    }
+    timeout = __any_sync(kFull, timeout);
+    bad = __any_sync(kFull, bad);
+    Rr = warp_max(Rr);
+    double S = 0.0;
+    if (!timeout && Rr != DSSD_NEG_INF) {
+        for (int k = lane; k < P.n_lse_runs; k += 32) {
+            const unsigned long long w = ld_relaxed_u64(part + k);
+            const float pr = __uint_as_float((unsigned)w), ps = __uint_as_float((unsigned)(w >> 32));
+            if (ps > 0.f) S += (double)ps * exp2((double)pr - (double)Rr);
+        }
+    }
+    S = warp_sum(S);
+    if (lane == 0) {
+        double lse2 = (double)Rr + log2(S);  // log2 sum_v 2^(l_v * c1)
+        const bool finite = !timeout && !bad && (lse2 == lse2) && (fabs(lse2) < INFINITY);
+        if (!finite) lse2 = NAN;
+        unsigned bits = (finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u);
+        if (timeout) *P.error = 1u;
+        if (P.lse) P.lse[row] = (float)(lse2 * 0.6931471805599453);
+        if (pos < P.gamma) {
+            double p = NAN;
+            bool accept = false;
+            if (x < 0 || x >= P.V) {
+                bits |= kBitBadToken;
+            } else {
+                // u < min(1, p(x)/q(x)), evaluated in float64
+                p = exp2((double)zx * c1 - lse2);
+                const double q = (double)qx;
+                const double u = (double)ux;
+                double ratio;
+                if (q != q) ratio = NAN;
+                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
+                else ratio = p / q;
+                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+            }
+            if (P.p_tok) P.p_tok[(size_t)b * P.gamma + pos] = (float)p;
+            bits |= accept ? kBitAccept : 0u;
+        }
+        const float invS = finite ? (float)(1.0 / S) : NAN;
+        const float Rs = finite ? Rr : 0.f;
+        unsigned long long *ri = reinterpret_cast<unsigned long long *>(P.row_info + row);
+        st_relaxed_u64(ri, (unsigned long long)__float_as_uint(Rs) | ((unsigned long long)__float_as_uint(invS) << 32));
+        st_relaxed_u64(ri + 1, (unsigned long long)bits);
+    }
+    unsigned arrival = 0;
+    if (lane == 0) arrival = logical(atomicAdd(&P.seq_cnt[b], 1u));
+    if (__shfl_sync(kFull, arrival, 0) == (unsigned)P.gamma) finish_sequence(P, b);
+}
+
+// One slice of an EMIT ticket: p_row[b, e] = 2^(l_e * c1 - ref2) * invS.
+template <int DT>
+__device__ __forceinline__ void emit_consume(const EdgeParams &P, const Slice &s, const Geo &g, uint32_t stage)
+{
+    using E = Elem<DT>;
+    if (s.b < 0) return;
+    const int lane = threadIdx.x & 31;
+    const float c1 = P.c1, nref = -s.ref2, invS = s.invS;
+    float *outp = P.p_row + (size_t)s.b * P.V;
+    float *body = outp + g.e0;
+    const int nelem = (int)(g.bulk / E::kBytes);
+    if ((reinterpret_cast<uintptr_t>(body) & 15u) == 0) {
+        const int nquad = nelem >> 2;  // bulk is a multiple of 16 bytes, so nelem is a multiple of 4
+        if (DT == DSSD_BF16) {
+            const uint32_t base = stage + (uint32_t)lane * 8u;
+#pragma unroll 4
+            for (int i = lane; i < nquad; i += 32) {
+                const uint2 w = lds8(base + (uint32_t)(i - lane) * 8u);
+                st_stream16(body + (size_t)i * 4, ex2(fmaf(bf16_lo(w.x), c1, nref)) * invS,
+                            ex2(fmaf(bf16_hi(w.x), c1, nref)) * invS, ex2(fmaf(bf16_lo(w.y), c1, nref)) * invS,
+                            ex2(fmaf(bf16_hi(w.y), c1, nref)) * invS);
+            }
+        } else {
+            const uint32_t base = stage + (uint32_t)lane * 16u;
+#pragma unroll 4
+            for (int i = lane; i < nquad; i += 32) {
+                const uint4 w = lds16(base + (uint32_t)(i - lane) * 16u);
+                st_stream16(body + (size_t)i * 4, ex2(fmaf(__uint_as_float(w.x), c1, nref)) * invS,
+                            ex2(fmaf(__uint_as_float(w.y), c1, nref)) * invS,
+                            ex2(fmaf(__uint_as_float(w.z), c1, nref)) * invS,
+                            ex2(fmaf(__uint_as_float(w.w), c1, nref)) * invS);
             }
         }
-        for (; i < nvec; i += 32) {
-            float f[E::kVec];
-            E::unpack(ld_stream16(body + i), f);
-#pragma unroll
-            for (int j = 0; j < E::kVec; ++j) f[j] = ex2((f[j] - M) * c1) * invS;
-            float *o = outp + e0 + (size_t)i * E::kVec;
-#pragma unroll
-            for (int j = 0; j < E::kVec; j += 4) st_stream16(o + j, f[j], f[j + 1], f[j + 2], f[j + 3]);
+    } else {
+        // output not 16-byte aligned at this slice: coalesced 4-byte stores
+        for (int i = lane; i < nelem; i += 32) {
+            float z;
+            if (DT == DSSD_BF16) {
+                unsigned short h;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(stage + (uint32_t)i * 2u));
+                z = __uint_as_float((uint32_t)h << 16);
+            } else {
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(z) : "r"(stage + (uint32_t)i * 4u));
+            }
+            body[i] = ex2(fmaf(z, c1, nref)) * invS;
         }
-        done = e0 + nvec * E::kVec;
     }
-    for (int e = done + lane; e < e1; e += 32) outp[e] = ex2((E::load(rowp, e) - M) * c1) * invS;
-    return true;
+    if (lane < g.head) outp[lane] = ex2(fmaf(E::load(g.rowp, lane), c1, nref)) * invS;
+    if (lane < g.tail) {
+        const int64_t e = (int64_t)g.e0 + nelem + lane;
+        outp[e] = ex2(fmaf(E::load(g.rowp, e), c1, nref)) * invS;
+    }
+}
+
+// lane 0 refreshes what it knows of the EMIT queue; the values are looked at one draw later,
+// so the loads' round trips are never waited for
+__device__ __forceinline__ void peek_queue(const EdgeParams &P, Cursor &c)
+{
+    if ((threadIdx.x & 31) == 0) {
+        c.tail_raw = ld_relaxed_u32(P.ready_tail);
+        c.head_raw = ld_relaxed_u64(P.emit_head);
+    }
+}
+
+// Starts the next ticket: an EMIT ticket if one can be had for a sequence already pushed, else
+// the LSE ticket in hand.  EMIT tickets are claimed with one atomic add when the queue seems to
+// hold unclaimed work; a claim that lands beyond the pushed sequences (several warps saw the same
+// work) is parked and served as soon as its sequence is pushed.  Never waits for other warps'
+// work: c.kind = kIdle means "nothing right now", kEnd "nothing ever again".
+__device__ __forceinline__ void draw(const EdgeParams &P, Cursor &c)
+{
+    const int lane = threadIdx.x & 31;
+    int got = 0;
+    unsigned long long t = 0;
+    if (lane == 0) {
+        const unsigned long long tail = (unsigned long long)logical(c.tail_raw);
+        if (c.parked == kNoTicket) {
+            const unsigned long long head = logical(c.head_raw);
+            if (head < tail * (unsigned long long)P.n_emit_runs) {
+                const unsigned long long claimed = logical(atomicAdd(P.emit_head, 1ull));
+                if (claimed < P.total_emit) c.parked = claimed;
+            }
+        }
+        if (c.parked != kNoTicket && c.parked / (unsigned)P.n_emit_runs < tail) {
+            got = 1;
+            t = c.parked;
+            c.parked = kNoTicket;
+        }
+    }
+    got = shfl0(got);
+    if (got) {
+        t = shfl0(t);
+        const unsigned long long slot = t / (unsigned)P.n_emit_runs;
+        c.run = (int)(t - slot * (unsigned)P.n_emit_runs);
+        int b = -1, n = -1;
+        float ref2 = 0.f, invS = 0.f;
+        if (lane == 0) {
+            const unsigned long long *rs = reinterpret_cast<const unsigned long long *>(P.ready + slot);
+            unsigned long long w0 = ld_relaxed_u64(rs), w1 = ld_relaxed_u64(rs + 1);
+            for (unsigned it = 0; ((unsigned)w0 == kFull || (unsigned)w1 == kFull) && it < P.spin_limit; ++it) {
+                __nanosleep(32);
+                w0 = ld_relaxed_u64(rs);
+                w1 = ld_relaxed_u64(rs + 1);
+            }
+            if ((unsigned)w0 == kFull || (unsigned)w1 == kFull) {
+                *P.error = 1u;  // the pusher's stores never landed: nothing can be written
+            } else {
+                b = (int)(unsigned)w0;
+                n = (int)(unsigned)(w0 >> 32);
+                ref2 = __uint_as_float((unsigned)w1);
+                invS = __uint_as_float((unsigned)(w1 >> 32));
+            }
+        }
+        b = shfl0(b);
+        n = shfl0(n);
+        c.ref2 = shfl0(ref2);
+        c.invS = shfl0(invS);
+        c.kind = kEmit;
+        c.b = (b >= 0 && n >= 0) ? (long long)b : -1ll;
+        c.row = (long long)(b < 0 ? 0 : b) * (P.gamma + 1) + (n < 0 ? 0 : n);
+        c.k_begin = c.run * P.emit_run;
+        c.k_end = min(P.n_slices, c.k_begin + P.emit_run);
+        c.k = c.k_begin;
+        peek_queue(P, c);
+        return;
+    }
+    const unsigned long long no = logical(shfl0(c.lse_raw));
+    if (no < P.total_lse) {
+        c.row = (long long)(no / (unsigned)P.n_lse_runs);
+        c.run = (int)(no - (unsigned long long)c.row * (unsigned)P.n_lse_runs);
+        c.kind = kLse;
+        c.k_begin = c.run * P.lse_run;
+        c.k_end = min(P.n_slices, c.k_begin + P.lse_run);
+        c.k = c.k_begin;
+        if (lane == 0) c.lse_raw = atomicAdd(P.lse_ticket, 1ull);
+        peek_queue(P, c);
+        return;
+    }
+    // no LSE ticket left: done once every EMIT ticket is claimed and none is parked here
+    int more = 0;
+    if (lane == 0) more = (c.parked != kNoTicket) || (logical(c.head_raw) < P.total_emit);
+    c.kind = shfl0(more) ? kIdle : kEnd;
+    if (c.kind == kIdle) peek_queue(P, c);
+}
+
+__device__ __forceinline__ Slice next_slice(const EdgeParams &P, Cursor &c)
+{
+    if (c.kind != kEnd && (c.kind == kIdle || c.k >= c.k_end)) draw(P, c);
+    Slice s;
+    s.kind = c.kind;
+    s.k = c.k;
+    s.first_last = (c.k == c.k_begin ? 1 : 0) | (c.k + 1 == c.k_end ? 2 : 0);
+    s.run = c.run;
+    s.row = c.row;
+    s.b = c.b;
+    s.ref2 = c.ref2;
+    s.invS = c.invS;
+    if (c.kind == kLse || c.kind == kEmit) ++c.k;
+    return s;
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, kEdgeCtasPerSm) edge_verify_kernel(const EdgeParams P)
+__global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __grid_constant__ EdgeParams P)
 {
-    const int lane = threadIdx.x & 31;
-    const float c1 = P.c1;
-    // two draws ahead: `cur` is being worked on, `nxt_no` is the number of the next ticket (drawn
-    // one ticket early so that the atomic's round trip is never waited for)
-    unsigned no = 0;
-    if (lane == 0) no = logical(atomicAdd(P.ticket, 1u));
-    Ticket cur = decode<DT>(P, __shfl_sync(kFull, no, 0));
-    unsigned nxt_no = 0;
-    if (lane == 0) nxt_no = logical(atomicAdd(P.ticket, 1u));
-    uint4 v[kVPL], w[kVPL];
-    if (cur.kind == kLseFast) load_half<DT>(P, cur, 0, v);
-    Ticket parked{kEnd, 0, 0};  // an EMIT ticket whose sequence was not folded yet
-    while (cur.kind != kEnd) {
-        Ticket nxt;
-        if (cur.kind == kLseFast) {
-            load_half<DT>(P, cur, 1, w);
-            // The slice is counted before its partial is stored: the count is back when the work
-            // is done, and whoever folds the row polls for partials that have not landed yet.
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring = smem_addr(smem) + (uint32_t)warp * (uint32_t)(kEdgeStages * kS);
+    const uint32_t bars = smem_addr(smem) + (uint32_t)(kEdgeWarps * kEdgeStages * kS) + (uint32_t)warp * (kEdgeStages * 8u);
+    if (lane == 0) {
+#pragma unroll
+        for (int st = 0; st < kEdgeStages; ++st) mbar_init(bars + 8u * st, 1u);
+        mbar_init_fence();
+    }
+    __syncwarp();
+    const uint64_t pol_emit = l2_policy_evict_first();
+
+    Cursor cur;
+    cur.kind = kIdle;
+    cur.k = cur.k_begin = cur.k_end = cur.run = 0;
+    cur.row = 0;
+    cur.b = -1;
+    cur.ref2 = cur.invS = 0.f;
+    cur.lse_raw = 0;
+    cur.head_raw = 0;
+    cur.tail_raw = 0;
+    cur.parked = kNoTicket;
+    if (lane == 0) cur.lse_raw = atomicAdd(P.lse_ticket, 1ull);
+    peek_queue(P, cur);
+
+    // D[0] is the oldest slice in flight and sits in ring stage `st`; the ring starts out idle
+    // and fills itself during the first kEdgeStages iterations
+    Slice D[kEdgeStages];
+#pragma unroll
+    for (int j = 0; j < kEdgeStages; ++j) {
+        D[j].kind = kIdle;
+        D[j].k = D[j].first_last = D[j].run = 0;
+        D[j].row = 0;
+        D[j].b = -1;
+        D[j].ref2 = D[j].invS = 0.f;
+    }
+    Online o;
+    online_reset(o);
+    unsigned parity = 0;  // bit s: parity of the phase that stage s completes next
+    unsigned idle = 0;    // consecutive iterations without work
+    int st = 0;
+    bool failed = false;
+    for (;;) {
+        const Slice s = D[0];
+        bool any = false;
+#pragma unroll
+        for (int j = 0; j < kEdgeStages; ++j) any = any || (D[j].kind != kEnd);
+        if (!any) break;
+        const uint32_t stage = ring + (uint32_t)st * kS, bar = bars + 8u * st;
+        if (s.kind == kLse || s.kind == kEmit) {
+            idle = 0;
+            const Geo g = slice_geo<DT>(P, s.row, s.k);
             unsigned arrival = 0;
-            if (lane == 0) arrival = logical(atomicAdd(&P.row_cnt[cur.index], 1u));
-            Online o{DSSD_NEG_INF, 0.f, 0.f};
-            accum_half<DT>(o, v, c1);
-            // the next ticket's number is back: request its first half before the second half
-            // of this slice is worked on
-            nxt = decode<DT>(P, __shfl_sync(kFull, nxt_no, 0));
-            if (lane == 0 && nxt.kind != kEnd) nxt_no = logical(atomicAdd(P.ticket, 1u));
-            if (nxt.kind == kLseFast) load_half<DT>(P, nxt, 0, v);
-            accum_half<DT>(o, w, c1);
-            publish_partial(P, cur, o.m, o.s0 + o.s1);
-            if (__shfl_sync(kFull, arrival, 0) == (unsigned)(P.n_lse_slices - 1)) fold_row<DT>(P, cur.index);
-        } else {
-            nxt = decode<DT>(P, __shfl_sync(kFull, nxt_no, 0));
-            if (lane == 0 && nxt.kind != kEnd) nxt_no = logical(atomicAdd(P.ticket, 1u));
-            if (nxt.kind == kLseFast) load_half<DT>(P, nxt, 0, v);
-            if (cur.kind == kLseSlow) {
-                unsigned arrival = 0;
-                if (lane == 0) arrival = logical(atomicAdd(&P.row_cnt[cur.index], 1u));
-                lse_slow<DT>(P, cur);
-                if (__shfl_sync(kFull, arrival, 0) == (unsigned)(P.n_lse_slices - 1)) fold_row<DT>(P, cur.index);
-            } else if (cur.kind == kEmit) {
-                if (!emit_slice<DT>(P, cur.index, cur.slice, false)) {
-                    if (parked.kind != kEnd) emit_slice<DT>(P, parked.index, parked.slice, true);  // older
-                    parked = cur;
+            if (s.kind == kLse) {
+                if (s.first_last & 1) online_reset(o);
+                // The ticket is counted before its partial is stored: the count is back by the
+                // time the slice is done, and whoever folds the row polls for late partials.
+                if ((s.first_last & 2) && lane == 0) arrival = atomicAdd(&P.row_cnt[s.row], 1u);  // raw
+            }
+            if (!mbar_wait(bar, (parity >> st) & 1u, P.spin_limit)) {
+                failed = true;  // a copy never completed
+                break;
+            }
+            parity ^= 1u << st;
+            if (s.kind == kLse) {
+                lse_consume<DT>(P, g, stage, o);
+                if (s.first_last & 2) {
+                    publish_partial(P, s.row, s.run, o);
+                    if (logical(__shfl_sync(kFull, arrival, 0)) == (unsigned)(P.n_lse_runs - 1)) fold_row<DT>(P, s.row);
+                }
+            } else {
+                emit_consume<DT>(P, s, g, stage);
+            }
+            __syncwarp();
+#if DSSD_EDGE_WAR == 1
+            fence_proxy_async();  // the stage is about to be overwritten by a bulk copy
+#endif
+        } else if (s.kind == kIdle) {
+            if (++idle > P.spin_limit) {
+                failed = true;
+                break;
+            }
+            if (idle > (unsigned)kEdgeStages) __nanosleep(200);  // the whole ring is idle
+        }
+        // refill the stage just freed with the warp's next slice
+        const Slice nw = next_slice(P, cur);
+        if (nw.kind == kLse || nw.kind == kEmit) {
+            const Geo g = slice_geo<DT>(P, nw.row, nw.k);
+            if (lane == 0) {
+                if (g.bulk) {
+                    mbar_arrive_expect_tx(bar, g.bulk);
+                    if (nw.kind == kEmit) bulk_g2s_hint(stage, g.src, g.bulk, bar, pol_emit);
+                    else bulk_g2s(stage, g.src, g.bulk, bar);
+                } else {
+                    mbar_arrive(bar);
                 }
             }
         }
-        if (parked.kind != kEnd && cur.kind != kEmit && emit_slice<DT>(P, parked.index, parked.slice, false))
-            parked.kind = kEnd;
-        cur = nxt;
+#pragma unroll
+        for (int j = 0; j + 1 < kEdgeStages; ++j) D[j] = D[j + 1];
+        D[kEdgeStages - 1] = nw;
+        st = (st + 1 == kEdgeStages) ? 0 : st + 1;
     }
-    if (parked.kind != kEnd) emit_slice<DT>(P, parked.index, parked.slice, true);
+    if (failed) {
+        // error exit: copies may still be in flight into this warp's ring; wait for them (bounded)
+        // before the CTA's shared memory can be handed to another CTA.  D[0] sits in stage st.
+        if (lane == 0) *P.error = 1u;
+#pragma unroll
+        for (int j = 0; j < kEdgeStages; ++j) {
+            if ((D[j].kind == kLse || D[j].kind == kEmit) && !(j == 0 && idle == 0))
+                mbar_wait(bars + 8u * st, (parity >> st) & 1u, P.spin_limit);
+            st = (st + 1 == kEdgeStages) ? 0 : st + 1;
+        }
+    }
 }
+
+constexpr size_t kEdgeSmemBytes = (size_t)kEdgeWarps * kEdgeStages * kS + (size_t)kEdgeWarps * kEdgeStages * 8;
 
 }  // namespace
 
-size_t edge_workspace_layout(int B, int gamma, int V, int n_lse_slices, EdgeParams *P, char *base)
+int edge_max_runs_per_row(int V)
+{
+    const long long n = ((long long)V * 4 + kS - 1) / kS;
+    return (int)(n < 1 ? 1 : n);
+}
+
+size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, char *base)
 {
     // all of it is filled with 0xFF before the launch: counters then read "logical 0", slots "not yet"
     const size_t R = (size_t)B * (size_t)(gamma + 1);
@@ -431,19 +671,24 @@ size_t edge_workspace_layout(int B, int gamma, int V, int n_lse_slices, EdgePara
         off += (bytes + 255) & ~(size_t)255;
         return o;
     };
-    const size_t o_err = take(256);  // ticket counter and error word on separate 128-byte lines
+    const size_t o_ctr = take(512);  // four counters, each on its own 128-byte line
     const size_t o_rowcnt = take(R * 4);
+    const size_t o_seqcnt = take((size_t)B * 4);
     const size_t o_info = take(R * sizeof(RowInfo));
-    const size_t o_part = take(R * (size_t)n_lse_slices * sizeof(float2));
+    const size_t o_ready = take((size_t)B * sizeof(ReadySlot));
+    const size_t o_part = take(R * (size_t)runs_per_row * 8);
     if (P) {
-        P->ticket = reinterpret_cast<unsigned *>(base + o_err);
-        P->error = reinterpret_cast<unsigned *>(base + o_err + 128);
+        P->lse_ticket = reinterpret_cast<unsigned long long *>(base + o_ctr);
+        P->emit_head = reinterpret_cast<unsigned long long *>(base + o_ctr + 128);
+        P->ready_tail = reinterpret_cast<unsigned *>(base + o_ctr + 256);
+        P->error = reinterpret_cast<unsigned *>(base + o_ctr + 384);
         P->row_cnt = reinterpret_cast<unsigned *>(base + o_rowcnt);
+        P->seq_cnt = reinterpret_cast<unsigned *>(base + o_seqcnt);
         P->row_info = reinterpret_cast<RowInfo *>(base + o_info);
-        P->part = reinterpret_cast<float2 *>(base + o_part);
+        P->ready = reinterpret_cast<ReadySlot *>(base + o_ready);
+        P->part = reinterpret_cast<unsigned long long *>(base + o_part);
         P->fill_bytes = off;
     }
-    (void)V;
     return off;
 }
 
@@ -460,39 +705,40 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     if (g_sm_count[dev] == 0) {
         int sms = 0, occ0 = 0, occ1 = 0;
         if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, edge_verify_kernel<DSSD_F32>, kThreads, 0)) != cudaSuccess) return err;
-        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, edge_verify_kernel<DSSD_BF16>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaFuncSetAttribute(edge_verify_kernel<DSSD_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEdgeSmemBytes)) != cudaSuccess) return err;
+        if ((err = cudaFuncSetAttribute(edge_verify_kernel<DSSD_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEdgeSmemBytes)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, edge_verify_kernel<DSSD_F32>, kEdgeThreads, kEdgeSmemBytes)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, edge_verify_kernel<DSSD_BF16>, kEdgeThreads, kEdgeSmemBytes)) != cudaSuccess) return err;
         if (occ0 < 1 || occ1 < 1) return cudaErrorLaunchOutOfResources;
-        g_edge_ctas_per_sm[dev][0] = occ0 < kEdgeCtasPerSm ? occ0 : kEdgeCtasPerSm;
-        g_edge_ctas_per_sm[dev][1] = occ1 < kEdgeCtasPerSm ? occ1 : kEdgeCtasPerSm;
+        g_edge_ctas_per_sm[dev][0] = occ0;
+        g_edge_ctas_per_sm[dev][1] = occ1;
         g_sm_count[dev] = sms;
     }
     const int esz = dtype == DSSD_BF16 ? 2 : 4;
-    P.lse_slice = kEdgeLseSliceBytes / esz;
-    P.emit_slice = kEdgeEmitSlice;
-    P.n_lse_slices = (P.V + P.lse_slice - 1) / P.lse_slice;
-    P.n_emit_slices = (P.V + P.emit_slice - 1) / P.emit_slice;
-    P.lse_tickets = (P.gamma + 1) * P.n_lse_slices;
-    const unsigned long long G = (unsigned long long)P.lse_tickets + (unsigned long long)P.n_emit_slices;
-    edge_workspace_layout(P.B, P.gamma, P.V, P.n_lse_slices, &P, static_cast<char *>(workspace));
+    const unsigned long long R = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);
+    const long long n_slices = ((long long)P.V * esz + kS - 1) / kS;
+    P.n_slices = (int)(n_slices < 1 ? 1 : n_slices);
     const unsigned long long resident_ctas = (unsigned long long)g_sm_count[dev] * g_edge_ctas_per_sm[dev][dtype == DSSD_BF16];
-    const unsigned long long resident_warps = resident_ctas * kWarps;
-    // EMIT trails its sequence's LSE tickets by kEdgeEmitLagSweeps times the number of resident
-    // warps: one such sweep covers the tickets still being worked on, the rest the fold.
-    P.lag = (int)((kEdgeEmitLagSweeps * resident_warps + G - 1) / G) + 1;
-    const unsigned long long total = ((unsigned long long)P.B + (unsigned long long)P.lag) * G;
-    if (total + 2 * resident_warps >= 0xffffffffull) return cudaErrorInvalidValue;
-    P.tickets_per_group = (unsigned)G;
-    P.total_tickets = (unsigned)total;
+    const unsigned long long resident_warps = resident_ctas * kEdgeWarps;
+    // run length: as long as every resident warp still gets about kEdgeTicketsPerWarp tickets
+    unsigned long long run = (R * (unsigned long long)P.n_slices) / (resident_warps * kEdgeTicketsPerWarp);
+    run = run < 1 ? 1 : (run > (unsigned long long)kEdgeMaxRun ? (unsigned long long)kEdgeMaxRun : run);
+    P.lse_run = (int)run;
+    P.emit_run = (int)run;
+    P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
+    P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
+    P.total_lse = R * (unsigned long long)P.n_lse_runs;
+    P.total_emit = (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
     P.spin_limit = 1u << 20;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
+    edge_workspace_layout(P.B, P.gamma, P.n_lse_runs, &P, static_cast<char *>(workspace));
     if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
-    const unsigned long long want = (total + 2 * kWarps - 1) / (2 * kWarps);
+    const unsigned long long tickets = P.total_lse + P.total_emit;
+    const unsigned long long want = (tickets + kEdgeWarps - 1) / kEdgeWarps;
     const unsigned grid = (unsigned)(want < resident_ctas ? want : resident_ctas);
-    void *args[] = {&P};
-    const void *fn = dtype == DSSD_BF16 ? reinterpret_cast<const void *>(edge_verify_kernel<DSSD_BF16>)
-                                        : reinterpret_cast<const void *>(edge_verify_kernel<DSSD_F32>);
-    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, 0, stream);
+    if (dtype == DSSD_BF16) edge_verify_kernel<DSSD_BF16><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
+    else edge_verify_kernel<DSSD_F32><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
+    return cudaGetLastError();
 }
 
 }  // namespace dssd
