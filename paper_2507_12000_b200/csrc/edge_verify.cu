@@ -52,25 +52,35 @@ __device__ __forceinline__ const char *row_ptr(const EdgeParams &P, long long ro
     return static_cast<const char *>(P.logits) + (size_t)row * (size_t)P.row_stride * Elem<DT>::kBytes;
 }
 
-// One slice of work, identical in every lane of the warp.
-struct Slice {
-    int kind;
-    int k;          // slice index within the row
-    int first_last; // bit0: first slice of its ticket, bit1: last
-    int run;        // ticket index within the row (LSE: partial slot)
-    long long row;  // LSE: the row; EMIT: row n of the sequence
-    long long b;    // EMIT: the sequence, -1 when nothing may be written
-    float ref2, invS;  // EMIT
+// A ticket as the warp keeps it in shared memory between the moment its first copy is issued
+// and the moment its last slice has been worked on.
+struct Ticket {
+    long long row;      // LSE: the row; EMIT: row n of the sequence
+    long long out_off;  // EMIT: b * V, offset of the output row in p_row; < 0: write nothing
+    int run;            // ticket index within the row (LSE: partial slot)
+    int head;           // bytes before the row's first 16-byte boundary (scalar head of slice 0)
+    float ref2, invS;   // EMIT
 };
+constexpr int kTq = 8;  // tickets a warp can have in flight (>= kEdgeStages + 1), a power of two
+static_assert(kTq > kEdgeStages && (kTq & (kTq - 1)) == 0, "ticket queue too small");
 
-// Where the warp is in its current ticket, and what lane 0 has fetched ahead.  Values fetched
-// ahead are kept raw (as loaded) and converted where they are used, so that nothing depends on
-// a load or atomic until its round trip is over.
-struct Cursor {
+// What the registers hold per ring stage: `bulk` bytes in flight and
+//   meta = kind | first << 2 | last << 3 | ragged << 4 | queue slot << 5 | slice index << 8
+// first/last: of its ticket; ragged: the slice has scalar elements outside the bulk copy.
+constexpr unsigned kMetaFirst = 4u, kMetaLast = 8u, kMetaRagged = 16u;
+
+// Where lane 0's copies are (the fetch side runs up to kEdgeStages slices ahead of the work),
+// and what lane 0 has loaded ahead.  Values loaded ahead are kept raw (as loaded) and
+// converted where they are used, so that nothing depends on a load or atomic until its round
+// trip is over.
+struct Fetch {
     int kind;
-    int k, k_begin, k_end, run;
-    long long row, b;
-    float ref2, invS;
+    int k, k_begin, k_end;  // next slice, first slice and end of the current ticket
+    int slot;               // ticket queue slot of the current ticket
+    int head;               // its row's head bytes
+    const char *src;        // source of slice k's bulk copy
+    long long remain;       // bytes of the row's body from slice k on (may be <= 0)
+    unsigned issued;        // tickets started so far (next queue slot = issued % kTq)
     unsigned long long lse_raw;   // lane 0: atomic result holding the LSE ticket in hand
     unsigned long long head_raw;  // lane 0: last value loaded from emit_head
     unsigned tail_raw;            // lane 0: last value loaded from ready_tail
@@ -78,35 +88,12 @@ struct Cursor {
 };
 constexpr unsigned long long kNoTicket = ~0ull;
 
-// Geometry of slice k of a row: an optional scalar head (up to the first 16-byte boundary, slice
-// 0 only), a 16-byte aligned body that one bulk copy brings in, a scalar tail (< 16 bytes).
-struct Geo {
-    const char *rowp;
-    const char *src;  // body start
-    uint32_t bulk;    // body bytes, a multiple of 16
-    int e0;           // element index of the body's first element
-    int head;         // scalar elements [0, head)
-    int tail;         // scalar elements [e0 + bulk / size, +tail)
-};
-
 template <int DT>
-__device__ __forceinline__ Geo slice_geo(const EdgeParams &P, long long row, int k)
+__device__ __forceinline__ int row_head_bytes(const EdgeParams &P, const char *rowp)
 {
-    using E = Elem<DT>;
-    Geo g;
-    g.rowp = row_ptr<DT>(P, row);
-    const long long rowbytes = (long long)P.V * E::kBytes;
-    long long h = (long long)((16u - (unsigned)(reinterpret_cast<uintptr_t>(g.rowp) & 15u)) & 15u);
-    if (h > rowbytes) h = rowbytes;
-    const long long off = (long long)k * kS;
-    long long len = rowbytes - h - off;
-    len = len < 0 ? 0 : (len > kS ? kS : len);
-    g.bulk = (uint32_t)len & ~15u;
-    g.src = g.rowp + h + off;
-    g.e0 = (int)((h + off) / E::kBytes);
-    g.head = k == 0 ? (int)(h / E::kBytes) : 0;
-    g.tail = (int)((len - g.bulk) / E::kBytes);
-    return g;
+    const long long rowbytes = (long long)P.V * Elem<DT>::kBytes;
+    const long long h = (long long)((16u - (unsigned)(reinterpret_cast<uintptr_t>(rowp) & 15u)) & 15u);
+    return (int)(h > rowbytes ? rowbytes : h);
 }
 
 // ---- per-lane online log-sum-exp state ---------------------------------------------------
@@ -195,15 +182,23 @@ __device__ __forceinline__ uint4 neg_inf_vec()
                            : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
 }
 
-// One slice of an LSE ticket: the stage's vectors, then the scalar head and tail from global.
+// One slice of an LSE ticket: the `bulk` bytes that the copy brought into the stage.
 template <int DT>
-__device__ __forceinline__ void lse_consume(const EdgeParams &P, const Geo &g, uint32_t stage, Online &o)
+__device__ __forceinline__ void lse_consume(uint32_t stage, uint32_t bulk, float c1, Online &o)
 {
-    using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    const float c1 = P.c1;
-    const int nvec = (int)(g.bulk >> 4);
     const uint32_t base = stage + (uint32_t)lane * 16u;
+    if (bulk == (uint32_t)kS && kS % 2048 == 0) {
+#pragma unroll
+        for (int blk = 0; blk < kS / 2048; ++blk) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = lds16(base + (uint32_t)(blk * 2048 + u * 512));
+            accum_block<DT>(o, v, c1);
+        }
+        return;
+    }
+    const int nvec = (int)(bulk >> 4);
     int i = lane;
     for (; i + 96 < nvec; i += 128) {
         uint4 v[4];
@@ -218,8 +213,23 @@ __device__ __forceinline__ void lse_consume(const EdgeParams &P, const Geo &g, u
             v[u] = (i + 32 * u < nvec) ? lds16(base + (uint32_t)(i - lane + 32 * u) * 16u) : neg_inf_vec<DT>();
         accum_block<DT>(o, v, c1);
     }
-    if (lane < g.head) online_add(o, E::load(g.rowp, lane), c1);
-    if (lane < g.tail) online_add(o, E::load(g.rowp, (int64_t)g.e0 + (int64_t)(g.bulk / E::kBytes) + lane), c1);
+}
+
+// Scalar elements of slice k that lie outside its bulk copy: the head of the row (slice 0) and
+// the tail of the row's last slice.  `fn(element index)` is called by one lane per element.
+template <int DT, class F>
+__device__ __forceinline__ void for_ragged(const EdgeParams &P, int head, int k, F fn)
+{
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    const long long rowbytes = (long long)P.V * E::kBytes;
+    const long long off = (long long)k * kS;
+    long long len = rowbytes - head - off;
+    len = len < 0 ? 0 : (len > kS ? kS : len);
+    const long long bulk = len & ~15ll;
+    if (k == 0 && lane < head / E::kBytes) fn((int64_t)lane);
+    const int tail = (int)((len - bulk) / E::kBytes);
+    if (lane < tail) fn((int64_t)((head + off + bulk) / E::kBytes) + lane);
 }
 
 // lane-local state -> the ticket's partial (ref2, sum), one 8-byte store
@@ -371,17 +381,13 @@ __device__ __noinline__ void fold_row(const EdgeParams &P, long long row)
     if (__shfl_sync(kFull, arrival, 0) == (unsigned)P.gamma) finish_sequence(P, b);
 }
 
-// One slice of an EMIT ticket: p_row[b, e] = 2^(l_e * c1 - ref2) * invS.
+// One slice of an EMIT ticket: body[e] = 2^(l_e * c1 - ref2) * invS for the elements of the stage.
 template <int DT>
-__device__ __forceinline__ void emit_consume(const EdgeParams &P, const Slice &s, const Geo &g, uint32_t stage)
+__device__ __forceinline__ void emit_consume(uint32_t stage, uint32_t bulk, float *body, float c1, float nref, float invS)
 {
     using E = Elem<DT>;
-    if (s.b < 0) return;
     const int lane = threadIdx.x & 31;
-    const float c1 = P.c1, nref = -s.ref2, invS = s.invS;
-    float *outp = P.p_row + (size_t)s.b * P.V;
-    float *body = outp + g.e0;
-    const int nelem = (int)(g.bulk / E::kBytes);
+    const int nelem = (int)(bulk / E::kBytes);
     if ((reinterpret_cast<uintptr_t>(body) & 15u) == 0) {
         const int nquad = nelem >> 2;  // bulk is a multiple of 16 bytes, so nelem is a multiple of 4
         if (DT == DSSD_BF16) {
@@ -418,20 +424,28 @@ __device__ __forceinline__ void emit_consume(const EdgeParams &P, const Slice &s
             body[i] = ex2(fmaf(z, c1, nref)) * invS;
         }
     }
-    if (lane < g.head) outp[lane] = ex2(fmaf(E::load(g.rowp, lane), c1, nref)) * invS;
-    if (lane < g.tail) {
-        const int64_t e = (int64_t)g.e0 + nelem + lane;
-        outp[e] = ex2(fmaf(E::load(g.rowp, e), c1, nref)) * invS;
-    }
 }
 
 // lane 0 refreshes what it knows of the EMIT queue; the values are looked at one draw later,
 // so the loads' round trips are never waited for
-__device__ __forceinline__ void peek_queue(const EdgeParams &P, Cursor &c)
+__device__ __forceinline__ void peek_queue(const EdgeParams &P, Fetch &f)
 {
     if ((threadIdx.x & 31) == 0) {
-        c.tail_raw = ld_relaxed_u32(P.ready_tail);
-        c.head_raw = ld_relaxed_u64(P.emit_head);
+        f.tail_raw = ld_relaxed_u32(P.ready_tail);
+        f.head_raw = ld_relaxed_u64(P.emit_head);
+    }
+}
+
+// ticket number -> (index / per, index % per); 32-bit arithmetic whenever the number fits
+__device__ __forceinline__ void split_ticket(unsigned long long t, int per, unsigned long long &q, int &r)
+{
+    if ((t >> 32) == 0) {
+        const unsigned q32 = (unsigned)t / (unsigned)per;
+        q = q32;
+        r = (int)((unsigned)t - q32 * (unsigned)per);
+    } else {
+        q = t / (unsigned)per;
+        r = (int)(t - q * (unsigned)per);
     }
 }
 
@@ -439,32 +453,40 @@ __device__ __forceinline__ void peek_queue(const EdgeParams &P, Cursor &c)
 // the LSE ticket in hand.  EMIT tickets are claimed with one atomic add when the queue seems to
 // hold unclaimed work; a claim that lands beyond the pushed sequences (several warps saw the same
 // work) is parked and served as soon as its sequence is pushed.  Never waits for other warps'
-// work: c.kind = kIdle means "nothing right now", kEnd "nothing ever again".
-__device__ __forceinline__ void draw(const EdgeParams &P, Cursor &c)
+// work: f.kind = kIdle means "nothing right now", kEnd "nothing ever again".
+template <int DT>
+__device__ __forceinline__ void draw(const EdgeParams &P, Fetch &f, Ticket *tq)
 {
+    using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
     int got = 0;
     unsigned long long t = 0;
     if (lane == 0) {
-        const unsigned long long tail = (unsigned long long)logical(c.tail_raw);
-        if (c.parked == kNoTicket) {
-            const unsigned long long head = logical(c.head_raw);
+        const unsigned long long tail = (unsigned long long)logical(f.tail_raw);
+        if (f.parked == kNoTicket) {
+            const unsigned long long head = logical(f.head_raw);
             if (head < tail * (unsigned long long)P.n_emit_runs) {
                 const unsigned long long claimed = logical(atomicAdd(P.emit_head, 1ull));
-                if (claimed < P.total_emit) c.parked = claimed;
+                if (claimed < P.total_emit) f.parked = claimed;
             }
         }
-        if (c.parked != kNoTicket && c.parked / (unsigned)P.n_emit_runs < tail) {
-            got = 1;
-            t = c.parked;
-            c.parked = kNoTicket;
+        if (f.parked != kNoTicket) {
+            unsigned long long slot;
+            int run;
+            split_ticket(f.parked, P.n_emit_runs, slot, run);
+            if (slot < tail) {
+                got = 1;
+                t = f.parked;
+                f.parked = kNoTicket;
+            }
         }
     }
     got = shfl0(got);
+    Ticket tk;
     if (got) {
         t = shfl0(t);
-        const unsigned long long slot = t / (unsigned)P.n_emit_runs;
-        c.run = (int)(t - slot * (unsigned)P.n_emit_runs);
+        unsigned long long slot;
+        split_ticket(t, P.n_emit_runs, slot, tk.run);
         int b = -1, n = -1;
         float ref2 = 0.f, invS = 0.f;
         if (lane == 0) {
@@ -486,59 +508,56 @@ __device__ __forceinline__ void draw(const EdgeParams &P, Cursor &c)
         }
         b = shfl0(b);
         n = shfl0(n);
-        c.ref2 = shfl0(ref2);
-        c.invS = shfl0(invS);
-        c.kind = kEmit;
-        c.b = (b >= 0 && n >= 0) ? (long long)b : -1ll;
-        c.row = (long long)(b < 0 ? 0 : b) * (P.gamma + 1) + (n < 0 ? 0 : n);
-        c.k_begin = c.run * P.emit_run;
-        c.k_end = min(P.n_slices, c.k_begin + P.emit_run);
-        c.k = c.k_begin;
-        peek_queue(P, c);
-        return;
+        tk.ref2 = shfl0(ref2);
+        tk.invS = shfl0(invS);
+        tk.out_off = (b >= 0 && n >= 0) ? (long long)b * P.V : -1ll;
+        tk.row = (long long)(b < 0 ? 0 : b) * (P.gamma + 1) + (n < 0 ? 0 : n);
+        f.kind = kEmit;
+        f.k_begin = tk.run * P.emit_run;
+        f.k_end = min(P.n_slices, f.k_begin + P.emit_run);
+    } else {
+        const unsigned long long no = logical(shfl0(f.lse_raw));
+        if (no >= P.total_lse) {
+            // no LSE ticket left: done once every EMIT ticket is claimed and none is parked here
+            int more = 0;
+            if (lane == 0) more = (f.parked != kNoTicket) || (logical(f.head_raw) < P.total_emit);
+            f.kind = shfl0(more) ? kIdle : kEnd;
+            if (f.kind == kIdle) peek_queue(P, f);
+            return;
+        }
+        unsigned long long row;
+        split_ticket(no, P.n_lse_runs, row, tk.run);
+        tk.row = (long long)row;
+        tk.out_off = -1;
+        tk.ref2 = tk.invS = 0.f;
+        f.kind = kLse;
+        f.k_begin = tk.run * P.lse_run;
+        f.k_end = min(P.n_slices, f.k_begin + P.lse_run);
+        if (lane == 0) f.lse_raw = atomicAdd(P.lse_ticket, 1ull);
     }
-    const unsigned long long no = logical(shfl0(c.lse_raw));
-    if (no < P.total_lse) {
-        c.row = (long long)(no / (unsigned)P.n_lse_runs);
-        c.run = (int)(no - (unsigned long long)c.row * (unsigned)P.n_lse_runs);
-        c.kind = kLse;
-        c.k_begin = c.run * P.lse_run;
-        c.k_end = min(P.n_slices, c.k_begin + P.lse_run);
-        c.k = c.k_begin;
-        if (lane == 0) c.lse_raw = atomicAdd(P.lse_ticket, 1ull);
-        peek_queue(P, c);
-        return;
-    }
-    // no LSE ticket left: done once every EMIT ticket is claimed and none is parked here
-    int more = 0;
-    if (lane == 0) more = (c.parked != kNoTicket) || (logical(c.head_raw) < P.total_emit);
-    c.kind = shfl0(more) ? kIdle : kEnd;
-    if (c.kind == kIdle) peek_queue(P, c);
-}
-
-__device__ __forceinline__ Slice next_slice(const EdgeParams &P, Cursor &c)
-{
-    if (c.kind != kEnd && (c.kind == kIdle || c.k >= c.k_end)) draw(P, c);
-    Slice s;
-    s.kind = c.kind;
-    s.k = c.k;
-    s.first_last = (c.k == c.k_begin ? 1 : 0) | (c.k + 1 == c.k_end ? 2 : 0);
-    s.run = c.run;
-    s.row = c.row;
-    s.b = c.b;
-    s.ref2 = c.ref2;
-    s.invS = c.invS;
-    if (c.kind == kLse || c.kind == kEmit) ++c.k;
-    return s;
+    peek_queue(P, f);
+    const char *rowp = row_ptr<DT>(P, tk.row);
+    tk.head = row_head_bytes<DT>(P, rowp);
+    f.head = tk.head;
+    f.k = f.k_begin;
+    f.src = rowp + tk.head + (long long)f.k_begin * kS;
+    f.remain = (long long)P.V * E::kBytes - tk.head - (long long)f.k_begin * kS;
+    f.slot = (int)(f.issued & (kTq - 1));
+    ++f.issued;
+    if (lane == 0) tq[f.slot] = tk;
+    __syncwarp();
 }
 
 template <int DT>
 __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __grid_constant__ EdgeParams P)
 {
+    using E = Elem<DT>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring = smem_addr(smem) + (uint32_t)warp * (uint32_t)(kEdgeStages * kS);
-    const uint32_t bars = smem_addr(smem) + (uint32_t)(kEdgeWarps * kEdgeStages * kS) + (uint32_t)warp * (kEdgeStages * 8u);
+    unsigned char *after_rings = smem + (size_t)kEdgeWarps * kEdgeStages * kS;
+    Ticket *tq = reinterpret_cast<Ticket *>(after_rings) + warp * kTq;
+    const uint32_t bars = smem_addr(after_rings + sizeof(Ticket) * kTq * kEdgeWarps) + (uint32_t)warp * (kEdgeStages * 8u);
     if (lane == 0) {
 #pragma unroll
         for (int st = 0; st < kEdgeStages; ++st) mbar_init(bars + 8u * st, 1u);
@@ -546,31 +565,34 @@ __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __gr
     }
     __syncwarp();
     const uint64_t pol_emit = l2_policy_evict_first();
+    const float c1 = P.c1;
 
-    Cursor cur;
-    cur.kind = kIdle;
-    cur.k = cur.k_begin = cur.k_end = cur.run = 0;
-    cur.row = 0;
-    cur.b = -1;
-    cur.ref2 = cur.invS = 0.f;
-    cur.lse_raw = 0;
-    cur.head_raw = 0;
-    cur.tail_raw = 0;
-    cur.parked = kNoTicket;
-    if (lane == 0) cur.lse_raw = atomicAdd(P.lse_ticket, 1ull);
-    peek_queue(P, cur);
+    Fetch f;
+    f.kind = kIdle;
+    f.k = f.k_begin = f.k_end = f.slot = f.head = 0;
+    f.src = nullptr;
+    f.remain = 0;
+    f.issued = 0;
+    f.lse_raw = 0;
+    f.head_raw = 0;
+    f.tail_raw = 0;
+    f.parked = kNoTicket;
+    if (lane == 0) f.lse_raw = atomicAdd(P.lse_ticket, 1ull);
+    peek_queue(P, f);
 
-    // D[0] is the oldest slice in flight and sits in ring stage `st`; the ring starts out idle
-    // and fills itself during the first kEdgeStages iterations
-    Slice D[kEdgeStages];
+    // meta[0] / bulk[0] describe the oldest slice in flight, which sits in ring stage `st`; the
+    // ring starts out idle and fills itself during the first kEdgeStages iterations
+    unsigned meta[kEdgeStages], bulk[kEdgeStages];
 #pragma unroll
     for (int j = 0; j < kEdgeStages; ++j) {
-        D[j].kind = kIdle;
-        D[j].k = D[j].first_last = D[j].run = 0;
-        D[j].row = 0;
-        D[j].b = -1;
-        D[j].ref2 = D[j].invS = 0.f;
+        meta[j] = kIdle;
+        bulk[j] = 0;
     }
+    Ticket cur;  // the ticket being worked on
+    cur.row = 0;
+    cur.out_off = -1;
+    cur.run = cur.head = 0;
+    cur.ref2 = cur.invS = 0.f;
     Online o;
     online_reset(o);
     unsigned parity = 0;  // bit s: parity of the phase that stage s completes next
@@ -578,41 +600,53 @@ __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __gr
     int st = 0;
     bool failed = false;
     for (;;) {
-        const Slice s = D[0];
-        bool any = false;
+        const unsigned m = meta[0], nb = bulk[0];
+        const int kind = (int)(m & 3u);
+        unsigned live = 0;
 #pragma unroll
-        for (int j = 0; j < kEdgeStages; ++j) any = any || (D[j].kind != kEnd);
-        if (!any) break;
+        for (int j = 0; j < kEdgeStages; ++j) live |= meta[j];
+        if ((live & 3u) == kEnd) break;  // kinds are 0 (end) .. 3: all stages at end
         const uint32_t stage = ring + (uint32_t)st * kS, bar = bars + 8u * st;
-        if (s.kind == kLse || s.kind == kEmit) {
+        if (kind == kLse || kind == kEmit) {
             idle = 0;
-            const Geo g = slice_geo<DT>(P, s.row, s.k);
-            unsigned arrival = 0;
-            if (s.kind == kLse) {
-                if (s.first_last & 1) online_reset(o);
-                // The ticket is counted before its partial is stored: the count is back by the
-                // time the slice is done, and whoever folds the row polls for late partials.
-                if ((s.first_last & 2) && lane == 0) arrival = atomicAdd(&P.row_cnt[s.row], 1u);  // raw
+            if (m & kMetaFirst) {
+                cur = tq[(m >> 5) & (kTq - 1)];
+                if (kind == kLse) online_reset(o);
             }
+            const int k = (int)(m >> 8);
+            unsigned arrival = 0;
+            // An LSE ticket is counted before its partial is stored: the count is back by the
+            // time the slice is done, and whoever folds the row polls for late partials.
+            if (kind == kLse && (m & kMetaLast) && lane == 0) arrival = atomicAdd(&P.row_cnt[cur.row], 1u);  // raw
             if (!mbar_wait(bar, (parity >> st) & 1u, P.spin_limit)) {
                 failed = true;  // a copy never completed
                 break;
             }
             parity ^= 1u << st;
-            if (s.kind == kLse) {
-                lse_consume<DT>(P, g, stage, o);
-                if (s.first_last & 2) {
-                    publish_partial(P, s.row, s.run, o);
-                    if (logical(__shfl_sync(kFull, arrival, 0)) == (unsigned)(P.n_lse_runs - 1)) fold_row<DT>(P, s.row);
+            if (kind == kLse) {
+                lse_consume<DT>(stage, nb, c1, o);
+                if (m & kMetaRagged) {
+                    const char *rowp = row_ptr<DT>(P, cur.row);
+                    for_ragged<DT>(P, cur.head, k, [&](int64_t e) { online_add(o, E::load(rowp, e), c1); });
                 }
-            } else {
-                emit_consume<DT>(P, s, g, stage);
+                if (m & kMetaLast) {
+                    publish_partial(P, cur.row, cur.run, o);
+                    if (logical(__shfl_sync(kFull, arrival, 0)) == (unsigned)(P.n_lse_runs - 1)) fold_row<DT>(P, cur.row);
+                }
+            } else if (cur.out_off >= 0) {
+                float *outp = P.p_row + cur.out_off;
+                const float nref = -cur.ref2, invS = cur.invS;
+                emit_consume<DT>(stage, nb, outp + (cur.head + (long long)k * kS) / E::kBytes, c1, nref, invS);
+                if (m & kMetaRagged) {
+                    const char *rowp = row_ptr<DT>(P, cur.row);
+                    for_ragged<DT>(P, cur.head, k, [&](int64_t e) { outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS; });
+                }
             }
             __syncwarp();
 #if DSSD_EDGE_WAR == 1
             fence_proxy_async();  // the stage is about to be overwritten by a bulk copy
 #endif
-        } else if (s.kind == kIdle) {
+        } else if (kind == kIdle) {
             if (++idle > P.spin_limit) {
                 failed = true;
                 break;
@@ -620,38 +654,54 @@ __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __gr
             if (idle > (unsigned)kEdgeStages) __nanosleep(200);  // the whole ring is idle
         }
         // refill the stage just freed with the warp's next slice
-        const Slice nw = next_slice(P, cur);
-        if (nw.kind == kLse || nw.kind == kEmit) {
-            const Geo g = slice_geo<DT>(P, nw.row, nw.k);
-            if (lane == 0) {
-                if (g.bulk) {
-                    mbar_arrive_expect_tx(bar, g.bulk);
-                    if (nw.kind == kEmit) bulk_g2s_hint(stage, g.src, g.bulk, bar, pol_emit);
-                    else bulk_g2s(stage, g.src, g.bulk, bar);
-                } else {
-                    mbar_arrive(bar);
+        unsigned nm = kEnd, nbulk = 0;
+        if (f.kind != kEnd) {
+            if (f.kind == kIdle || f.k >= f.k_end) draw<DT>(P, f, tq);
+            nm = (unsigned)f.kind;
+            if (f.kind == kLse || f.kind == kEmit) {
+                const long long len = f.remain < 0 ? 0 : (f.remain > kS ? kS : f.remain);
+                nbulk = (unsigned)len & ~15u;
+                const bool ragged = (f.k == 0 && f.head != 0) || (len & 15);
+                nm |= (f.k == f.k_begin ? kMetaFirst : 0u) | (f.k + 1 == f.k_end ? kMetaLast : 0u) |
+                      (ragged ? kMetaRagged : 0u) | ((unsigned)f.slot << 5) | ((unsigned)f.k << 8);
+                if (lane == 0) {
+                    if (nbulk) {
+                        mbar_arrive_expect_tx(bar, nbulk);
+                        if (f.kind == kEmit) bulk_g2s_hint(stage, f.src, nbulk, bar, pol_emit);
+                        else bulk_g2s(stage, f.src, nbulk, bar);
+                    } else {
+                        mbar_arrive(bar);
+                    }
                 }
+                f.src += kS;
+                f.remain -= kS;
+                ++f.k;
             }
         }
 #pragma unroll
-        for (int j = 0; j + 1 < kEdgeStages; ++j) D[j] = D[j + 1];
-        D[kEdgeStages - 1] = nw;
+        for (int j = 0; j + 1 < kEdgeStages; ++j) {
+            meta[j] = meta[j + 1];
+            bulk[j] = bulk[j + 1];
+        }
+        meta[kEdgeStages - 1] = nm;
+        bulk[kEdgeStages - 1] = nbulk;
         st = (st + 1 == kEdgeStages) ? 0 : st + 1;
     }
     if (failed) {
         // error exit: copies may still be in flight into this warp's ring; wait for them (bounded)
-        // before the CTA's shared memory can be handed to another CTA.  D[0] sits in stage st.
+        // before the CTA's shared memory can be handed to another CTA.  Slice j sits in stage st + j;
+        // the wait on slice 0 is the one that has just run out, if it was work at all.
         if (lane == 0) *P.error = 1u;
 #pragma unroll
         for (int j = 0; j < kEdgeStages; ++j) {
-            if ((D[j].kind == kLse || D[j].kind == kEmit) && !(j == 0 && idle == 0))
-                mbar_wait(bars + 8u * st, (parity >> st) & 1u, P.spin_limit);
+            const int kind = (int)(meta[j] & 3u);
+            if (j > 0 && (kind == kLse || kind == kEmit)) mbar_wait(bars + 8u * st, (parity >> st) & 1u, P.spin_limit);
             st = (st + 1 == kEdgeStages) ? 0 : st + 1;
         }
     }
 }
 
-constexpr size_t kEdgeSmemBytes = (size_t)kEdgeWarps * kEdgeStages * kS + (size_t)kEdgeWarps * kEdgeStages * 8;
+constexpr size_t kEdgeSmemBytes = (size_t)kEdgeWarps * kEdgeStages * kS + sizeof(Ticket) * kTq * kEdgeWarps + (size_t)kEdgeWarps * kEdgeStages * 8;
 
 }  // namespace
 
