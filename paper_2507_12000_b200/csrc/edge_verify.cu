@@ -1,24 +1,30 @@
-// Edge half of the verification round as one persistent streaming kernel.
+// Edge half of the verification round as one persistent, warp-specialised streaming kernel.
 //
-// Every warp is an independent worker with a private ring of shared-memory stages.  Logits
-// travel global -> shared memory as bulk asynchronous copies (TMA, untiled) that the warp's
-// lane 0 issues up to kEdgeStages slices ahead; a stage's arrival is signalled on an mbarrier.
-// Work comes as tickets drawn from global counters:
-//   LSE(row, run)    a run of consecutive slices of one target row: online maximum and sum of
-//                    2^(l * c1 - ref2) in float32 -> one 8-byte partial (ref2, sum).  ref2 is an
+// One CTA per SM.  Warp 0 is the producer: its lane 0 draws tickets from global counters and
+// streams the logits global -> shared memory with bulk asynchronous copies (TMA, untiled) into a
+// ring of kEdgeStages stages, each guarded by a "full" mbarrier (armed with the copy's bytes) and
+// an "empty" mbarrier (one arrival per consumer warp).  Warps 1..kEdgeConsumers are consumers:
+// every consumer takes a fixed 1/kEdgeConsumers share of each stage.  The last warp is the fold
+// warp, which serves a mailbox in shared memory.
+//   LSE(row, run)    a run of consecutive stages of one target row: every consumer keeps an online
+//                    maximum and sum of 2^(l * c1 - ref2) in float32 over its shares; at the run's
+//                    last stage the consumers' results meet in shared memory and the last to
+//                    arrive posts the ticket's partial (ref2, sum) to the fold warp.  ref2 is an
 //                    integer, so partials combine by exact power-of-two scaling.
-//   EMIT(slot, run)  a run of slices of row n of a sequence taken from the `ready` queue: the row
+//   EMIT(slot, run)  a run of stages of row n of a sequence taken from the `ready` queue: the row
 //                    is streamed again (from L2) and p_row = 2^(l * c1 - ref2) / S is written.
-// The warp that brings a row's last partial folds the row (float64 log-sum-exp, acceptance test
-// of that position); the warp that folds a sequence's last row runs the first-rejection scan
-// (ballot + find-first-set) and pushes the sequence to `ready`.  EMIT tickets are claimed, by
-// compare-and-swap, only for sequences already pushed, and are preferred over LSE tickets, so the
-// second read of row n follows the first closely and hits L2.
-// Nothing on this path waits on a fence: results travel through 8-byte slots that the host
-// pre-filled with all ones and that carry their own validity; a consumer that sees the fill
-// pattern polls (bounded) for a store that a running warp has already issued.  A warp only ever
-// waits for work held by running warps, and never while its own ring holds unprocessed slices,
-// so the kernel needs no co-residency guarantee.
+// The fold warp stores each partial to global memory and counts it; the fold warp that brings a
+// row's last partial folds the row (float64 log-sum-exp, acceptance test of that position); the
+// one that folds a sequence's last row runs the first-rejection scan (ballot + find-first-set)
+// and pushes the sequence to `ready`.  EMIT tickets are claimed only for sequences already
+// pushed and are preferred over LSE tickets, so the second read of row n follows the first
+// closely and hits L2.
+// Nothing on the global path waits on a fence: results travel through 8-byte slots that the
+// host pre-filled with all ones and that carry their own validity; a consumer of such a slot
+// that sees the fill pattern polls (bounded) for a store that a running warp has already issued.
+// A producer only ever waits for work held by running CTAs, and never while its own CTA holds
+// unprocessed stages, so the kernel needs no co-residency guarantee.  Every wait is bounded;
+// when one runs out the error word is set and the warps wind down.
 #include "edge_verify.h"
 
 #include <math.h>
@@ -29,22 +35,24 @@ namespace dssd {
 
 namespace {
 
-#ifndef DSSD_EDGE_WAR
-#define DSSD_EDGE_WAR 1
-#endif
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kS = kEdgeSliceBytes;
+constexpr int kS = kEdgeStageBytes;
+constexpr int kNC = kEdgeConsumers;
+constexpr int kVecPerWarp = kS / 16 / kNC;  // 16-byte vectors of a full stage per consumer warp
+static_assert(kVecPerWarp >= 128 && kVecPerWarp % 128 == 0, "a consumer's share must be whole blocks of 4 vectors per lane");
+constexpr int kBlocksPerWarp = kVecPerWarp / 128;
+constexpr int kComb = 16;  // ticket records; tickets in flight in a CTA <= kEdgeStages + 1
+static_assert(kComb >= kEdgeStages + 2 && kComb <= 16 && (kComb & (kComb - 1)) == 0, "ticket records");
+constexpr int kMeet = 4;   // meeting areas where the consumers leave an LSE ticket's per-lane results for the fold warp
+constexpr int kMail = 32;  // mailbox entries of the fold warp, a power of two
 constexpr unsigned kBitAccept = 1u, kBitBadToken = 2u, kBitNonFinite = 4u, kBitTimeout = 8u;
 
-enum Kind : int { kEnd = 0, kIdle = 1, kLse = 2, kEmit = 3 };
+enum Kind : unsigned { kEnd = 0, kIdle = 1, kLse = 2, kEmit = 3 };
+constexpr unsigned kMetaFirst = 4u, kMetaLast = 8u, kMetaRagged = 16u;  // first / last stage of its ticket; scalars outside the copy
 
 // counters start at all ones (the workspace fill pattern): logical value = raw + 1
 __device__ __forceinline__ unsigned logical(unsigned raw) { return raw + 1u; }
 __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
-
-__device__ __forceinline__ unsigned long long shfl0(unsigned long long v) { return __shfl_sync(kFull, v, 0); }
-__device__ __forceinline__ int shfl0(int v) { return __shfl_sync(kFull, v, 0); }
-__device__ __forceinline__ float shfl0(float v) { return __shfl_sync(kFull, v, 0); }
 
 template <int DT>
 __device__ __forceinline__ const char *row_ptr(const EdgeParams &P, long long row)
@@ -52,41 +60,49 @@ __device__ __forceinline__ const char *row_ptr(const EdgeParams &P, long long ro
     return static_cast<const char *>(P.logits) + (size_t)row * (size_t)P.row_stride * Elem<DT>::kBytes;
 }
 
-// A ticket as the warp keeps it in shared memory between the moment its first copy is issued
-// and the moment its last slice has been worked on.
-struct Ticket {
+// A ticket as the CTA keeps it in shared memory, written by the producer before the ticket's
+// first stage is armed and read by every consumer at that stage.
+struct __align__(16) Ticket {
     long long row;      // LSE: the row; EMIT: row n of the sequence
+    long long seq;      // the row's sequence
     long long out_off;  // EMIT: b * V, offset of the output row in p_row; < 0: write nothing
     int run;            // ticket index within the row (LSE: partial slot)
-    int head;           // bytes before the row's first 16-byte boundary (scalar head of slice 0)
+    int head;           // bytes before the row's first 16-byte boundary (scalar head of stage 0)
     float ref2, invS;   // EMIT
+    int meet;           // LSE: meeting area of this ticket
+    unsigned gen;       // LSE: number of earlier tickets of this CTA that used the same area
 };
-constexpr int kTq = 8;  // tickets a warp can have in flight (>= kEdgeStages + 1), a power of two
-static_assert(kTq > kEdgeStages && (kTq & (kTq - 1)) == 0, "ticket queue too small");
+static_assert(sizeof(Ticket) == 48, "Ticket layout");
 
-// What the registers hold per ring stage: `bulk` bytes in flight and
-//   meta = kind | first << 2 | last << 3 | ragged << 4 | queue slot << 5 | slice index << 8
-// first/last: of its ticket; ragged: the slice has scalar elements outside the bulk copy.
-constexpr unsigned kMetaFirst = 4u, kMetaLast = 8u, kMetaRagged = 16u;
+// What the producer writes for each stage before it arms the stage's full barrier:
+//   x = kind | kMeta* | ticket slot << 5 | stage index within the row << 9
+//   y = bytes that the copy brings into the stage, a multiple of 16
+typedef uint2 StageDesc;
+constexpr unsigned kMetaSlotShift = 5, kMetaKShift = 9;
 
-// Where lane 0's copies are (the fetch side runs up to kEdgeStages slices ahead of the work),
-// and what lane 0 has loaded ahead.  Values loaded ahead are kept raw (as loaded) and
-// converted where they are used, so that nothing depends on a load or atomic until its round
-// trip is over.
-struct Fetch {
-    int kind;
-    int k, k_begin, k_end;  // next slice, first slice and end of the current ticket
-    int slot;               // ticket queue slot of the current ticket
-    int head;               // its row's head bytes
-    const char *src;        // source of slice k's bulk copy
-    long long remain;       // bytes of the row's body from slice k on (may be <= 0)
-    unsigned issued;        // tickets started so far (next queue slot = issued % kTq)
-    unsigned long long lse_raw;   // lane 0: atomic result holding the LSE ticket in hand
-    unsigned long long head_raw;  // lane 0: last value loaded from emit_head
-    unsigned tail_raw;            // lane 0: last value loaded from ready_tail
-    unsigned long long parked;    // lane 0: EMIT ticket claimed ahead of its sequence, or kNoTicket
+// A ticket's partial on its way to the fold warp.
+struct __align__(16) Mail {
+    long long row;
+    long long seq;
+    int run;
+    int meet;   // meeting area holding the consumers' results
+    int valid;  // 0: free, 1: posted
+    int pad;
 };
-constexpr unsigned long long kNoTicket = ~0ull;
+static_assert(sizeof(Mail) == 32, "Mail layout");
+
+struct Shared {  // carved from dynamic shared memory behind the ring
+    Ticket ticket[kComb];
+    StageDesc desc[kEdgeStages];
+    unsigned long long full[kEdgeStages];
+    unsigned long long empty[kEdgeStages];
+    float2 lane_part[kMeet][kNC][32];  // per-lane (reference exponent or -inf, sum) of every consumer warp
+    unsigned meet_cnt[kMeet];          // consumer warps that have left their results
+    unsigned meet_gen[kMeet];          // tickets the fold warp has taken out of the area
+    Mail mail[kMail];
+    unsigned mail_tail;
+    unsigned cons_done;
+};
 
 template <int DT>
 __device__ __forceinline__ int row_head_bytes(const EdgeParams &P, const char *rowp)
@@ -101,14 +117,21 @@ __device__ __forceinline__ int row_head_bytes(const EdgeParams &P, const char *r
 struct Online {
     float m;    // running maximum of the raw logits (-inf: nothing seen)
     float ref;  // rint(m * c1), or 0 while m == -inf: terms are 2^(l * c1 - ref) <= 2^0.5
-    float s0, s1, s2, s3;
+    f32x2 s0, s1, s2, s3;  // eight running sums, as four packed pairs
 };
 
 __device__ __forceinline__ void online_reset(Online &o)
 {
     o.m = DSSD_NEG_INF;
     o.ref = 0.f;
-    o.s0 = o.s1 = o.s2 = o.s3 = 0.f;
+    o.s0 = o.s1 = o.s2 = o.s3 = 0ull;
+}
+
+__device__ __forceinline__ float online_total(const Online &o)
+{
+    float a, b;
+    unpack2(add2(add2(o.s0, o.s1), add2(o.s2, o.s3)), a, b);
+    return a + b;
 }
 
 __device__ __forceinline__ void online_raise(Online &o, float bm, float c1)
@@ -116,10 +139,11 @@ __device__ __forceinline__ void online_raise(Online &o, float bm, float c1)
     if (bm > o.m) {
         const float nref = rintf(bm * c1);
         const float f = (o.m == DSSD_NEG_INF) ? 0.f : ex2(o.ref - nref);  // an exact power of two
-        o.s0 *= f;
-        o.s1 *= f;
-        o.s2 *= f;
-        o.s3 *= f;
+        const f32x2 ff = pack2(f, f);
+        o.s0 = mul2(o.s0, ff);
+        o.s1 = mul2(o.s1, ff);
+        o.s2 = mul2(o.s2, ff);
+        o.s3 = mul2(o.s3, ff);
         o.m = bm;
         o.ref = nref;
     }
@@ -128,7 +152,15 @@ __device__ __forceinline__ void online_raise(Online &o, float bm, float c1)
 __device__ __forceinline__ void online_add(Online &o, float z, float c1)
 {
     online_raise(o, z, c1);
-    o.s0 += ex2(fmaf(z, c1, -o.ref));
+    o.s0 = add2(o.s0, pack2(ex2(fmaf(z, c1, -o.ref)), 0.f));
+}
+
+// acc += 2^(a * c1 - ref), 2^(b * c1 - ref)
+__device__ __forceinline__ void add_pair(f32x2 &acc, float a, float b, f32x2 cc, f32x2 nn)
+{
+    float x, y;
+    unpack2(fma2(pack2(a, b), cc, nn), x, y);
+    acc = add2(acc, pack2(ex2(x), ex2(y)));
 }
 
 template <int DT>
@@ -142,17 +174,13 @@ __device__ __forceinline__ void accum_block<DSSD_BF16>(Online &o, const uint4 (&
     for (int u = 1; u < 4; ++u)
         mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(v[u].x, v[u].y), max_bf16x2(v[u].z, v[u].w)));
     online_raise(o, fmaxf(bf16_lo(mx), bf16_hi(mx)), c1);
-    const float nref = -o.ref;
+    const f32x2 cc = pack2(c1, c1), nn = pack2(-o.ref, -o.ref);
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-        o.s0 += ex2(fmaf(bf16_lo(v[u].x), c1, nref));
-        o.s1 += ex2(fmaf(bf16_hi(v[u].x), c1, nref));
-        o.s2 += ex2(fmaf(bf16_lo(v[u].y), c1, nref));
-        o.s3 += ex2(fmaf(bf16_hi(v[u].y), c1, nref));
-        o.s0 += ex2(fmaf(bf16_lo(v[u].z), c1, nref));
-        o.s1 += ex2(fmaf(bf16_hi(v[u].z), c1, nref));
-        o.s2 += ex2(fmaf(bf16_lo(v[u].w), c1, nref));
-        o.s3 += ex2(fmaf(bf16_hi(v[u].w), c1, nref));
+        add_pair(o.s0, bf16_lo(v[u].x), bf16_hi(v[u].x), cc, nn);
+        add_pair(o.s1, bf16_lo(v[u].y), bf16_hi(v[u].y), cc, nn);
+        add_pair(o.s2, bf16_lo(v[u].z), bf16_hi(v[u].z), cc, nn);
+        add_pair(o.s3, bf16_lo(v[u].w), bf16_hi(v[u].w), cc, nn);
     }
 }
 
@@ -165,13 +193,13 @@ __device__ __forceinline__ void accum_block<DSSD_F32>(Online &o, const uint4 (&v
         bm = fmaxf(bm, fmaxf(fmaxf(__uint_as_float(v[u].x), __uint_as_float(v[u].y)),
                              fmaxf(__uint_as_float(v[u].z), __uint_as_float(v[u].w))));
     online_raise(o, bm, c1);
-    const float nref = -o.ref;
+    const f32x2 cc = pack2(c1, c1), nn = pack2(-o.ref, -o.ref);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        o.s0 += ex2(fmaf(__uint_as_float(v[u].x), c1, nref));
-        o.s1 += ex2(fmaf(__uint_as_float(v[u].y), c1, nref));
-        o.s2 += ex2(fmaf(__uint_as_float(v[u].z), c1, nref));
-        o.s3 += ex2(fmaf(__uint_as_float(v[u].w), c1, nref));
+    for (int u = 0; u < 4; u += 2) {
+        add_pair(o.s0, __uint_as_float(v[u].x), __uint_as_float(v[u].y), cc, nn);
+        add_pair(o.s1, __uint_as_float(v[u].z), __uint_as_float(v[u].w), cc, nn);
+        add_pair(o.s2, __uint_as_float(v[u + 1].x), __uint_as_float(v[u + 1].y), cc, nn);
+        add_pair(o.s3, __uint_as_float(v[u + 1].z), __uint_as_float(v[u + 1].w), cc, nn);
     }
 }
 
@@ -182,15 +210,15 @@ __device__ __forceinline__ uint4 neg_inf_vec()
                            : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
 }
 
-// One slice of an LSE ticket: the `bulk` bytes that the copy brought into the stage.
+// A consumer's share of one stage of an LSE ticket: vectors [v0, v1) of the stage.
 template <int DT>
-__device__ __forceinline__ void lse_consume(uint32_t stage, uint32_t bulk, float c1, Online &o)
+__device__ __forceinline__ void lse_consume(uint32_t stage, int v0, int v1, float c1, Online &o)
 {
     const int lane = threadIdx.x & 31;
-    const uint32_t base = stage + (uint32_t)lane * 16u;
-    if (bulk == (uint32_t)kS && kS % 2048 == 0) {
+    const uint32_t base = stage + (uint32_t)(v0 + lane) * 16u;
+    if (v1 - v0 == kVecPerWarp) {
 #pragma unroll
-        for (int blk = 0; blk < kS / 2048; ++blk) {
+        for (int blk = 0; blk < kBlocksPerWarp; ++blk) {
             uint4 v[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) v[u] = lds16(base + (uint32_t)(blk * 2048 + u * 512));
@@ -198,7 +226,7 @@ __device__ __forceinline__ void lse_consume(uint32_t stage, uint32_t bulk, float
         }
         return;
     }
-    const int nvec = (int)(bulk >> 4);
+    const int nvec = v1 - v0;
     int i = lane;
     for (; i + 96 < nvec; i += 128) {
         uint4 v[4];
@@ -215,8 +243,8 @@ __device__ __forceinline__ void lse_consume(uint32_t stage, uint32_t bulk, float
     }
 }
 
-// Scalar elements of slice k that lie outside its bulk copy: the head of the row (slice 0) and
-// the tail of the row's last slice.  `fn(element index)` is called by one lane per element.
+// Scalar elements of stage k that lie outside its bulk copy: the head of the row (stage 0) and
+// the tail of the row's last stage.  `fn(element index)` is called by one lane per element.
 template <int DT, class F>
 __device__ __forceinline__ void for_ragged(const EdgeParams &P, int head, int k, F fn)
 {
@@ -232,186 +260,46 @@ __device__ __forceinline__ void for_ragged(const EdgeParams &P, int head, int k,
     if (lane < tail) fn((int64_t)((head + off + bulk) / E::kBytes) + lane);
 }
 
-// lane-local state -> the ticket's partial (ref2, sum), one 8-byte store
-__device__ __forceinline__ void publish_partial(const EdgeParams &P, long long row, int run, const Online &o)
+// out[0..3] = 2^(z * c1 - ref2) * invS for four logits, as two packed pairs
+__device__ __forceinline__ void emit_quad(float *out, float z0, float z1, float z2, float z3, f32x2 cc, f32x2 nn, f32x2 ss)
 {
-    const bool empty = (o.m == DSSD_NEG_INF);
-    const float R = warp_max(empty ? DSSD_NEG_INF : o.ref);
-    float s = (o.s0 + o.s1) + (o.s2 + o.s3);
-    s = empty ? 0.f : s * ex2(o.ref - R);  // exact scaling
-    s = warp_sum(s);
-    if ((threadIdx.x & 31) == 0) {
-        const float Rp = (R == DSSD_NEG_INF) ? 0.f : R;
-        st_relaxed_u64(&P.part[(size_t)row * P.n_lse_runs + run],
-                       (unsigned long long)__float_as_uint(Rp) | ((unsigned long long)__float_as_uint(s) << 32));
-    }
+    float a, b, c, d;
+    unpack2(fma2(pack2(z0, z1), cc, nn), a, b);
+    unpack2(fma2(pack2(z2, z3), cc, nn), c, d);
+    unpack2(mul2(pack2(ex2(a), ex2(b)), ss), a, b);
+    unpack2(mul2(pack2(ex2(c), ex2(d)), ss), c, d);
+    st_stream16(out, a, b, c, d);
 }
 
-// Run by the warp that folded the last row of sequence b: first-rejection scan over the
-// acceptance bits (one row per lane, ballot + find-first-set), then the push to `ready`.
-__device__ __noinline__ void finish_sequence(const EdgeParams &P, long long b)
-{
-    const int lane = threadIdx.x & 31;
-    int n = P.gamma;
-    unsigned fl = 0;
-    unsigned long long w0n = 0;
-    bool timeout = false;
-    for (int base = 0; base <= P.gamma; base += 32) {
-        const int i = base + lane;
-        unsigned bits = kBitAccept;
-        unsigned long long w0 = 0;
-        if (i <= P.gamma) {
-            const unsigned long long *ri = reinterpret_cast<const unsigned long long *>(P.row_info + b * (P.gamma + 1) + i);
-            w0 = ld_relaxed_u64(ri);
-            bits = (unsigned)ld_relaxed_u64(ri + 1);
-            for (unsigned it = 0; (bits == kFull || (unsigned)w0 == kFull) && it < P.spin_limit; ++it) {
-                __nanosleep(64);
-                w0 = ld_relaxed_u64(ri);
-                bits = (unsigned)ld_relaxed_u64(ri + 1);
-            }
-            if (bits == kFull || (unsigned)w0 == kFull) {
-                timeout = true;
-                bits = kBitTimeout;
-            }
-        }
-        const unsigned rej = __ballot_sync(kFull, i < P.gamma && !(bits & kBitAccept));
-        if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
-        fl |= (__ballot_sync(kFull, bits & kBitBadToken) ? DSSD_EDGE_FLAG_BAD_TOKEN : 0u) |
-              (__ballot_sync(kFull, bits & kBitNonFinite) ? DSSD_EDGE_FLAG_NONFINITE : 0u) |
-              (__ballot_sync(kFull, bits & kBitTimeout) ? DSSD_EDGE_FLAG_TIMEOUT : 0u);
-        if (n >= base && n < base + 32) w0n = __shfl_sync(kFull, w0, n - base);
-    }
-    timeout = __any_sync(kFull, timeout);
-    if (lane == 0) {
-        P.accept_len[b] = timeout ? -1 : n;
-        if (P.flags) P.flags[b] = fl;
-        if (timeout) *P.error = 1u;
-        const unsigned slot = logical(atomicAdd(P.ready_tail, 1u));
-        unsigned long long *rs = reinterpret_cast<unsigned long long *>(P.ready + slot);
-        st_relaxed_u64(rs, (unsigned long long)(unsigned)b | ((unsigned long long)(unsigned)(timeout ? -1 : n) << 32));
-        st_relaxed_u64(rs + 1, timeout ? 0ull : w0n);
-    }
-}
-
-// Run by the warp that brought a row's last partial: partials -> log-sum-exp (float64),
-// acceptance test of the position, RowInfo; then the sequence's arrival count.
+// A consumer's share of one stage of an EMIT ticket: body[e] = 2^(l_e * c1 - ref2) * invS for
+// the `nbytes` bytes of logits at `stage`.
 template <int DT>
-__device__ __noinline__ void fold_row(const EdgeParams &P, long long row)
+__device__ __forceinline__ void emit_consume(uint32_t stage, int nbytes, float *body, float c1, float nref, float invS)
 {
     using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    const double c1 = (double)P.c1;
-    const unsigned long long *part = P.part + (size_t)row * P.n_lse_runs;
-    const long long b = row / (P.gamma + 1);
-    const int pos = (int)(row - b * (P.gamma + 1));
-    // lane 0 starts on the drafted token early: its loads overlap the partials'
-    int x = -1;
-    float zx = 0.f, qx = 0.f, ux = 0.f;
-    if (lane == 0 && pos < P.gamma) {
-        const size_t di = (size_t)b * P.gamma + pos;
-        x = P.draft_tokens[di];
-        qx = P.draft_q_tok[di];
-        ux = P.uniforms[di];
-        if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
-    }
-    // The arrival counter says every ticket of the row has been counted; a partial whose store
-    // has not landed yet still shows the fill pattern and is polled for.
-    float Rr = DSSD_NEG_INF;
-    bool bad = false, timeout = false;
-    for (int k = lane; k < P.n_lse_runs; k += 32) {
-        unsigned long long w = ld_relaxed_u64(part + k);
-        for (unsigned it = 0; (unsigned)w == kFull && it < P.spin_limit; ++it) {
-            __nanosleep(32);
-            w = ld_relaxed_u64(part + k);
-        }
-        if ((unsigned)w == kFull) {
-            timeout = true;
-        } else {
-            const float ps = __uint_as_float((unsigned)(w >> 32));
-            if (ps != ps) bad = true;
-            if (ps > 0.f) Rr = fmaxf(Rr, __uint_as_float((unsigned)w));
-        }
-    }
-    timeout = __any_sync(kFull, timeout);
-    bad = __any_sync(kFull, bad);
-    Rr = warp_max(Rr);
-    double S = 0.0;
-    if (!timeout && Rr != DSSD_NEG_INF) {
-        for (int k = lane; k < P.n_lse_runs; k += 32) {
-            const unsigned long long w = ld_relaxed_u64(part + k);
-            const float pr = __uint_as_float((unsigned)w), ps = __uint_as_float((unsigned)(w >> 32));
-            if (ps > 0.f) S += (double)ps * exp2((double)pr - (double)Rr);
-        }
-    }
-    S = warp_sum(S);
-    if (lane == 0) {
-        double lse2 = (double)Rr + log2(S);  // log2 sum_v 2^(l_v * c1)
-        const bool finite = !timeout && !bad && (lse2 == lse2) && (fabs(lse2) < INFINITY);
-        if (!finite) lse2 = NAN;
-        unsigned bits = (finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u);
-        if (timeout) *P.error = 1u;
-        if (P.lse) P.lse[row] = (float)(lse2 * 0.6931471805599453);
-        if (pos < P.gamma) {
-            double p = NAN;
-            bool accept = false;
-            if (x < 0 || x >= P.V) {
-                bits |= kBitBadToken;
-            } else {
-                // u < min(1, p(x)/q(x)), evaluated in float64
-                p = exp2((double)zx * c1 - lse2);
-                const double q = (double)qx;
-                const double u = (double)ux;
-                double ratio;
-                if (q != q) ratio = NAN;
-                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
-                else ratio = p / q;
-                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
-            }
-            if (P.p_tok) P.p_tok[(size_t)b * P.gamma + pos] = (float)p;
-            bits |= accept ? kBitAccept : 0u;
-        }
-        const float invS = finite ? (float)(1.0 / S) : NAN;
-        const float Rs = finite ? Rr : 0.f;
-        unsigned long long *ri = reinterpret_cast<unsigned long long *>(P.row_info + row);
-        st_relaxed_u64(ri, (unsigned long long)__float_as_uint(Rs) | ((unsigned long long)__float_as_uint(invS) << 32));
-        st_relaxed_u64(ri + 1, (unsigned long long)bits);
-    }
-    unsigned arrival = 0;
-    if (lane == 0) arrival = logical(atomicAdd(&P.seq_cnt[b], 1u));
-    if (__shfl_sync(kFull, arrival, 0) == (unsigned)P.gamma) finish_sequence(P, b);
-}
-
-// One slice of an EMIT ticket: body[e] = 2^(l_e * c1 - ref2) * invS for the elements of the stage.
-template <int DT>
-__device__ __forceinline__ void emit_consume(uint32_t stage, uint32_t bulk, float *body, float c1, float nref, float invS)
-{
-    using E = Elem<DT>;
-    const int lane = threadIdx.x & 31;
-    const int nelem = (int)(bulk / E::kBytes);
+    const int nelem = nbytes / E::kBytes;
+    const f32x2 cc = pack2(c1, c1), nn = pack2(nref, nref), ss = pack2(invS, invS);
     if ((reinterpret_cast<uintptr_t>(body) & 15u) == 0) {
-        const int nquad = nelem >> 2;  // bulk is a multiple of 16 bytes, so nelem is a multiple of 4
+        const int nquad = nelem >> 2;  // nbytes is a multiple of 16, so nelem is a multiple of 4
         if (DT == DSSD_BF16) {
             const uint32_t base = stage + (uint32_t)lane * 8u;
 #pragma unroll 4
             for (int i = lane; i < nquad; i += 32) {
                 const uint2 w = lds8(base + (uint32_t)(i - lane) * 8u);
-                st_stream16(body + (size_t)i * 4, ex2(fmaf(bf16_lo(w.x), c1, nref)) * invS,
-                            ex2(fmaf(bf16_hi(w.x), c1, nref)) * invS, ex2(fmaf(bf16_lo(w.y), c1, nref)) * invS,
-                            ex2(fmaf(bf16_hi(w.y), c1, nref)) * invS);
+                emit_quad(body + (size_t)i * 4, bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y), cc, nn, ss);
             }
         } else {
             const uint32_t base = stage + (uint32_t)lane * 16u;
 #pragma unroll 4
             for (int i = lane; i < nquad; i += 32) {
                 const uint4 w = lds16(base + (uint32_t)(i - lane) * 16u);
-                st_stream16(body + (size_t)i * 4, ex2(fmaf(__uint_as_float(w.x), c1, nref)) * invS,
-                            ex2(fmaf(__uint_as_float(w.y), c1, nref)) * invS,
-                            ex2(fmaf(__uint_as_float(w.z), c1, nref)) * invS,
-                            ex2(fmaf(__uint_as_float(w.w), c1, nref)) * invS);
+                emit_quad(body + (size_t)i * 4, __uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z),
+                          __uint_as_float(w.w), cc, nn, ss);
             }
         }
     } else {
-        // output not 16-byte aligned at this slice: coalesced 4-byte stores
+        // output not 16-byte aligned here: coalesced 4-byte stores
         for (int i = lane; i < nelem; i += 32) {
             float z;
             if (DT == DSSD_BF16) {
@@ -426,282 +314,599 @@ __device__ __forceinline__ void emit_consume(uint32_t stage, uint32_t bulk, floa
     }
 }
 
-// lane 0 refreshes what it knows of the EMIT queue; the values are looked at one draw later,
-// so the loads' round trips are never waited for
-__device__ __forceinline__ void peek_queue(const EdgeParams &P, Fetch &f)
-{
-    if ((threadIdx.x & 31) == 0) {
-        f.tail_raw = ld_relaxed_u32(P.ready_tail);
-        f.head_raw = ld_relaxed_u64(P.emit_head);
-    }
-}
+// ---- the fold warp -------------------------------------------------------------------------
 
-// ticket number -> (index / per, index % per); 32-bit arithmetic whenever the number fits
-__device__ __forceinline__ void split_ticket(unsigned long long t, int per, unsigned long long &q, int &r)
-{
-    if ((t >> 32) == 0) {
-        const unsigned q32 = (unsigned)t / (unsigned)per;
-        q = q32;
-        r = (int)((unsigned)t - q32 * (unsigned)per);
-    } else {
-        q = t / (unsigned)per;
-        r = (int)(t - q * (unsigned)per);
-    }
-}
-
-// Starts the next ticket: an EMIT ticket if one can be had for a sequence already pushed, else
-// the LSE ticket in hand.  EMIT tickets are claimed with one atomic add when the queue seems to
-// hold unclaimed work; a claim that lands beyond the pushed sequences (several warps saw the same
-// work) is parked and served as soon as its sequence is pushed.  Never waits for other warps'
-// work: f.kind = kIdle means "nothing right now", kEnd "nothing ever again".
+// Run by the fold warp that brought the last partial of sequence b.  One lane per position
+// i = 0..gamma: the row's partials -> log-sum-exp (float64) -> acceptance test
+//   u_i < min(1, p_i(x_i) / q_i(x_i));
+// then the first-rejection scan over the lanes' acceptance bits (ballot + find-first-set) and
+// the push of the sequence to `ready`.
 template <int DT>
-__device__ __forceinline__ void draw(const EdgeParams &P, Fetch &f, Ticket *tq)
+__device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
 {
     using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    int got = 0;
-    unsigned long long t = 0;
-    if (lane == 0) {
-        const unsigned long long tail = (unsigned long long)logical(f.tail_raw);
-        if (f.parked == kNoTicket) {
-            const unsigned long long head = logical(f.head_raw);
-            if (head < tail * (unsigned long long)P.n_emit_runs) {
-                const unsigned long long claimed = logical(atomicAdd(P.emit_head, 1ull));
-                if (claimed < P.total_emit) f.parked = claimed;
+    const double c1 = (double)P.c1;
+    int n = P.gamma;
+    unsigned fl = 0;
+    float ref2_n = 0.f, invS_n = 0.f;
+    bool any_timeout = false;
+    for (int base = 0; base <= P.gamma; base += 32) {
+        const int i = base + lane;
+        const bool live = i <= P.gamma;
+        const long long row = b * (P.gamma + 1) + (live ? i : 0);
+        const unsigned long long *part = P.part + (size_t)row * P.n_lse_runs;
+        // Everything this position needs is requested at once: the drafted token with its
+        // probability and uniform, and the row's first partials; the logit of the drafted token
+        // follows as soon as the token id is back.
+        constexpr int kAhead = 4;
+        unsigned long long pw[kAhead];
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k) pw[k] = (live && k < P.n_lse_runs) ? ld_relaxed_u64(part + k) : 0ull;
+        int x = -1;
+        float zx = 0.f, qx = 0.f, ux = 0.f;
+        if (live && i < P.gamma) {
+            const size_t di = (size_t)b * P.gamma + i;
+            x = P.draft_tokens[di];
+            qx = P.draft_q_tok[di];
+            ux = P.uniforms[di];
+            if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
+        }
+        // The sequence's arrival counter says every ticket has been counted; a partial whose
+        // store has not landed yet still shows the fill pattern and is polled for.
+        float Rr = DSSD_NEG_INF;
+        double S = 0.0;
+        bool bad = false, timeout = false;
+        if (live) {
+            for (int k = 0; k < P.n_lse_runs; ++k) {
+                unsigned long long w = 0;
+                if (k < kAhead) {
+#pragma unroll
+                    for (int j = 0; j < kAhead; ++j)
+                        if (j == k) w = pw[j];
+                } else {
+                    w = ld_relaxed_u64(part + k);
+                }
+                for (unsigned it = 0; (unsigned)w == kFull && it < P.spin_limit; ++it) {
+                    __nanosleep(32);
+                    w = ld_relaxed_u64(part + k);
+                }
+                if ((unsigned)w == kFull) {
+                    timeout = true;
+                    continue;
+                }
+                const float pr = __uint_as_float((unsigned)w), ps = __uint_as_float((unsigned)(w >> 32));
+                if (ps != ps) bad = true;
+                if (ps > 0.f) {  // S is kept relative to the largest reference seen so far
+                    if (pr > Rr) {
+                        S = (Rr == DSSD_NEG_INF) ? 0.0 : S * exp2((double)Rr - (double)pr);
+                        Rr = pr;
+                    }
+                    S += (double)ps * exp2((double)pr - (double)Rr);
+                }
             }
         }
-        if (f.parked != kNoTicket) {
-            unsigned long long slot;
-            int run;
-            split_ticket(f.parked, P.n_emit_runs, slot, run);
-            if (slot < tail) {
-                got = 1;
-                t = f.parked;
-                f.parked = kNoTicket;
+        double lse2 = (double)Rr + log2(S);  // log2 sum_v 2^(l_v * c1)
+        const bool finite = !timeout && !bad && (lse2 == lse2) && (fabs(lse2) < INFINITY);
+        if (!finite) lse2 = NAN;
+        unsigned bits = live ? ((finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u)) : kBitAccept;
+        if (live && P.lse) P.lse[row] = (float)(lse2 * 0.6931471805599453);
+        if (live && i < P.gamma) {
+            double p = NAN;
+            bool accept = false;
+            if (x < 0 || x >= P.V) {
+                bits |= kBitBadToken;
+            } else {
+                p = exp2((double)zx * c1 - lse2);  // float64 throughout
+                const double q = (double)qx;
+                const double u = (double)ux;
+                double ratio;
+                if (q != q) ratio = NAN;
+                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
+                else ratio = p / q;
+                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
             }
+            if (P.p_tok) P.p_tok[(size_t)b * P.gamma + i] = (float)p;
+            bits |= accept ? kBitAccept : 0u;
+        }
+        const float invS = finite ? (float)(1.0 / S) : __int_as_float(0x7fc00000);
+        const float Rs = finite ? Rr : 0.f;
+        const unsigned rej = __ballot_sync(kFull, live && i < P.gamma && !(bits & kBitAccept));
+        if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
+        fl |= (__ballot_sync(kFull, bits & kBitBadToken) ? DSSD_EDGE_FLAG_BAD_TOKEN : 0u) |
+              (__ballot_sync(kFull, bits & kBitNonFinite) ? DSSD_EDGE_FLAG_NONFINITE : 0u) |
+              (__ballot_sync(kFull, bits & kBitTimeout) ? DSSD_EDGE_FLAG_TIMEOUT : 0u);
+        any_timeout = any_timeout || __any_sync(kFull, timeout);
+        if (n >= base && n < base + 32) {
+            ref2_n = __shfl_sync(kFull, Rs, n - base);
+            invS_n = __shfl_sync(kFull, invS, n - base);
         }
     }
-    got = shfl0(got);
-    Ticket tk;
-    if (got) {
-        t = shfl0(t);
-        unsigned long long slot;
-        split_ticket(t, P.n_emit_runs, slot, tk.run);
-        int b = -1, n = -1;
-        float ref2 = 0.f, invS = 0.f;
-        if (lane == 0) {
-            const unsigned long long *rs = reinterpret_cast<const unsigned long long *>(P.ready + slot);
-            unsigned long long w0 = ld_relaxed_u64(rs), w1 = ld_relaxed_u64(rs + 1);
-            for (unsigned it = 0; ((unsigned)w0 == kFull || (unsigned)w1 == kFull) && it < P.spin_limit; ++it) {
-                __nanosleep(32);
-                w0 = ld_relaxed_u64(rs);
-                w1 = ld_relaxed_u64(rs + 1);
+    if (lane == 0) {
+        P.accept_len[b] = any_timeout ? -1 : n;
+        if (P.flags) P.flags[b] = fl;
+        if (any_timeout) *P.error = 1u;
+        // the sequence's entry, then the count of ready sequences (nobody waits for either)
+        unsigned long long *rs = reinterpret_cast<unsigned long long *>(P.ready + b);
+        st_relaxed_u64(rs, (unsigned long long)(unsigned)b | ((unsigned long long)(unsigned)(any_timeout ? -1 : n) << 32));
+        st_relaxed_u64(rs + 1, any_timeout ? 0ull
+                                           : ((unsigned long long)__float_as_uint(ref2_n) |
+                                              ((unsigned long long)__float_as_uint(invS_n) << 32)));
+        atomicAdd(P.ready_count, 1u);
+    }
+}
+
+// Serves the CTA's mailbox.  For each posted ticket: reduce the meeting area to the ticket's
+// partial (ref2, sum), store it to global memory and count it on its sequence.  The count's
+// result is not waited for: up to two are in flight, and they are looked at when no mail is
+// waiting (or a third count is due), so posting partials always comes before folding.  Whoever
+// brought a sequence's last partial folds it.
+template <int DT>
+__device__ __forceinline__ void fold_warp(const EdgeParams &P, Shared *sh)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned per_seq = (unsigned)(P.gamma + 1) * (unsigned)P.n_lse_runs;
+    int npend = 0;
+    long long pend_b0 = 0, pend_b1 = 0;
+    unsigned pend_raw0 = 0, pend_raw1 = 0;  // lane 0: raw results of the counts, oldest first
+    auto resolve_oldest = [&]() {
+        const bool last = logical(__shfl_sync(kFull, pend_raw0, 0)) == per_seq - 1u;
+        const long long b = pend_b0;
+        pend_b0 = pend_b1;
+        pend_raw0 = pend_raw1;
+        --npend;
+        if (last) fold_sequence<DT>(P, b);
+    };
+    unsigned idle = 0;
+    for (unsigned head = 0;;) {
+        Mail *e = &sh->mail[head & (kMail - 1)];
+        volatile int *valid = &e->valid;
+        if (*valid) {
+            idle = 0;
+            if (npend == 2) resolve_oldest();
+            __threadfence_block();
+            const long long row = e->row, b = e->seq;
+            const int run = e->run, meet = e->meet;
+            // this lane's column of the meeting area, then across the lanes: the ticket's (ref2, sum)
+            float2 c[kNC];
+#pragma unroll
+            for (int w = 0; w < kNC; ++w) {
+                const volatile float *cp = reinterpret_cast<const volatile float *>(&sh->lane_part[meet][w][lane]);
+                c[w].x = cp[0];
+                c[w].y = cp[1];
             }
-            if ((unsigned)w0 == kFull || (unsigned)w1 == kFull) {
-                *P.error = 1u;  // the pusher's stores never landed: nothing can be written
+            float R = DSSD_NEG_INF;
+            bool nan = false;
+#pragma unroll
+            for (int w = 0; w < kNC; ++w) {
+                nan = nan || (c[w].y != c[w].y);
+                if (c[w].y > 0.f) R = fmaxf(R, c[w].x);
+            }
+            float S = 0.f;
+#pragma unroll
+            for (int w = 0; w < kNC; ++w)
+                if (c[w].y > 0.f) S += c[w].y * ex2(c[w].x - R);  // exact scaling
+            const float Rt = warp_max(R);
+            float sum = warp_sum(R == DSSD_NEG_INF ? 0.f : S * ex2(R - Rt));
+            if (__any_sync(kFull, nan)) sum = __int_as_float(0x7fc00000);
+            const float ref2 = Rt == DSSD_NEG_INF ? 0.f : Rt;
+            __syncwarp();
+            unsigned raw = 0;
+            if (lane == 0) {
+                __threadfence_block();
+                *valid = 0;
+                ++*(volatile unsigned *)&sh->meet_gen[meet];  // the area may be used again
+                st_relaxed_u64(&P.part[(size_t)row * P.n_lse_runs + run],
+                               (unsigned long long)__float_as_uint(ref2) | ((unsigned long long)__float_as_uint(sum) << 32));
+                raw = atomicAdd(&P.seq_cnt[b], 1u);
+            }
+            if (npend == 0) {
+                pend_b0 = b;
+                pend_raw0 = raw;
             } else {
-                b = (int)(unsigned)w0;
-                n = (int)(unsigned)(w0 >> 32);
-                ref2 = __uint_as_float((unsigned)w1);
-                invS = __uint_as_float((unsigned)(w1 >> 32));
+                pend_b1 = b;
+                pend_raw1 = raw;
             }
+            ++npend;
+            ++head;
+            continue;
         }
-        b = shfl0(b);
-        n = shfl0(n);
-        tk.ref2 = shfl0(ref2);
-        tk.invS = shfl0(invS);
-        tk.out_off = (b >= 0 && n >= 0) ? (long long)b * P.V : -1ll;
-        tk.row = (long long)(b < 0 ? 0 : b) * (P.gamma + 1) + (n < 0 ? 0 : n);
-        f.kind = kEmit;
-        f.k_begin = tk.run * P.emit_run;
-        f.k_end = min(P.n_slices, f.k_begin + P.emit_run);
-    } else {
-        const unsigned long long no = logical(shfl0(f.lse_raw));
-        if (no >= P.total_lse) {
-            // no LSE ticket left: done once every EMIT ticket is claimed and none is parked here
-            int more = 0;
-            if (lane == 0) more = (f.parked != kNoTicket) || (logical(f.head_raw) < P.total_emit);
-            f.kind = shfl0(more) ? kIdle : kEnd;
-            if (f.kind == kIdle) peek_queue(P, f);
+        if (npend) {
+            resolve_oldest();
+            continue;
+        }
+        if (*(volatile unsigned *)&sh->cons_done == (unsigned)kNC) {
+            // every consumer has left; anything they posted is visible by now
+            __threadfence_block();
+            if (*valid) continue;
             return;
         }
-        unsigned long long row;
-        split_ticket(no, P.n_lse_runs, row, tk.run);
-        tk.row = (long long)row;
-        tk.out_off = -1;
-        tk.ref2 = tk.invS = 0.f;
-        f.kind = kLse;
-        f.k_begin = tk.run * P.lse_run;
-        f.k_end = min(P.n_slices, f.k_begin + P.lse_run);
-        if (lane == 0) f.lse_raw = atomicAdd(P.lse_ticket, 1ull);
+        if (++idle > P.spin_limit) {
+            if (lane == 0) *P.error = 1u;  // waited too long
+            return;
+        }
+        __nanosleep(200);
     }
-    peek_queue(P, f);
-    const char *rowp = row_ptr<DT>(P, tk.row);
-    tk.head = row_head_bytes<DT>(P, rowp);
-    f.head = tk.head;
-    f.k = f.k_begin;
-    f.src = rowp + tk.head + (long long)f.k_begin * kS;
-    f.remain = (long long)P.V * E::kBytes - tk.head - (long long)f.k_begin * kS;
-    f.slot = (int)(f.issued & (kTq - 1));
-    ++f.issued;
-    if (lane == 0) tq[f.slot] = tk;
+}
+
+// ---- the consumers -------------------------------------------------------------------------
+
+// At an LSE ticket's last stage every consumer warp leaves its lanes' running (reference, sum)
+// pairs in the ticket's meeting area - plain stores, no shuffles on the streaming warps - and the
+// last warp to arrive posts the ticket to the fold warp, which does the reduction.
+__device__ __forceinline__ void leave_and_post(const EdgeParams &P, Shared *sh, int w, const Ticket &t, const Online &o)
+{
+    const int lane = threadIdx.x & 31;
+    // the area is free once the fold warp has taken out every earlier ticket that used it
+    volatile unsigned *gen = &sh->meet_gen[t.meet];
+    for (unsigned it = 0; *gen != t.gen && it < P.spin_limit; ++it) __nanosleep(64);
+    if (*gen != t.gen) {
+        if (lane == 0) *P.error = 1u;  // the fold warp is not keeping up: this ticket's partial is lost
+        return;
+    }
+    sh->lane_part[t.meet][w][lane] = make_float2(o.m == DSSD_NEG_INF ? DSSD_NEG_INF : o.ref, online_total(o));
     __syncwarp();
+    if (lane == 0) {
+        __threadfence_block();
+        if (atomicAdd(&sh->meet_cnt[t.meet], 1u) == (unsigned)(kNC - 1)) {
+            sh->meet_cnt[t.meet] = 0;
+            const unsigned ms = atomicAdd(&sh->mail_tail, 1u) & (kMail - 1);
+            Mail *e = &sh->mail[ms];
+            volatile int *valid = &e->valid;
+            unsigned it = 0;
+            while (*valid && it < P.spin_limit) {  // the fold warp is a whole mailbox behind
+                __nanosleep(100);
+                ++it;
+            }
+            if (*valid) {
+                *P.error = 1u;
+            } else {
+                e->row = t.row;
+                e->seq = t.seq;
+                e->run = t.run;
+                e->meet = t.meet;
+                __threadfence_block();
+                *valid = 1;
+            }
+        }
+    }
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __grid_constant__ EdgeParams P)
+__device__ __forceinline__ void consumer_warp(const EdgeParams &P, Shared *sh, uint32_t ring, int w)
 {
     using E = Elem<DT>;
-    extern __shared__ __align__(128) unsigned char smem[];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t ring = smem_addr(smem) + (uint32_t)warp * (uint32_t)(kEdgeStages * kS);
-    unsigned char *after_rings = smem + (size_t)kEdgeWarps * kEdgeStages * kS;
-    Ticket *tq = reinterpret_cast<Ticket *>(after_rings) + warp * kTq;
-    const uint32_t bars = smem_addr(after_rings + sizeof(Ticket) * kTq * kEdgeWarps) + (uint32_t)warp * (kEdgeStages * 8u);
-    if (lane == 0) {
-#pragma unroll
-        for (int st = 0; st < kEdgeStages; ++st) mbar_init(bars + 8u * st, 1u);
-        mbar_init_fence();
-    }
-    __syncwarp();
-    const uint64_t pol_emit = l2_policy_evict_first();
+    const int lane = threadIdx.x & 31;
     const float c1 = P.c1;
-
-    Fetch f;
-    f.kind = kIdle;
-    f.k = f.k_begin = f.k_end = f.slot = f.head = 0;
-    f.src = nullptr;
-    f.remain = 0;
-    f.issued = 0;
-    f.lse_raw = 0;
-    f.head_raw = 0;
-    f.tail_raw = 0;
-    f.parked = kNoTicket;
-    if (lane == 0) f.lse_raw = atomicAdd(P.lse_ticket, 1ull);
-    peek_queue(P, f);
-
-    // meta[0] / bulk[0] describe the oldest slice in flight, which sits in ring stage `st`; the
-    // ring starts out idle and fills itself during the first kEdgeStages iterations
-    unsigned meta[kEdgeStages], bulk[kEdgeStages];
-#pragma unroll
-    for (int j = 0; j < kEdgeStages; ++j) {
-        meta[j] = kIdle;
-        bulk[j] = 0;
-    }
-    Ticket cur;  // the ticket being worked on
-    cur.row = 0;
-    cur.out_off = -1;
-    cur.run = cur.head = 0;
-    cur.ref2 = cur.invS = 0.f;
+    const int v0 = w * kVecPerWarp;
     Online o;
     online_reset(o);
-    unsigned parity = 0;  // bit s: parity of the phase that stage s completes next
-    unsigned idle = 0;    // consecutive iterations without work
-    int st = 0;
+    // the LSE and the EMIT ticket in progress: an EMIT ticket may run between two stages of an LSE ticket
+    Ticket lt, et;
+    lt.row = lt.seq = 0;
+    lt.out_off = -1;
+    lt.run = lt.head = lt.meet = 0;
+    lt.gen = 0;
+    lt.ref2 = lt.invS = 0.f;
+    et = lt;
+    unsigned st = 0, par = 0;
+    for (;;) {
+        if (!mbar_wait(smem_addr(&sh->full[st]), par, P.spin_limit)) {
+            if (lane == 0) *P.error = 1u;  // the producer went silent
+            break;
+        }
+        const StageDesc d = sh->desc[st];
+        const unsigned meta = d.x;
+        const unsigned kind = meta & 3u;
+        if (kind == kEnd) break;
+        const unsigned slot = (meta >> kMetaSlotShift) & (kComb - 1);
+        if (meta & kMetaFirst) {
+            if (kind == kLse) {
+                lt = sh->ticket[slot];
+                online_reset(o);
+            } else {
+                et = sh->ticket[slot];
+            }
+        }
+        const uint32_t stage = ring + st * (uint32_t)kS;
+        const int k = (int)(meta >> kMetaKShift);
+        const int nvec = (int)(d.y >> 4);
+        const int v1 = min(nvec, v0 + kVecPerWarp);
+        if (kind == kLse) {
+            if (v1 > v0) lse_consume<DT>(stage, v0, v1, c1, o);
+            if ((meta & kMetaRagged) && w == 0) {
+                const char *rowp = row_ptr<DT>(P, lt.row);
+                for_ragged<DT>(P, lt.head, k, [&](int64_t e) { online_add(o, E::load(rowp, e), c1); });
+            }
+        } else if (et.out_off >= 0) {
+            float *outp = P.p_row + et.out_off;
+            const float nref = -et.ref2, invS = et.invS;
+            if (v1 > v0)
+                emit_consume<DT>(stage + (uint32_t)v0 * 16u, (v1 - v0) * 16,
+                                 outp + (et.head + (long long)k * kS + (long long)v0 * 16) / E::kBytes, c1, nref, invS);
+            if ((meta & kMetaRagged) && w == 0) {
+                const char *rowp = row_ptr<DT>(P, et.row);
+                for_ragged<DT>(P, et.head, k, [&](int64_t e) { outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS; });
+            }
+        }
+        // release the stage: the arrival orders this warp's reads before the producer's next copy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(&sh->empty[st]));
+        if (kind == kLse && (meta & kMetaLast)) leave_and_post(P, sh, w, lt, o);
+        if (++st == (unsigned)kEdgeStages) {
+            st = 0;
+            par ^= 1u;
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        __threadfence_block();
+        atomicAdd(&sh->cons_done, 1u);
+    }
+}
+
+// ---- the producer --------------------------------------------------------------------------
+
+// ticket number -> (t / per, t % per).  `magic` = ceil(2^64 / per) when the host has checked
+// that the multiply-high is exact for every ticket number of this launch, else 0.
+__device__ __forceinline__ void split_ticket(unsigned long long t, int per, unsigned long long magic,
+                                             unsigned long long &q, int &r)
+{
+    if (per == 1) {
+        q = t;
+        r = 0;
+        return;
+    }
+    q = magic ? __umul64hi(t, magic) : t / (unsigned)per;
+    r = (int)(t - q * (unsigned)per);
+}
+
+// A run of stages that the producer is issuing.
+struct Run {
+    unsigned kind;  // kEnd: none
+    unsigned slot;  // ticket record
+    int k, k_begin, k_end;
+    const char *src;   // source of stage k's copy
+    long long remain;  // bytes of the row's body from stage k on (may be <= 0)
+    int head;
+};
+
+// The producer's claim on EMIT work advances one step per stage issued, and no step waits for
+// memory: a value requested in one step is looked at in the next.
+//   kWatch    nothing claimed; the counters of ready sequences and of claimed tickets are watched
+//   kClaimed  one atomic add on emit_head is in flight
+//   kLooking  the ticket is known; its sequence's `ready` entry has been requested
+// A ticket whose sequence is not ready yet (claims are handed out in sequence order, sequences
+// become ready in any order) simply stays in kLooking while the LSE work goes on.
+enum ClaimState : int { kWatch = 0, kClaimed = 1, kLooking = 2 };
+struct Claim {
+    int state;
+    unsigned ready_raw;           // last value loaded from ready_count
+    unsigned long long head_raw;  // last value loaded from emit_head
+    unsigned long long claim_raw; // result of the atomic add in flight
+    unsigned long long ticket;    // kLooking: the claimed ticket
+    unsigned long long w0, w1;    // kLooking: the two words of ready[sequence], as loaded
+    bool exhausted;               // a claim came back beyond the last EMIT ticket
+};
+
+__device__ __forceinline__ void claim_watch(const EdgeParams &P, Claim &c)
+{
+    c.ready_raw = ld_relaxed_u32(P.ready_count);
+    c.head_raw = ld_relaxed_u64(P.emit_head);
+}
+
+__device__ __forceinline__ void claim_look(const EdgeParams &P, Claim &c)
+{
+    unsigned long long b;
+    int run;
+    split_ticket(c.ticket, P.n_emit_runs, P.emit_magic, b, run);
+    const unsigned long long *rs = reinterpret_cast<const unsigned long long *>(P.ready + b);
+    c.w0 = ld_relaxed_u64(rs);
+    c.w1 = ld_relaxed_u64(rs + 1);
+}
+
+// One step of the claim.  Returns true, with the ticket's fields of `t` and its stage range
+// filled in, when an EMIT ticket can start now.
+__device__ __forceinline__ bool claim_step(const EdgeParams &P, Claim &c, Ticket &t, int &k_begin, int &k_end)
+{
+    if (c.state == kWatch) {
+        const unsigned long long ready = (unsigned long long)logical(c.ready_raw);
+        const unsigned long long head = logical(c.head_raw);
+        if (!c.exhausted && head < ready * (unsigned long long)P.n_emit_runs) {
+            c.claim_raw = atomicAdd(P.emit_head, 1ull);
+            c.state = kClaimed;
+        } else {
+            claim_watch(P, c);
+        }
+        return false;
+    }
+    if (c.state == kClaimed) {
+        c.ticket = logical(c.claim_raw);
+        if (c.ticket >= P.total_emit) {
+            c.exhausted = true;
+            c.state = kWatch;
+            claim_watch(P, c);
+            return false;
+        }
+        c.state = kLooking;
+        claim_look(P, c);
+        return false;
+    }
+    // kLooking
+    if ((unsigned)c.w0 == kFull || (unsigned)c.w1 == kFull) {
+        claim_look(P, c);  // not ready (or a store still on its way): ask again
+        return false;
+    }
+    unsigned long long b;
+    split_ticket(c.ticket, P.n_emit_runs, P.emit_magic, b, t.run);
+    const int n = (int)(unsigned)(c.w0 >> 32);
+    t.ref2 = __uint_as_float((unsigned)c.w1);
+    t.invS = __uint_as_float((unsigned)(c.w1 >> 32));
+    t.seq = (long long)b;
+    t.out_off = n >= 0 ? (long long)b * P.V : -1ll;  // n < 0: a wait ran out while folding, nothing can be written
+    t.row = t.seq * (P.gamma + 1) + (n < 0 ? 0 : n);
+    k_begin = t.run * P.emit_run;
+    k_end = min(P.n_slices, k_begin + P.emit_run);
+    c.state = kWatch;
+    claim_watch(P, c);
+    return true;
+}
+
+template <int DT>
+__device__ __forceinline__ void start_run(const EdgeParams &P, Shared *sh, Run &r, unsigned kind, Ticket &t, int k_begin,
+                                          int k_end, unsigned &tickets, unsigned &lse_tickets)
+{
+    using E = Elem<DT>;
+    const char *rowp = row_ptr<DT>(P, t.row);
+    t.head = row_head_bytes<DT>(P, rowp);
+    t.meet = 0;
+    t.gen = 0;
+    if (kind == kLse) {
+        t.meet = (int)(lse_tickets % kMeet);
+        t.gen = lse_tickets / kMeet;
+        ++lse_tickets;
+    }
+    r.kind = kind;
+    r.slot = tickets++ & (kComb - 1);
+    // The record's previous ticket was started kComb tickets ago; every consumer read it at that
+    // ticket's first stage, which has been released since (more than kEdgeStages stages ago).
+    sh->ticket[r.slot] = t;
+    r.k = r.k_begin = k_begin;
+    r.k_end = k_end;
+    r.head = t.head;
+    r.src = rowp + t.head + (long long)k_begin * kS;
+    r.remain = (long long)P.V * E::kBytes - t.head - (long long)k_begin * kS;
+}
+
+template <int DT>
+__device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh, uint32_t ring)
+{
+    const uint64_t pol_emit = l2_policy_evict_first();
+    Claim c;
+    c.state = kWatch;
+    c.exhausted = false;
+    c.claim_raw = c.ticket = c.w0 = c.w1 = 0;
+    claim_watch(P, c);
+    unsigned long long lse_raw = atomicAdd(P.lse_ticket, 1ull);  // the LSE ticket in hand, drawn one ticket early
+    bool lse_left = true;
+    Run lr, er;  // the LSE and the EMIT run in progress; an EMIT run goes first
+    lr.kind = er.kind = kEnd;
+    unsigned st = 0, par = 1;  // a fresh barrier passes a wait on parity 1: the ring starts out empty
+    unsigned issued = 0, tickets = 0, lse_tickets = 0, idle = 0;
     bool failed = false;
     for (;;) {
-        const unsigned m = meta[0], nb = bulk[0];
-        const int kind = (int)(m & 3u);
-        unsigned live = 0;
-#pragma unroll
-        for (int j = 0; j < kEdgeStages; ++j) live |= meta[j];
-        if ((live & 3u) == kEnd) break;  // kinds are 0 (end) .. 3: all stages at end
-        const uint32_t stage = ring + (uint32_t)st * kS, bar = bars + 8u * st;
-        if (kind == kLse || kind == kEmit) {
-            idle = 0;
-            if (m & kMetaFirst) {
-                cur = tq[(m >> 5) & (kTq - 1)];
-                if (kind == kLse) online_reset(o);
+        Ticket t;
+        int k_begin = 0, k_end = 0;
+        if (er.kind == kEnd && claim_step(P, c, t, k_begin, k_end)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
+        if (er.kind == kEnd && lr.kind == kEnd && lse_left) {
+            const unsigned long long no = logical(lse_raw);
+            if (no < P.total_lse) {
+                unsigned long long row;
+                split_ticket(no, P.n_lse_runs, P.lse_magic, row, t.run);
+                t.row = (long long)row;
+                t.seq = (row >> 32) == 0 ? (long long)((unsigned)row / (unsigned)(P.gamma + 1))
+                                         : (long long)(row / (unsigned)(P.gamma + 1));
+                t.out_off = -1;
+                t.ref2 = t.invS = 0.f;
+                k_begin = t.run * P.lse_run;
+                k_end = min(P.n_slices, k_begin + P.lse_run);
+                lse_raw = atomicAdd(P.lse_ticket, 1ull);
+                start_run<DT>(P, sh, lr, kLse, t, k_begin, k_end, tickets, lse_tickets);
+            } else {
+                lse_left = false;
             }
-            const int k = (int)(m >> 8);
-            unsigned arrival = 0;
-            // An LSE ticket is counted before its partial is stored: the count is back by the
-            // time the slice is done, and whoever folds the row polls for late partials.
-            if (kind == kLse && (m & kMetaLast) && lane == 0) arrival = atomicAdd(&P.row_cnt[cur.row], 1u);  // raw
-            if (!mbar_wait(bar, (parity >> st) & 1u, P.spin_limit)) {
-                failed = true;  // a copy never completed
-                break;
-            }
-            parity ^= 1u << st;
-            if (kind == kLse) {
-                lse_consume<DT>(stage, nb, c1, o);
-                if (m & kMetaRagged) {
-                    const char *rowp = row_ptr<DT>(P, cur.row);
-                    for_ragged<DT>(P, cur.head, k, [&](int64_t e) { online_add(o, E::load(rowp, e), c1); });
-                }
-                if (m & kMetaLast) {
-                    publish_partial(P, cur.row, cur.run, o);
-                    if (logical(__shfl_sync(kFull, arrival, 0)) == (unsigned)(P.n_lse_runs - 1)) fold_row<DT>(P, cur.row);
-                }
-            } else if (cur.out_off >= 0) {
-                float *outp = P.p_row + cur.out_off;
-                const float nref = -cur.ref2, invS = cur.invS;
-                emit_consume<DT>(stage, nb, outp + (cur.head + (long long)k * kS) / E::kBytes, c1, nref, invS);
-                if (m & kMetaRagged) {
-                    const char *rowp = row_ptr<DT>(P, cur.row);
-                    for_ragged<DT>(P, cur.head, k, [&](int64_t e) { outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS; });
-                }
-            }
-            __syncwarp();
-#if DSSD_EDGE_WAR == 1
-            fence_proxy_async();  // the stage is about to be overwritten by a bulk copy
-#endif
-        } else if (kind == kIdle) {
+        }
+        Run &r = er.kind != kEnd ? er : lr;
+        if (r.kind == kEnd) {
+            // nothing to issue: done once no LSE ticket is left, no claim is under way and every
+            // EMIT ticket has been claimed by someone
+            if (!lse_left && c.state == kWatch && (c.exhausted || logical(c.head_raw) >= P.total_emit)) break;
             if (++idle > P.spin_limit) {
                 failed = true;
                 break;
             }
-            if (idle > (unsigned)kEdgeStages) __nanosleep(200);  // the whole ring is idle
+            __nanosleep(200);
+            continue;
         }
-        // refill the stage just freed with the warp's next slice
-        unsigned nm = kEnd, nbulk = 0;
-        if (f.kind != kEnd) {
-            if (f.kind == kIdle || f.k >= f.k_end) draw<DT>(P, f, tq);
-            nm = (unsigned)f.kind;
-            if (f.kind == kLse || f.kind == kEmit) {
-                const long long len = f.remain < 0 ? 0 : (f.remain > kS ? kS : f.remain);
-                nbulk = (unsigned)len & ~15u;
-                const bool ragged = (f.k == 0 && f.head != 0) || (len & 15);
-                nm |= (f.k == f.k_begin ? kMetaFirst : 0u) | (f.k + 1 == f.k_end ? kMetaLast : 0u) |
-                      (ragged ? kMetaRagged : 0u) | ((unsigned)f.slot << 5) | ((unsigned)f.k << 8);
-                if (lane == 0) {
-                    if (nbulk) {
-                        mbar_arrive_expect_tx(bar, nbulk);
-                        if (f.kind == kEmit) bulk_g2s_hint(stage, f.src, nbulk, bar, pol_emit);
-                        else bulk_g2s(stage, f.src, nbulk, bar);
-                    } else {
-                        mbar_arrive(bar);
-                    }
-                }
-                f.src += kS;
-                f.remain -= kS;
-                ++f.k;
-            }
+        idle = 0;
+        if (!mbar_wait(smem_addr(&sh->empty[st]), par, P.spin_limit)) {
+            failed = true;  // the consumers went silent
+            break;
         }
-#pragma unroll
-        for (int j = 0; j + 1 < kEdgeStages; ++j) {
-            meta[j] = meta[j + 1];
-            bulk[j] = bulk[j + 1];
+        const unsigned len = r.remain <= 0 ? 0u : (r.remain >= kS ? (unsigned)kS : (unsigned)r.remain);
+        const unsigned bulk = len & ~15u;
+        const bool ragged = (r.k == 0 && r.head != 0) || (len & 15u);
+        const unsigned meta = r.kind | (r.k == r.k_begin ? kMetaFirst : 0u) | (r.k + 1 == r.k_end ? kMetaLast : 0u) |
+                              (ragged ? kMetaRagged : 0u) | (r.slot << kMetaSlotShift) | ((unsigned)r.k << kMetaKShift);
+        sh->desc[st] = make_uint2(meta, bulk);
+        const uint32_t bar = smem_addr(&sh->full[st]);
+        if (bulk) {
+            mbar_arrive_expect_tx(bar, bulk);
+            if (r.kind == kEmit) bulk_g2s_hint(ring + st * (uint32_t)kS, r.src, bulk, bar, pol_emit);
+            else bulk_g2s(ring + st * (uint32_t)kS, r.src, bulk, bar);
+        } else {
+            mbar_arrive(bar);
         }
-        meta[kEdgeStages - 1] = nm;
-        bulk[kEdgeStages - 1] = nbulk;
-        st = (st + 1 == kEdgeStages) ? 0 : st + 1;
+        ++issued;
+        r.src += kS;
+        r.remain -= kS;
+        if (++r.k == r.k_end) r.kind = kEnd;
+        if (++st == (unsigned)kEdgeStages) {
+            st = 0;
+            par ^= 1u;
+        }
     }
-    if (failed) {
-        // error exit: copies may still be in flight into this warp's ring; wait for them (bounded)
-        // before the CTA's shared memory can be handed to another CTA.  Slice j sits in stage st + j;
-        // the wait on slice 0 is the one that has just run out, if it was work at all.
-        if (lane == 0) *P.error = 1u;
-#pragma unroll
-        for (int j = 0; j < kEdgeStages; ++j) {
-            const int kind = (int)(meta[j] & 3u);
-            if (j > 0 && (kind == kLse || kind == kEmit)) mbar_wait(bars + 8u * st, (parity >> st) & 1u, P.spin_limit);
-            st = (st + 1 == kEdgeStages) ? 0 : st + 1;
+    if (!failed && mbar_wait(smem_addr(&sh->empty[st]), par, P.spin_limit)) {
+        // tell the consumers that nothing follows
+        sh->desc[st] = make_uint2(kEnd, 0u);
+        mbar_arrive(smem_addr(&sh->full[st]));
+        return;
+    }
+    // error exit: the consumers will run out of patience on their own.  Copies may still be in
+    // flight into the ring; wait for them (bounded) before the CTA's shared memory can be handed
+    // to another CTA.  The last min(issued, kEdgeStages) stages armed are st - 1, st - 2, ...
+    *P.error = 1u;
+    unsigned s2 = st, p2 = par;
+    for (unsigned j = 0; j < (unsigned)kEdgeStages && j < issued; ++j) {
+        if (s2 == 0) {
+            s2 = kEdgeStages;
+            p2 ^= 1u;
         }
+        --s2;
+        mbar_wait(smem_addr(&sh->full[s2]), p2 ^ 1u, P.spin_limit);  // armed in the pass whose empty parity was p2
     }
 }
 
-constexpr size_t kEdgeSmemBytes = (size_t)kEdgeWarps * kEdgeStages * kS + sizeof(Ticket) * kTq * kEdgeWarps + (size_t)kEdgeWarps * kEdgeStages * 8;
+constexpr size_t kEdgeSmemBytes = (size_t)kEdgeStages * kS + sizeof(Shared);
+
+template <int DT>
+__global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __grid_constant__ EdgeParams P)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ring = smem_addr(smem);
+    Shared *sh = reinterpret_cast<Shared *>(smem + (size_t)kEdgeStages * kS);
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int st = 0; st < kEdgeStages; ++st) {
+            mbar_init(smem_addr(&sh->full[st]), 1u);
+            mbar_init(smem_addr(&sh->empty[st]), (unsigned)kNC);
+        }
+        for (int i = 0; i < kMeet; ++i) sh->meet_cnt[i] = sh->meet_gen[i] = 0;
+        for (int i = 0; i < kMail; ++i) sh->mail[i].valid = 0;
+        sh->mail_tail = 0;
+        sh->cons_done = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        if (lane == 0) producer_thread<DT>(P, sh, ring);
+    } else if (warp <= kNC) {
+        consumer_warp<DT>(P, sh, ring, warp - 1);
+    } else {
+        fold_warp<DT>(P, sh);
+    }
+}
 
 }  // namespace
 
@@ -722,19 +927,15 @@ size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, 
         return o;
     };
     const size_t o_ctr = take(512);  // four counters, each on its own 128-byte line
-    const size_t o_rowcnt = take(R * 4);
     const size_t o_seqcnt = take((size_t)B * 4);
-    const size_t o_info = take(R * sizeof(RowInfo));
     const size_t o_ready = take((size_t)B * sizeof(ReadySlot));
     const size_t o_part = take(R * (size_t)runs_per_row * 8);
     if (P) {
         P->lse_ticket = reinterpret_cast<unsigned long long *>(base + o_ctr);
         P->emit_head = reinterpret_cast<unsigned long long *>(base + o_ctr + 128);
-        P->ready_tail = reinterpret_cast<unsigned *>(base + o_ctr + 256);
+        P->ready_count = reinterpret_cast<unsigned *>(base + o_ctr + 256);
         P->error = reinterpret_cast<unsigned *>(base + o_ctr + 384);
-        P->row_cnt = reinterpret_cast<unsigned *>(base + o_rowcnt);
         P->seq_cnt = reinterpret_cast<unsigned *>(base + o_seqcnt);
-        P->row_info = reinterpret_cast<RowInfo *>(base + o_info);
         P->ready = reinterpret_cast<ReadySlot *>(base + o_ready);
         P->part = reinterpret_cast<unsigned long long *>(base + o_part);
         P->fill_bytes = off;
@@ -769,23 +970,31 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     const long long n_slices = ((long long)P.V * esz + kS - 1) / kS;
     P.n_slices = (int)(n_slices < 1 ? 1 : n_slices);
     const unsigned long long resident_ctas = (unsigned long long)g_sm_count[dev] * g_edge_ctas_per_sm[dev][dtype == DSSD_BF16];
-    const unsigned long long resident_warps = resident_ctas * kEdgeWarps;
-    // run length: as long as every resident warp still gets about kEdgeTicketsPerWarp tickets
-    unsigned long long run = (R * (unsigned long long)P.n_slices) / (resident_warps * kEdgeTicketsPerWarp);
+    // Stages per ticket: as long as every resident CTA still gets about kEdgeTicketsPerCta
+    // tickets, at most kEdgeMaxRun, and then evened out so that a row splits into equal tickets.
+    unsigned long long run = (R * (unsigned long long)P.n_slices) / (resident_ctas * kEdgeTicketsPerCta);
     run = run < 1 ? 1 : (run > (unsigned long long)kEdgeMaxRun ? (unsigned long long)kEdgeMaxRun : run);
+    const int runs_per_row = (int)((P.n_slices + run - 1) / run);
+    run = (unsigned long long)((P.n_slices + runs_per_row - 1) / runs_per_row);
     P.lse_run = (int)run;
     P.emit_run = (int)run;
     P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
     P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
     P.total_lse = R * (unsigned long long)P.n_lse_runs;
     P.total_emit = (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
+    // t / d == mulhi64(t, ceil(2^64 / d)) for every t with t * d * d < 2^64
+    auto magic = [](unsigned long long total, int d) -> unsigned long long {
+        if (d < 2 || d > (1 << 15) || total > (1ull << 33)) return 0ull;
+        return ~0ull / (unsigned long long)d + 1ull;
+    };
+    P.lse_magic = magic(P.total_lse, P.n_lse_runs);
+    P.emit_magic = magic(P.total_emit, P.n_emit_runs);
     P.spin_limit = 1u << 20;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
     edge_workspace_layout(P.B, P.gamma, P.n_lse_runs, &P, static_cast<char *>(workspace));
     if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long tickets = P.total_lse + P.total_emit;
-    const unsigned long long want = (tickets + kEdgeWarps - 1) / kEdgeWarps;
-    const unsigned grid = (unsigned)(want < resident_ctas ? want : resident_ctas);
+    const unsigned grid = (unsigned)(tickets < resident_ctas ? tickets : resident_ctas);
     if (dtype == DSSD_BF16) edge_verify_kernel<DSSD_BF16><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
     else edge_verify_kernel<DSSD_F32><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
     return cudaGetLastError();

@@ -7,44 +7,36 @@
 
 namespace dssd {
 
-#ifndef DSSD_EDGE_WARPS
-#define DSSD_EDGE_WARPS 8
+#ifndef DSSD_EDGE_CONSUMERS
+#define DSSD_EDGE_CONSUMERS 16
 #endif
-#ifndef DSSD_EDGE_SLICE_BYTES
-#define DSSD_EDGE_SLICE_BYTES 8192
+#ifndef DSSD_EDGE_STAGE_BYTES
+#define DSSD_EDGE_STAGE_BYTES 32768
 #endif
 #ifndef DSSD_EDGE_STAGES
-#define DSSD_EDGE_STAGES 3
+#define DSSD_EDGE_STAGES 6
 #endif
 #ifndef DSSD_EDGE_MAX_RUN
-#define DSSD_EDGE_MAX_RUN 4
+#define DSSD_EDGE_MAX_RUN 8
 #endif
-#ifndef DSSD_EDGE_TICKETS_PER_WARP
-#define DSSD_EDGE_TICKETS_PER_WARP 16
+#ifndef DSSD_EDGE_TICKETS_PER_CTA
+#define DSSD_EDGE_TICKETS_PER_CTA 8
 #endif
 
-constexpr int kEdgeWarps = DSSD_EDGE_WARPS;            // warps per CTA; each owns a private ring
-constexpr int kEdgeThreads = 32 * kEdgeWarps;
-constexpr int kEdgeSliceBytes = DSSD_EDGE_SLICE_BYTES;  // logits bytes per ring stage (one bulk copy)
-constexpr int kEdgeStages = DSSD_EDGE_STAGES;           // ring stages per warp
-constexpr int kEdgeMaxRun = DSSD_EDGE_MAX_RUN;          // most consecutive slices of a row in one ticket
-constexpr int kEdgeTicketsPerWarp = DSSD_EDGE_TICKETS_PER_WARP;  // tickets aimed at per resident warp
+constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
+constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 2);  // + the producer warp and the fold warp
+constexpr int kEdgeStageBytes = DSSD_EDGE_STAGE_BYTES;   // logits bytes per ring stage (one bulk copy)
+constexpr int kEdgeStages = DSSD_EDGE_STAGES;            // ring stages per CTA
+constexpr int kEdgeMaxRun = DSSD_EDGE_MAX_RUN;           // most consecutive stages of a row in one ticket
+constexpr int kEdgeTicketsPerCta = DSSD_EDGE_TICKETS_PER_CTA;  // tickets aimed at per resident CTA
 
-// Result of folding one target row; two 8-byte slots, each valid once it differs from the
-// all-ones pattern the workspace is filled with before the launch.
-struct RowInfo {
-    float ref2;     // integer-valued reference exponent: terms are 2^(l * c1 - ref2); never NaN
-    float invS;     // 1 / sum_v 2^(l_v * c1 - ref2)   (NaN for a row without finite log-sum-exp)
-    unsigned bits;  // bit0 accepted, bit1 bad token id, bit2 non-finite row, bit3 wait ran out
-    unsigned pad;
-};
-
-// One entry of the queue of sequences whose row P_n can be emitted; two self-validating 8-byte slots.
+// What the emission of row P_n needs to know about a folded sequence: two 8-byte slots, each
+// valid once it differs from the all-ones pattern the workspace is filled with before the launch.
 struct ReadySlot {
-    int b;  // sequence (>= 0)
-    int n;  // accepted length, or -1 if a wait ran out
-    float ref2;
-    float invS;
+    int b;       // sequence (>= 0)
+    int n;       // accepted length, or -1 if a wait ran out
+    float ref2;  // row n's integer-valued reference exponent: terms are 2^(l * c1 - ref2); never NaN
+    float invS;  // 1 / sum_v 2^(l_v * c1 - ref2)   (NaN for a row without finite log-sum-exp)
 };
 
 struct EdgeParams {
@@ -63,23 +55,22 @@ struct EdgeParams {
     float *lse;
     uint32_t *flags;
     // ticket geometry
-    int n_slices;                  // slices per row
-    int lse_run, emit_run;         // slices per LSE / EMIT ticket
+    int n_slices;                  // stages per row
+    int lse_run, emit_run;         // stages per LSE / EMIT ticket
     int n_lse_runs, n_emit_runs;   // tickets per row
     unsigned long long total_lse;  // rows * n_lse_runs
     unsigned long long total_emit; // B * n_emit_runs
+    unsigned long long lse_magic, emit_magic;  // ceil(2^64 / n_*_runs) when multiply-high division is exact, else 0
     unsigned spin_limit;
     // workspace, filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
     // and 8-byte slots read "not yet" until their one store has landed
     unsigned long long *lse_ticket;  // next LSE ticket
     unsigned long long *emit_head;   // next EMIT ticket
-    unsigned *ready_tail;            // sequences pushed to `ready`
+    unsigned *ready_count;           // sequences whose `ready` entry has been written
     unsigned *error;                 // all ones = no error
-    unsigned *row_cnt;               // [rows] LSE tickets of the row that have arrived
-    unsigned *seq_cnt;               // [B] rows of the sequence that have been folded
-    RowInfo *row_info;               // [rows]
+    unsigned *seq_cnt;               // [B] LSE tickets of the sequence that have arrived
     unsigned long long *part;        // [rows, n_lse_runs] (ref2, sum) of one ticket
-    ReadySlot *ready;                // [B]
+    ReadySlot *ready;                // [B] indexed by sequence
     size_t fill_bytes;
 };
 
