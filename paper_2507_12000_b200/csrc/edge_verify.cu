@@ -316,6 +316,35 @@ __device__ __forceinline__ void emit_consume(uint32_t stage, int nbytes, float *
 
 // ---- the fold warp -------------------------------------------------------------------------
 
+// v * 2^d for an integer d <= 0 and a normal, positive v of float32 range: exponent arithmetic,
+// exact; anything below 2^-900 of v counts as nothing
+__device__ __forceinline__ double scale_pow2(double v, float d)
+{
+    if (!(d > -900.f)) return 0.0;
+    return __hiloint2double(__double2hiint(v) + ((int)d << 20), __double2loint(v));
+}
+
+// 2^x in float64 for x <= about 1 (relative error below 1e-11): x = n + f, |f| <= 1/2, and the
+// degree-9 Taylor polynomial of e^(f ln 2); 0 below 2^-1000, NaN for NaN
+__device__ __forceinline__ double exp2_small(double x)
+{
+    if (x != x) return x;
+    if (!(x > -1000.0)) return 0.0;
+    const int n = __double2int_rn(x);
+    const double y = (x - (double)n) * 0.6931471805599453;
+    double p = 2.7557319223985893e-6;
+    p = fma(p, y, 2.48015873015873e-5);
+    p = fma(p, y, 1.984126984126984e-4);
+    p = fma(p, y, 1.388888888888889e-3);
+    p = fma(p, y, 8.333333333333333e-3);
+    p = fma(p, y, 4.1666666666666664e-2);
+    p = fma(p, y, 1.6666666666666666e-1);
+    p = fma(p, y, 0.5);
+    p = fma(p, y, 1.0);
+    p = fma(p, y, 1.0);
+    return __hiloint2double(__double2hiint(p) + (n << 20), __double2loint(p));
+}
+
 // Run by the fold warp that brought the last partial of sequence b.  One lane per position
 // i = 0..gamma: the row's partials -> log-sum-exp (float64) -> acceptance test
 //   u_i < min(1, p_i(x_i) / q_i(x_i));
@@ -379,37 +408,41 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
                 if (ps != ps) bad = true;
                 if (ps > 0.f) {  // S is kept relative to the largest reference seen so far
                     if (pr > Rr) {
-                        S = (Rr == DSSD_NEG_INF) ? 0.0 : S * exp2((double)Rr - (double)pr);
+                        S = (Rr == DSSD_NEG_INF || S == 0.0) ? 0.0 : scale_pow2(S, Rr - pr);
                         Rr = pr;
                     }
-                    S += (double)ps * exp2((double)pr - (double)Rr);
+                    S += scale_pow2((double)ps, pr - Rr);
                 }
             }
         }
-        double lse2 = (double)Rr + log2(S);  // log2 sum_v 2^(l_v * c1)
-        const bool finite = !timeout && !bad && (lse2 == lse2) && (fabs(lse2) < INFINITY);
-        if (!finite) lse2 = NAN;
+        // sum_v 2^(l_v * c1) = S * 2^Rr; it has a finite logarithm iff S is positive and finite
+        const bool finite = !timeout && !bad && (S > 0.0) && (S < INFINITY) && (Rr != DSSD_NEG_INF);
         unsigned bits = live ? ((finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u)) : kBitAccept;
-        if (live && P.lse) P.lse[row] = (float)(lse2 * 0.6931471805599453);
+        if (live && P.lse) P.lse[row] = finite ? (Rr + __log2f((float)S)) * 0.6931471805599453f : __int_as_float(0x7fc00000);
+        // 1 / S in float64: the float32 reciprocal refined by one Newton step
+        double invS_d = NAN;
+        if (finite) {
+            const double r0 = (double)(1.0f / (float)S);
+            invS_d = r0 * (2.0 - S * r0);
+        }
         if (live && i < P.gamma) {
             double p = NAN;
             bool accept = false;
             if (x < 0 || x >= P.V) {
                 bits |= kBitBadToken;
             } else {
-                p = exp2((double)zx * c1 - lse2);  // float64 throughout
+                // u < min(1, p(x)/q(x)) in float64, as  u < 1  and  u * q < p  (u * q is exact)
+                p = finite ? exp2_small((double)zx * c1 - (double)Rr) * invS_d : NAN;
                 const double q = (double)qx;
                 const double u = (double)ux;
-                double ratio;
-                if (q != q) ratio = NAN;
-                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
-                else ratio = p / q;
-                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+                if (q != q || p != p) accept = false;
+                else if (q <= 0.0) accept = (p > 0.0) && (u < 1.0);
+                else accept = (u < 1.0) && (u * q < p);
             }
             if (P.p_tok) P.p_tok[(size_t)b * P.gamma + i] = (float)p;
             bits |= accept ? kBitAccept : 0u;
         }
-        const float invS = finite ? (float)(1.0 / S) : __int_as_float(0x7fc00000);
+        const float invS = finite ? (float)invS_d : __int_as_float(0x7fc00000);
         const float Rs = finite ? Rr : 0.f;
         const unsigned rej = __ballot_sync(kFull, live && i < P.gamma && !(bits & kBitAccept));
         if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
