@@ -146,6 +146,35 @@ dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
                                  int gamma, int V, int32_t *token, uint32_t *flags,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * dssd_device_resample without a caller-provided workspace.  (The paper has no counterpart: this
+ * entry point exists for the library's users, not for the method.)
+ *
+ * Some callers cannot allocate device memory at the point where they sample: code running inside
+ * a serving loop whose memory pool is frozen after start-up, a plugin that is handed input and
+ * output buffers by its host framework and nothing else, or a process whose allocator must not be
+ * touched while other work is in flight.  For them the scratch lives inside the library: a fixed
+ * array of DSSD_STATIC_SCRATCH_BYTES bytes in the library's device image, which every GPU that
+ * loads the library holds until the process exits.  The call itself allocates nothing and frees
+ * nothing.
+ *
+ * Same inputs, outputs and results as dssd_device_resample (the two share the kernel).
+ *   - Sizes whose scratch need (dssd_device_resample_workspace_bytes) exceeds
+ *     DSSD_STATIC_SCRATCH_BYTES are refused with DSSD_ERR_UNSUPPORTED before anything is enqueued;
+ *     use dssd_device_resample for those.
+ *   - The first call made with a given device current looks up the array's device address (once
+ *     per device).  Make that first call during set-up, before any stream capture is begun.
+ *   - Every call on a device uses the same array.  Each call clears the counters it needs and
+ *     overwrites the rest before reading it, so calls that follow one another on a stream are
+ *     independent; two calls that run on the GPU at the same time (different streams, or
+ *     different host threads without ordering) race on the array and give undefined results.
+ */
+#define DSSD_STATIC_SCRATCH_BYTES (1 << 20)
+dssd_status dssd_device_resample_static(const float *p_row, const float *draft_q,
+                                        const int32_t *accept_len, const float *uniforms, int B,
+                                        int gamma, int V, int32_t *token, uint32_t *flags,
+                                        void *cuda_stream);
+
 /* Bytes of device memory that dssd_round_host needs as its arena (0 if the sizes are invalid). */
 size_t dssd_round_host_arena_bytes(int B, int gamma, int V, dssd_dtype dtype);
 

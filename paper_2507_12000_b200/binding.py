@@ -65,6 +65,10 @@ def _load() -> ctypes.CDLL:
     L.dssd_device_resample.argtypes = [
         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
         c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_device_resample_static.restype = c.c_int
+    L.dssd_device_resample_static.argtypes = [
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
+        c.c_void_p, c.c_void_p, c.c_void_p]
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -167,6 +171,26 @@ def dssd_device_resample(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], a
         _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_device_resample")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def dssd_device_resample_static(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], accept_len: torch.Tensor,
+                                uniforms_rs: torch.Tensor, gamma: int, *, out: Dict[str, torch.Tensor],
+                                stream=None) -> Dict[str, torch.Tensor]:
+    """Device half of one round for callers that cannot allocate: the scratch is a fixed array
+    inside the library, and `out` (token, flags: int32 [B]) must be passed in, so that neither
+    the library nor this wrapper allocates anything.  Sizes beyond the built-in scratch raise
+    DssdError(DSSD_ERR_UNSUPPORTED).  Calls that overlap on the GPU race on the shared scratch."""
+    assert p_row.is_cuda and p_row.dim() == 2 and p_row.is_contiguous() and p_row.dtype == torch.float32
+    B, V = p_row.shape
+    st = lib.dssd_device_resample_static(
+        p_row.data_ptr(), _ptr(draft_q) if gamma > 0 else None, accept_len.data_ptr(), uniforms_rs.data_ptr(),
+        B, gamma, V, out["token"].data_ptr(), _ptr(out.get("flags")), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_device_resample_static")
     return out
 
 

@@ -29,6 +29,11 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 }  // namespace
 
+namespace dssd {
+// lets entry points defined in other files of the library report through dssd_last_cuda_error()
+void set_last_cuda_error(int e) { t_last_cuda_error = e; }
+}  // namespace dssd
+
 extern "C" {
 
 const char *dssd_status_string(int status)

@@ -9,6 +9,8 @@
 // lies within rounding (about 1e-13 relative) of a CDF step.
 #include "device_resample.h"
 
+#include <mutex>
+
 #include <math.h>
 
 #include "dssd_device.cuh"
@@ -290,3 +292,71 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
 }
 
 }  // namespace dssd
+
+// ---- dssd_device_resample_static: the same draw, with its scratch inside the library ----------
+//
+// The scratch of this entry point is a fixed array in the library's device image.  Host code
+// cannot use the array's name as an address: the address is looked up once per device with
+// cudaGetSymbolAddress, with that device current, and handed to the kernel like any workspace.
+
+static __device__ __align__(256) unsigned char g_static_scratch[DSSD_STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_mutex;
+void *g_static_ptr[64];  // per device, filled on the first call made with that device current
+}  // namespace
+
+extern "C" dssd_status dssd_device_resample_static(const float *p_row, const float *draft_q,
+                                                   const int32_t *accept_len, const float *uniforms, int B,
+                                                   int gamma, int V, int32_t *token, uint32_t *flags,
+                                                   void *cuda_stream)
+{
+    dssd::set_last_cuda_error(0);
+    if (B < 1 || gamma < 0 || V < 1) return DSSD_ERR_INVALID_ARG;
+    if (V > DSSD_MAX_V || (long long)B * ((long long)gamma + 1) > (long long)DSSD_MAX_ROWS) return DSSD_ERR_UNSUPPORTED;
+    if (!p_row || !accept_len || !uniforms || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft_q) return DSSD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(p_row) % 4) || (reinterpret_cast<uintptr_t>(draft_q) % 4)) return DSSD_ERR_INVALID_ARG;
+    // the built-in scratch has a fixed size: larger batches must use dssd_device_resample
+    if (dssd::resample_workspace_layout(B, V, nullptr, nullptr) > (size_t)DSSD_STATIC_SCRATCH_BYTES) return DSSD_ERR_UNSUPPORTED;
+
+    cudaError_t e;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) {
+        dssd::set_last_cuda_error((int)e);
+        return DSSD_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= 64) return DSSD_ERR_UNSUPPORTED;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            void *ptr = nullptr;
+            if ((e = cudaGetSymbolAddress(&ptr, g_static_scratch)) != cudaSuccess || !ptr) {
+                dssd::set_last_cuda_error((int)e);
+                return DSSD_ERR_CUDA;
+            }
+            g_static_ptr[dev] = ptr;
+        }
+        scratch = g_static_ptr[dev];
+    }
+
+    dssd::ResampleParams P{};
+    P.p_row = p_row;
+    P.draft_q = draft_q;
+    P.accept_len = accept_len;
+    P.uniforms = uniforms;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V;
+    P.token = token;
+    P.flags = flags;
+    // resample_launch clears the counters that must start at zero; the rest of the scratch is
+    // written before it is read, so what the previous call left behind does not matter
+    e = dssd::resample_launch(P, scratch, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        dssd::set_last_cuda_error((int)e);
+        return DSSD_ERR_CUDA;
+    }
+    return DSSD_OK;
+}

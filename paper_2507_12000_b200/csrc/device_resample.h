@@ -30,4 +30,6 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base);
 
 cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream);
 
+void set_last_cuda_error(int e);  // defined with the C ABI
+
 }  // namespace dssd
