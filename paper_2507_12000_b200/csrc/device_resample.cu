@@ -1,10 +1,13 @@
 // Device half of the verification round: residual (or bonus) inverse-CDF draw.
 //
 // Pass A, ticket (b, c): stream chunk c of p_row[b] and of Q_n[b], form r = max(0, p - q) (or
-// r = p for the bonus draw) and add it up in float64 -> chunk_sum[b, c].
-// Pass B, run by the CTA that completes the last chunk of sequence b: prefix over the chunk sums
-// gives Z and the chunk holding u' * Z; that one chunk is read again (from L2), a block-wide
-// prefix sum over per-thread runs finds the thread, and the thread walks its run.
+// r = p for the bonus draw) and add it up in float64 -> chunk_sum[b, c], an 8-byte slot that is
+// valid once it differs from the all-ones pattern the workspace is filled with.  The ticket is
+// then counted on its sequence; the count's result is looked at one ticket later, so a CTA has
+// one barrier per ticket and waits for no round trip.
+// Pass B, run by the CTA that brought the last chunk of sequence b: a block-wide float64 prefix
+// over the chunk sums gives Z and the chunk holding u' * Z; that one chunk is read again (from
+// L2), a block-wide prefix sum over per-thread runs finds the thread, and the thread walks its run.
 // All sums are float64, so the token differs from an index-order float64 scan only when u' * Z
 // lies within rounding (about 1e-13 relative) of a CDF step.
 #include "device_resample.h"
@@ -105,38 +108,107 @@ struct Pick {  // what thread 0 hands to the CTA for pass B
     double target; // u' * Z
 };
 
+constexpr unsigned long long kFill64 = ~0ull;
+
+__device__ __forceinline__ unsigned logical(unsigned raw) { return raw + 1u; }
+__device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
+
+// chunk sum (b, c); a sum whose store has not landed yet still shows the fill pattern and is
+// polled for (bounded); NaN when the wait runs out
+__device__ __forceinline__ double load_chunk_sum(const ResampleParams &P, const unsigned long long *cs, int c)
+{
+    unsigned long long w = ld_relaxed_u64(cs + c);
+    for (unsigned it = 0; w == kFill64 && it < P.spin_limit; ++it) {
+        __nanosleep(32);
+        w = ld_relaxed_u64(cs + c);
+    }
+    return __longlong_as_double((long long)w);
+}
+
+// CTA-wide inclusive prefix sum in index order of the threads; `total` is the sum over the CTA
+__device__ __forceinline__ double block_scan(double x, double *s_scan, double &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    double before = 0.0, all = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        const double v = s_scan[w];
+        if (w < warp) before += v;
+        all += v;
+    }
+    total = all;
+    return before + incl;
+}
+
 // pass B for sequence b; q == nullptr means r = p
 __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const float *q, unsigned fl,
                      double *s_w, Pick *s_pick, int *s_i)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    double *cs = P.chunk_sum + (size_t)b * P.n_chunks;
+    unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_chunks;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        if (tid == 0) {
-            double Z = 0.0;
-            for (int c = 0; c < P.n_chunks; ++c) Z += __ldcg(cs + c);
-            Pick pk;
-            pk.ok = (Z > 0.0) && (Z < INFINITY);
-            pk.chunk = 0;
-            pk.beyond = 1;
-            pk.base = 0.0;
-            pk.target = (double)__ldg(P.uniforms + b) * Z;
-            if (pk.ok) {
-                double C = 0.0;
-                int last_pos = 0;
-                double last_base = 0.0;
-                for (int c = 0; c < P.n_chunks; ++c) {
-                    const double m = __ldcg(cs + c);
-                    if (m > 0.0) { last_pos = c; last_base = C; }
-                    if (C + m > pk.target) { pk.chunk = c; pk.base = C; pk.beyond = 0; break; }
-                    C += m;
-                }
-                if (pk.beyond) { pk.chunk = last_pos; pk.base = last_base; }
-            }
-            *s_pick = pk;
+        // Z = sum of the chunk sums, in groups of one chunk per thread
+        double Z = 0.0;
+        for (int base = 0; base < P.n_chunks; base += kThreads) {
+            const int c = base + tid;
+            double tot;
+            block_scan(c < P.n_chunks ? load_chunk_sum(P, cs, c) : 0.0, s_w, tot);
+            Z += tot;
+            __syncthreads();
         }
-        __syncthreads();
-        if (s_pick->ok) break;
+        const bool ok = (Z > 0.0) && (Z < INFINITY);
+        if (ok) {
+            // the first chunk whose inclusive prefix exceeds the target, else the last chunk with mass
+            const double target = (double)__ldg(P.uniforms + b) * Z;
+            if (tid == 0) {
+                s_i[0] = 0x7fffffff;
+                s_i[1] = -1;
+            }
+            __syncthreads();
+            double carry = 0.0;
+            double my_base_first = 0.0, my_base_last = 0.0;
+            int my_first = 0x7fffffff, my_last = -1;
+            for (int base = 0; base < P.n_chunks; base += kThreads) {
+                const int c = base + tid;
+                const double m = c < P.n_chunks ? load_chunk_sum(P, cs, c) : 0.0;
+                double tot;
+                const double incl = carry + block_scan(m, s_w, tot);
+                if (c < P.n_chunks && incl > target && my_first == 0x7fffffff) {
+                    my_first = c;
+                    my_base_first = incl - m;
+                }
+                if (c < P.n_chunks && m > 0.0) {
+                    my_last = c;
+                    my_base_last = incl - m;
+                }
+                carry += tot;
+                __syncthreads();
+            }
+            if (my_first != 0x7fffffff) atomicMin(&s_i[0], my_first);
+            if (my_last >= 0) atomicMax(&s_i[1], my_last);
+            __syncthreads();
+            const int first = s_i[0], last = s_i[1];
+            if (first != 0x7fffffff ? (my_first == first) : (my_last == last && last >= 0)) {
+                Pick pk;
+                pk.ok = 1;
+                pk.beyond = first == 0x7fffffff;
+                pk.chunk = pk.beyond ? last : first;
+                pk.base = pk.beyond ? my_base_last : my_base_first;
+                pk.target = target;
+                *s_pick = pk;
+            }
+            __syncthreads();
+            break;
+        }
         if (q == nullptr) {  // already drawing from p: the row has no usable mass
             if (tid == 0) {
                 P.token[b] = -1;
@@ -150,9 +222,8 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
         for (int c = 0; c < P.n_chunks; ++c) {
             const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
             const double tot = block_sum(chunk_mass(p, nullptr, e0, e1), s_w);
-            if (tid == 0) cs[c] = tot;
+            if (tid == 0) st_relaxed_u64(cs + c, (unsigned long long)__double_as_longlong(tot));
         }
-        __threadfence();
         __syncthreads();
     }
     const Pick pk = *s_pick;
@@ -160,10 +231,36 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
     const int r0 = min(e1, e0 + tid * kRun), r1 = min(e1, r0 + kRun);
     double mine = 0.0;
     int last_pos = -1;
-    for (int e = r0; e < r1; ++e) {
-        const double r = q ? res(__ldg(p + e), __ldg(q + e)) : (double)__ldg(p + e);
-        mine += r;
-        if (r > 0.0) last_pos = e;
+    // The run is fetched in groups of 16 entries whose loads are all issued before the first is
+    // used (two round trips for the run, not one per entry); entries past the row's end read as 0.
+    const bool vec = (r1 - r0 == kRun) &&
+                     (((reinterpret_cast<uintptr_t>(p + r0) | (q ? reinterpret_cast<uintptr_t>(q + r0) : 0)) & 15u) == 0);
+#pragma unroll
+    for (int g = 0; g < kRun; g += 16) {
+        float pv[16], qv[16];
+        if (vec) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 a = __ldg(reinterpret_cast<const float4 *>(p + r0 + g) + j);
+                pv[4 * j] = a.x, pv[4 * j + 1] = a.y, pv[4 * j + 2] = a.z, pv[4 * j + 3] = a.w;
+                float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q) c = __ldg(reinterpret_cast<const float4 *>(q + r0 + g) + j);
+                qv[4 * j] = c.x, qv[4 * j + 1] = c.y, qv[4 * j + 2] = c.z, qv[4 * j + 3] = c.w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int e = r0 + g + j;
+                pv[j] = e < r1 ? __ldg(p + e) : 0.f;
+                qv[j] = (q && e < r1) ? __ldg(q + e) : 0.f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const double r = q ? res(pv[j], qv[j]) : (double)pv[j];
+            mine += r;
+            if (r > 0.0) last_pos = r0 + g + j;
+        }
     }
     // exclusive prefix of the per-thread run sums across the CTA
     double incl = mine;
@@ -203,49 +300,79 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const ResampleParams P)
+__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ ResampleParams P)
 {
-    __shared__ double s_w[kWarps];
+    __shared__ double s_w[2][kWarps];
+    __shared__ double s_scan[kWarps];
     __shared__ Pick s_pick;
     __shared__ int s_i[2];
-    __shared__ int s_last;
-    __shared__ unsigned long long s_ticket;
-    const int tid = threadIdx.x;
-    if (tid == 0) s_ticket = atomicAdd(P.ticket, 1ull);
+    __shared__ int s_last[2];
+    __shared__ unsigned long long s_ticket[2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long next_raw = 0;  // thread 0: the ticket after the next one, drawn early
+    if (tid == 0) {
+        s_ticket[1] = logical(atomicAdd(P.ticket, 1ull));
+        next_raw = atomicAdd(P.ticket, 1ull);
+    }
     __syncthreads();
-    unsigned long long t = s_ticket;
-    while (t < P.total_tickets) {
-        __syncthreads();
-        unsigned long long nxt = 0;
-        if (tid == 0) nxt = atomicAdd(P.ticket, 1ull);
-        const int64_t b = (int64_t)(t / (unsigned)P.n_chunks);
-        const int c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
-        const int n = __ldg(P.accept_len + b);
-        const bool valid = n >= 0 && n <= P.gamma;
-        const float *p = P.p_row + (size_t)b * P.V;
-        const float *q = (valid && n < P.gamma) ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-        const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
-        const double tot = block_sum(valid ? chunk_mass(p, q, e0, e1) : 0.0, s_w);
-        if (tid == 0) {
-            P.chunk_sum[(size_t)b * P.n_chunks + c] = tot;
-            __threadfence();
-            s_last = (atomicAdd(&P.seq_cnt[b], 1u) == (unsigned)(P.n_chunks - 1));
-        }
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            if (!valid) {
-                if (tid == 0) {
-                    P.token[b] = -1;
-                    if (P.flags) P.flags[b] = DSSD_RS_FLAG_INVALID;
-                }
-            } else {
-                draw(P, b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_w, &s_pick, s_i);
+    unsigned long long t = s_ticket[1];
+    bool pending = false;   // the previous ticket's count has not been looked at yet
+    int64_t pend_b = 0;
+    unsigned pend_raw = 0;  // thread 0: raw result of that count
+    for (int it = 0;; ++it) {
+        const int buf = it & 1;
+        const bool have = t < P.total_tickets;
+        int64_t b = 0;
+        int c = 0;
+        double acc = 0.0;
+        if (have) {
+            b = (int64_t)(t / (unsigned)P.n_chunks);
+            c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
+            const int n = __ldg(P.accept_len + b);
+            if (n >= 0 && n <= P.gamma) {
+                const float *p = P.p_row + (size_t)b * P.V;
+                const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
+                const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
+                acc = chunk_mass(p, q, e0, e1);
             }
         }
-        if (tid == 0) s_ticket = nxt;
+        acc = warp_sum(acc);
+        if (lane == 0) s_w[buf][warp] = acc;
+        if (tid == 0) {
+            s_last[buf] = pending && logical(pend_raw) == (unsigned)(P.n_chunks - 1);
+            s_ticket[buf] = logical(next_raw);
+            if (have) next_raw = atomicAdd(P.ticket, 1ull);
+        }
         __syncthreads();
-        t = s_ticket;
+        const unsigned long long t_next = s_ticket[buf];
+        const bool last = s_last[buf] != 0;
+        unsigned new_raw = 0;
+        if (tid == 0 && have) {
+            double tot = 0.0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) tot += s_w[buf][w];
+            st_relaxed_u64(reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_chunks + c,
+                           (unsigned long long)__double_as_longlong(tot));
+            new_raw = atomicAdd(&P.seq_cnt[b], 1u);
+        }
+        if (last) {
+            const int n = __ldg(P.accept_len + pend_b);
+            if (n < 0 || n > P.gamma) {
+                if (tid == 0) {
+                    P.token[pend_b] = -1;
+                    if (P.flags) P.flags[pend_b] = DSSD_RS_FLAG_INVALID;
+                }
+            } else {
+                const float *p = P.p_row + (size_t)pend_b * P.V;
+                const float *q = n < P.gamma ? P.draft_q + ((size_t)pend_b * P.gamma + n) * (size_t)P.V : nullptr;
+                draw(P, pend_b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
+            }
+        }
+        if (!have) break;  // the count of the last ticket was looked at in this round
+        pending = true;
+        pend_b = b;
+        pend_raw = new_raw;
+        t = t_next;
     }
 }
 
@@ -253,6 +380,8 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const ResamplePar
 
 size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
 {
+    // all of it is filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
+    // and the chunk sums read "not yet"
     const int n_chunks = (V + kResampleChunk - 1) / kResampleChunk;
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -262,13 +391,12 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
     };
     const size_t o_ticket = take(16);
     const size_t o_cnt = take((size_t)B * 4);
-    const size_t zero_bytes = off;
     const size_t o_sum = take((size_t)B * (size_t)n_chunks * sizeof(double));
     if (P) {
         P->ticket = reinterpret_cast<unsigned long long *>(base + o_ticket);
         P->seq_cnt = reinterpret_cast<unsigned *>(base + o_cnt);
         P->chunk_sum = reinterpret_cast<double *>(base + o_sum);
-        P->zero_bytes = zero_bytes;
+        P->fill_bytes = off;
         P->n_chunks = n_chunks;
         P->total_tickets = (unsigned long long)B * (unsigned long long)n_chunks;
     }
@@ -284,7 +412,8 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, resample_kernel, kThreads, 0)) != cudaSuccess) return err;
     if (occ < 1) occ = 1;
     resample_workspace_layout(P.B, P.V, &P, static_cast<char *>(workspace));
-    if ((err = cudaMemsetAsync(workspace, 0, P.zero_bytes, stream)) != cudaSuccess) return err;
+    P.spin_limit = 1u << 20;
+    if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long resident = (unsigned long long)sms * (unsigned long long)occ;
     const unsigned grid = (unsigned)(P.total_tickets < resident ? P.total_tickets : resident);
     resample_kernel<<<grid, kThreads, 0, stream>>>(P);
@@ -351,8 +480,8 @@ extern "C" dssd_status dssd_device_resample_static(const float *p_row, const flo
     P.V = V;
     P.token = token;
     P.flags = flags;
-    // resample_launch clears the counters that must start at zero; the rest of the scratch is
-    // written before it is read, so what the previous call left behind does not matter
+    // resample_launch refills the part of the scratch it uses (counters and validity patterns),
+    // so what the previous call left behind does not matter
     e = dssd::resample_launch(P, scratch, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) {
         dssd::set_last_cuda_error((int)e);

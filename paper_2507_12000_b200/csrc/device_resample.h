@@ -23,7 +23,8 @@ struct ResampleParams {
     unsigned long long *ticket;
     unsigned *seq_cnt;   // [B]
     double *chunk_sum;   // [B, n_chunks]
-    size_t zero_bytes;
+    size_t fill_bytes;
+    unsigned spin_limit;
 };
 
 size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base);
