@@ -22,7 +22,9 @@ namespace dssd {
 
 namespace {
 
-constexpr int kRun = kResampleChunk / kThreads;  // contiguous entries per thread in pass B
+constexpr int kSub = kResampleChunk / 2;  // entries per chunk sum: a ticket covers two of them
+constexpr int kRun = kSub / kThreads;      // contiguous entries per thread in pass B
+static_assert(kRun == 16, "pass B fetches a run as one group of 16 entries");
 
 __device__ __forceinline__ double res(float p, float q) { return fmax(0.0, (double)p - (double)q); }
 
@@ -154,18 +156,52 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
                      double *s_w, Pick *s_pick, int *s_i)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_chunks;
+    unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub;
     for (int attempt = 0; attempt < 2; ++attempt) {
+        bool ok;
+        if (P.n_sub <= kThreads) {
+            // one chunk per thread: a single scan gives Z and every inclusive prefix
+            const double m = tid < P.n_sub ? load_chunk_sum(P, cs, tid) : 0.0;
+            double Z;
+            const double incl = block_scan(m, s_w, Z);
+            ok = (Z > 0.0) && (Z < INFINITY);
+            if (ok) {
+                const double target = (double)__ldg(P.uniforms + b) * Z;
+                if (tid == 0) {
+                    s_i[0] = 0x7fffffff;
+                    s_i[1] = -1;
+                }
+                __syncthreads();
+                const bool crosses = tid < P.n_sub && incl > target;
+                const unsigned bal = __ballot_sync(0xffffffffu, crosses);
+                if (lane == 0 && bal) atomicMin(&s_i[0], warp * 32 + __ffs(bal) - 1);
+                const unsigned pos = __ballot_sync(0xffffffffu, tid < P.n_sub && m > 0.0);
+                if (lane == 0 && pos) atomicMax(&s_i[1], warp * 32 + 31 - __clz(pos));
+                __syncthreads();
+                const int first = s_i[0], last = s_i[1];
+                if (tid == (first != 0x7fffffff ? first : last)) {
+                    Pick pk;
+                    pk.ok = 1;
+                    pk.beyond = first == 0x7fffffff;
+                    pk.chunk = tid;
+                    pk.base = incl - m;
+                    pk.target = target;
+                    *s_pick = pk;
+                }
+                __syncthreads();
+                break;
+            }
+        } else {
         // Z = sum of the chunk sums, in groups of one chunk per thread
         double Z = 0.0;
-        for (int base = 0; base < P.n_chunks; base += kThreads) {
+        for (int base = 0; base < P.n_sub; base += kThreads) {
             const int c = base + tid;
             double tot;
-            block_scan(c < P.n_chunks ? load_chunk_sum(P, cs, c) : 0.0, s_w, tot);
+            block_scan(c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0, s_w, tot);
             Z += tot;
             __syncthreads();
         }
-        const bool ok = (Z > 0.0) && (Z < INFINITY);
+        ok = (Z > 0.0) && (Z < INFINITY);
         if (ok) {
             // the first chunk whose inclusive prefix exceeds the target, else the last chunk with mass
             const double target = (double)__ldg(P.uniforms + b) * Z;
@@ -177,16 +213,16 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
             double carry = 0.0;
             double my_base_first = 0.0, my_base_last = 0.0;
             int my_first = 0x7fffffff, my_last = -1;
-            for (int base = 0; base < P.n_chunks; base += kThreads) {
+            for (int base = 0; base < P.n_sub; base += kThreads) {
                 const int c = base + tid;
-                const double m = c < P.n_chunks ? load_chunk_sum(P, cs, c) : 0.0;
+                const double m = c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0;
                 double tot;
                 const double incl = carry + block_scan(m, s_w, tot);
-                if (c < P.n_chunks && incl > target && my_first == 0x7fffffff) {
+                if (c < P.n_sub && incl > target && my_first == 0x7fffffff) {
                     my_first = c;
                     my_base_first = incl - m;
                 }
-                if (c < P.n_chunks && m > 0.0) {
+                if (c < P.n_sub && m > 0.0) {
                     my_last = c;
                     my_base_last = incl - m;
                 }
@@ -209,6 +245,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
             __syncthreads();
             break;
         }
+        }
         if (q == nullptr) {  // already drawing from p: the row has no usable mass
             if (tid == 0) {
                 P.token[b] = -1;
@@ -219,20 +256,20 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
         // residual has no mass (p == q): draw from p instead
         q = nullptr;
         fl |= DSSD_RS_FLAG_FALLBACK;
-        for (int c = 0; c < P.n_chunks; ++c) {
-            const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
+        for (int c = 0; c < P.n_sub; ++c) {
+            const int e0 = c * kSub, e1 = min(P.V, e0 + kSub);
             const double tot = block_sum(chunk_mass(p, nullptr, e0, e1), s_w);
             if (tid == 0) st_relaxed_u64(cs + c, (unsigned long long)__double_as_longlong(tot));
         }
         __syncthreads();
     }
     const Pick pk = *s_pick;
-    const int e0 = pk.chunk * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
+    const int e0 = pk.chunk * kSub, e1 = min(P.V, e0 + kSub);
     const int r0 = min(e1, e0 + tid * kRun), r1 = min(e1, r0 + kRun);
     double mine = 0.0;
     int last_pos = -1;
-    // The run is fetched in groups of 16 entries whose loads are all issued before the first is
-    // used (two round trips for the run, not one per entry); entries past the row's end read as 0.
+    // The run's 16 entries are all requested before the first is used (one round trip for the
+    // run, not one per entry); entries past the row's end read as 0.
     const bool vec = (r1 - r0 == kRun) &&
                      (((reinterpret_cast<uintptr_t>(p + r0) | (q ? reinterpret_cast<uintptr_t>(q + r0) : 0)) & 15u) == 0);
 #pragma unroll
@@ -302,7 +339,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
 
 __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ ResampleParams P)
 {
-    __shared__ double s_w[2][kWarps];
+    __shared__ double s_w[2][kWarps][2];
     __shared__ double s_scan[kWarps];
     __shared__ Pick s_pick;
     __shared__ int s_i[2];
@@ -318,26 +355,32 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     unsigned long long t = s_ticket[1];
     bool pending = false;   // the previous ticket's count has not been looked at yet
     int64_t pend_b = 0;
+    int pend_n = -1;        // that ticket's sequence and its accepted length
     unsigned pend_raw = 0;  // thread 0: raw result of that count
     for (int it = 0;; ++it) {
         const int buf = it & 1;
         const bool have = t < P.total_tickets;
         int64_t b = 0;
-        int c = 0;
-        double acc = 0.0;
+        int c = 0, n = -1;
+        double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
         if (have) {
             b = (int64_t)(t / (unsigned)P.n_chunks);
             c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
-            const int n = __ldg(P.accept_len + b);
+            n = __ldg(P.accept_len + b);
             if (n >= 0 && n <= P.gamma) {
                 const float *p = P.p_row + (size_t)b * P.V;
                 const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-                const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kResampleChunk);
-                acc = chunk_mass(p, q, e0, e1);
+                const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
+                acc0 = chunk_mass(p, q, e0, e1);
+                if (e2 > e1) acc1 = chunk_mass(p, q, e1, e2);
             }
         }
-        acc = warp_sum(acc);
-        if (lane == 0) s_w[buf][warp] = acc;
+        acc0 = warp_sum(acc0);
+        acc1 = warp_sum(acc1);
+        if (lane == 0) {
+            s_w[buf][warp][0] = acc0;
+            s_w[buf][warp][1] = acc1;
+        }
         if (tid == 0) {
             s_last[buf] = pending && logical(pend_raw) == (unsigned)(P.n_chunks - 1);
             s_ticket[buf] = logical(next_raw);
@@ -348,15 +391,19 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         const bool last = s_last[buf] != 0;
         unsigned new_raw = 0;
         if (tid == 0 && have) {
-            double tot = 0.0;
+            double tot0 = 0.0, tot1 = 0.0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) tot += s_w[buf][w];
-            st_relaxed_u64(reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_chunks + c,
-                           (unsigned long long)__double_as_longlong(tot));
+            for (int w = 0; w < kWarps; ++w) {
+                tot0 += s_w[buf][w][0];
+                tot1 += s_w[buf][w][1];
+            }
+            unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub + 2 * c;
+            st_relaxed_u64(cs, (unsigned long long)__double_as_longlong(tot0));
+            if (2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
             new_raw = atomicAdd(&P.seq_cnt[b], 1u);
         }
         if (last) {
-            const int n = __ldg(P.accept_len + pend_b);
+            const int n = pend_n;
             if (n < 0 || n > P.gamma) {
                 if (tid == 0) {
                     P.token[pend_b] = -1;
@@ -371,6 +418,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         if (!have) break;  // the count of the last ticket was looked at in this round
         pending = true;
         pend_b = b;
+        pend_n = n;
         pend_raw = new_raw;
         t = t_next;
     }
@@ -391,13 +439,15 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
     };
     const size_t o_ticket = take(16);
     const size_t o_cnt = take((size_t)B * 4);
-    const size_t o_sum = take((size_t)B * (size_t)n_chunks * sizeof(double));
+    const int n_sub = (V + kResampleChunk / 2 - 1) / (kResampleChunk / 2);
+    const size_t o_sum = take((size_t)B * (size_t)n_sub * sizeof(double));
     if (P) {
         P->ticket = reinterpret_cast<unsigned long long *>(base + o_ticket);
         P->seq_cnt = reinterpret_cast<unsigned *>(base + o_cnt);
         P->chunk_sum = reinterpret_cast<double *>(base + o_sum);
         P->fill_bytes = off;
         P->n_chunks = n_chunks;
+        P->n_sub = n_sub;
         P->total_tickets = (unsigned long long)B * (unsigned long long)n_chunks;
     }
     return off;

@@ -17,12 +17,13 @@ struct ResampleParams {
     int B, gamma, V;
     int32_t *token;
     uint32_t *flags;
-    int n_chunks;
+    int n_chunks;   // tickets per sequence (kResampleChunk entries each)
+    int n_sub;      // chunk sums per sequence (two per ticket)
     unsigned long long total_tickets;
     // scratch
     unsigned long long *ticket;
     unsigned *seq_cnt;   // [B]
-    double *chunk_sum;   // [B, n_chunks]
+    double *chunk_sum;   // [B, n_sub]
     size_t fill_bytes;
     unsigned spin_limit;
 };
