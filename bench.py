@@ -37,7 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/edge_verify_kernel_c4.md: 443.4 MB read + 100.5 MB written
+    "c4": {"bytes": 543948800, "kernel_hash": "64db35991aeadefe"},
+}
 
 
 def _kernel_hash() -> str:
@@ -132,18 +135,21 @@ def _torch_inputs(d, device=None, pin=False):
     return out
 
 
-def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, repeats: int = 1):
-    """rows/s of the CPU oracle (both halves) on the first n_seq sequences."""
+def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float = 1.5):
+    """rows/s of the CPU oracle (both halves) on the first n_seq sequences: whole passes are
+    repeated until about `min_seconds` of wall time (some 10-30 s of CPU work on all cores) have gone."""
     from oracle import oracle as O
 
     sub = {k: v[:n_seq] for k, v in d.items()}
-    best = None
-    for _ in range(repeats):
-        t0 = time.perf_counter()
+    passes = 0
+    t0 = time.perf_counter()
+    while True:
         O.verify_round(sub, w.temperature, threads=threads)
+        passes += 1
         dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    return n_seq * (w.gamma + 1) / best, best
+        if dt >= min_seconds or passes >= 64:
+            break
+    return passes * n_seq * (w.gamma + 1) / dt, dt, passes
 
 
 def run_reference(args, w: di.Workload):
@@ -184,6 +190,20 @@ def _config(w: di.Workload, args):
             "parallelism": f"batch-sharded x{args.gpus}, no collective"}
 
 
+def rank_workload(w: di.Workload, rank: int) -> di.Workload:
+    """Weak scaling: every rank verifies its own batch of the same shape, drawn from its own seed."""
+    return di.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+
+
+def max_over_ranks(value_ms: float, dist, device) -> float:
+    """The job's time is the slowest rank's (device-timed) time."""
+    import torch
+
+    t = torch.tensor([value_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args, w: di.Workload):
     import torch
     import torch.distributed as dist
@@ -201,8 +221,7 @@ def run_ours(args, w: di.Workload):
         dist.init_process_group("nccl", device_id=dev)
     from paper_2507_12000_b200 import binding as B
 
-    # every rank draws its own batch (weak scaling): same shape, different seed
-    wr = di.Workload(**{**w.__dict__, "seed": w.seed + 7919 * rank})
+    wr = rank_workload(w, rank)
     d = di.generate(wr, threads=max(1, cores // max(1, min(world, 8))))
     logit_bytes = d["target_logits"].nbytes
     # inputs smaller than L2 rotate through enough copies to exceed it
@@ -250,9 +269,7 @@ def run_ours(args, w: di.Workload):
     edge_ms = [e[0].elapsed_time(e[1]) for e in ev]
     rs_ms = [e[1].elapsed_time(e[2]) for e in ev]
     if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+        total_ms = max_over_ranks(total_ms, dist, dev)
     sampler.stop_flag = True
     sampler.join(timeout=1.0)
     clocks = sampler.summary(t_host0, t_host1)
@@ -278,9 +295,7 @@ def run_ours(args, w: di.Workload):
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
     if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = sum(host[k].numel() * host[k].element_size() for k in
               ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs"))
     d2h = 4 * Bn * 4
@@ -307,10 +322,10 @@ def run_ours(args, w: di.Workload):
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         n_seq = min(Bn, args.ref_sequences)
-        rate, secs = oracle_rate(w, d, n_seq, cores)
+        rate, secs, passes = oracle_rate(w, d, n_seq, cores)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"first {n_seq} of {Bn} sequences of {w.name}, both halves, one pass of {secs:.2f} s wall "
-                         f"on {cores} threads"}
+               "sample": f"first {n_seq} of {Bn} sequences of {w.name}, both halves, {passes} passes in {secs:.2f} s "
+                         f"wall on {cores} threads"}
         ref = O.verify_round({k: v[:n_seq] for k, v in d.items()}, w.temperature, threads=cores)
         near = ref["margin_acc"] < 1e-6
         parity = {"sequences_checked": n_seq,

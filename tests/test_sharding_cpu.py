@@ -1,0 +1,48 @@
+"""The multi-GPU path shards the batch by sequence with no exchange step.  Two gloo ranks on the
+CPU check what that rests on: a rank's slice of a workload, generated and verified on its own,
+equals the same slice of the whole batch (sequences are independent and individually seeded), and
+the job's time is the maximum over the ranks."""
+import os
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _rank_main(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    import dssd_inputs as di
+    from oracle import oracle as O
+
+    w = di.custom(B=6, gamma=3, V=4099, dtype="bf16", temperature=0.8, sigma_d=0.8, seed=99)
+    per = w.B // world
+    d = di.generate(w, rank * per, (rank + 1) * per)      # this rank's sequences only
+    ref = O.verify_round(d, w.temperature)
+    mine = torch.from_numpy(np.stack([ref["accept_len"], ref["token"]]).astype(np.int64))
+    gathered = [torch.zeros_like(mine) for _ in range(world)]
+    dist.all_gather(gathered, mine)                          # only to check: the path itself needs no collective
+    slowest = bench.max_over_ranks(10.0 + rank, dist, torch.device("cpu"))
+    seeds = [bench.rank_workload(w, r).seed for r in range(world)]
+    if rank == 0:
+        whole = O.verify_round(di.generate(w), w.temperature)
+        got = torch.cat(gathered, dim=1).numpy()
+        np.save(os.path.join(out_dir, "ok.npy"),
+                np.array([int((got[0] == whole["accept_len"]).all() and (got[1] == whole["token"]).all()),
+                          int(slowest == 10.0 + world - 1), int(len(set(seeds)) == world)]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_by_sequence(tmp_path, oracle_mod):
+    port = 29500 + (os.getpid() % 2000)
+    mp.spawn(_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    ok = np.load(tmp_path / "ok.npy")
+    assert ok.tolist() == [1, 1, 1]
