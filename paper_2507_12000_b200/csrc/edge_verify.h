@@ -17,10 +17,10 @@ namespace dssd {
 #define DSSD_EDGE_STAGES 6
 #endif
 #ifndef DSSD_EDGE_MAX_RUN
-#define DSSD_EDGE_MAX_RUN 8
+#define DSSD_EDGE_MAX_RUN 16
 #endif
 #ifndef DSSD_EDGE_TICKETS_PER_CTA
-#define DSSD_EDGE_TICKETS_PER_CTA 8
+#define DSSD_EDGE_TICKETS_PER_CTA 4
 #endif
 
 constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
