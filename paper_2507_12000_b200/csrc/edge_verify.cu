@@ -740,12 +740,14 @@ __device__ __forceinline__ void claim_look(const EdgeParams &P, Claim &c)
 
 // One step of the claim.  Returns true, with the ticket's fields of `t` and its stage range
 // filled in, when an EMIT ticket can start now.
-__device__ __forceinline__ bool claim_step(const EdgeParams &P, Claim &c, Ticket &t, int &k_begin, int &k_end)
+__device__ __forceinline__ bool claim_step(const EdgeParams &P, Claim &c, Ticket &t, int &k_begin, int &k_end, bool eager)
 {
     if (c.state == kWatch) {
         const unsigned long long ready = (unsigned long long)logical(c.ready_raw);
         const unsigned long long head = logical(c.head_raw);
-        if (!c.exhausted && head < ready * (unsigned long long)P.n_emit_runs) {
+        // `eager` (nothing else left to do): claim the next ticket even before its sequence is
+        // ready and watch its entry, which saves the round trips of noticing and claiming later
+        if (!c.exhausted && (head < ready * (unsigned long long)P.n_emit_runs || (eager && head < P.total_emit))) {
             c.claim_raw = atomicAdd(P.emit_head, 1ull);
             c.state = kClaimed;
         } else {
@@ -830,7 +832,7 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     for (;;) {
         Ticket t;
         int k_begin = 0, k_end = 0;
-        if (er.kind == kEnd && claim_step(P, c, t, k_begin, k_end)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
+        if (er.kind == kEnd && claim_step(P, c, t, k_begin, k_end, !lse_left && lr.kind == kEnd)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
         if (er.kind == kEnd && lr.kind == kEnd && lse_left) {
             const unsigned long long no = logical(lse_raw);
             if (no < P.total_lse) {
@@ -1010,7 +1012,9 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     const int runs_per_row = (int)((P.n_slices + run - 1) / run);
     run = (unsigned long long)((P.n_slices + runs_per_row - 1) / runs_per_row);
     P.lse_run = (int)run;
-    P.emit_run = (int)run;
+    // EMIT tickets stay short: they cost the consumers nothing per ticket, and at the end of the
+    // launch the last sequences' rows are then written by several CTAs at once
+    P.emit_run = (int)(run < 2 ? run : 2);
     P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
     P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
     P.total_lse = R * (unsigned long long)P.n_lse_runs;
