@@ -1014,7 +1014,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     P.lse_run = (int)run;
     // EMIT tickets stay short: they cost the consumers nothing per ticket, and at the end of the
     // launch the last sequences' rows are then written by several CTAs at once
-    P.emit_run = (int)(run < 2 ? run : 2);
+    P.emit_run = (int)(run < (unsigned long long)kEdgeEmitRun ? run : (unsigned long long)kEdgeEmitRun);
     P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
     P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
     P.total_lse = R * (unsigned long long)P.n_lse_runs;

@@ -17,10 +17,13 @@ namespace dssd {
 #define DSSD_EDGE_STAGES 6
 #endif
 #ifndef DSSD_EDGE_MAX_RUN
-#define DSSD_EDGE_MAX_RUN 16
+#define DSSD_EDGE_MAX_RUN 32
+#endif
+#ifndef DSSD_EDGE_EMIT_RUN
+#define DSSD_EDGE_EMIT_RUN 2
 #endif
 #ifndef DSSD_EDGE_TICKETS_PER_CTA
-#define DSSD_EDGE_TICKETS_PER_CTA 4
+#define DSSD_EDGE_TICKETS_PER_CTA 2
 #endif
 
 constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
@@ -28,6 +31,7 @@ constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 2);  // + the producer warp 
 constexpr int kEdgeStageBytes = DSSD_EDGE_STAGE_BYTES;   // logits bytes per ring stage (one bulk copy)
 constexpr int kEdgeStages = DSSD_EDGE_STAGES;            // ring stages per CTA
 constexpr int kEdgeMaxRun = DSSD_EDGE_MAX_RUN;           // most consecutive stages of a row in one ticket
+constexpr int kEdgeEmitRun = DSSD_EDGE_EMIT_RUN;        // most stages of row n in one EMIT ticket
 constexpr int kEdgeTicketsPerCta = DSSD_EDGE_TICKETS_PER_CTA;  // tickets aimed at per resident CTA
 
 // What the emission of row P_n needs to know about a folded sequence: two 8-byte slots, each
