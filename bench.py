@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 443.4 MB read + 100.5 MB written
-    "c4": {"bytes": 543948800, "kernel_hash": "64db35991aeadefe"},
+    # profiles/edge_verify_kernel_c4.md: 446.0 MB read + 98.3 MB written
+    "c4": {"bytes": 544329472, "kernel_hash": "d59083ef4c8f7c4c"},
 }
 
 
