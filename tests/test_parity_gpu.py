@@ -56,6 +56,31 @@ def test_full_size_configs(B, oracle_mod, name):
     assert rep["mismatch_token_iso"] <= rep["near_cdf"]
 
 
+def test_largest_sweep_point_sampled(B, oracle_mod):
+    """B=1024, gamma=16, V=50272 float32 (3.5 GB of logits) in the benchmark's launch configuration;
+    the oracle checks a sample of the sequences one by one."""
+    w = di.sweep_max()
+    d = di.generate(w, threads=16)
+    g = to_device(d)
+    ev = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"], w.temperature)
+    rs = B.dssd_device_resample(ev["p_row"], g["draft_q"], ev["accept_len"], g["uniforms_rs"], w.gamma)
+    torch.cuda.synchronize()
+    n_gpu = ev["accept_len"].cpu().numpy()
+    tok_gpu = rs["token"].cpu().numpy()
+    assert (ev["flags"].cpu().numpy() == 0).all()
+    assert ((n_gpu >= 0) & (n_gpu <= w.gamma)).all() and ((tok_gpu >= 0) & (tok_gpu < w.V)).all()
+    sample = np.r_[0:24, 500:524, w.B - 24:w.B]
+    sub = {k: np.ascontiguousarray(v[sample]) for k, v in d.items()}
+    ref = oracle_mod.verify_round(sub, w.temperature, threads=8)
+    near = (ref["margin_acc"] < 1e-6)
+    assert ((n_gpu[sample] == ref["accept_len"]) | near).all()
+    same = n_gpu[sample] == ref["accept_len"]
+    p_gpu = ev["p_row"][torch.from_numpy(sample).cuda()].cpu().numpy()
+    assert prob_close(p_gpu[same], ref["p_row"][same]).all()
+    slack = np.maximum(1e-6, 2e-5 / np.maximum(ref["Z"], 1e-30))
+    assert ((tok_gpu[sample] == ref["token"]) | ~same | (ref["margin_cdf"] < slack)).all()
+
+
 def test_sweep_points_sampled(B, oracle_mod):
     """A spread of the V=50272 sweep (largest batch sizes run on a slice of their sequences)."""
     for w in di.sweep_points():
