@@ -1,13 +1,14 @@
 // Device half of the verification round: residual (or bonus) inverse-CDF draw.
 //
 // Pass A, ticket (b, c): stream chunk c of p_row[b] and of Q_n[b], form r = max(0, p - q) (or
-// r = p for the bonus draw) and add it up in float64 -> chunk_sum[b, c], an 8-byte slot that is
-// valid once it differs from the all-ones pattern the workspace is filled with.  The ticket is
-// then counted on its sequence; the count's result is looked at one ticket later, so a CTA has
-// one barrier per ticket and waits for no round trip.
-// Pass B, run by the CTA that brought the last chunk of sequence b: a block-wide float64 prefix
-// over the chunk sums gives Z and the chunk holding u' * Z; that one chunk is read again (from
-// L2), a block-wide prefix sum over per-thread runs finds the thread, and the thread walks its run.
+// r = p for the bonus draw) and add it up in float64 -> two chunk sums, 8-byte slots that are
+// valid once they differ from the all-ones pattern the workspace is filled with.  A ticket costs
+// one barrier and waits for no round trip.
+// Pass B, ticket b, taken by a CTA once no chunk is left for it: a block-wide float64 prefix over
+// the sequence's chunk sums gives Z and the chunk holding u' * Z; every thread fetches its run of
+// that chunk (from L2 or HBM), a second prefix finds the thread, and the thread walks its run.
+// The draws run after the streams because their dependent round trips are several times longer
+// while the memory system is saturated.
 // All sums are float64, so the token differs from an index-order float64 scan only when u' * Z
 // lies within rounding (about 1e-13 relative) of a CDF step.
 #include "device_resample.h"
@@ -112,7 +113,6 @@ struct Pick {  // what thread 0 hands to the CTA for pass B
 
 constexpr unsigned long long kFill64 = ~0ull;
 
-__device__ __forceinline__ unsigned logical(unsigned raw) { return raw + 1u; }
 __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
 
 // chunk sum (b, c); a sum whose store has not landed yet still shows the fill pattern and is
@@ -343,9 +343,10 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     __shared__ double s_scan[kWarps];
     __shared__ Pick s_pick;
     __shared__ int s_i[2];
-    __shared__ int s_last[2];
     __shared__ unsigned long long s_ticket[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---- pass A: chunk sums.  One barrier per ticket, no round trip waited for. ----
     unsigned long long next_raw = 0;  // thread 0: the ticket after the next one, drawn early
     if (tid == 0) {
         s_ticket[1] = logical(atomicAdd(P.ticket, 1ull));
@@ -353,27 +354,18 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     }
     __syncthreads();
     unsigned long long t = s_ticket[1];
-    bool pending = false;   // the previous ticket's count has not been looked at yet
-    int64_t pend_b = 0;
-    int pend_n = -1;        // that ticket's sequence and its accepted length
-    unsigned pend_raw = 0;  // thread 0: raw result of that count
-    for (int it = 0;; ++it) {
+    for (int it = 0; t < P.total_tickets; ++it) {
         const int buf = it & 1;
-        const bool have = t < P.total_tickets;
-        int64_t b = 0;
-        int c = 0, n = -1;
+        const int64_t b = (int64_t)(t / (unsigned)P.n_chunks);
+        const int c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
+        const int n = __ldg(P.accept_len + b);
         double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
-        if (have) {
-            b = (int64_t)(t / (unsigned)P.n_chunks);
-            c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
-            n = __ldg(P.accept_len + b);
-            if (n >= 0 && n <= P.gamma) {
-                const float *p = P.p_row + (size_t)b * P.V;
-                const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-                const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
-                acc0 = chunk_mass(p, q, e0, e1);
-                if (e2 > e1) acc1 = chunk_mass(p, q, e1, e2);
-            }
+        if (n >= 0 && n <= P.gamma) {
+            const float *p = P.p_row + (size_t)b * P.V;
+            const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
+            const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
+            acc0 = chunk_mass(p, q, e0, e1);
+            if (e2 > e1) acc1 = chunk_mass(p, q, e1, e2);
         }
         acc0 = warp_sum(acc0);
         acc1 = warp_sum(acc1);
@@ -382,15 +374,11 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
             s_w[buf][warp][1] = acc1;
         }
         if (tid == 0) {
-            s_last[buf] = pending && logical(pend_raw) == (unsigned)(P.n_chunks - 1);
             s_ticket[buf] = logical(next_raw);
-            if (have) next_raw = atomicAdd(P.ticket, 1ull);
+            next_raw = atomicAdd(P.ticket, 1ull);
         }
         __syncthreads();
-        const unsigned long long t_next = s_ticket[buf];
-        const bool last = s_last[buf] != 0;
-        unsigned new_raw = 0;
-        if (tid == 0 && have) {
+        if (tid == 0) {
             double tot0 = 0.0, tot1 = 0.0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
@@ -400,27 +388,40 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
             unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub + 2 * c;
             st_relaxed_u64(cs, (unsigned long long)__double_as_longlong(tot0));
             if (2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
-            new_raw = atomicAdd(&P.seq_cnt[b], 1u);
         }
-        if (last) {
-            const int n = pend_n;
-            if (n < 0 || n > P.gamma) {
-                if (tid == 0) {
-                    P.token[pend_b] = -1;
-                    if (P.flags) P.flags[pend_b] = DSSD_RS_FLAG_INVALID;
-                }
-            } else {
-                const float *p = P.p_row + (size_t)pend_b * P.V;
-                const float *q = n < P.gamma ? P.draft_q + ((size_t)pend_b * P.gamma + n) * (size_t)P.V : nullptr;
-                draw(P, pend_b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
+        t = s_ticket[buf];
+    }
+
+    // ---- pass B: the draws, one sequence per ticket, once this CTA has no chunk left.  By then
+    // the memory system is no longer saturated by the streams, so a draw's two round trips are
+    // short; a chunk sum that has not landed yet is polled for (its CTA is still running). ----
+    __syncthreads();
+    if (tid == 0) {
+        s_ticket[0] = logical(atomicAdd(P.draw_ticket, 1ull));
+        next_raw = atomicAdd(P.draw_ticket, 1ull);
+    }
+    __syncthreads();
+    unsigned long long d = s_ticket[0];
+    for (int it = 1; d < (unsigned long long)P.B; ++it) {
+        const int buf = it & 1;
+        if (tid == 0) {
+            s_ticket[buf] = logical(next_raw);
+            next_raw = atomicAdd(P.draw_ticket, 1ull);
+        }
+        const int64_t b = (int64_t)d;
+        const int n = __ldg(P.accept_len + b);
+        if (n < 0 || n > P.gamma) {
+            if (tid == 0) {
+                P.token[b] = -1;
+                if (P.flags) P.flags[b] = DSSD_RS_FLAG_INVALID;
             }
+        } else {
+            const float *p = P.p_row + (size_t)b * P.V;
+            const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
+            draw(P, b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
         }
-        if (!have) break;  // the count of the last ticket was looked at in this round
-        pending = true;
-        pend_b = b;
-        pend_n = n;
-        pend_raw = new_raw;
-        t = t_next;
+        __syncthreads();
+        d = s_ticket[buf];
     }
 }
 
@@ -437,13 +438,12 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
         off += (bytes + 255) & ~(size_t)255;
         return o;
     };
-    const size_t o_ticket = take(16);
-    const size_t o_cnt = take((size_t)B * 4);
+    const size_t o_ticket = take(256);  // the two ticket counters, on separate 128-byte lines
     const int n_sub = (V + kResampleChunk / 2 - 1) / (kResampleChunk / 2);
     const size_t o_sum = take((size_t)B * (size_t)n_sub * sizeof(double));
     if (P) {
         P->ticket = reinterpret_cast<unsigned long long *>(base + o_ticket);
-        P->seq_cnt = reinterpret_cast<unsigned *>(base + o_cnt);
+        P->draw_ticket = reinterpret_cast<unsigned long long *>(base + o_ticket + 128);
         P->chunk_sum = reinterpret_cast<double *>(base + o_sum);
         P->fill_bytes = off;
         P->n_chunks = n_chunks;

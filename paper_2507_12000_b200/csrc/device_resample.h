@@ -21,8 +21,8 @@ struct ResampleParams {
     int n_sub;      // chunk sums per sequence (two per ticket)
     unsigned long long total_tickets;
     // scratch
-    unsigned long long *ticket;
-    unsigned *seq_cnt;   // [B]
+    unsigned long long *ticket;       // next chunk ticket
+    unsigned long long *draw_ticket;  // next sequence to draw
     double *chunk_sum;   // [B, n_sub]
     size_t fill_bytes;
     unsigned spin_limit;
