@@ -6,22 +6,28 @@
 // an "empty" mbarrier (one arrival per consumer warp).  Warps 1..kEdgeConsumers are consumers:
 // every consumer takes a fixed 1/kEdgeConsumers share of each stage.  The last warp is the fold
 // warp, which serves a mailbox in shared memory.
-//   LSE(row, run)    a run of consecutive stages of one target row: every consumer keeps an online
-//                    maximum and sum of 2^(l * c1 - ref2) in float32 over its shares; at the run's
-//                    last stage the consumers' results meet in shared memory and the last to
-//                    arrive posts the ticket's partial (ref2, sum) to the fold warp.  ref2 is an
+//   LSE(row, run)    a run of consecutive stages of one target row (the whole row when it is
+//                    short enough): every consumer keeps, per lane, an online maximum and sum of
+//                    2^(l * c1 - ref2) in float32 over its shares.  At the run's last stage the
+//                    consumers leave these per-lane pairs in a meeting area in shared memory
+//                    (plain stores) and the last to arrive posts the ticket to the fold warp,
+//                    which reduces the area to the ticket's partial (ref2, sum).  ref2 is an
 //                    integer, so partials combine by exact power-of-two scaling.
-//   EMIT(slot, run)  a run of stages of row n of a sequence taken from the `ready` queue: the row
-//                    is streamed again (from L2) and p_row = 2^(l * c1 - ref2) / S is written.
-// The fold warp stores each partial to global memory and counts it; the fold warp that brings a
-// row's last partial folds the row (float64 log-sum-exp, acceptance test of that position); the
-// one that folds a sequence's last row runs the first-rejection scan (ballot + find-first-set)
-// and pushes the sequence to `ready`.  EMIT tickets are claimed only for sequences already
-// pushed and are preferred over LSE tickets, so the second read of row n follows the first
-// closely and hits L2.
+//   EMIT(seq, run)   at most kEdgeEmitRun stages of row n of a folded sequence: the row is
+//                    streamed again and p_row = 2^(l * c1 - ref2) / S is written.
+// The fold warp stores each partial to global memory and counts it on its sequence; the fold
+// warp that brings a sequence's last partial folds the sequence: one lane per position adds up
+// the row's partials in float64 and evaluates the acceptance test, a ballot + find-first-set
+// over the lanes gives the accepted length n, and the sequence's `ready` entry (n and row n's
+// reference and 1/S) is written.  Producers claim EMIT tickets with one atomic add when ready
+// sequences have unclaimed tickets (or eagerly once they have no LSE work left); an EMIT ticket
+// goes before the next LSE stage, so the second read of row n follows the first as closely as
+// the fold allows.
 // Nothing on the global path waits on a fence: results travel through 8-byte slots that the
-// host pre-filled with all ones and that carry their own validity; a consumer of such a slot
-// that sees the fill pattern polls (bounded) for a store that a running warp has already issued.
+// host pre-filled with all ones and that carry their own validity; a reader that sees the fill
+// pattern asks again (bounded) for a store that a running warp has already issued.  Values that
+// a thread will need later (ticket numbers, counters, `ready` entries) are requested one step
+// ahead and looked at one step later, so no round trip is waited for while streaming.
 // A producer only ever waits for work held by running CTAs, and never while its own CTA holds
 // unprocessed stages, so the kernel needs no co-residency guarantee.  Every wait is bounded;
 // when one runs out the error word is set and the warps wind down.
