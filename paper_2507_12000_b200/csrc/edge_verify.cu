@@ -351,6 +351,47 @@ __device__ __forceinline__ double exp2_small(double x)
     return __hiloint2double(__double2hiint(p) + (n << 20), __double2loint(p));
 }
 
+// One position i of sequence b, given its row's sum_v 2^(l_v * c1) = S * 2^Rr (float64 S, integer
+// Rr): writes lse and p_i(x_i), evaluates the acceptance test and returns the position's bits;
+// Rs, invS are what the emission of this row would need.  A lane that is not live returns "accepted".
+__device__ __forceinline__ unsigned judge_position(const EdgeParams &P, long long b, int i, bool live, float Rr, double S,
+                                                   bool bad, bool timeout, int x, float zx, float qx, float ux,
+                                                   float &Rs, float &invS)
+{
+    const double c1 = (double)P.c1;
+    // the sum has a finite logarithm iff S is positive and finite
+    const bool finite = !timeout && !bad && (S > 0.0) && (S < INFINITY) && (Rr != DSSD_NEG_INF);
+    unsigned bits = live ? ((finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u)) : kBitAccept;
+    if (live && P.lse)
+        P.lse[b * (P.gamma + 1) + i] = finite ? (Rr + __log2f((float)S)) * 0.6931471805599453f : __int_as_float(0x7fc00000);
+    // 1 / S in float64: the float32 reciprocal refined by one Newton step
+    double invS_d = NAN;
+    if (finite) {
+        const double r0 = (double)(1.0f / (float)S);
+        invS_d = r0 * (2.0 - S * r0);
+    }
+    if (live && i < P.gamma) {
+        double p = NAN;
+        bool accept = false;
+        if (x < 0 || x >= P.V) {
+            bits |= kBitBadToken;
+        } else {
+            // u < min(1, p(x)/q(x)) in float64, as  u < 1  and  u * q < p  (u * q is exact)
+            p = finite ? exp2_small((double)zx * c1 - (double)Rr) * invS_d : NAN;
+            const double q = (double)qx;
+            const double u = (double)ux;
+            if (q != q || p != p) accept = false;
+            else if (q <= 0.0) accept = (p > 0.0) && (u < 1.0);
+            else accept = (u < 1.0) && (u * q < p);
+        }
+        if (P.p_tok) P.p_tok[(size_t)b * P.gamma + i] = (float)p;
+        bits |= accept ? kBitAccept : 0u;
+    }
+    invS = finite ? (float)invS_d : __int_as_float(0x7fc00000);
+    Rs = finite ? Rr : 0.f;
+    return bits;
+}
+
 // Run by the fold warp that brought the last partial of sequence b.  One lane per position
 // i = 0..gamma: the row's partials -> log-sum-exp (float64) -> acceptance test
 //   u_i < min(1, p_i(x_i) / q_i(x_i));
@@ -361,7 +402,6 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
 {
     using E = Elem<DT>;
     const int lane = threadIdx.x & 31;
-    const double c1 = (double)P.c1;
     int n = P.gamma;
     unsigned fl = 0;
     float ref2_n = 0.f, invS_n = 0.f;
@@ -421,35 +461,8 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
                 }
             }
         }
-        // sum_v 2^(l_v * c1) = S * 2^Rr; it has a finite logarithm iff S is positive and finite
-        const bool finite = !timeout && !bad && (S > 0.0) && (S < INFINITY) && (Rr != DSSD_NEG_INF);
-        unsigned bits = live ? ((finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u)) : kBitAccept;
-        if (live && P.lse) P.lse[row] = finite ? (Rr + __log2f((float)S)) * 0.6931471805599453f : __int_as_float(0x7fc00000);
-        // 1 / S in float64: the float32 reciprocal refined by one Newton step
-        double invS_d = NAN;
-        if (finite) {
-            const double r0 = (double)(1.0f / (float)S);
-            invS_d = r0 * (2.0 - S * r0);
-        }
-        if (live && i < P.gamma) {
-            double p = NAN;
-            bool accept = false;
-            if (x < 0 || x >= P.V) {
-                bits |= kBitBadToken;
-            } else {
-                // u < min(1, p(x)/q(x)) in float64, as  u < 1  and  u * q < p  (u * q is exact)
-                p = finite ? exp2_small((double)zx * c1 - (double)Rr) * invS_d : NAN;
-                const double q = (double)qx;
-                const double u = (double)ux;
-                if (q != q || p != p) accept = false;
-                else if (q <= 0.0) accept = (p > 0.0) && (u < 1.0);
-                else accept = (u < 1.0) && (u * q < p);
-            }
-            if (P.p_tok) P.p_tok[(size_t)b * P.gamma + i] = (float)p;
-            bits |= accept ? kBitAccept : 0u;
-        }
-        const float invS = finite ? (float)invS_d : __int_as_float(0x7fc00000);
-        const float Rs = finite ? Rr : 0.f;
+        float Rs, invS;
+        const unsigned bits = judge_position(P, b, i, live, Rr, S, bad, timeout, x, zx, qx, ux, Rs, invS);
         const unsigned rej = __ballot_sync(kFull, live && i < P.gamma && !(bits & kBitAccept));
         if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
         fl |= (__ballot_sync(kFull, bits & kBitBadToken) ? DSSD_EDGE_FLAG_BAD_TOKEN : 0u) |
@@ -918,6 +931,175 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     }
 }
 
+// ---- small launches: one CTA per sequence, no workspace ---------------------------------------
+//
+// When a sequence's rows are short and the batch is at most one CTA per SM, the hand-offs of the
+// streaming kernel (tickets, partials in global memory, the workspace fill) cost more than the
+// streaming itself.  Here one CTA of 1024 threads does a whole sequence: every row is streamed
+// with 16-byte loads into the same per-lane online sums, the warps' results meet in shared
+// memory, warp 0 judges the positions (same arithmetic as the fold warp) and finds n, and the CTA
+// streams row n again (from L1/L2) to write p_row.  Same results as the streaming kernel up to
+// the order of the float32 sums.
+
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallWarps = kSmallThreads / 32;
+constexpr int kSmallMaxRows = 64;                 // gamma + 1 at most
+#ifndef DSSD_EDGE_SMALL_SEQ_BYTES
+#define DSSD_EDGE_SMALL_SEQ_BYTES (512 << 10)
+#endif
+constexpr long long kSmallMaxSeqBytes = DSSD_EDGE_SMALL_SEQ_BYTES;  // logits bytes of one sequence at most
+
+template <int DT>
+__global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __grid_constant__ EdgeParams P)
+{
+    using E = Elem<DT>;
+    __shared__ float2 s_part[kSmallMaxRows][kSmallWarps];
+    __shared__ int s_x[kSmallMaxRows];
+    __shared__ float s_zx[kSmallMaxRows], s_q[kSmallMaxRows], s_u[kSmallMaxRows];
+    __shared__ int s_n;
+    __shared__ float s_ref2, s_invS;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long b = blockIdx.x;
+    const float c1 = P.c1;
+    const long long rowbytes = (long long)P.V * E::kBytes;
+    // The rows are streamed side by side, a group of `wpr` warps per row, so that the loads of
+    // all rows are in flight together; the first lane of each group also fetches the row's
+    // drafted token, its probability and uniform, and (once the token id is back) its logit.
+    const int rows = P.gamma + 1;
+    const int wpr = rows >= kSmallWarps ? 1 : kSmallWarps / rows;  // warps per row
+    const int groups = kSmallWarps / wpr;                           // rows in flight at once
+    const int g = warp / wpr, wi = warp - g * wpr, gthreads = wpr * 32, t = wi * 32 + lane;
+    for (int i = g; i < rows && g < groups; i += groups) {
+        const char *rowp = row_ptr<DT>(P, b * rows + i);
+        const int head = row_head_bytes<DT>(P, rowp);
+        const long long body = rowbytes - head;
+        const int nvec = (int)(body >> 4);
+        const uint4 *v4 = reinterpret_cast<const uint4 *>(rowp + head);
+        const bool scout = t == 0 && i < P.gamma;
+        int x = -1;
+        float qx = 0.f, ux = 0.f, zx = 0.f;
+        if (scout) {
+            const size_t di = (size_t)b * P.gamma + i;
+            x = P.draft_tokens[di];
+            qx = P.draft_q_tok[di];
+            ux = P.uniforms[di];
+        }
+        Online o;
+        online_reset(o);
+        bool asked = false;
+        for (int j = t; j < nvec; j += 4 * gthreads) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = (j + u * gthreads < nvec) ? ld_stream16(v4 + j + u * gthreads) : neg_inf_vec<DT>();
+            if (scout && !asked) {  // the token id is back by now: its logit travels with the next loads
+                if (x >= 0 && x < P.V) zx = E::load(rowp, x);
+                asked = true;
+            }
+            accum_block<DT>(o, v, c1);
+        }
+        if (scout && !asked && x >= 0 && x < P.V) zx = E::load(rowp, x);
+        if (wi == 0) {  // the scalars before the first and after the last 16-byte vector
+            if (lane < head / E::kBytes) online_add(o, E::load(rowp, lane), c1);
+            const int tail = (int)((body - ((long long)nvec << 4)) / E::kBytes);
+            if (lane < tail) online_add(o, E::load(rowp, (int64_t)((head + ((long long)nvec << 4)) / E::kBytes) + lane), c1);
+        }
+        const bool empty = (o.m == DSSD_NEG_INF);
+        const float R = warp_max(empty ? DSSD_NEG_INF : o.ref);
+        float sum = online_total(o);
+        sum = warp_sum(empty ? 0.f : sum * ex2(o.ref - R));  // exact scaling
+        if (lane == 0) s_part[i][wi] = make_float2(R == DSSD_NEG_INF ? 0.f : R, sum);
+        if (scout) {
+            s_x[i] = x;
+            s_zx[i] = zx;
+            s_q[i] = qx;
+            s_u[i] = ux;
+        }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int n = P.gamma;
+        unsigned fl = 0;
+        float ref2_n = 0.f, invS_n = 0.f;
+        for (int base = 0; base <= P.gamma; base += 32) {
+            const int i = base + lane;
+            const bool live = i <= P.gamma;
+            int x = -1;
+            float zx = 0.f, qx = 0.f, ux = 0.f;
+            if (live && i < P.gamma) {
+                x = s_x[i];
+                zx = s_zx[i];
+                qx = s_q[i];
+                ux = s_u[i];
+            }
+            float Rr = DSSD_NEG_INF;
+            double S = 0.0;
+            bool bad = false;
+            if (live) {
+                for (int k = 0; k < wpr; ++k) {
+                    const float2 c = s_part[i][k];
+                    if (c.y != c.y) bad = true;
+                    if (c.y > 0.f) {
+                        if (c.x > Rr) {
+                            S = (Rr == DSSD_NEG_INF || S == 0.0) ? 0.0 : scale_pow2(S, Rr - c.x);
+                            Rr = c.x;
+                        }
+                        S += scale_pow2((double)c.y, c.x - Rr);
+                    }
+                }
+            }
+            float Rs, invS;
+            const unsigned bits = judge_position(P, b, i, live, Rr, S, bad, false, x, zx, qx, ux, Rs, invS);
+            const unsigned rej = __ballot_sync(kFull, live && i < P.gamma && !(bits & kBitAccept));
+            if (rej && n == P.gamma) n = base + __ffs(rej) - 1;
+            fl |= (__ballot_sync(kFull, bits & kBitBadToken) ? DSSD_EDGE_FLAG_BAD_TOKEN : 0u) |
+                  (__ballot_sync(kFull, bits & kBitNonFinite) ? DSSD_EDGE_FLAG_NONFINITE : 0u);
+            if (n >= base && n < base + 32) {
+                ref2_n = __shfl_sync(kFull, Rs, n - base);
+                invS_n = __shfl_sync(kFull, invS, n - base);
+            }
+        }
+        if (lane == 0) {
+            P.accept_len[b] = n;
+            if (P.flags) P.flags[b] = fl;
+            s_n = n;
+            s_ref2 = ref2_n;
+            s_invS = invS_n;
+        }
+    }
+    __syncthreads();
+    // row n once more: p_row[b, v] = 2^(l_v * c1 - ref2) / S
+    {
+        const char *rowp = row_ptr<DT>(P, b * (P.gamma + 1) + s_n);
+        const int head = row_head_bytes<DT>(P, rowp);
+        const long long body = rowbytes - head;
+        const int nvec = (int)(body >> 4);
+        const uint4 *v4 = reinterpret_cast<const uint4 *>(rowp + head);
+        float *outp = P.p_row + (size_t)b * P.V;
+        float *bodyp = outp + head / E::kBytes;
+        const float nref = -s_ref2, invS = s_invS;
+        const f32x2 cc = pack2(c1, c1), nn = pack2(nref, nref), ss = pack2(invS, invS);
+        const bool vec_out = (reinterpret_cast<uintptr_t>(bodyp) & 15u) == 0;
+        for (int j = tid; j < nvec; j += kSmallThreads) {
+            float f[E::kVec];
+            E::unpack(ld_stream16(v4 + j), f);
+            float *o = bodyp + (size_t)j * E::kVec;
+            if (vec_out) {
+#pragma unroll
+                for (int q = 0; q < E::kVec; q += 4) emit_quad(o + q, f[q], f[q + 1], f[q + 2], f[q + 3], cc, nn, ss);
+            } else {
+#pragma unroll
+                for (int q = 0; q < E::kVec; ++q) o[q] = ex2(fmaf(f[q], c1, nref)) * invS;
+            }
+        }
+        if (warp == 0) {
+            if (lane < head / E::kBytes) outp[lane] = ex2(fmaf(E::load(rowp, lane), c1, nref)) * invS;
+            const int tail = (int)((body - ((long long)nvec << 4)) / E::kBytes);
+            const int64_t e = (int64_t)((head + ((long long)nvec << 4)) / E::kBytes) + lane;
+            if (lane < tail) outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS;
+        }
+    }
+}
+
 constexpr size_t kEdgeSmemBytes = (size_t)kEdgeStages * kS + sizeof(Shared);
 
 template <int DT>
@@ -1007,6 +1189,14 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
         g_sm_count[dev] = sms;
     }
     const int esz = dtype == DSSD_BF16 ? 2 : 4;
+    P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
+    // small launches: one CTA per sequence, no workspace, one launch
+    if (P.gamma + 1 <= kSmallMaxRows && P.B <= g_sm_count[dev] &&
+        (long long)(P.gamma + 1) * P.V * esz <= kSmallMaxSeqBytes) {
+        if (dtype == DSSD_BF16) edge_small_kernel<DSSD_BF16><<<P.B, kSmallThreads, 0, stream>>>(P);
+        else edge_small_kernel<DSSD_F32><<<P.B, kSmallThreads, 0, stream>>>(P);
+        return cudaGetLastError();
+    }
     const unsigned long long R = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);
     const long long n_slices = ((long long)P.V * esz + kS - 1) / kS;
     P.n_slices = (int)(n_slices < 1 ? 1 : n_slices);

@@ -30,6 +30,18 @@ def test_tiny_grid(B, oracle_mod, dtype):
                 compare_round(B, oracle_mod, di.generate(w), w.temperature, threads=1)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_tiny_vocabularies_through_the_streaming_kernel(B, oracle_mod, dtype):
+    """More sequences than SMs, so that the persistent streaming kernel (not the one-CTA-per-
+    sequence kernel of small launches) sees vocabularies around vector and stage boundaries."""
+    seed = 900
+    for V in (1, 7, 33, 1025, 16389):
+        for gamma in (0, 3):
+            seed += 1
+            w = di.custom(B=150, gamma=gamma, V=V, dtype=dtype, temperature=0.9, sigma_d=1.0, zipf=V > 8, seed=seed)
+            compare_round(B, oracle_mod, di.generate(w, threads=4), w.temperature, threads=4)
+
+
 @pytest.mark.parametrize("name", ["c1", "c2"])
 def test_small_configs(B, oracle_mod, name):
     w = di.get_workload(name)
@@ -88,15 +100,16 @@ def test_sweep_points_sampled(B, oracle_mod):
             compare_round(B, oracle_mod, di.generate(w, threads=8), w.temperature)
 
 
-def test_strided_and_unaligned_rows(B, oracle_mod):
+@pytest.mark.parametrize("Bn", [3, 151])  # one CTA per sequence / the streaming kernel
+def test_strided_and_unaligned_rows(B, oracle_mod, Bn):
     for dtype, V, off in (("f32", 1000, 1), ("bf16", 4097, 3), ("bf16", 20000, 1), ("f32", 9001, 2)):
-        w = di.custom(B=3, gamma=2, V=V, dtype=dtype, seed=V)
+        w = di.custom(B=Bn, gamma=2, V=V, dtype=dtype, seed=V)
         d = di.generate(w)
         ref = oracle_mod.verify_round(d, w.temperature)
         g = to_device(d)
         stride = V + 5
-        buf = torch.zeros(3 * 3 * stride + 16, dtype=g["target_logits"].dtype, device="cuda")
-        view = buf[off:off + 3 * 3 * stride].view(3, 3, stride)[:, :, :V]
+        buf = torch.zeros(Bn * 3 * stride + 16, dtype=g["target_logits"].dtype, device="cuda")
+        view = buf[off:off + Bn * 3 * stride].view(Bn, 3, stride)[:, :, :V]
         view.copy_(g["target_logits"])
         assert view.data_ptr() % 16 != 0
         ev = B.dssd_edge_verify(view, g["draft_tokens"], g["draft_q_tok"], g["uniforms"], w.temperature)
