@@ -35,6 +35,8 @@
 
 #include <math.h>
 
+#include <cooperative_groups.h>
+
 #include "dssd_device.cuh"
 
 namespace dssd {
@@ -931,37 +933,45 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     }
 }
 
-// ---- small launches: one CTA per sequence, no workspace ---------------------------------------
+// ---- small launches: one thread-block cluster per sequence, no workspace -----------------------
 //
-// When a sequence's rows are short and the batch is at most one CTA per SM, the hand-offs of the
-// streaming kernel (tickets, partials in global memory, the workspace fill) cost more than the
-// streaming itself.  Here one CTA of 1024 threads does a whole sequence: every row is streamed
-// with 16-byte loads into the same per-lane online sums, the warps' results meet in shared
-// memory, warp 0 judges the positions (same arithmetic as the fold warp) and finds n, and the CTA
-// streams row n again (from L1/L2) to write p_row.  Same results as the streaming kernel up to
-// the order of the float32 sums.
+// When the whole batch fits one CTA per SM with a small share each, the hand-offs of the streaming
+// kernel (tickets, partials in global memory, the workspace fill) cost more than the streaming
+// itself.  Here a cluster of 1, 2, 4 or 8 CTAs of 1024 threads does a whole sequence: every CTA
+// streams its share of every row with 16-byte loads into the same per-lane online sums, the
+// CTAs' per-row results meet in the shared memory of the cluster's first CTA (distributed shared
+// memory, hardware cluster barrier), whose warp 0 judges the positions (same arithmetic as the
+// fold warp) and finds n; then every CTA streams its share of row n again (from L2) and writes
+// p_row.  Same results as the streaming kernel up to the order of the float32 sums.
 
 constexpr int kSmallThreads = 1024;
 constexpr int kSmallWarps = kSmallThreads / 32;
 constexpr int kSmallMaxRows = 64;                 // gamma + 1 at most
-#ifndef DSSD_EDGE_SMALL_SEQ_BYTES
-#define DSSD_EDGE_SMALL_SEQ_BYTES (512 << 10)
+constexpr int kSmallMaxCluster = 8;               // CTAs per sequence at most (the portable cluster size)
+#ifndef DSSD_EDGE_SMALL_CTA_BYTES
+#define DSSD_EDGE_SMALL_CTA_BYTES (128 << 10)
 #endif
-constexpr long long kSmallMaxSeqBytes = DSSD_EDGE_SMALL_SEQ_BYTES;  // logits bytes of one sequence at most
+constexpr long long kSmallCtaBytes = 32 << 10;                        // share of a sequence aimed at per CTA
+constexpr long long kSmallMaxCtaBytes = DSSD_EDGE_SMALL_CTA_BYTES;   // ... and the most a CTA takes
 
 template <int DT>
 __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __grid_constant__ EdgeParams P)
 {
     using E = Elem<DT>;
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank(), csize = (int)cluster.num_blocks();  // CTAs sharing this sequence
     __shared__ float2 s_part[kSmallMaxRows][kSmallWarps];
+    __shared__ float2 s_clu[kSmallMaxRows][kSmallMaxCluster];  // rank 0: every CTA's (ref2, sum) per row
     __shared__ int s_x[kSmallMaxRows];
     __shared__ float s_zx[kSmallMaxRows], s_q[kSmallMaxRows], s_u[kSmallMaxRows];
     __shared__ int s_n;
     __shared__ float s_ref2, s_invS;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const long long b = blockIdx.x;
+    const long long b = blockIdx.x / csize;
     const float c1 = P.c1;
     const long long rowbytes = (long long)P.V * E::kBytes;
+    // Every CTA of the cluster takes a contiguous 1/csize of each row's 16-byte vectors.
     // The rows are streamed side by side, a group of `wpr` warps per row, so that the loads of
     // all rows are in flight together; the first lane of each group also fetches the row's
     // drafted token, its probability and uniform, and (once the token id is back) its logit.
@@ -975,7 +985,8 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         const long long body = rowbytes - head;
         const int nvec = (int)(body >> 4);
         const uint4 *v4 = reinterpret_cast<const uint4 *>(rowp + head);
-        const bool scout = t == 0 && i < P.gamma;
+        const int vbeg = (int)((long long)nvec * crank / csize), vend = (int)((long long)nvec * (crank + 1) / csize);
+        const bool scout = t == 0 && i < P.gamma && crank == 0;
         int x = -1;
         float qx = 0.f, ux = 0.f, zx = 0.f;
         if (scout) {
@@ -987,10 +998,10 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         Online o;
         online_reset(o);
         bool asked = false;
-        for (int j = t; j < nvec; j += 4 * gthreads) {
+        for (int j = vbeg + t; j < vend; j += 4 * gthreads) {
             uint4 v[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = (j + u * gthreads < nvec) ? ld_stream16(v4 + j + u * gthreads) : neg_inf_vec<DT>();
+            for (int u = 0; u < 4; ++u) v[u] = (j + u * gthreads < vend) ? ld_stream16(v4 + j + u * gthreads) : neg_inf_vec<DT>();
             if (scout && !asked) {  // the token id is back by now: its logit travels with the next loads
                 if (x >= 0 && x < P.V) zx = E::load(rowp, x);
                 asked = true;
@@ -998,7 +1009,7 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
             accum_block<DT>(o, v, c1);
         }
         if (scout && !asked && x >= 0 && x < P.V) zx = E::load(rowp, x);
-        if (wi == 0) {  // the scalars before the first and after the last 16-byte vector
+        if (wi == 0 && crank == 0) {  // the scalars before the first and after the last 16-byte vector
             if (lane < head / E::kBytes) online_add(o, E::load(rowp, lane), c1);
             const int tail = (int)((body - ((long long)nvec << 4)) / E::kBytes);
             if (lane < tail) online_add(o, E::load(rowp, (int64_t)((head + ((long long)nvec << 4)) / E::kBytes) + lane), c1);
@@ -1016,7 +1027,27 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         }
     }
     __syncthreads();
-    if (warp == 0) {
+    // each CTA's result per row goes to rank 0's shared memory (distributed shared memory)
+    if (tid < rows) {
+        float R = DSSD_NEG_INF;
+        bool nan = false;
+        for (int k = 0; k < wpr; ++k) {
+            const float2 c = s_part[tid][k];
+            nan = nan || (c.y != c.y);
+            if (c.y > 0.f) R = fmaxf(R, c.x);
+        }
+        float S = 0.f;
+        for (int k = 0; k < wpr; ++k) {
+            const float2 c = s_part[tid][k];
+            if (c.y > 0.f) S += c.y * ex2(c.x - R);  // exact scaling
+        }
+        if (nan) S = __int_as_float(0x7fc00000);
+        float2 *dst = cluster.map_shared_rank(&s_clu[tid][crank], 0);
+        *dst = make_float2(R == DSSD_NEG_INF ? 0.f : R, S);
+    }
+    if (csize == 1) __syncthreads();
+    else cluster.sync();
+    if (warp == 0 && crank == 0) {
         int n = P.gamma;
         unsigned fl = 0;
         float ref2_n = 0.f, invS_n = 0.f;
@@ -1035,8 +1066,8 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
             double S = 0.0;
             bool bad = false;
             if (live) {
-                for (int k = 0; k < wpr; ++k) {
-                    const float2 c = s_part[i][k];
+                for (int k = 0; k < csize; ++k) {
+                    const float2 c = s_clu[i][k];
                     if (c.y != c.y) bad = true;
                     if (c.y > 0.f) {
                         if (c.x > Rr) {
@@ -1061,25 +1092,32 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         if (lane == 0) {
             P.accept_len[b] = n;
             if (P.flags) P.flags[b] = fl;
-            s_n = n;
-            s_ref2 = ref2_n;
-            s_invS = invS_n;
+            for (int r = 0; r < csize; ++r) {  // the verdict goes to every CTA of the cluster
+                *cluster.map_shared_rank(&s_n, r) = n;
+                *cluster.map_shared_rank(&s_ref2, r) = ref2_n;
+                *cluster.map_shared_rank(&s_invS, r) = invS_n;
+            }
         }
     }
-    __syncthreads();
-    // row n once more: p_row[b, v] = 2^(l_v * c1 - ref2) / S
+    if (csize == 1) __syncthreads();
+    else cluster.sync();
+    // row n once more, every CTA its share: p_row[b, v] = 2^(l_v * c1 - ref2) / S.  No CTA reads
+    // another CTA's shared memory from here on, so the CTAs may leave in any order.
     {
-        const char *rowp = row_ptr<DT>(P, b * (P.gamma + 1) + s_n);
+        const int n = s_n;
+        const float ref2 = s_ref2, invS = s_invS;
+        const char *rowp = row_ptr<DT>(P, b * (P.gamma + 1) + n);
         const int head = row_head_bytes<DT>(P, rowp);
         const long long body = rowbytes - head;
         const int nvec = (int)(body >> 4);
         const uint4 *v4 = reinterpret_cast<const uint4 *>(rowp + head);
         float *outp = P.p_row + (size_t)b * P.V;
         float *bodyp = outp + head / E::kBytes;
-        const float nref = -s_ref2, invS = s_invS;
+        const float nref = -ref2;
         const f32x2 cc = pack2(c1, c1), nn = pack2(nref, nref), ss = pack2(invS, invS);
         const bool vec_out = (reinterpret_cast<uintptr_t>(bodyp) & 15u) == 0;
-        for (int j = tid; j < nvec; j += kSmallThreads) {
+        const int vbeg = (int)((long long)nvec * crank / csize), vend = (int)((long long)nvec * (crank + 1) / csize);
+        for (int j = vbeg + tid; j < vend; j += kSmallThreads) {
             float f[E::kVec];
             E::unpack(ld_stream16(v4 + j), f);
             float *o = bodyp + (size_t)j * E::kVec;
@@ -1091,7 +1129,7 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
                 for (int q = 0; q < E::kVec; ++q) o[q] = ex2(fmaf(f[q], c1, nref)) * invS;
             }
         }
-        if (warp == 0) {
+        if (warp == 0 && crank == 0) {
             if (lane < head / E::kBytes) outp[lane] = ex2(fmaf(E::load(rowp, lane), c1, nref)) * invS;
             const int tail = (int)((body - ((long long)nvec << 4)) / E::kBytes);
             const int64_t e = (int64_t)((head + ((long long)nvec << 4)) / E::kBytes) + lane;
@@ -1190,12 +1228,29 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     }
     const int esz = dtype == DSSD_BF16 ? 2 : 4;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
-    // small launches: one CTA per sequence, no workspace, one launch
-    if (P.gamma + 1 <= kSmallMaxRows && P.B <= g_sm_count[dev] &&
-        (long long)(P.gamma + 1) * P.V * esz <= kSmallMaxSeqBytes) {
-        if (dtype == DSSD_BF16) edge_small_kernel<DSSD_BF16><<<P.B, kSmallThreads, 0, stream>>>(P);
-        else edge_small_kernel<DSSD_F32><<<P.B, kSmallThreads, 0, stream>>>(P);
-        return cudaGetLastError();
+    // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
+    {
+        const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
+        int csize = 1;
+        while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;
+        while (csize > 1 && (long long)P.B * csize > g_sm_count[dev]) csize /= 2;
+        if (P.gamma + 1 <= kSmallMaxRows && seq_bytes / csize <= kSmallMaxCtaBytes &&
+            (long long)P.B * csize <= g_sm_count[dev]) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(P.B * csize));
+            cfg.blockDim = dim3(kSmallThreads);
+            cfg.dynamicSmemBytes = 0;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)csize;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            if (dtype == DSSD_BF16) return cudaLaunchKernelEx(&cfg, edge_small_kernel<DSSD_BF16>, P);
+            return cudaLaunchKernelEx(&cfg, edge_small_kernel<DSSD_F32>, P);
+        }
     }
     const unsigned long long R = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);
     const long long n_slices = ((long long)P.V * esz + kS - 1) / kS;
