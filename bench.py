@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 446.0 MB read + 98.3 MB written
-    "c4": {"bytes": 544329472, "kernel_hash": "d59083ef4c8f7c4c"},
+    # profiles/edge_verify_kernel_c4.md: 445.8 MB read + 98.0 MB written
+    "c4": {"bytes": 543830016, "kernel_hash": "e57acd19c795ee01"},
 }
 
 
