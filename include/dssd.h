@@ -62,6 +62,7 @@ typedef enum {
 #define DSSD_RS_FLAG_BONUS 1u    /* n == gamma: token drawn from P_{gamma+1}                       */
 #define DSSD_RS_FLAG_FALLBACK 2u /* residual mass sum max(0, p - q) <= 0: token drawn from p instead */
 #define DSSD_RS_FLAG_INVALID 4u  /* no positive mass at all, or n outside [0, gamma]: token = -1    */
+#define DSSD_RS_FLAG_TIMEOUT 8u  /* internal wait ran out: token = -1 (set together with INVALID)    */
 
 /* Human-readable name of a status (static storage, never NULL). */
 const char *dssd_status_string(int status);

@@ -30,6 +30,7 @@ EDGE_FLAG_TIMEOUT = 4
 RS_FLAG_BONUS = 1
 RS_FLAG_FALLBACK = 2
 RS_FLAG_INVALID = 4
+RS_FLAG_TIMEOUT = 8
 
 
 class DssdError(RuntimeError):

@@ -116,7 +116,7 @@ constexpr unsigned long long kFill64 = ~0ull;
 __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
 
 // chunk sum (b, c); a sum whose store has not landed yet still shows the fill pattern and is
-// polled for (bounded); NaN when the wait runs out
+// polled for (bounded); when the wait runs out the fill pattern itself comes back (see timed_out)
 __device__ __forceinline__ double load_chunk_sum(const ResampleParams &P, const unsigned long long *cs, int c)
 {
     unsigned long long w = ld_relaxed_u64(cs + c);
@@ -125,6 +125,19 @@ __device__ __forceinline__ double load_chunk_sum(const ResampleParams &P, const 
         w = ld_relaxed_u64(cs + c);
     }
     return __longlong_as_double((long long)w);
+}
+
+__device__ __forceinline__ bool timed_out(double m) { return (unsigned long long)__double_as_longlong(m) == kFill64; }
+
+// every thread's verdict on its chunk sums; on a timeout the sequence gets no token
+__device__ __forceinline__ bool give_up(const ResampleParams &P, int64_t b, bool mine, unsigned fl)
+{
+    if (!__syncthreads_or(mine)) return false;
+    if (threadIdx.x == 0) {
+        P.token[b] = -1;
+        if (P.flags) P.flags[b] = fl | DSSD_RS_FLAG_INVALID | DSSD_RS_FLAG_TIMEOUT;
+    }
+    return true;
 }
 
 // CTA-wide inclusive prefix sum in index order of the threads; `total` is the sum over the CTA
@@ -162,6 +175,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
         if (P.n_sub <= kThreads) {
             // one chunk per thread: a single scan gives Z and every inclusive prefix
             const double m = tid < P.n_sub ? load_chunk_sum(P, cs, tid) : 0.0;
+            if (give_up(P, b, timed_out(m), fl)) return;
             double Z;
             const double incl = block_scan(m, s_w, Z);
             ok = (Z > 0.0) && (Z < INFINITY);
@@ -194,13 +208,17 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
         } else {
         // Z = sum of the chunk sums, in groups of one chunk per thread
         double Z = 0.0;
+        bool late = false;
         for (int base = 0; base < P.n_sub; base += kThreads) {
             const int c = base + tid;
+            const double m = c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0;
+            late |= timed_out(m);
             double tot;
-            block_scan(c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0, s_w, tot);
+            block_scan(m, s_w, tot);
             Z += tot;
             __syncthreads();
         }
+        if (give_up(P, b, late, fl)) return;
         ok = (Z > 0.0) && (Z < INFINITY);
         if (ok) {
             // the first chunk whose inclusive prefix exceeds the target, else the last chunk with mass
