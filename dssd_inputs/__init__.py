@@ -6,6 +6,7 @@ from .generator import (  # noqa: F401
     custom,
     f32_to_bf16_bits,
     generate,
+    generate_topk,
     get_workload,
     sweep_max,
     sweep_points,

@@ -23,6 +23,11 @@ Recipe (per sequence b, position i, vocabulary entry v):
   q_i(x_i)      = the stored float32 entry of Q_i at x_i
   u_i, u'       = (32 random bits >> 8) * 2**-24, i.e. uniform on [0,1)
 
+Truncated-support batches (the experiments' top-k sampler, Section 4, k = 10): the draft side
+keeps only the k largest entries of each Q_i (equal entries: lower index first), renormalises
+them in float64, stores them as float32 (index, value) pairs and draws x_i from those; the
+target logits, the uniforms and their streams are the ones of the dense batch.
+
 Every array has its own counter-based (Philox) stream keyed by
 (seed, array id, sequence index), so changing B or gamma never perturbs the
 leading values of another array.
@@ -219,4 +224,72 @@ def generate(w: Workload, b0: int = 0, b1: Optional[int] = None, threads: int = 
 
         with ThreadPoolExecutor(max_workers=threads) as ex:
             list(ex.map(lambda s: _gen_sequence(w, b0 + s, beta, out, s), range(n)))
+    return out
+
+
+def generate_topk(w: Workload, k: int, b0: int = 0, b1: Optional[int] = None,
+                  threads: int = 1) -> Dict[str, np.ndarray]:
+    """Sequences [b0, b1) of workload `w` with the draft side truncated to its top k.
+
+    Returns target_logits, uniforms, uniforms_rs as `generate` does, and
+      q_idx        [n, gamma, k]  int32    support of the truncated Q_i, most likely first
+      q_val        [n, gamma, k]  float32  its renormalised probabilities
+      draft_tokens [n, gamma]     int32    x_i drawn from the truncated Q_i
+      draft_q_tok  [n, gamma]     float32  the stored q_val entry of x_i
+    """
+    if b1 is None:
+        b1 = w.B
+    n, g = b1 - b0, w.gamma
+    assert 1 <= k <= w.V
+    out = {
+        "q_idx": np.zeros((n, g, k), dtype=np.int32),
+        "q_val": np.zeros((n, g, k), dtype=np.float32),
+        "draft_tokens": np.zeros((n, g), dtype=np.int32),
+        "draft_q_tok": np.zeros((n, g), dtype=np.float32),
+    }
+    ldt = np.uint16 if w.dtype == "bf16" else np.float32
+    out["target_logits"] = np.empty((n, g + 1, w.V), dtype=ldt)
+    out["uniforms"] = np.zeros((n, g), dtype=np.float32)
+    out["uniforms_rs"] = np.zeros((n,), dtype=np.float32)
+    beta = zipf_bias(w)
+
+    def one(s: int) -> None:
+        dense = {
+            "target_logits": out["target_logits"][s:s + 1],
+            "draft_q": np.empty((1, g, w.V), dtype=np.float32),
+            "draft_tokens": np.zeros((1, g), dtype=np.int32),
+            "draft_q_tok": np.zeros((1, g), dtype=np.float32),
+            "uniforms": out["uniforms"][s:s + 1],
+            "uniforms_rs": out["uniforms_rs"][s:s + 1],
+        }
+        _gen_sequence(w, b0 + s, beta, dense, 0)
+        if g == 0:
+            return
+        ud = _unit_uniform(_rng(w.seed, _ARR_DRAFT_U, b0 + s), g)
+        for i in range(g):
+            q = dense["draft_q"][0, i]
+            # the k largest entries, equal entries by increasing index
+            cand = np.argpartition(-q, min(k, w.V - 1))[:k] if k < w.V else np.arange(w.V)
+            kth = q[cand].min()
+            pool = np.flatnonzero(q >= kth)
+            order = pool[np.argsort(-q[pool], kind="stable")][:k]
+            vals = q[order].astype(np.float64)
+            vals /= vals.sum()
+            v32 = vals.astype(np.float32)
+            out["q_idx"][s, i] = order
+            out["q_val"][s, i] = v32
+            cs = np.cumsum(v32, dtype=np.float64)
+            r = int(np.searchsorted(cs, np.float64(ud[i]) * cs[-1], side="right"))
+            r = min(r, k - 1)
+            out["draft_tokens"][s, i] = order[r]
+            out["draft_q_tok"][s, i] = v32[r]
+
+    if threads <= 1 or n <= 1:
+        for s in range(n):
+            one(s)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(one, range(n)))
     return out

@@ -234,3 +234,221 @@ int dssd_oracle_device_resample(const float *p_row, const float *draft_q,
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Truncated-support variant (Section 4: the experiments sample with top-k, k = 10, T = 1).
+ *
+ * Reading: "top-k sampling" restricts a model's distribution to its k most likely tokens and
+ * renormalises over them.  The support of a row is its k largest logits; equal logits are
+ * ordered by vocabulary index, lower index first, so the support is unique.  Inside the
+ * support P(v) = exp(l_v/T - m) / sum_{w in support} exp(l_w/T - m), outside it P(v) = 0.
+ * The draft side truncates its own distributions the same way before it samples, so the
+ * scalars q_i(x_i) it uploads and the rows Q_i it keeps are truncated ones; Algorithm 2 then
+ * runs unchanged on the truncated P and Q, and the downlink carries k (index, value) pairs
+ * instead of |V| values.
+ * ------------------------------------------------------------------------------------------ */
+
+#define TOPK_MAX 32
+
+/*
+ * Support and probabilities of one row.  Selection by k successive maxima: pick r is the
+ * largest element that comes strictly after pick r-1 in the order (logit descending, index
+ * ascending).  idx/prob are in that order.  *ok = 0 (idx = -1, prob = NaN) when the row
+ * holds a NaN or +inf, or has no entry above -inf.
+ */
+static void row_topk(const void *row, int dtype, int V, int k, double T,
+                     int32_t *idx, double *prob, int *ok)
+{
+    double val[TOPK_MAX];
+    int bad = 0;
+    double top = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        double l = load_logit(row, dtype, v);
+        if (l != l || l == INFINITY) bad = 1;
+        if (l > top) top = l;
+    }
+    if (bad || !(top > -INFINITY)) {
+        for (int r = 0; r < k; ++r) { idx[r] = -1; prob[r] = NAN; }
+        *ok = 0;
+        return;
+    }
+    double prev_val = INFINITY;
+    int32_t prev_idx = -1;
+    for (int r = 0; r < k; ++r) {
+        double best = 0.0;
+        int32_t best_idx = -1;
+        for (int v = 0; v < V; ++v) {
+            double l = load_logit(row, dtype, v);
+            int after_prev = (l < prev_val) || (l == prev_val && v > prev_idx);
+            if (!after_prev) continue;
+            if (best_idx < 0 || l > best) { best = l; best_idx = v; }
+        }
+        idx[r] = best_idx;
+        val[r] = best;
+        prev_val = best;
+        prev_idx = best_idx;
+    }
+    {
+        double m = val[0] / T, S = 0.0;
+        for (int r = 0; r < k; ++r) S += exp(val[r] / T - m);
+        for (int r = 0; r < k; ++r) prob[r] = exp(val[r] / T - m) / S;
+    }
+    *ok = 1;
+}
+
+/*
+ * Edge half of Algorithm 2 on truncated distributions.
+ *
+ * inputs as dssd_oracle_edge_verify, plus k (1 <= k <= min(V, 32)); draft_q_tok holds the
+ * draft's truncated q_i(x_i).
+ * outputs:
+ *   accept_len [B]
+ *   p_idx  [B, k]   support of row n in (logit descending, index ascending) order; -1 for a
+ *                   row without a finite distribution
+ *   p_val  [B, k]   its probabilities rounded to float32 (the downlink payload)
+ *   p_val64 [B, k]  before rounding (may be NULL)
+ *   p_tok  [B, gamma]  P_i(x_i): 0 outside the support (may be NULL)
+ *   flags  [B], margin_acc [B]  as in dssd_oracle_edge_verify (may be NULL)
+ */
+int dssd_oracle_edge_verify_topk(const void *target_logits, int dtype, int64_t row_stride,
+                                 const int32_t *draft_tokens, const float *draft_q_tok,
+                                 const float *uniforms, float temperature,
+                                 int B, int gamma, int V, int k,
+                                 int32_t *accept_len, int32_t *p_idx, float *p_val, double *p_val64,
+                                 double *p_tok, uint32_t *flags, double *margin_acc)
+{
+    const double T = (double)temperature;
+    const size_t esz = (dtype == ORACLE_BF16) ? 2 : 4;
+    if (B < 1 || gamma < 0 || V < 1 || !(T > 0.0) || row_stride < V) return 1;
+    if (k < 1 || k > V || k > TOPK_MAX) return 1;
+    for (int b = 0; b < B; ++b) {
+        uint32_t fl = 0;
+        int n = gamma;
+        int flag_open = 1;
+        double margin = INFINITY;
+        int32_t idx[TOPK_MAX];
+        double prob[TOPK_MAX];
+        for (int i = 0; i <= gamma; ++i) {
+            const char *row = (const char *)target_logits +
+                              ((size_t)b * (size_t)(gamma + 1) + (size_t)i) * (size_t)row_stride * esz;
+            int ok;
+            row_topk(row, dtype, V, k, T, idx, prob, &ok);
+            if (!ok) fl |= FLAG_NONFINITE;
+            if (i == gamma) break;
+            int32_t x = draft_tokens[(size_t)b * gamma + i];
+            double u = (double)uniforms[(size_t)b * gamma + i];
+            double q = (double)draft_q_tok[(size_t)b * gamma + i];
+            double p, ratio;
+            int accept;
+            if (x < 0 || x >= V) {
+                fl |= FLAG_BAD_TOKEN;
+                p = NAN;
+                accept = 0;
+                ratio = NAN;
+            } else {
+                if (!ok) p = NAN;
+                else {
+                    p = 0.0;
+                    for (int r = 0; r < k; ++r) if (idx[r] == x) p = prob[r];
+                }
+                if (q != q || p != p) ratio = NAN;
+                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
+                else ratio = p / q;
+                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+            }
+            if (p_tok) p_tok[(size_t)b * gamma + i] = p;
+            if (flag_open) {
+                if (ratio == ratio) {
+                    double d = fabs(u - (ratio < 1.0 ? ratio : 1.0));
+                    if (d < margin) margin = d;
+                }
+                if (!accept) { n = i; flag_open = 0; }
+            }
+        }
+        accept_len[b] = n;
+        if (flags) flags[b] = fl;
+        if (margin_acc) margin_acc[b] = margin;
+        {
+            const char *row = (const char *)target_logits +
+                              ((size_t)b * (size_t)(gamma + 1) + (size_t)n) * (size_t)row_stride * esz;
+            int ok;
+            row_topk(row, dtype, V, k, T, idx, prob, &ok);
+            for (int r = 0; r < k; ++r) {
+                p_idx[(size_t)b * k + r] = idx[r];
+                p_val[(size_t)b * k + r] = (float)prob[r];
+                if (p_val64) p_val64[(size_t)b * k + r] = prob[r];
+            }
+        }
+    }
+    return 0;
+}
+
+/*
+ * Device half on truncated distributions: the residual max(0, P - Q_n) lives on P's support,
+ * so the draw walks P's k entries in increasing vocabulary index (the order the dense draw
+ * walks the vocabulary in) with Q_n looked up by index (0 where Q_n has no such entry; the
+ * first match if an index is listed twice).
+ *
+ * p_idx, p_val [B, k]; q_idx, q_val [B, gamma, k] (only row n is read); accept_len, uniforms [B].
+ * A negative p_idx marks a sequence without a row: token = -1, RS_FLAG_INVALID.
+ */
+int dssd_oracle_device_resample_topk(const int32_t *p_idx, const float *p_val,
+                                     const int32_t *q_idx, const float *q_val,
+                                     const int32_t *accept_len, const float *uniforms,
+                                     int B, int gamma, int k,
+                                     int32_t *token, uint32_t *flags, double *margin_cdf, double *Z_out)
+{
+    if (B < 1 || gamma < 0 || k < 1 || k > TOPK_MAX) return 1;
+    for (int b = 0; b < B; ++b) {
+        int n = accept_len[b];
+        double u = (double)uniforms[b];
+        double Z = 0.0, mg = 0.0;
+        uint32_t fl = 0;
+        int32_t tok = -1;
+        int32_t sid[TOPK_MAX];
+        float sp[TOPK_MAX], sq[TOPK_MAX];
+        int has_row = 1;
+        for (int e = 0; e < k; ++e) if (p_idx[(size_t)b * k + e] < 0) has_row = 0;
+        if (n < 0 || n > gamma || !has_row) {
+            fl = RS_FLAG_INVALID;
+        } else {
+            /* P's entries in increasing index (insertion sort) */
+            for (int e = 0; e < k; ++e) {
+                int32_t id = p_idx[(size_t)b * k + e];
+                float pv = p_val[(size_t)b * k + e];
+                int pos = e;
+                while (pos > 0 && sid[pos - 1] > id) {
+                    sid[pos] = sid[pos - 1];
+                    sp[pos] = sp[pos - 1];
+                    --pos;
+                }
+                sid[pos] = id;
+                sp[pos] = pv;
+            }
+            int pos_tok;
+            if (n == gamma) {
+                fl |= RS_FLAG_BONUS;
+                pos_tok = inverse_cdf(sp, NULL, 1, k, u, &Z, &mg);
+            } else {
+                const int32_t *qi = q_idx + ((size_t)b * gamma + n) * (size_t)k;
+                const float *qv = q_val + ((size_t)b * gamma + n) * (size_t)k;
+                for (int e = 0; e < k; ++e) {
+                    sq[e] = 0.0f;
+                    for (int f = k - 1; f >= 0; --f) if (qi[f] == sid[e]) sq[e] = qv[f];
+                }
+                pos_tok = inverse_cdf(sp, sq, 0, k, u, &Z, &mg);
+                if (pos_tok < 0) {
+                    fl |= RS_FLAG_FALLBACK;
+                    pos_tok = inverse_cdf(sp, NULL, 1, k, u, &Z, &mg);
+                }
+            }
+            if (pos_tok < 0) { fl |= RS_FLAG_INVALID; mg = 0.0; }
+            else tok = sid[pos_tok];
+        }
+        token[b] = tok;
+        if (flags) flags[b] = fl;
+        if (margin_cdf) margin_cdf[b] = mg;
+        if (Z_out) Z_out[b] = Z;
+    }
+    return 0;
+}

@@ -57,6 +57,15 @@ def _load():
         lib.dssd_oracle_device_resample.argtypes = [
             c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
             c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.dssd_oracle_edge_verify_topk.restype = c.c_int
+        lib.dssd_oracle_edge_verify_topk.argtypes = [
+            c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+            c.c_int, c.c_int, c.c_int, c.c_int,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.dssd_oracle_device_resample_topk.restype = c.c_int
+        lib.dssd_oracle_device_resample_topk.argtypes = [
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+            c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         _lib = lib
     return _lib
 
@@ -160,6 +169,97 @@ def verify_round(inputs: Dict[str, np.ndarray], temperature: float, threads: int
     gamma = inputs["target_logits"].shape[1] - 1
     rs = device_resample(ev["p_row"], inputs["draft_q"], ev["accept_len"], inputs["uniforms_rs"],
                          gamma, threads=threads)
+    out = dict(ev)
+    out["token"] = rs["token"]
+    out["rs_flags"] = rs["flags"]
+    out["margin_cdf"] = rs["margin_cdf"]
+    out["Z"] = rs["Z"]
+    return out
+
+
+TOPK_MAX = 32
+
+
+def edge_verify_topk(target_logits: np.ndarray, draft_tokens: np.ndarray, draft_q_tok: np.ndarray,
+                     uniforms: np.ndarray, temperature: float, k: int,
+                     threads: int = 1) -> Dict[str, np.ndarray]:
+    """Edge half on distributions truncated to their k largest entries (Section 4, top-k sampling)."""
+    lib = _load()
+    tl = np.ascontiguousarray(target_logits)
+    assert tl.ndim == 3 and tl.dtype in (np.float32, np.uint16)
+    dtype = BF16 if tl.dtype == np.uint16 else F32
+    B, g1, V = tl.shape
+    gamma = g1 - 1
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32).reshape(B, gamma)
+    qt = np.ascontiguousarray(draft_q_tok, dtype=np.float32).reshape(B, gamma)
+    u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, gamma)
+    out = {
+        "accept_len": np.zeros(B, np.int32),
+        "p_idx": np.zeros((B, k), np.int32),
+        "p_val": np.zeros((B, k), np.float32),
+        "p_val64": np.zeros((B, k), np.float64),
+        "p_tok": np.zeros((B, gamma), np.float64),
+        "flags": np.zeros(B, np.uint32),
+        "margin_acc": np.zeros(B, np.float64),
+    }
+
+    def run(rng):
+        b0, b1 = rng
+        rc = lib.dssd_oracle_edge_verify_topk(
+            _ptr(tl[b0:b1]), dtype, V, _ptr(tok[b0:b1]), _ptr(qt[b0:b1]), _ptr(u[b0:b1]),
+            ctypes.c_float(temperature), b1 - b0, gamma, V, k,
+            _ptr(out["accept_len"][b0:b1]), _ptr(out["p_idx"][b0:b1]), _ptr(out["p_val"][b0:b1]),
+            _ptr(out["p_val64"][b0:b1]), _ptr(out["p_tok"][b0:b1]), _ptr(out["flags"][b0:b1]),
+            _ptr(out["margin_acc"][b0:b1]))
+        if rc != 0:
+            raise ValueError("dssd_oracle_edge_verify_topk: invalid arguments")
+
+    parts = _chunks(B, threads)
+    if len(parts) == 1:
+        run(parts[0])
+    else:
+        with ThreadPoolExecutor(len(parts)) as ex:
+            list(ex.map(run, parts))
+    return out
+
+
+def device_resample_topk(p_idx: np.ndarray, p_val: np.ndarray, q_idx: Optional[np.ndarray],
+                         q_val: Optional[np.ndarray], accept_len: np.ndarray,
+                         uniforms_rs: np.ndarray, gamma: int) -> Dict[str, np.ndarray]:
+    """Device half on truncated distributions: p_* [B, k], q_* [B, gamma, k]."""
+    lib = _load()
+    pi = np.ascontiguousarray(p_idx, dtype=np.int32)
+    pv = np.ascontiguousarray(p_val, dtype=np.float32)
+    B, k = pi.shape
+    if gamma > 0:
+        qi = np.ascontiguousarray(q_idx, dtype=np.int32).reshape(B, gamma, k)
+        qv = np.ascontiguousarray(q_val, dtype=np.float32).reshape(B, gamma, k)
+    else:
+        qi = qv = None
+    n = np.ascontiguousarray(accept_len, dtype=np.int32).reshape(B)
+    u = np.ascontiguousarray(uniforms_rs, dtype=np.float32).reshape(B)
+    out = {
+        "token": np.zeros(B, np.int32),
+        "flags": np.zeros(B, np.uint32),
+        "margin_cdf": np.zeros(B, np.float64),
+        "Z": np.zeros(B, np.float64),
+    }
+    rc = lib.dssd_oracle_device_resample_topk(
+        _ptr(pi), _ptr(pv), _ptr(qi), _ptr(qv), _ptr(n), _ptr(u), B, gamma, k,
+        _ptr(out["token"]), _ptr(out["flags"]), _ptr(out["margin_cdf"]), _ptr(out["Z"]))
+    if rc != 0:
+        raise ValueError("dssd_oracle_device_resample_topk: invalid arguments")
+    return out
+
+
+def verify_round_topk(inputs: Dict[str, np.ndarray], temperature: float, k: int,
+                      threads: int = 1) -> Dict[str, np.ndarray]:
+    """Both halves on one generated truncated-support batch."""
+    ev = edge_verify_topk(inputs["target_logits"], inputs["draft_tokens"], inputs["draft_q_tok"],
+                          inputs["uniforms"], temperature, k, threads=threads)
+    gamma = inputs["target_logits"].shape[1] - 1
+    rs = device_resample_topk(ev["p_idx"], ev["p_val"], inputs["q_idx"], inputs["q_val"],
+                              ev["accept_len"], inputs["uniforms_rs"], gamma)
     out = dict(ev)
     out["token"] = rs["token"]
     out["rs_flags"] = rs["flags"]
