@@ -9,7 +9,10 @@
  *   dssd_device_resample  the device half: "Resample" (Section 3, Algorithm 2), plus the
  *                         bonus draw x_{gamma+1} ~ P_{gamma+1} that Algorithm 2 performs when
  *                         every draft token was accepted;
- *   dssd_round_host       both halves on host buffers, with the copies to and from the GPU.
+ *   dssd_round_host       both halves on host buffers, with the copies to and from the GPU;
+ *   dssd_edge_verify_topk, dssd_device_resample_topk
+ *                         the same round on distributions truncated to their k most likely
+ *                         tokens, the sampler of the paper's experiments (Section 4).
  *
  * Notation follows the paper: gamma draft tokens x_1..x_gamma with draft probabilities
  * q_i(x_i), target distributions P_1..P_{gamma+1} over a vocabulary of V entries, uniforms
@@ -198,6 +201,75 @@ dssd_status dssd_round_host(const void *target_logits, dssd_dtype dtype,
                             int32_t *token, uint32_t *edge_flags, uint32_t *rs_flags,
                             float *p_row, void *device_arena, size_t arena_bytes,
                             void *cuda_stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------
+ * Truncated-support round (Section 4: the experiments sample with top-k, k = 10, T = 1).
+ *
+ * Reading of "top-k sampling": a model's distribution is restricted to its k most likely tokens
+ * and renormalised over them.  The support of a target row is its k largest logits; equal logits
+ * are ordered by vocabulary index, lower index first, so the support is unique.  Inside it
+ *   P(v) = exp(l_v / T - m) / sum_{w in support} exp(l_w / T - m),   m = max_w l_w / T,
+ * outside it P(v) = 0.  The draft side truncates its own distributions the same way before it
+ * samples.  Algorithm 2 then runs unchanged on the truncated P and Q; the downlink payload of
+ * Section 3.1 shrinks from |V| values to k (index, value) pairs.
+ * ---------------------------------------------------------------------------------------------
+ */
+#define DSSD_TOPK_MAX 32
+
+/* Bytes of scratch that dssd_edge_verify_topk needs (0 if the sizes are invalid). */
+size_t dssd_edge_verify_topk_workspace_bytes(int B, int gamma, int V, int k);
+
+/*
+ * Edge half of one round on truncated target distributions (Algorithm 2, "Verification Process"
+ * and the payload of "Downlink Transmission", with the sampler of Section 4).
+ *
+ * Inputs as dssd_edge_verify; draft_q_tok holds the draft's truncated q_i(x_i).  A drafted token
+ * outside the target row's support has p_i(x_i) = 0 and is rejected.  All probabilities and the
+ * acceptance test are evaluated in float64; the logits are read exactly once.
+ *
+ * k           1 <= k <= min(V, DSSD_TOPK_MAX)
+ * accept_len  [B] int32        out: n in [0, gamma]
+ * p_idx       [B, k] int32     out: support of row n, most likely first (equal logits: lower
+ *                              index first); -1 everywhere for a row flagged NONFINITE
+ * p_val       [B, k] float32   out: its probabilities, same order (NaN for a NONFINITE row)
+ * p_tok       [B, gamma] float32 out, optional (NULL ok): p_i(x_i)
+ * flags       [B] uint32       out, optional (NULL ok): DSSD_EDGE_FLAG_BAD_TOKEN / _NONFINITE
+ *                              (a row holding NaN or +inf, or nothing above -inf)
+ * workspace   >= dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k) bytes, 256-byte aligned;
+ *             contents need not be initialised and are garbage afterwards
+ */
+dssd_status dssd_edge_verify_topk(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                  const int32_t *draft_tokens, const float *draft_q_tok,
+                                  const float *uniforms, float temperature, int B, int gamma,
+                                  int V, int k, int32_t *accept_len, int32_t *p_idx, float *p_val,
+                                  float *p_tok, uint32_t *flags, void *workspace,
+                                  size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Device half on truncated distributions (Algorithm 2, "Resample", and the bonus draw).
+ *
+ * The residual max(0, P_n - Q_n) lives on P_n's support, so the draw walks P_n's k entries in
+ * increasing vocabulary index - the order dssd_device_resample walks the vocabulary in - with
+ * Q_n looked up by index (0 where Q_n has no such entry; the first listed if an index occurs
+ * twice):  r_e = max(0, p_e - q_n(idx_e)),  Z = sum r_e,  token = idx of the first entry whose
+ * running sum exceeds u' * Z; for n == gamma the same with r = p.  Fallback and flags as in
+ * dssd_device_resample.  Sums run sequentially in float64, so results are reproducible bit for bit.
+ *
+ * p_idx, p_val  [B, k]         the pairs dssd_edge_verify_topk wrote; the indices of a sequence
+ *                              must be distinct; a negative index marks a sequence without a row
+ *                              (token = -1, DSSD_RS_FLAG_INVALID)
+ * q_idx, q_val  [B, gamma, k]  the draft's truncated Q_i; only row n is read (may be NULL iff
+ *                              gamma == 0)
+ * accept_len    [B] int32;  uniforms [B] float32 u' in [0,1)
+ * token         [B] int32 out;  flags [B] uint32 out, optional (NULL ok): DSSD_RS_FLAG_*
+ * Needs no workspace.
+ */
+dssd_status dssd_device_resample_topk(const int32_t *p_idx, const float *p_val,
+                                      const int32_t *q_idx, const float *q_val,
+                                      const int32_t *accept_len, const float *uniforms, int B,
+                                      int gamma, int k, int32_t *token, uint32_t *flags,
+                                      void *cuda_stream);
 
 #ifdef __cplusplus
 }

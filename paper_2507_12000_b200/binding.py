@@ -70,6 +70,17 @@ def _load() -> ctypes.CDLL:
     L.dssd_device_resample_static.argtypes = [
         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
         c.c_void_p, c.c_void_p, c.c_void_p]
+    L.dssd_edge_verify_topk_workspace_bytes.restype = c.c_size_t
+    L.dssd_edge_verify_topk_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int]
+    L.dssd_edge_verify_topk.restype = c.c_int
+    L.dssd_edge_verify_topk.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_device_resample_topk.restype = c.c_int
+    L.dssd_device_resample_topk.argtypes = [
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -192,6 +203,72 @@ def dssd_device_resample_static(p_row: torch.Tensor, draft_q: Optional[torch.Ten
         B, gamma, V, out["token"].data_ptr(), _ptr(out.get("flags")), _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_device_resample_static")
+    return out
+
+
+TOPK_MAX = 32
+
+
+def dssd_edge_verify_topk_workspace_bytes(B: int, gamma: int, V: int, k: int) -> int:
+    return int(lib.dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k))
+
+
+def dssd_edge_verify_topk(target_logits: torch.Tensor, draft_tokens: torch.Tensor, draft_q_tok: torch.Tensor,
+                          uniforms: torch.Tensor, temperature: float, k: int, *,
+                          out: Optional[Dict[str, torch.Tensor]] = None, want_p_tok: bool = True,
+                          workspace: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """Edge half of one round on target distributions truncated to their k largest entries.
+    Returns accept_len [B], p_idx / p_val [B, k], flags and, if asked, p_tok."""
+    assert target_logits.is_cuda and target_logits.dim() == 3
+    B, g1, V = target_logits.shape
+    gamma = g1 - 1
+    assert target_logits.stride(2) == 1 or V == 1
+    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
+    if B > 1 and target_logits.stride(0) != g1 * row_stride:
+        raise ValueError("rows of target_logits must be equally spaced")
+    dev = target_logits.device
+    if out is None:
+        kk = max(0, min(k, TOPK_MAX))
+        out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_idx": torch.empty(B, kk, dtype=torch.int32, device=dev),
+            "p_val": torch.empty(B, kk, dtype=torch.float32, device=dev),
+            "flags": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_tok": torch.empty(B, gamma, dtype=torch.float32, device=dev) if want_p_tok else None,
+        }
+    if workspace is None:
+        workspace = _workspace(dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k), dev)
+    st = lib.dssd_edge_verify_topk(
+        target_logits.data_ptr(), _dtype_code(target_logits), row_stride,
+        _ptr(draft_tokens), _ptr(draft_q_tok), _ptr(uniforms), ctypes.c_float(temperature), B, gamma, V, k,
+        out["accept_len"].data_ptr(), out["p_idx"].data_ptr(), out["p_val"].data_ptr(), _ptr(out.get("p_tok")),
+        _ptr(out.get("flags")), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_verify_topk")
+    return out
+
+
+def dssd_device_resample_topk(p_idx: torch.Tensor, p_val: torch.Tensor, q_idx: Optional[torch.Tensor],
+                              q_val: Optional[torch.Tensor], accept_len: torch.Tensor,
+                              uniforms_rs: torch.Tensor, gamma: int, *,
+                              out: Optional[Dict[str, torch.Tensor]] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """Device half on truncated distributions: p_* [B, k], q_* [B, gamma, k] (contiguous)."""
+    assert p_idx.is_cuda and p_idx.dim() == 2 and p_idx.is_contiguous() and p_idx.dtype == torch.int32
+    assert p_val.is_contiguous() and p_val.dtype == torch.float32 and p_val.shape == p_idx.shape
+    B, k = p_idx.shape
+    if gamma > 0:
+        assert q_idx.is_contiguous() and q_idx.dtype == torch.int32 and q_idx.numel() == B * gamma * k
+        assert q_val.is_contiguous() and q_val.dtype == torch.float32 and q_val.numel() == B * gamma * k
+    dev = p_idx.device
+    if out is None:
+        out = {"token": torch.empty(B, dtype=torch.int32, device=dev),
+               "flags": torch.empty(B, dtype=torch.int32, device=dev)}
+    st = lib.dssd_device_resample_topk(
+        p_idx.data_ptr(), p_val.data_ptr(), _ptr(q_idx) if gamma > 0 else None,
+        _ptr(q_val) if gamma > 0 else None, accept_len.data_ptr(), uniforms_rs.data_ptr(), B, gamma, k,
+        out["token"].data_ptr(), _ptr(out.get("flags")), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_device_resample_topk")
     return out
 
 

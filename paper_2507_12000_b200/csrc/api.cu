@@ -5,6 +5,7 @@
 #include "device_resample.h"
 #include "dssd.h"
 #include "edge_verify.h"
+#include "topk_verify.h"
 
 namespace {
 
@@ -132,6 +133,83 @@ dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
     P.token = token;
     P.flags = flags;
     cudaError_t e = dssd::resample_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+size_t dssd_edge_verify_topk_workspace_bytes(int B, int gamma, int V, int k)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    if (k < 1 || k > V || k > DSSD_TOPK_MAX) return 0;
+    return dssd::topk_workspace_layout(B, gamma, k, nullptr, nullptr);
+}
+
+dssd_status dssd_edge_verify_topk(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                  const int32_t *draft_tokens, const float *draft_q_tok,
+                                  const float *uniforms, float temperature, int B, int gamma,
+                                  int V, int k, int32_t *accept_len, int32_t *p_idx, float *p_val,
+                                  float *p_tok, uint32_t *flags, void *workspace,
+                                  size_t workspace_bytes, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (k < 1 || k > V) return DSSD_ERR_INVALID_ARG;
+    if (k > DSSD_TOPK_MAX) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !accept_len || !p_idx || !p_val) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if (reinterpret_cast<uintptr_t>(target_logits) % esz) return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k))
+        return DSSD_ERR_WORKSPACE;
+
+    dssd::TopkParams P{};
+    P.logits = target_logits;
+    P.row_stride = row_stride;
+    P.draft_tokens = draft_tokens;
+    P.draft_q_tok = draft_q_tok;
+    P.uniforms = uniforms;
+    P.temperature = temperature;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V;
+    P.k = k;
+    P.accept_len = accept_len;
+    P.p_idx = p_idx;
+    P.p_val = p_val;
+    P.p_tok = p_tok;
+    P.flags = flags;
+    cudaError_t e = dssd::topk_verify_launch(P, (int)dtype, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+dssd_status dssd_device_resample_topk(const int32_t *p_idx, const float *p_val,
+                                      const int32_t *q_idx, const float *q_val,
+                                      const int32_t *accept_len, const float *uniforms, int B,
+                                      int gamma, int k, int32_t *token, uint32_t *flags,
+                                      void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    if (B < 1 || gamma < 0 || k < 1) return DSSD_ERR_INVALID_ARG;
+    if (k > DSSD_TOPK_MAX) return DSSD_ERR_UNSUPPORTED;
+    if (!p_idx || !p_val || !accept_len || !uniforms || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!q_idx || !q_val)) return DSSD_ERR_INVALID_ARG;
+    dssd::TopkResampleParams P{};
+    P.p_idx = p_idx;
+    P.p_val = p_val;
+    P.q_idx = q_idx;
+    P.q_val = q_val;
+    P.accept_len = accept_len;
+    P.uniforms = uniforms;
+    P.B = B;
+    P.gamma = gamma;
+    P.k = k;
+    P.token = token;
+    P.flags = flags;
+    cudaError_t e = dssd::topk_resample_launch(P, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
 }
 

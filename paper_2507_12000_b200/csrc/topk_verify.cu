@@ -1,0 +1,598 @@
+// Truncated-support (top-k) verification round for sm_100a: the sampler of the paper's
+// experiments (Section 4) applied to Algorithm 2.
+//
+// Edge kernel.  The work is one pass over the logits, so the kernel is a pure HBM read stream
+// with a selection riding on it:
+//
+//   * Rows are cut into blocks of kTopkBlock entries; the blocks of all rows are numbered row
+//     by row and divided evenly over the CTAs (4 per SM), each CTA owning one contiguous span.
+//     A span crosses row boundaries, so a CTA works through a few "pieces" (row, first block,
+//     last block); no tickets, no atomics on the streaming path, every CTA ends at the same time.
+//   * A piece is scanned with 16-byte loads, kU vectors per thread in flight plus the next kU
+//     prefetched.  Each vector is reduced to its maximum with NaN-propagating max instructions
+//     and compared with the CTA's threshold tau, a lower bound on the piece's k-th largest
+//     logit; only a vector that reaches tau is taken apart.  Its elements that beat the
+//     current k-th key are appended to a candidate buffer in shared memory.
+//   * A key is 64 bits: the logit mapped to an unsigned integer that sorts like the float
+//     (with -0 folded into +0), then the complemented index - larger key = earlier in the order
+//     (logit descending, index ascending), and all keys of a row are distinct.
+//   * After every iteration the CTA meets at a barrier; when enough candidates have gathered
+//     it merges them with its current list by rank counting (each key counts the keys above
+//     it; rank < k writes itself to that slot), which needs no sorting network and no second
+//     barrier round.  The threshold lives in registers and is refreshed from the new list.
+//   * tau starts from the first iteration: the 256 threads form 32 groups of 8, each group's
+//     maximum is one distinct element, so the k-th largest group maximum (k <= 32) is a valid
+//     lower bound.  A candidate buffer that overflows anyway (ascending input) is handled by
+//     merging and resuming the same registers from where each thread stopped.
+//   * The piece's list goes to the workspace; the CTA that completes a sequence (a counter of
+//     scanned blocks per sequence tells) folds it: one warp per row merges the row's pieces,
+//     turns the k logits into probabilities in float64, applies the acceptance test; the first
+//     rejection is an atomicMin in shared memory; warp 0 then writes row n's k pairs.
+//
+// Device kernel: one warp per sequence, everything in registers and shuffles, sums strictly
+// sequential in float64 so that the draw is reproducible bit for bit.
+#include "topk_verify.h"
+
+#include <math.h>
+
+#include "dssd_device.cuh"
+
+namespace dssd {
+namespace {
+
+constexpr int kU = 4;          // 16-byte vectors per thread per iteration
+constexpr int kCap = 512;      // candidate buffer entries
+constexpr int kMergeAt = 24;   // merge once this many candidates wait
+constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
+constexpr unsigned kFullMask = 0xffffffffu;
+
+__device__ __forceinline__ float max_nan(float a, float b)
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t r;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// unsigned integers that sort like the floats they come from (NaN excluded by the callers)
+__device__ __forceinline__ uint32_t ord(float f)
+{
+    uint32_t b = __float_as_uint(f);
+    if (b == 0x80000000u) b = 0u;  // -0 and +0 are the same logit
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ float unord(uint32_t o)
+{
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+}
+
+__device__ __forceinline__ unsigned long long make_key(float f, int idx)
+{
+    return ((unsigned long long)ord(f) << 32) | (unsigned long long)(~(uint32_t)idx);
+}
+
+__device__ __forceinline__ int key_index(unsigned long long key) { return (int)(~(uint32_t)key); }
+__device__ __forceinline__ float key_value(unsigned long long key) { return unord((uint32_t)(key >> 32)); }
+
+template <int DT>
+struct Vec;
+template <>
+struct Vec<DSSD_F32> {
+    static constexpr int E = 4;
+    static constexpr int kEsz = 4;
+    __device__ static __forceinline__ uint4 fill() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    __device__ static __forceinline__ float vmax(const uint4 &v)
+    {
+        return max_nan(max_nan(__uint_as_float(v.x), __uint_as_float(v.y)),
+                       max_nan(__uint_as_float(v.z), __uint_as_float(v.w)));
+    }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
+    {
+        f[0] = __uint_as_float(v.x), f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z), f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float load(const void *row, int64_t i) { return reinterpret_cast<const float *>(row)[i]; }
+};
+template <>
+struct Vec<DSSD_BF16> {
+    static constexpr int E = 8;
+    static constexpr int kEsz = 2;
+    __device__ static __forceinline__ uint4 fill() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    __device__ static __forceinline__ float vmax(const uint4 &v)
+    {
+        const uint32_t w = max_nan_bf16x2(max_nan_bf16x2(v.x, v.y), max_nan_bf16x2(v.z, v.w));
+        return max_nan(bf16_lo(w), bf16_hi(w));
+    }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
+    {
+        f[0] = bf16_lo(v.x), f[1] = bf16_hi(v.x), f[2] = bf16_lo(v.y), f[3] = bf16_hi(v.y);
+        f[4] = bf16_lo(v.z), f[5] = bf16_hi(v.z), f[6] = bf16_lo(v.w), f[7] = bf16_hi(v.w);
+    }
+    __device__ static __forceinline__ float load(const void *row, int64_t i)
+    {
+        return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short *>(row)[i] << 16);
+    }
+};
+
+struct Smem {
+    unsigned long long list[2][32];  // the piece's current top-k, best first; two buffers, swapped by each merge
+    unsigned long long cand[kCap];   // candidates since the last merge
+    float grp[32];                   // group maxima of the first iteration
+    int n[2];                        // candidates appended (may run past kCap: overflow)
+    int bad;                         // the piece holds a NaN or +inf
+    int last;                        // this CTA scanned the last block of a sequence
+    int first_reject;                // fold: first rejected position
+    unsigned fl;                     // fold: flags of the sequence
+    unsigned long long fold_keys[kWarps][kTopkMergeKeys];  // fold: one row's pieces, per warp
+    unsigned long long fold_top[kWarps][32];               // fold: the row's top-k, best first
+};
+
+// One element that reached tau: reject it by key, flag it, or append it.  Returns false when the
+// candidate buffer is full (the caller stops and resumes after the next merge).
+__device__ __forceinline__ bool offer(Smem &S, int nbuf, float f, int idx, unsigned long long taukey)
+{
+    if (f != f || f == INFINITY) {
+        S.bad = 1;
+        return true;
+    }
+    const unsigned long long key = make_key(f, idx);
+    if (key > taukey) {
+        const int slot = atomicAdd(&S.n[nbuf], 1);
+        if (slot >= kCap) return false;
+        S.cand[slot] = key;
+    }
+    return true;
+}
+
+// Scans this thread's kU vectors from element ordinal `pos` on; returns the ordinal it stopped
+// at (kU * E when done).  vi0 = index of the thread's first vector within the piece's vector
+// body, idx0 = vocabulary index of the body's first element.
+template <int DT>
+__device__ __forceinline__ int scan(const uint4 (&a)[kU], int pos, int vi0, int nvec, int idx0, float tau,
+                                    unsigned long long taukey, Smem &S, int nbuf)
+{
+    constexpr int E = Vec<DT>::E;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const int vi = vi0 + u * kThreads;
+        if (pos < (u + 1) * E && vi < nvec && !(Vec<DT>::vmax(a[u]) < tau)) {
+            float f[E];
+            Vec<DT>::unpack(a[u], f);
+#pragma unroll
+            for (int j = 0; j < E; ++j) {
+                const int o = u * E + j;
+                if (o >= pos && !(f[j] < tau)) {
+                    if (!offer(S, nbuf, f[j], idx0 + vi * E + j, taukey)) return o;
+                }
+            }
+        }
+    }
+    return kU * E;
+}
+
+// Merges the candidates with the current list by rank counting; the new list lands in the
+// other buffer.  All keys involved are distinct.  Ends with a barrier.
+__device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n_raw, int k)
+{
+    const int n = min(n_raw, kCap), m = k + n;
+    const unsigned long long *top = S.list[cur];
+    unsigned long long *out = S.list[cur ^ 1];
+    if (threadIdx.x == 0) S.n[nbuf ^ 1] = 0;
+    for (int i = threadIdx.x; i < m; i += kThreads) {
+        const unsigned long long x = i < k ? top[i] : S.cand[i - k];
+        int rank = 0;
+        for (int j = 0; j < k; ++j) rank += top[j] > x;
+        for (int j = 0; j < n; ++j) rank += S.cand[j] > x;
+        if (rank < k) out[rank] = x;
+    }
+    __syncthreads();
+}
+
+// Top-k of elements [e0, e1) of one row into S.list[returned buffer]; S.bad tells whether the
+// piece held a NaN or +inf.  Called by the whole CTA.
+template <int DT>
+__device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
+{
+    constexpr int E = Vec<DT>::E;
+    constexpr int kEsz = Vec<DT>::kEsz;
+    const int tid = threadIdx.x, lane = tid & 31;
+    // empty slots hold distinct small keys (k - r in slot r), below every real key
+    if (tid < 32) S.list[0][tid] = tid < k ? (unsigned long long)(k - tid) : 0ull;
+    if (tid == 0) {
+        S.n[0] = 0;
+        S.n[1] = 0;
+        S.bad = 0;
+    }
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(rowp) + (uintptr_t)e0 * kEsz;
+    const int head = min(e1 - e0, (int)(((16u - (unsigned)(addr & 15u)) & 15u) / kEsz));
+    const int nvec = (e1 - e0 - head) / E;
+    const int idx0 = e0 + head;
+    const int tail0 = idx0 + nvec * E;
+    const uint4 *vp = reinterpret_cast<const uint4 *>(rowp + (size_t)idx0 * kEsz);
+    const int iters = (nvec + kThreads * kU - 1) / (kThreads * kU);
+
+    uint4 a[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const int vi = tid + u * kThreads;
+        a[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
+    }
+    // tau from the first iteration: k-th largest of the 32 group maxima
+    float tm = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const float v = Vec<DT>::vmax(a[u]);
+        tm = fmaxf(tm, v == v ? v : -INFINITY);
+    }
+    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 1));
+    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 2));
+    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 4));
+    __syncthreads();  // the previous piece's readers of S are done; the init above is visible after the next barrier
+    if ((tid & 7) == 0) S.grp[tid >> 3] = tm;
+    __syncthreads();
+    float tau;
+    {
+        const float g = S.grp[lane];
+        int rank = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float o = __shfl_sync(kFullMask, g, j);
+            rank += (o > g) || (o == g && j < lane);
+        }
+        const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
+        tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
+    }
+    unsigned long long taukey = (unsigned long long)ord(tau) << 32;
+    int cur = 0, nbuf = 0;
+
+    // the ragged ends of the piece, one element per thread
+    if (tid < head) offer(S, nbuf, Vec<DT>::load(rowp, e0 + tid), e0 + tid, taukey);
+    if (tid >= 32 && tid - 32 < e1 - tail0) offer(S, nbuf, Vec<DT>::load(rowp, tail0 + tid - 32), tail0 + tid - 32, taukey);
+
+    for (int it = 0; it < iters; ++it) {
+        uint4 nx[kU];
+        const int vnext = (it + 1) * kThreads * kU + tid;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int vi = vnext + u * kThreads;
+            nx[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
+        }
+        const int vi0 = it * kThreads * kU + tid;
+        int pos = 0;
+        for (;;) {
+            pos = scan<DT>(a, pos, vi0, nvec, idx0, tau, taukey, S, nbuf);
+            __syncthreads();
+            const int n = S.n[nbuf];
+            if (n >= kMergeAt || n > kCap || it + 1 == iters) {
+                merge(S, cur, nbuf, n, k);
+                cur ^= 1;
+                nbuf ^= 1;
+                const unsigned long long kth = S.list[cur][k - 1];
+                if (kth > taukey) {
+                    taukey = kth;
+                    tau = key_value(kth);
+                }
+            }
+            if (n <= kCap) break;
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) a[u] = nx[u];
+    }
+    if (iters == 0) {  // only ragged elements
+        __syncthreads();
+        merge(S, cur, nbuf, S.n[nbuf], k);
+        cur ^= 1;
+    }
+    return cur;
+}
+
+// CTA that owns block `blk` when `total` blocks are divided over `grid` CTAs
+__device__ __forceinline__ unsigned long long owner_of(unsigned long long blk, unsigned long long grid, unsigned long long total)
+{
+    return ((blk + 1ull) * grid - 1ull) / total;
+}
+
+struct RowDist {   // per lane r < k: entry r of the row's support, best first
+    int idx;
+    double prob;
+    bool bad;      // the row has no distribution (warp-uniform)
+};
+
+// One warp: merges the pieces of `row`, then turns the k logits into probabilities (float64,
+// summed in rank order).
+__device__ RowDist row_dist(const TopkParams &P, int64_t row, unsigned long long *keys, unsigned long long *top)
+{
+    const int lane = threadIdx.x & 31, k = P.k;
+    const unsigned long long first_blk = (unsigned long long)row * (unsigned long long)P.nb;
+    const int pieces = (int)(owner_of(first_blk + P.nb - 1, P.grid, P.total_blocks) - owner_of(first_blk, P.grid, P.total_blocks)) + 1;
+    const int m = pieces * k;
+    const unsigned long long *src = P.lists + (size_t)row * P.max_pieces * k;
+    bool bad = false;
+    for (int i = lane; i < m; i += 32) {
+        const unsigned long long x = __ldcg(src + i);
+        bad |= (x == kBadList);
+        keys[i] = x;
+    }
+    bad = __any_sync(kFullMask, bad);
+    __syncwarp();
+    RowDist d;
+    d.idx = -1;
+    d.prob = NAN;
+    d.bad = bad;
+    if (bad) return d;
+    if (pieces == 1) {
+        if (lane < k) top[lane] = keys[lane];
+    } else {
+        for (int i = lane; i < m; i += 32) {
+            const unsigned long long x = keys[i];
+            int rank = 0;
+            for (int j = 0; j < m; ++j) rank += keys[j] > x;
+            if (rank < k) top[rank] = x;  // keys below rank k include every empty slot
+        }
+    }
+    __syncwarp();
+    const unsigned long long key = lane < k ? top[lane] : 0ull;
+    __syncwarp();
+    const float val = key_value(key);
+    const float best = __shfl_sync(kFullMask, val, 0);
+    if (!(best > -INFINITY)) {  // nothing above -inf
+        d.bad = true;
+        return d;
+    }
+    const double T = (double)P.temperature;
+    const double z = (double)val / T;
+    const double mx = __shfl_sync(kFullMask, z, 0);
+    const double e = lane < k ? exp(z - mx) : 0.0;
+    double S = 0.0;
+    for (int r = 0; r < k; ++r) S += __shfl_sync(kFullMask, e, r);
+    d.idx = lane < k ? key_index(key) : -1;
+    d.prob = e / S;
+    return d;
+}
+
+// The CTA that scanned a sequence's last block: acceptance tests, first rejection, row n's pairs.
+__device__ void fold_sequence(const TopkParams &P, int b, Smem &S)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gamma = P.gamma, k = P.k;
+    if (tid == 0) {
+        S.first_reject = gamma;
+        S.fl = 0u;
+    }
+    __syncthreads();
+    for (int j = warp; j <= gamma; j += kWarps) {
+        const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + j, S.fold_keys[warp], S.fold_top[warp]);
+        if (d.bad && lane == 0) atomicOr(&S.fl, DSSD_EDGE_FLAG_NONFINITE);
+        if (j == gamma) continue;
+        const size_t o = (size_t)b * gamma + j;
+        const int x = __ldg(P.draft_tokens + o);
+        const unsigned holds = __ballot_sync(kFullMask, lane < k && !d.bad && d.idx == x);
+        const double p_in = __shfl_sync(kFullMask, d.prob, holds ? __ffs(holds) - 1 : 0);
+        if (lane == 0) {
+            const double u = (double)__ldg(P.uniforms + o), q = (double)__ldg(P.draft_q_tok + o);
+            double p;
+            bool accept = false;
+            if (x < 0 || x >= P.V) {
+                atomicOr(&S.fl, DSSD_EDGE_FLAG_BAD_TOKEN);
+                p = NAN;
+            } else {
+                p = d.bad ? NAN : (holds ? p_in : 0.0);
+                double ratio;
+                if (q != q || p != p) ratio = NAN;
+                else if (q <= 0.0) ratio = p > 0.0 ? INFINITY : 0.0;
+                else ratio = p / q;
+                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+            }
+            if (P.p_tok) P.p_tok[o] = (float)p;
+            if (!accept) atomicMin(&S.first_reject, j);
+        }
+    }
+    __syncthreads();
+    const int n = S.first_reject;
+    if (warp == 0) {
+        const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + n, S.fold_keys[0], S.fold_top[0]);
+        if (lane < k) {
+            P.p_idx[(size_t)b * k + lane] = d.bad ? -1 : d.idx;
+            P.p_val[(size_t)b * k + lane] = d.bad ? NAN : (float)d.prob;
+        }
+        if (lane == 0) {
+            P.accept_len[b] = n;
+            if (P.flags) P.flags[b] = S.fl;
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4) topk_verify_kernel(const __grid_constant__ TopkParams P)
+{
+    __shared__ Smem S;
+    const int tid = threadIdx.x, k = P.k;
+    const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
+    const unsigned long long blk_end = (c + 1ull) * TB / G;
+    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
+    unsigned long long blk = c * TB / G;
+    while (blk < blk_end) {
+        const int64_t row = (int64_t)(blk / (unsigned long long)P.nb);
+        const int fb = (int)(blk - (unsigned long long)row * P.nb);
+        const int lb = (int)min((unsigned long long)P.nb, fb + (blk_end - blk));
+        const int e0 = fb * kTopkBlock, e1 = (int)min((long long)P.V, (long long)lb * kTopkBlock);
+        const char *rowp = reinterpret_cast<const char *>(P.logits) + (size_t)row * (size_t)P.row_stride * Vec<DT>::kEsz;
+        const int cur = piece_topk<DT>(rowp, e0, e1, k, S);
+        const int slot = (int)(c - owner_of((unsigned long long)row * P.nb, G, TB));
+        if (tid < k) {
+            unsigned long long key = S.list[cur][tid];
+            if (S.bad) key = tid == 0 ? kBadList : 0ull;
+            __stcg(P.lists + ((size_t)row * P.max_pieces + slot) * k + tid, key);
+        }
+        __threadfence();
+        __syncthreads();
+        const int b = (int)(row / (P.gamma + 1));
+        if (tid == 0) {
+            const unsigned long long done = (unsigned long long)(lb - fb);
+            const unsigned long long old = atomicAdd(P.seq_done + b, done);
+            S.last = (old + done == per_seq);
+        }
+        __syncthreads();
+        if (S.last) {
+            __threadfence();
+            fold_sequence(P, b, S);
+        }
+        __syncthreads();
+        blk += (unsigned long long)(lb - fb);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// device half: one warp per sequence
+
+__device__ __forceinline__ double shfl_f64(double v, int src) { return __shfl_sync(kFullMask, v, src); }
+
+// inverse CDF over the warp's k entries (lane e holds r_e, entries in increasing index);
+// returns the position, or -1 when the mass is not positive and finite
+__device__ __forceinline__ int warp_inverse_cdf(double r, int k, double u)
+{
+    double Z = 0.0;
+    for (int e = 0; e < k; ++e) Z += shfl_f64(r, e);
+    if (!(Z > 0.0) || !(Z < INFINITY)) return -1;
+    const double t = u * Z;
+    double C = 0.0;
+    int last_pos = -1, hit = -1;
+    for (int e = 0; e < k; ++e) {
+        const double re = shfl_f64(r, e);
+        C += re;
+        if (re > 0.0) last_pos = e;
+        if (hit < 0 && C > t) hit = e;
+    }
+    return hit >= 0 ? hit : last_pos;
+}
+
+__global__ void __launch_bounds__(kThreads) topk_resample_kernel(const TopkResampleParams P)
+{
+    __shared__ int s_idx[kWarps][32];
+    __shared__ float s_val[kWarps][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, k = P.k;
+    const int b = blockIdx.x * kWarps + warp;
+    if (b >= P.B) return;
+    const int n = __ldg(P.accept_len + b);
+    const double u = (double)__ldg(P.uniforms + b);
+    const int pi = lane < k ? __ldg(P.p_idx + (size_t)b * k + lane) : 0;
+    const float pv = lane < k ? __ldg(P.p_val + (size_t)b * k + lane) : 0.f;
+    const bool has_row = !__any_sync(kFullMask, lane < k && pi < 0);
+    unsigned fl = 0u;
+    int tok = -1;
+    if (n < 0 || n > P.gamma || !has_row) {
+        fl = DSSD_RS_FLAG_INVALID;
+    } else {
+        // P's entries in increasing vocabulary index (indices are distinct)
+        int rank = 0;
+        for (int e = 0; e < k; ++e) rank += __shfl_sync(kFullMask, pi, e) < pi;
+        if (lane < k) {
+            s_idx[warp][rank] = pi;
+            s_val[warp][rank] = pv;
+        }
+        __syncwarp();
+        const int sid = lane < k ? s_idx[warp][lane] : -1;
+        const double sp = lane < k ? (double)s_val[warp][lane] : 0.0;
+        int pos;
+        if (n == P.gamma) {
+            fl |= DSSD_RS_FLAG_BONUS;
+            pos = warp_inverse_cdf(sp, k, u);
+        } else {
+            const size_t qo = ((size_t)b * P.gamma + n) * (size_t)k;
+            const int qi = lane < k ? __ldg(P.q_idx + qo + lane) : -1;
+            const float qv = lane < k ? __ldg(P.q_val + qo + lane) : 0.f;
+            float sq = 0.f;
+            for (int f = k - 1; f >= 0; --f) {  // the first listed match wins
+                const int fi = __shfl_sync(kFullMask, qi, f);
+                const float fv = __shfl_sync(kFullMask, qv, f);
+                if (fi == sid) sq = fv;
+            }
+            const double r = lane < k ? fmax(0.0, sp - (double)sq) : 0.0;
+            pos = warp_inverse_cdf(r, k, u);
+            if (pos < 0) {
+                fl |= DSSD_RS_FLAG_FALLBACK;
+                pos = warp_inverse_cdf(sp, k, u);
+            }
+        }
+        if (pos < 0) fl |= DSSD_RS_FLAG_INVALID;
+        else tok = __shfl_sync(kFullMask, sid, pos);
+    }
+    if (lane == 0) {
+        P.token[b] = tok;
+        if (P.flags) P.flags[b] = fl;
+    }
+}
+
+}  // namespace
+
+int topk_max_pieces(int k)
+{
+    const int byk = kTopkMergeKeys / (k < 1 ? 1 : k);
+    return byk < kTopkMaxPieces ? byk : kTopkMaxPieces;
+}
+
+size_t topk_workspace_layout(int B, int gamma, int k, TopkParams *P, char *base)
+{
+    const size_t rows = (size_t)B * (size_t)(gamma + 1);
+    const size_t cnt = ((size_t)B * 8 + 255) & ~(size_t)255;
+    const size_t lists = rows * (size_t)topk_max_pieces(k) * (size_t)k * 8;
+    if (P) {
+        P->seq_done = reinterpret_cast<unsigned long long *>(base);
+        P->lists = reinterpret_cast<unsigned long long *>(base + cnt);
+        P->zero_bytes = (size_t)B * 8;
+        P->max_pieces = topk_max_pieces(k);
+    }
+    return cnt + ((lists + 255) & ~(size_t)255);
+}
+
+static int g_topk_ctas[64];  // resident CTAs of the kernel per device (0 = not asked yet)
+
+cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaStream_t stream)
+{
+    cudaError_t err;
+    int dev = 0;
+    if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
+    int ctas = (dev >= 0 && dev < 64) ? g_topk_ctas[dev] : 0;
+    if (ctas == 0) {
+        int sms = 0, occ0 = 0, occ1 = 0;
+        if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, topk_verify_kernel<DSSD_F32>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, topk_verify_kernel<DSSD_BF16>, kThreads, 0)) != cudaSuccess) return err;
+        const int occ = occ0 < occ1 ? occ0 : occ1;
+        ctas = sms * (occ < 1 ? 1 : occ);
+        if (dev >= 0 && dev < 64) g_topk_ctas[dev] = ctas;
+    }
+    topk_workspace_layout(P.B, P.gamma, P.k, &P, static_cast<char *>(workspace));
+    const unsigned long long rows = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);
+    P.nb = (P.V + kTopkBlock - 1) / kTopkBlock;
+    P.total_blocks = rows * (unsigned long long)P.nb;
+    // every span must hold at least ceil(nb / (max_pieces - 1)) blocks, so that no row is shared
+    // by more than max_pieces CTAs
+    const unsigned long long wmin = ((unsigned long long)P.nb + P.max_pieces - 2) / (unsigned long long)(P.max_pieces - 1);
+    unsigned long long grid = P.total_blocks / wmin;
+    if (grid > (unsigned long long)ctas) grid = (unsigned long long)ctas;
+    if (grid < 1) grid = 1;
+    P.grid = (int)grid;
+    if ((err = cudaMemsetAsync(P.seq_done, 0, P.zero_bytes, stream)) != cudaSuccess) return err;
+    if (dtype == DSSD_BF16)
+        topk_verify_kernel<DSSD_BF16><<<P.grid, kThreads, 0, stream>>>(P);
+    else
+        topk_verify_kernel<DSSD_F32><<<P.grid, kThreads, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+cudaError_t topk_resample_launch(const TopkResampleParams &P, cudaStream_t stream)
+{
+    const int grid = (P.B + kWarps - 1) / kWarps;
+    topk_resample_kernel<<<grid, kThreads, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+}  // namespace dssd

@@ -49,6 +49,11 @@ def test_workspace_sizes(B):
     assert 0 < a < b < c < 64 << 20 and a % 256 == 0
     r = B.dssd_device_resample_workspace_bytes(256, 4, 151936)
     assert 0 < r < 4 << 20
+    assert B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 0) == 0
+    assert B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 33) == 0
+    assert B.dssd_edge_verify_topk_workspace_bytes(1, 0, 8, 9) == 0
+    t = B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 10)
+    assert 0 < t < 4 << 20 and t % 256 == 0
     assert B.dssd_round_host_arena_bytes(8, 4, 32000, B.DSSD_BF16) > 8 * 5 * 32000 * 2 + 8 * 4 * 32000 * 4
     assert B.dssd_round_host_arena_bytes(8, 4, 32000, 7) == 0
 
@@ -93,6 +98,34 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
     assert rs(Bn=-3) == B.DSSD_ERR_INVALID_ARG
     assert rs(wsb=8) == B.DSSD_ERR_WORKSPACE
     assert rs(ws=None) == B.DSSD_ERR_WORKSPACE
+
+    def evk(logits=p, dtype=0, stride=64, tok=p, qt=p, u=p, T=1.0, Bn=1, g=2, V=64, k=10, n=p, pi=p, pv=p, ws=p,
+            wsb=ok_ws):
+        return L.dssd_edge_verify_topk(logits, dtype, stride, tok, qt, u, f(T), Bn, g, V, k, n, pi, pv, None, None,
+                                       ws, wsb, None)
+
+    assert evk(logits=None) == B.DSSD_ERR_INVALID_ARG
+    assert evk(pi=None) == B.DSSD_ERR_INVALID_ARG
+    assert evk(pv=None) == B.DSSD_ERR_INVALID_ARG
+    assert evk(u=None) == B.DSSD_ERR_INVALID_ARG
+    assert evk(k=0) == B.DSSD_ERR_INVALID_ARG
+    assert evk(k=20, V=16, stride=16) == B.DSSD_ERR_INVALID_ARG
+    assert evk(k=33) == B.DSSD_ERR_UNSUPPORTED
+    assert evk(T=0.0) == B.DSSD_ERR_INVALID_ARG
+    assert evk(stride=63) == B.DSSD_ERR_INVALID_ARG
+    assert evk(dtype=2) == B.DSSD_ERR_UNSUPPORTED
+    assert evk(ws=None) == B.DSSD_ERR_WORKSPACE
+    assert evk(wsb=8) == B.DSSD_ERR_WORKSPACE
+
+    def rsk(pi=p, pv=p, qi=p, qv=p, n=p, u=p, Bn=1, g=2, k=10, tok=p):
+        return L.dssd_device_resample_topk(pi, pv, qi, qv, n, u, Bn, g, k, tok, None, None)
+
+    assert rsk(pi=None) == B.DSSD_ERR_INVALID_ARG
+    assert rsk(qv=None) == B.DSSD_ERR_INVALID_ARG
+    assert rsk(tok=None) == B.DSSD_ERR_INVALID_ARG
+    assert rsk(Bn=0) == B.DSSD_ERR_INVALID_ARG
+    assert rsk(k=0) == B.DSSD_ERR_INVALID_ARG
+    assert rsk(k=33) == B.DSSD_ERR_UNSUPPORTED
 
     assert L.dssd_round_host(None, 0, p, p, p, p, p, f(1.0), 1, 2, 16, p, p, None, None, None, p, ok_ws, None) \
         == B.DSSD_ERR_INVALID_ARG
