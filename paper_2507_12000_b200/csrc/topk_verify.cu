@@ -40,9 +40,19 @@
 namespace dssd {
 namespace {
 
-constexpr int kU = 4;          // 16-byte vectors per thread per iteration
-constexpr int kCap = 512;      // candidate buffer entries
-constexpr int kMergeAt = 24;   // merge once this many candidates wait
+#ifndef DSSD_TOPK_U
+#define DSSD_TOPK_U 4
+#endif
+#ifndef DSSD_TOPK_CTAS
+#define DSSD_TOPK_CTAS 4
+#endif
+#ifndef DSSD_TOPK_MERGE_AT
+#define DSSD_TOPK_MERGE_AT 24
+#endif
+constexpr int kU = DSSD_TOPK_U;                // 16-byte vectors per thread per iteration
+constexpr int kCtasPerSm = DSSD_TOPK_CTAS;     // resident CTAs per SM the kernel is compiled for
+constexpr int kCap = 512;                      // candidate buffer entries
+constexpr int kMergeAt = DSSD_TOPK_MERGE_AT;   // merge once this many candidates wait
 constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
 constexpr unsigned kFullMask = 0xffffffffu;
 
@@ -99,6 +109,11 @@ struct Vec<DSSD_F32> {
         f[2] = __uint_as_float(v.z), f[3] = __uint_as_float(v.w);
     }
     __device__ static __forceinline__ float load(const void *row, int64_t i) { return reinterpret_cast<const float *>(row)[i]; }
+    // element j of the vector (j < E)
+    __device__ static __forceinline__ float elem(const uint4 &v, int j)
+    {
+        return __uint_as_float(j < 2 ? (j == 0 ? v.x : v.y) : (j == 2 ? v.z : v.w));
+    }
 };
 template <>
 struct Vec<DSSD_BF16> {
@@ -119,72 +134,113 @@ struct Vec<DSSD_BF16> {
     {
         return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short *>(row)[i] << 16);
     }
+    __device__ static __forceinline__ float elem(const uint4 &v, int j)
+    {
+        const uint32_t w = j < 4 ? (j < 2 ? v.x : v.y) : (j < 6 ? v.z : v.w);
+        return (j & 1) ? bf16_hi(w) : bf16_lo(w);
+    }
 };
 
 struct Smem {
-    unsigned long long list[2][32];  // the piece's current top-k, best first; two buffers, swapped by each merge
-    unsigned long long cand[kCap];   // candidates since the last merge
-    float grp[32];                   // group maxima of the first iteration
-    int n[2];                        // candidates appended (may run past kCap: overflow)
-    int bad;                         // the piece holds a NaN or +inf
-    int last;                        // this CTA scanned the last block of a sequence
-    int first_reject;                // fold: first rejected position
-    unsigned fl;                     // fold: flags of the sequence
+    unsigned long long list[2][32];    // the piece's current top-k, best first; two buffers, swapped by each merge
+    unsigned long long cand[kCap + 8]; // candidates since the last merge (a vector reserved below kCap may end past it)
+    float grp[32];                     // group maxima of the first iteration
+    int n[2];                          // candidate slots reserved (runs past kCap on overflow)
+    int nvalid[2];                     // first slot of the first refused reservation (INT_MAX: none)
+    int bad;                           // the piece holds a NaN or +inf
+    int last;                          // this CTA scanned the last block of a sequence
+    int first_reject;                  // fold: first rejected position
+    unsigned fl;                       // fold: flags of the sequence
     unsigned long long fold_keys[kWarps][kTopkMergeKeys];  // fold: one row's pieces, per warp
     unsigned long long fold_top[kWarps][32];               // fold: the row's top-k, best first
 };
 
-// One element that reached tau: reject it by key, flag it, or append it.  Returns false when the
-// candidate buffer is full (the caller stops and resumes after the next merge).
-__device__ __forceinline__ bool offer(Smem &S, int nbuf, float f, int idx, unsigned long long taukey)
+constexpr int kNone = 0x7fffffff;
+
+// One element of a piece's ragged ends (called before the first scan, when the buffer is empty)
+__device__ __forceinline__ void offer(Smem &S, int nbuf, float f, int idx, unsigned long long taukey)
 {
     if (f != f || f == INFINITY) {
         S.bad = 1;
-        return true;
+        return;
     }
     const unsigned long long key = make_key(f, idx);
-    if (key > taukey) {
-        const int slot = atomicAdd(&S.n[nbuf], 1);
-        if (slot >= kCap) return false;
-        S.cand[slot] = key;
+    if (key > taukey) S.cand[atomicAdd(&S.n[nbuf], 1)] = key;
+}
+
+// Where a warp stopped when the candidate buffer was full
+struct Resume {
+    int u;          // vector of the iteration (kU: the warp is done)
+    unsigned hot;   // lanes of that vector still to be taken apart
+};
+
+// Scans the warp's kU x 32 vectors.  A vector whose maximum reaches tau is taken apart by the
+// whole warp: its 16 bytes are broadcast and lane j judges element j, so a hit costs a few
+// instructions instead of a divergent per-element loop; the slots of a vector are reserved with
+// one shared-memory atomic.  Returns false when a reservation was refused (buffer full): `r`
+// then tells where to resume after the merge.  vi0 = this lane's first vector within the
+// piece's vector body, idx0 = vocabulary index of the body's first element.
+template <int DT>
+__device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resuming, int vi0, int nvec, int idx0,
+                                     float tau, unsigned long long taukey, Smem &S, int nbuf)
+{
+    constexpr int E = Vec<DT>::E;
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        if (u < r.u) continue;
+        const int vi = vi0 + u * kThreads;
+        unsigned hot = __ballot_sync(kFullMask, vi < nvec && !(Vec<DT>::vmax(a[u]) < tau));
+        if (resuming && u == r.u) hot = r.hot;
+        while (hot) {
+            const int src = __ffs(hot) - 1;
+            uint4 v;
+            v.x = __shfl_sync(kFullMask, a[u].x, src);
+            v.y = __shfl_sync(kFullMask, a[u].y, src);
+            v.z = __shfl_sync(kFullMask, a[u].z, src);
+            v.w = __shfl_sync(kFullMask, a[u].w, src);
+            const float f = Vec<DT>::elem(v, lane);
+            bool want = false;
+            unsigned long long key = 0ull;
+            if (lane < E && !(f < tau)) {
+                if (f != f || f == INFINITY) {
+                    S.bad = 1;
+                } else {
+                    key = make_key(f, idx0 + (vi - lane + src) * E + lane);
+                    want = key > taukey;
+                }
+            }
+            const unsigned wm = __ballot_sync(kFullMask, want);
+            if (wm) {
+                int base = 0;
+                if (lane == 0) base = atomicAdd(&S.n[nbuf], __popc(wm));
+                base = __shfl_sync(kFullMask, base, 0);
+                if (base >= kCap) {
+                    if (lane == 0) atomicMin(&S.nvalid[nbuf], base);
+                    r.u = u;
+                    r.hot = hot;
+                    return false;
+                }
+                if (want) S.cand[base + __popc(wm & ((1u << lane) - 1u))] = key;
+            }
+            hot &= hot - 1u;
+        }
     }
+    r.u = kU;
     return true;
 }
 
-// Scans this thread's kU vectors from element ordinal `pos` on; returns the ordinal it stopped
-// at (kU * E when done).  vi0 = index of the thread's first vector within the piece's vector
-// body, idx0 = vocabulary index of the body's first element.
-template <int DT>
-__device__ __forceinline__ int scan(const uint4 (&a)[kU], int pos, int vi0, int nvec, int idx0, float tau,
-                                    unsigned long long taukey, Smem &S, int nbuf)
+// Merges n candidates with the current list by rank counting; the new list lands in the other
+// buffer.  All keys involved are distinct.  Ends with a barrier.
+__device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n, int k)
 {
-    constexpr int E = Vec<DT>::E;
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const int vi = vi0 + u * kThreads;
-        if (pos < (u + 1) * E && vi < nvec && !(Vec<DT>::vmax(a[u]) < tau)) {
-            float f[E];
-            Vec<DT>::unpack(a[u], f);
-#pragma unroll
-            for (int j = 0; j < E; ++j) {
-                const int o = u * E + j;
-                if (o >= pos && !(f[j] < tau)) {
-                    if (!offer(S, nbuf, f[j], idx0 + vi * E + j, taukey)) return o;
-                }
-            }
-        }
-    }
-    return kU * E;
-}
-
-// Merges the candidates with the current list by rank counting; the new list lands in the
-// other buffer.  All keys involved are distinct.  Ends with a barrier.
-__device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n_raw, int k)
-{
-    const int n = min(n_raw, kCap), m = k + n;
+    const int m = k + n;
     const unsigned long long *top = S.list[cur];
     unsigned long long *out = S.list[cur ^ 1];
-    if (threadIdx.x == 0) S.n[nbuf ^ 1] = 0;
+    if (threadIdx.x == 0) {
+        S.n[nbuf ^ 1] = 0;
+        S.nvalid[nbuf ^ 1] = kNone;
+    }
     for (int i = threadIdx.x; i < m; i += kThreads) {
         const unsigned long long x = i < k ? top[i] : S.cand[i - k];
         int rank = 0;
@@ -195,19 +251,68 @@ __device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n_raw, int
     __syncthreads();
 }
 
+// State of a piece's scan that the iterations share
+struct PieceState {
+    int cur, nbuf;              // list / counter buffers in use
+    float tau;                  // value of the threshold key
+    unsigned long long taukey;  // a key must exceed this to be a candidate
+};
+
+// One iteration: scan the registers, meet, merge when worthwhile; repeats while the buffer overflows.
+template <int DT>
+__device__ __forceinline__ void iteration(const uint4 (&a)[kU], int vi0, int nvec, int idx0, bool last_it, int k,
+                                          PieceState &st, Smem &S)
+{
+    Resume r;
+    r.u = 0;
+    r.hot = 0u;
+    bool resuming = false;
+    for (;;) {
+        resuming = !scan<DT>(a, r, resuming, vi0, nvec, idx0, st.tau, st.taukey, S, st.nbuf);
+        __syncthreads();
+        const int n_raw = S.n[st.nbuf], n_ok = S.nvalid[st.nbuf];
+        const bool overflow = n_ok != kNone;
+        if (n_raw >= kMergeAt || overflow || last_it) {
+            merge(S, st.cur, st.nbuf, overflow ? n_ok : n_raw, k);
+            st.cur ^= 1;
+            st.nbuf ^= 1;
+            const unsigned long long kth = S.list[st.cur][k - 1];
+            if (kth > st.taukey) {
+                st.taukey = kth;
+                st.tau = key_value(kth);
+            }
+        }
+        if (!overflow) break;
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ void load_set(uint4 (&a)[kU], const uint4 *vp, int vfirst, int nvec)
+{
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const int vi = vfirst + u * kThreads;
+        a[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
+    }
+}
+
 // Top-k of elements [e0, e1) of one row into S.list[returned buffer]; S.bad tells whether the
-// piece held a NaN or +inf.  Called by the whole CTA.
+// piece held a NaN or +inf.  Called by the whole CTA, which has met at a barrier since it last
+// touched S.
 template <int DT>
 __device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
 {
     constexpr int E = Vec<DT>::E;
     constexpr int kEsz = Vec<DT>::kEsz;
+    constexpr int kSet = kThreads * kU;  // vectors per iteration
     const int tid = threadIdx.x, lane = tid & 31;
     // empty slots hold distinct small keys (k - r in slot r), below every real key
     if (tid < 32) S.list[0][tid] = tid < k ? (unsigned long long)(k - tid) : 0ull;
     if (tid == 0) {
         S.n[0] = 0;
         S.n[1] = 0;
+        S.nvalid[0] = kNone;
+        S.nvalid[1] = kNone;
         S.bad = 0;
     }
     const uintptr_t addr = reinterpret_cast<uintptr_t>(rowp) + (uintptr_t)e0 * kEsz;
@@ -216,14 +321,10 @@ __device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
     const int idx0 = e0 + head;
     const int tail0 = idx0 + nvec * E;
     const uint4 *vp = reinterpret_cast<const uint4 *>(rowp + (size_t)idx0 * kEsz);
-    const int iters = (nvec + kThreads * kU - 1) / (kThreads * kU);
+    const int iters = (nvec + kSet - 1) / kSet;
 
-    uint4 a[kU];
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const int vi = tid + u * kThreads;
-        a[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
-    }
+    uint4 a[kU], b[kU];
+    load_set<DT>(a, vp, tid, nvec);
     // tau from the first iteration: k-th largest of the 32 group maxima
     float tm = -INFINITY;
 #pragma unroll
@@ -234,10 +335,9 @@ __device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
     tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 1));
     tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 2));
     tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 4));
-    __syncthreads();  // the previous piece's readers of S are done; the init above is visible after the next barrier
     if ((tid & 7) == 0) S.grp[tid >> 3] = tm;
     __syncthreads();
-    float tau;
+    PieceState st;
     {
         const float g = S.grp[lane];
         int rank = 0;
@@ -247,50 +347,30 @@ __device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
             rank += (o > g) || (o == g && j < lane);
         }
         const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
-        tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
+        st.tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
     }
-    unsigned long long taukey = (unsigned long long)ord(tau) << 32;
-    int cur = 0, nbuf = 0;
+    st.taukey = (unsigned long long)ord(st.tau) << 32;
+    st.cur = 0;
+    st.nbuf = 0;
 
     // the ragged ends of the piece, one element per thread
-    if (tid < head) offer(S, nbuf, Vec<DT>::load(rowp, e0 + tid), e0 + tid, taukey);
-    if (tid >= 32 && tid - 32 < e1 - tail0) offer(S, nbuf, Vec<DT>::load(rowp, tail0 + tid - 32), tail0 + tid - 32, taukey);
+    if (tid < head) offer(S, 0, Vec<DT>::load(rowp, e0 + tid), e0 + tid, st.taukey);
+    if (tid >= 32 && tid - 32 < e1 - tail0) offer(S, 0, Vec<DT>::load(rowp, tail0 + tid - 32), tail0 + tid - 32, st.taukey);
 
-    for (int it = 0; it < iters; ++it) {
-        uint4 nx[kU];
-        const int vnext = (it + 1) * kThreads * kU + tid;
-#pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            const int vi = vnext + u * kThreads;
-            nx[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
+    for (int it = 0; it < iters; it += 2) {
+        load_set<DT>(b, vp, (it + 1) * kSet + tid, nvec);
+        iteration<DT>(a, it * kSet + tid, nvec, idx0, it + 1 == iters, k, st, S);
+        if (it + 1 < iters) {
+            load_set<DT>(a, vp, (it + 2) * kSet + tid, nvec);
+            iteration<DT>(b, (it + 1) * kSet + tid, nvec, idx0, it + 2 == iters, k, st, S);
         }
-        const int vi0 = it * kThreads * kU + tid;
-        int pos = 0;
-        for (;;) {
-            pos = scan<DT>(a, pos, vi0, nvec, idx0, tau, taukey, S, nbuf);
-            __syncthreads();
-            const int n = S.n[nbuf];
-            if (n >= kMergeAt || n > kCap || it + 1 == iters) {
-                merge(S, cur, nbuf, n, k);
-                cur ^= 1;
-                nbuf ^= 1;
-                const unsigned long long kth = S.list[cur][k - 1];
-                if (kth > taukey) {
-                    taukey = kth;
-                    tau = key_value(kth);
-                }
-            }
-            if (n <= kCap) break;
-        }
-#pragma unroll
-        for (int u = 0; u < kU; ++u) a[u] = nx[u];
     }
     if (iters == 0) {  // only ragged elements
         __syncthreads();
-        merge(S, cur, nbuf, S.n[nbuf], k);
-        cur ^= 1;
+        merge(S, st.cur, st.nbuf, S.n[st.nbuf], k);
+        st.cur ^= 1;
     }
-    return cur;
+    return st.cur;
 }
 
 // CTA that owns block `blk` when `total` blocks are divided over `grid` CTAs
@@ -358,7 +438,7 @@ __device__ RowDist row_dist(const TopkParams &P, int64_t row, unsigned long long
 }
 
 // The CTA that scanned a sequence's last block: acceptance tests, first rejection, row n's pairs.
-__device__ void fold_sequence(const TopkParams &P, int b, Smem &S)
+__device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gamma = P.gamma, k = P.k;
@@ -410,7 +490,7 @@ __device__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 4) topk_verify_kernel(const __grid_constant__ TopkParams P)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) topk_verify_kernel(const __grid_constant__ TopkParams P)
 {
     __shared__ Smem S;
     const int tid = threadIdx.x, k = P.k;
