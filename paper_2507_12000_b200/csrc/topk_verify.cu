@@ -5,29 +5,38 @@
 // with a selection riding on it:
 //
 //   * Rows are cut into blocks of kTopkBlock entries; the blocks of all rows are numbered row
-//     by row and divided evenly over the CTAs (4 per SM), each CTA owning one contiguous span.
+//     by row and divided evenly over the resident CTAs, each CTA owning one contiguous span.
 //     A span crosses row boundaries, so a CTA works through a few "pieces" (row, first block,
 //     last block); no tickets, no atomics on the streaming path, every CTA ends at the same time.
-//   * A piece is scanned with 16-byte loads, kU vectors per thread in flight plus the next kU
-//     prefetched.  Each vector is reduced to its maximum with NaN-propagating max instructions
-//     and compared with the CTA's threshold tau, a lower bound on the piece's k-th largest
-//     logit; only a vector that reaches tau is taken apart.  Its elements that beat the
-//     current k-th key are appended to a candidate buffer in shared memory.
+//   * Warp specialisation.  One producer thread streams the CTA's span through a ring of
+//     kStages shared-memory stages with bulk asynchronous copies (TMA, untiled) that complete
+//     on "full" mbarriers; the consumer warps read a stage into registers (kU vectors of 16
+//     bytes per thread), scan them and release the stage through an "empty" mbarrier.  Memory
+//     latency is hidden by the rings, not by the consumers; several CTAs share an SM so that
+//     one CTA's barriers and merges overlap with the others' streaming.
+//   * Each vector is reduced to its maximum with NaN-propagating max instructions and compared
+//     with the CTA's threshold tau, a lower bound on the piece's k-th largest logit.  A vector
+//     that reaches tau is taken apart by the whole warp: its 16 bytes are broadcast and lane j
+//     judges element j; the elements that beat the current k-th key are appended to a candidate
+//     buffer in shared memory (one atomic per vector).
 //   * A key is 64 bits: the logit mapped to an unsigned integer that sorts like the float
 //     (with -0 folded into +0), then the complemented index - larger key = earlier in the order
 //     (logit descending, index ascending), and all keys of a row are distinct.
-//   * After every iteration the CTA meets at a barrier; when enough candidates have gathered
-//     it merges them with its current list by rank counting (each key counts the keys above
-//     it; rank < k writes itself to that slot), which needs no sorting network and no second
-//     barrier round.  The threshold lives in registers and is refreshed from the new list.
-//   * tau starts from the first iteration: the 256 threads form 32 groups of 8, each group's
-//     maximum is one distinct element, so the k-th largest group maximum (k <= 32) is a valid
-//     lower bound.  A candidate buffer that overflows anyway (ascending input) is handled by
-//     merging and resuming the same registers from where each thread stopped.
+//   * After every stage the consumers meet at a named barrier; when enough candidates have
+//     gathered they merge them with the current list by rank counting (each key counts the keys
+//     above it; rank < k writes itself to that slot), which needs no sorting network.  The
+//     threshold lives in registers and is refreshed from the new list.
+//   * tau starts from the piece's first stage: the consumer threads form 32 groups,
+//     each group's maximum is one distinct element, so the k-th largest group maximum (k <= 32)
+//     is a valid lower bound.  A candidate buffer that overflows anyway (ascending input) is
+//     handled by merging and resuming the same registers from where each warp stopped.
 //   * The piece's list goes to the workspace; the CTA that completes a sequence (a counter of
 //     scanned blocks per sequence tells) folds it: one warp per row merges the row's pieces,
 //     turns the k logits into probabilities in float64, applies the acceptance test; the first
 //     rejection is an atomicMin in shared memory; warp 0 then writes row n's k pairs.
+//   * Every wait on an mbarrier is bounded; a wait that runs out raises an error word in the
+//     workspace, the kernel runs to its end without faulting and every sequence folded after
+//     that carries DSSD_EDGE_FLAG_TIMEOUT.
 //
 // Device kernel: one warp per sequence, everything in registers and shuffles, sums strictly
 // sequential in float64 so that the draw is reproducible bit for bit.
@@ -40,19 +49,34 @@
 namespace dssd {
 namespace {
 
-#ifndef DSSD_TOPK_U
-#define DSSD_TOPK_U 4
+#ifndef DSSD_TOPK_CONS_WARPS
+#define DSSD_TOPK_CONS_WARPS 8
 #endif
-#ifndef DSSD_TOPK_CTAS
-#define DSSD_TOPK_CTAS 4
+#ifndef DSSD_TOPK_STAGE_BYTES
+#define DSSD_TOPK_STAGE_BYTES 32768
+#endif
+#ifndef DSSD_TOPK_STAGES
+#define DSSD_TOPK_STAGES 3
+#endif
+#ifndef DSSD_TOPK_MIN_CTAS
+#define DSSD_TOPK_MIN_CTAS 2
 #endif
 #ifndef DSSD_TOPK_MERGE_AT
 #define DSSD_TOPK_MERGE_AT 24
 #endif
-constexpr int kU = DSSD_TOPK_U;                // 16-byte vectors per thread per iteration
-constexpr int kCtasPerSm = DSSD_TOPK_CTAS;     // resident CTAs per SM the kernel is compiled for
-constexpr int kCap = 512;                      // candidate buffer entries
-constexpr int kMergeAt = DSSD_TOPK_MERGE_AT;   // merge once this many candidates wait
+constexpr int kConsWarps = DSSD_TOPK_CONS_WARPS;      // consumer warps per CTA (a power of two, 4..16)
+constexpr int kConsThreads = 32 * kConsWarps;
+constexpr int kTkThreads = kConsThreads + 32;        // + the producer warp
+constexpr int kStages = DSSD_TOPK_STAGES;            // ring stages per CTA
+constexpr int kStageBytes = DSSD_TOPK_STAGE_BYTES;   // logits bytes per stage (one bulk copy)
+constexpr int kStageVecs = kStageBytes / 16;         // 16-byte vectors per stage
+constexpr int kU = kStageVecs / kConsThreads;        // vectors per consumer thread per stage
+constexpr int kGroup = kConsThreads / 32;            // threads per group of the first threshold
+static_assert(kU >= 1 && kU * kConsThreads == kStageVecs && kGroup >= 4 && kGroup <= 16, "stage / consumer shape");
+constexpr int kCap = 512;                            // candidate buffer entries
+constexpr int kMergeAt = DSSD_TOPK_MERGE_AT;         // merge once this many candidates wait
+constexpr unsigned kSpinLimit = 1u << 16;            // tries of a bounded wait (about 4 us each)
+constexpr unsigned kSpinLimitAborted = 8u;           // after a wait has run out
 constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
 constexpr unsigned kFullMask = 0xffffffffu;
 
@@ -142,18 +166,38 @@ struct Vec<DSSD_BF16> {
 };
 
 struct Smem {
+    unsigned long long full[kStages];  // mbarriers: stage filled by the copy engine
+    unsigned long long empty[kStages]; // mbarriers: stage read by all consumer warps
     unsigned long long list[2][32];    // the piece's current top-k, best first; two buffers, swapped by each merge
     unsigned long long cand[kCap + 8]; // candidates since the last merge (a vector reserved below kCap may end past it)
-    float grp[32];                     // group maxima of the first iteration
+    float grp[32];                     // group maxima of the piece's first stage
     int n[2];                          // candidate slots reserved (runs past kCap on overflow)
     int nvalid[2];                     // first slot of the first refused reservation (INT_MAX: none)
     int bad;                           // the piece holds a NaN or +inf
-    int last;                          // this CTA scanned the last block of a sequence
+    int fold_b;                        // sequence that this CTA completed and now folds (-1: none)
+    int abort;                         // a bounded wait ran out
     int first_reject;                  // fold: first rejected position
     unsigned fl;                       // fold: flags of the sequence
-    unsigned long long fold_keys[kWarps][kTopkMergeKeys];  // fold: one row's pieces, per warp
-    unsigned long long fold_top[kWarps][32];               // fold: the row's top-k, best first
+    unsigned long long fold_keys[kConsWarps][kTopkMergeKeys];  // fold: one row's pieces, per warp
+    unsigned long long fold_top[kConsWarps][32];               // fold: the row's top-k, best first
 };
+
+// barrier among the consumer warps only (the producer warp never joins)
+__device__ __forceinline__ void cons_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory"); }
+
+// the same barrier, returning to every consumer the number of them that passed a true predicate
+__device__ __forceinline__ int cons_sync_count(bool pred)
+{
+    unsigned r;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.popc.u32 %0, 1, %2, p;\n\t}"
+        : "=r"(r)
+        : "r"((unsigned)pred), "n"(kConsThreads)
+        : "memory");
+    return (int)r;
+}
 
 constexpr int kNone = 0x7fffffff;
 
@@ -178,18 +222,18 @@ struct Resume {
 // whole warp: its 16 bytes are broadcast and lane j judges element j, so a hit costs a few
 // instructions instead of a divergent per-element loop; the slots of a vector are reserved with
 // one shared-memory atomic.  Returns false when a reservation was refused (buffer full): `r`
-// then tells where to resume after the merge.  vi0 = this lane's first vector within the
+// then tells where to resume after the merge.  `asked` grows by the slots the warp asked for.  vi0 = this lane's first vector within the
 // piece's vector body, idx0 = vocabulary index of the body's first element.
 template <int DT>
 __device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resuming, int vi0, int nvec, int idx0,
-                                     float tau, unsigned long long taukey, Smem &S, int nbuf)
+                                     float tau, unsigned long long taukey, Smem &S, int nbuf, int &asked)
 {
     constexpr int E = Vec<DT>::E;
     const int lane = threadIdx.x & 31;
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
         if (u < r.u) continue;
-        const int vi = vi0 + u * kThreads;
+        const int vi = vi0 + u * kConsThreads;
         unsigned hot = __ballot_sync(kFullMask, vi < nvec && !(Vec<DT>::vmax(a[u]) < tau));
         if (resuming && u == r.u) hot = r.hot;
         while (hot) {
@@ -212,6 +256,7 @@ __device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resum
             }
             const unsigned wm = __ballot_sync(kFullMask, want);
             if (wm) {
+                asked += __popc(wm);
                 int base = 0;
                 if (lane == 0) base = atomicAdd(&S.n[nbuf], __popc(wm));
                 base = __shfl_sync(kFullMask, base, 0);
@@ -231,24 +276,29 @@ __device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resum
 }
 
 // Merges n candidates with the current list by rank counting; the new list lands in the other
-// buffer.  All keys involved are distinct.  Ends with a barrier.
+// buffer.  All keys involved are distinct.  One warp per key: the lanes compare 32 keys at a time
+// with it and a ballot counts the larger ones, so there is no chain of dependent loads.  Called
+// by all consumers; ends with their barrier.
 __device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n, int k)
 {
-    const int m = k + n;
+    const int m = k + n, lane = threadIdx.x & 31;
     const unsigned long long *top = S.list[cur];
     unsigned long long *out = S.list[cur ^ 1];
     if (threadIdx.x == 0) {
         S.n[nbuf ^ 1] = 0;
         S.nvalid[nbuf ^ 1] = kNone;
     }
-    for (int i = threadIdx.x; i < m; i += kThreads) {
+    for (int i = threadIdx.x >> 5; i < m; i += kConsWarps) {
         const unsigned long long x = i < k ? top[i] : S.cand[i - k];
         int rank = 0;
-        for (int j = 0; j < k; ++j) rank += top[j] > x;
-        for (int j = 0; j < n; ++j) rank += S.cand[j] > x;
-        if (rank < k) out[rank] = x;
+        for (int j0 = 0; j0 < m; j0 += 32) {
+            const int j = j0 + lane;
+            const unsigned long long y = j < k ? top[j] : (j < m ? S.cand[j - k] : 0ull);
+            rank += __popc(__ballot_sync(kFullMask, y > x));
+        }
+        if (lane == 0 && rank < k) out[rank] = x;
     }
-    __syncthreads();
+    cons_sync();
 }
 
 // State of a piece's scan that the iterations share
@@ -256,55 +306,112 @@ struct PieceState {
     int cur, nbuf;              // list / counter buffers in use
     float tau;                  // value of the threshold key
     unsigned long long taukey;  // a key must exceed this to be a candidate
+    int pending;                // slots asked for since the last merge (the same in every consumer)
 };
 
-// One iteration: scan the registers, meet, merge when worthwhile; repeats while the buffer overflows.
+// One stage: scan the registers, meet, merge when worthwhile; repeats while the buffer overflows.
+// Every decision that the consumers must take alike comes out of the barrier itself (the count
+// of slots asked for, capped at 32 per warp, summed by the barrier) or is read from shared
+// memory at a point where no consumer can be writing it, so that a fast warp that has moved on
+// to the next stage never changes what a slow warp sees.  A refused reservation implies that
+// at least kCap slots were asked for since the last merge, so it always falls in a merge round.
 template <int DT>
 __device__ __forceinline__ void iteration(const uint4 (&a)[kU], int vi0, int nvec, int idx0, bool last_it, int k,
                                           PieceState &st, Smem &S)
 {
+    const int lane = threadIdx.x & 31;
     Resume r;
     r.u = 0;
     r.hot = 0u;
     bool resuming = false;
     for (;;) {
-        resuming = !scan<DT>(a, r, resuming, vi0, nvec, idx0, st.tau, st.taukey, S, st.nbuf);
-        __syncthreads();
+        int asked = 0;
+        resuming = !scan<DT>(a, r, resuming, vi0, nvec, idx0, st.tau, st.taukey, S, st.nbuf, asked);
+        st.pending += cons_sync_count(lane < asked);
+        if (st.pending < kMergeAt && !last_it) break;
         const int n_raw = S.n[st.nbuf], n_ok = S.nvalid[st.nbuf];
         const bool overflow = n_ok != kNone;
-        if (n_raw >= kMergeAt || overflow || last_it) {
-            merge(S, st.cur, st.nbuf, overflow ? n_ok : n_raw, k);
-            st.cur ^= 1;
-            st.nbuf ^= 1;
-            const unsigned long long kth = S.list[st.cur][k - 1];
-            if (kth > st.taukey) {
-                st.taukey = kth;
-                st.tau = key_value(kth);
-            }
+        merge(S, st.cur, st.nbuf, overflow ? n_ok : n_raw, k);
+        st.cur ^= 1;
+        st.nbuf ^= 1;
+        st.pending = 0;
+        const unsigned long long kth = S.list[st.cur][k - 1];
+        if (kth > st.taukey) {
+            st.taukey = kth;
+            st.tau = key_value(kth);
         }
         if (!overflow) break;
     }
 }
 
-template <int DT>
-__device__ __forceinline__ void load_set(uint4 (&a)[kU], const uint4 *vp, int vfirst, int nvec)
-{
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const int vi = vfirst + u * kThreads;
-        a[u] = vi < nvec ? ld_stream16(vp + vi) : Vec<DT>::fill();
-    }
-}
+// Geometry of one piece: elements [e0, e1) of a row = ragged head (up to the first 16-byte
+// boundary), `nvec` whole vectors streamed through the ring in `stages` bulk copies, ragged tail.
+struct Piece {
+    const char *rowp;
+    const uint4 *vp;   // first whole vector
+    int64_t row;
+    int fb, lb;        // blocks [fb, lb) of the row
+    int e0, e1, head, nvec, idx0, tail0, stages;
+};
 
-// Top-k of elements [e0, e1) of one row into S.list[returned buffer]; S.bad tells whether the
-// piece held a NaN or +inf.  Called by the whole CTA, which has met at a barrier since it last
-// touched S.
 template <int DT>
-__device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
+__device__ __forceinline__ Piece piece_at(const TopkParams &P, unsigned long long blk, unsigned long long blk_end)
 {
     constexpr int E = Vec<DT>::E;
     constexpr int kEsz = Vec<DT>::kEsz;
-    constexpr int kSet = kThreads * kU;  // vectors per iteration
+    Piece pc;
+    pc.row = (int64_t)(blk / (unsigned long long)P.nb);
+    pc.fb = (int)(blk - (unsigned long long)pc.row * P.nb);
+    pc.lb = (int)min((unsigned long long)P.nb, pc.fb + (blk_end - blk));
+    pc.e0 = pc.fb * kTopkBlock;
+    pc.e1 = (int)min((long long)P.V, (long long)pc.lb * kTopkBlock);
+    pc.rowp = reinterpret_cast<const char *>(P.logits) + (size_t)pc.row * (size_t)P.row_stride * kEsz;
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(pc.rowp) + (uintptr_t)pc.e0 * kEsz;
+    pc.head = min(pc.e1 - pc.e0, (int)(((16u - (unsigned)(addr & 15u)) & 15u) / kEsz));
+    pc.nvec = (pc.e1 - pc.e0 - pc.head) / E;
+    pc.idx0 = pc.e0 + pc.head;
+    pc.tail0 = pc.idx0 + pc.nvec * E;
+    pc.vp = reinterpret_cast<const uint4 *>(pc.rowp + (size_t)pc.idx0 * kEsz);
+    pc.stages = (pc.nvec + kStageVecs - 1) / kStageVecs;
+    return pc;
+}
+
+// Bounded wait on a ring barrier.  Once a wait has run out the CTA keeps going with short
+// waits, so that it still ends, and reports through the error word.
+__device__ __forceinline__ void ring_wait(const TopkParams &P, Smem &S, unsigned long long *bar, uint32_t parity)
+{
+    const unsigned limit = *reinterpret_cast<volatile int *>(&S.abort) ? kSpinLimitAborted : kSpinLimit;
+    if (!mbar_wait(smem_addr(bar), parity, limit)) {
+        *reinterpret_cast<volatile int *>(&S.abort) = 1;
+        atomicExch(P.error, 1u);
+    }
+}
+
+// The producer thread: streams the CTA's span, stage by stage, in the order the consumers read it.
+template <int DT>
+__device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, unsigned long long blk, unsigned long long blk_end)
+{
+    unsigned q = 0;  // stages issued so far
+    while (blk < blk_end) {
+        const Piece pc = piece_at<DT>(P, blk, blk_end);
+        for (int s = 0; s < pc.stages; ++s, ++q) {
+            const unsigned slot = q % kStages, pass = q / kStages;
+            if (pass > 0) ring_wait(P, S, &S.empty[slot], (pass - 1u) & 1u);
+            const uint32_t bytes = (uint32_t)min(kStageVecs, pc.nvec - s * kStageVecs) * 16u;
+            const uint32_t bar = smem_addr(&S.full[slot]);
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_g2s(ring + slot * (uint32_t)kStageBytes, pc.vp + (size_t)s * kStageVecs, bytes, bar);
+        }
+        blk += (unsigned long long)(pc.lb - pc.fb);
+    }
+}
+
+// Top-k of one piece into S.list[returned buffer]; S.bad tells whether the piece held a NaN or
+// +inf.  Called by all consumers, which have met at their barrier since they last touched S.
+// `q` counts the stages consumed so far (the ring position), as the producer counts them.
+template <int DT>
+__device__ int piece_topk(const TopkParams &P, const Piece &pc, int k, Smem &S, uint32_t ring, unsigned &q)
+{
     const int tid = threadIdx.x, lane = tid & 31;
     // empty slots hold distinct small keys (k - r in slot r), below every real key
     if (tid < 32) S.list[0][tid] = tid < k ? (unsigned long long)(k - tid) : 0ull;
@@ -315,58 +422,59 @@ __device__ int piece_topk(const char *rowp, int e0, int e1, int k, Smem &S)
         S.nvalid[1] = kNone;
         S.bad = 0;
     }
-    const uintptr_t addr = reinterpret_cast<uintptr_t>(rowp) + (uintptr_t)e0 * kEsz;
-    const int head = min(e1 - e0, (int)(((16u - (unsigned)(addr & 15u)) & 15u) / kEsz));
-    const int nvec = (e1 - e0 - head) / E;
-    const int idx0 = e0 + head;
-    const int tail0 = idx0 + nvec * E;
-    const uint4 *vp = reinterpret_cast<const uint4 *>(rowp + (size_t)idx0 * kEsz);
-    const int iters = (nvec + kSet - 1) / kSet;
-
-    uint4 a[kU], b[kU];
-    load_set<DT>(a, vp, tid, nvec);
-    // tau from the first iteration: k-th largest of the 32 group maxima
-    float tm = -INFINITY;
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const float v = Vec<DT>::vmax(a[u]);
-        tm = fmaxf(tm, v == v ? v : -INFINITY);
-    }
-    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 1));
-    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 2));
-    tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, 4));
-    if ((tid & 7) == 0) S.grp[tid >> 3] = tm;
-    __syncthreads();
     PieceState st;
-    {
-        const float g = S.grp[lane];
-        int rank = 0;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float o = __shfl_sync(kFullMask, g, j);
-            rank += (o > g) || (o == g && j < lane);
-        }
-        const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
-        st.tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
-    }
-    st.taukey = (unsigned long long)ord(st.tau) << 32;
     st.cur = 0;
     st.nbuf = 0;
-
-    // the ragged ends of the piece, one element per thread
-    if (tid < head) offer(S, 0, Vec<DT>::load(rowp, e0 + tid), e0 + tid, st.taukey);
-    if (tid >= 32 && tid - 32 < e1 - tail0) offer(S, 0, Vec<DT>::load(rowp, tail0 + tid - 32), tail0 + tid - 32, st.taukey);
-
-    for (int it = 0; it < iters; it += 2) {
-        load_set<DT>(b, vp, (it + 1) * kSet + tid, nvec);
-        iteration<DT>(a, it * kSet + tid, nvec, idx0, it + 1 == iters, k, st, S);
-        if (it + 1 < iters) {
-            load_set<DT>(a, vp, (it + 2) * kSet + tid, nvec);
-            iteration<DT>(b, (it + 1) * kSet + tid, nvec, idx0, it + 2 == iters, k, st, S);
+    st.pending = 0;
+    st.tau = -INFINITY;
+    for (int s = 0; s < pc.stages; ++s, ++q) {
+        const unsigned slot = q % kStages, pass = q / kStages;
+        ring_wait(P, S, &S.full[slot], pass & 1u);
+        uint4 a[kU];
+        const int vi0 = s * kStageVecs + tid;
+        const uint32_t src = ring + slot * (uint32_t)kStageBytes + (uint32_t)tid * 16u;
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+            a[u] = vi0 + u * kConsThreads < pc.nvec ? lds16(src + (uint32_t)u * kConsThreads * 16u) : Vec<DT>::fill();
+        if (s == 0) {
+            // tau from the first stage: k-th largest of the 32 group maxima
+            float tm = -INFINITY;
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const float v = Vec<DT>::vmax(a[u]);
+                tm = fmaxf(tm, v == v ? v : -INFINITY);
+            }
+#pragma unroll
+            for (int o = 1; o < kGroup; o <<= 1) tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, o));
+            if ((tid & (kGroup - 1)) == 0) S.grp[tid / kGroup] = tm;
+            cons_sync();
+            const float g = S.grp[lane];
+            int rank = 0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float o = __shfl_sync(kFullMask, g, j);
+                rank += (o > g) || (o == g && j < lane);
+            }
+            const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
+            st.tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
+            st.taukey = (unsigned long long)ord(st.tau) << 32;
+            // the ragged ends of the piece, one element per thread
+            if (tid < pc.head) offer(S, 0, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, st.taukey);
+            if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
+                offer(S, 0, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, st.taukey);
         }
+        iteration<DT>(a, vi0, pc.nvec, pc.idx0, s + 1 == pc.stages, k, st, S);
+        // the stage has been consumed from registers: hand the buffer back to the producer
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_addr(&S.empty[slot]));
     }
-    if (iters == 0) {  // only ragged elements
-        __syncthreads();
+    if (pc.stages == 0) {  // only ragged elements
+        cons_sync();
+        st.taukey = 0ull;
+        if (tid < pc.head) offer(S, 0, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, st.taukey);
+        if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
+            offer(S, 0, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, st.taukey);
+        cons_sync();
         merge(S, st.cur, st.nbuf, S.n[st.nbuf], k);
         st.cur ^= 1;
     }
@@ -438,16 +546,17 @@ __device__ RowDist row_dist(const TopkParams &P, int64_t row, unsigned long long
 }
 
 // The CTA that scanned a sequence's last block: acceptance tests, first rejection, row n's pairs.
+// Called by all consumers.
 __device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gamma = P.gamma, k = P.k;
     if (tid == 0) {
         S.first_reject = gamma;
-        S.fl = 0u;
+        S.fl = ld_relaxed_u32(P.error) ? DSSD_EDGE_FLAG_TIMEOUT : 0u;
     }
-    __syncthreads();
-    for (int j = warp; j <= gamma; j += kWarps) {
+    cons_sync();
+    for (int j = warp; j <= gamma; j += kConsWarps) {
         const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + j, S.fold_keys[warp], S.fold_top[warp]);
         if (d.bad && lane == 0) atomicOr(&S.fl, DSSD_EDGE_FLAG_NONFINITE);
         if (j == gamma) continue;
@@ -474,7 +583,7 @@ __device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
             if (!accept) atomicMin(&S.first_reject, j);
         }
     }
-    __syncthreads();
+    cons_sync();
     const int n = S.first_reject;
     if (warp == 0) {
         const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + n, S.fold_keys[0], S.fold_top[0]);
@@ -490,42 +599,68 @@ __device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) topk_verify_kernel(const __grid_constant__ TopkParams P)
+__global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_kernel(const __grid_constant__ TopkParams P)
 {
-    __shared__ Smem S;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Smem &S = *reinterpret_cast<Smem *>(smem_raw + (size_t)kStages * kStageBytes);
+    const uint32_t ring = smem_addr(smem_raw);
     const int tid = threadIdx.x, k = P.k;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_addr(&S.full[s]), 1u);
+            mbar_init(smem_addr(&S.empty[s]), (uint32_t)kConsWarps);
+        }
+        S.abort = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
     const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
     const unsigned long long blk_end = (c + 1ull) * TB / G;
-    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
     unsigned long long blk = c * TB / G;
+    if (tid >= kConsThreads) {
+        if (tid == kConsThreads) producer<DT>(P, S, ring, blk, blk_end);
+        return;
+    }
+    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
+    unsigned q = 0;
+    // The sequence counter's answer is not waited for: thread 0 looks at it one piece later.
+    unsigned long long prev_sum = 0ull;  // thread 0: counter value after the previous piece's blocks
+    int prev_b = -1;
     while (blk < blk_end) {
-        const int64_t row = (int64_t)(blk / (unsigned long long)P.nb);
-        const int fb = (int)(blk - (unsigned long long)row * P.nb);
-        const int lb = (int)min((unsigned long long)P.nb, fb + (blk_end - blk));
-        const int e0 = fb * kTopkBlock, e1 = (int)min((long long)P.V, (long long)lb * kTopkBlock);
-        const char *rowp = reinterpret_cast<const char *>(P.logits) + (size_t)row * (size_t)P.row_stride * Vec<DT>::kEsz;
-        const int cur = piece_topk<DT>(rowp, e0, e1, k, S);
-        const int slot = (int)(c - owner_of((unsigned long long)row * P.nb, G, TB));
-        if (tid < k) {
-            unsigned long long key = S.list[cur][tid];
-            if (S.bad) key = tid == 0 ? kBadList : 0ull;
-            __stcg(P.lists + ((size_t)row * P.max_pieces + slot) * k + tid, key);
-        }
-        __threadfence();
-        __syncthreads();
-        const int b = (int)(row / (P.gamma + 1));
-        if (tid == 0) {
-            const unsigned long long done = (unsigned long long)(lb - fb);
-            const unsigned long long old = atomicAdd(P.seq_done + b, done);
-            S.last = (old + done == per_seq);
-        }
-        __syncthreads();
-        if (S.last) {
+        const Piece pc = piece_at<DT>(P, blk, blk_end);
+        const int cur = piece_topk<DT>(P, pc, k, S, ring, q);
+        const int b = (int)(pc.row / (P.gamma + 1));
+        if (tid < 32) {
+            // warp 0 publishes the piece: list, fence, then the blocks are counted
+            const int slot = (int)(c - owner_of((unsigned long long)pc.row * P.nb, G, TB));
+            if (tid < k) {
+                unsigned long long key = S.list[cur][tid];
+                if (S.bad) key = tid == 0 ? kBadList : 0ull;
+                __stcg(P.lists + ((size_t)pc.row * P.max_pieces + slot) * k + tid, key);
+            }
             __threadfence();
-            fold_sequence(P, b, S);
+            __syncwarp();
+            if (tid == 0) {
+                S.fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
+                const unsigned long long done = (unsigned long long)(pc.lb - pc.fb);
+                prev_sum = atomicAdd(P.seq_done + b, done) + done;
+                prev_b = b;
+            }
         }
-        __syncthreads();
-        blk += (unsigned long long)(lb - fb);
+        cons_sync();
+        const int fb = S.fold_b;
+        if (fb >= 0) {
+            __threadfence();
+            fold_sequence(P, fb, S);
+            cons_sync();
+        }
+        blk += (unsigned long long)(pc.lb - pc.fb);
+    }
+    if (tid == 0) S.fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
+    cons_sync();
+    if (S.fold_b >= 0) {
+        __threadfence();
+        fold_sequence(P, S.fold_b, S);
     }
 }
 
@@ -621,18 +756,20 @@ int topk_max_pieces(int k)
 size_t topk_workspace_layout(int B, int gamma, int k, TopkParams *P, char *base)
 {
     const size_t rows = (size_t)B * (size_t)(gamma + 1);
-    const size_t cnt = ((size_t)B * 8 + 255) & ~(size_t)255;
+    const size_t cnt = (8 + (size_t)B * 8 + 255) & ~(size_t)255;
     const size_t lists = rows * (size_t)topk_max_pieces(k) * (size_t)k * 8;
     if (P) {
-        P->seq_done = reinterpret_cast<unsigned long long *>(base);
+        P->error = reinterpret_cast<unsigned *>(base);
+        P->seq_done = reinterpret_cast<unsigned long long *>(base + 8);
         P->lists = reinterpret_cast<unsigned long long *>(base + cnt);
-        P->zero_bytes = (size_t)B * 8;
+        P->zero_bytes = 8 + (size_t)B * 8;
         P->max_pieces = topk_max_pieces(k);
     }
     return cnt + ((lists + 255) & ~(size_t)255);
 }
 
-static int g_topk_ctas[64];  // resident CTAs of the kernel per device (0 = not asked yet)
+static int g_topk_ctas[64];  // CTAs resident on the device at once (0 = not asked yet)
+constexpr size_t kTopkSmemBytes = (size_t)kStages * kStageBytes + sizeof(Smem);
 
 cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaStream_t stream)
 {
@@ -641,12 +778,15 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     int ctas = (dev >= 0 && dev < 64) ? g_topk_ctas[dev] : 0;
     if (ctas == 0) {
-        int sms = 0, occ0 = 0, occ1 = 0;
+        int sms = 0;
         if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, topk_verify_kernel<DSSD_F32>, kThreads, 0)) != cudaSuccess) return err;
-        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, topk_verify_kernel<DSSD_BF16>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaFuncSetAttribute(topk_verify_kernel<DSSD_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmemBytes)) != cudaSuccess) return err;
+        if ((err = cudaFuncSetAttribute(topk_verify_kernel<DSSD_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTopkSmemBytes)) != cudaSuccess) return err;
+        int occ0 = 0, occ1 = 0;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, topk_verify_kernel<DSSD_F32>, kTkThreads, kTopkSmemBytes)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, topk_verify_kernel<DSSD_BF16>, kTkThreads, kTopkSmemBytes)) != cudaSuccess) return err;
         const int occ = occ0 < occ1 ? occ0 : occ1;
-        ctas = sms * (occ < 1 ? 1 : occ);
+        ctas = (sms < 1 ? 1 : sms) * (occ < 1 ? 1 : occ);
         if (dev >= 0 && dev < 64) g_topk_ctas[dev] = ctas;
     }
     topk_workspace_layout(P.B, P.gamma, P.k, &P, static_cast<char *>(workspace));
@@ -660,11 +800,11 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
     if (grid > (unsigned long long)ctas) grid = (unsigned long long)ctas;
     if (grid < 1) grid = 1;
     P.grid = (int)grid;
-    if ((err = cudaMemsetAsync(P.seq_done, 0, P.zero_bytes, stream)) != cudaSuccess) return err;
+    if ((err = cudaMemsetAsync(P.error, 0, P.zero_bytes, stream)) != cudaSuccess) return err;
     if (dtype == DSSD_BF16)
-        topk_verify_kernel<DSSD_BF16><<<P.grid, kThreads, 0, stream>>>(P);
+        topk_verify_kernel<DSSD_BF16><<<P.grid, kTkThreads, kTopkSmemBytes, stream>>>(P);
     else
-        topk_verify_kernel<DSSD_F32><<<P.grid, kThreads, 0, stream>>>(P);
+        topk_verify_kernel<DSSD_F32><<<P.grid, kTkThreads, kTopkSmemBytes, stream>>>(P);
     return cudaGetLastError();
 }
 
