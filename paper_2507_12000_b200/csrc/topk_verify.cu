@@ -15,28 +15,30 @@
 //     latency is hidden by the rings, not by the consumers; several CTAs share an SM so that
 //     one CTA's barriers and merges overlap with the others' streaming.
 //   * Each vector is reduced to its maximum with NaN-propagating max instructions and compared
-//     with the CTA's threshold tau, a lower bound on the piece's k-th largest logit.  A vector
+//     with the warp's threshold tau, a lower bound on the piece's k-th largest logit.  A vector
 //     that reaches tau is taken apart by the whole warp: its 16 bytes are broadcast and lane j
-//     judges element j; the elements that beat the current k-th key are appended to a candidate
-//     buffer in shared memory (one atomic per vector).
+//     judges element j; the elements that beat the threshold key go into a queue in shared
+//     memory (one atomic per vector).  The consumers never meet at a barrier within a piece.
 //   * A key is 64 bits: the logit mapped to an unsigned integer that sorts like the float
 //     (with -0 folded into +0), then the complemented index - larger key = earlier in the order
 //     (logit descending, index ascending), and all keys of a row are distinct.
-//   * After every stage the consumers meet at a named barrier; when enough candidates have
-//     gathered they merge them with the current list by rank counting (each key counts the keys
-//     above it; rank < k writes itself to that slot), which needs no sorting network.  The
-//     threshold lives in registers and is refreshed from the new list.
-//   * tau starts from the piece's first stage: the consumer threads form 32 groups,
-//     each group's maximum is one distinct element, so the k-th largest group maximum (k <= 32)
-//     is a valid lower bound.  A candidate buffer that overflows anyway (ascending input) is
-//     handled by merging and resuming the same registers from where each warp stopped.
-//   * The piece's list goes to the workspace; the CTA that completes a sequence (a counter of
-//     scanned blocks per sequence tells) folds it: one warp per row merges the row's pieces,
-//     turns the k logits into probabilities in float64, applies the acceptance test; the first
-//     rejection is an atomicMin in shared memory; warp 0 then writes row n's k pairs.
-//   * Every wait on an mbarrier is bounded; a wait that runs out raises an error word in the
-//     workspace, the kernel runs to its end without faulting and every sequence folded after
-//     that carries DSSD_EDGE_FLAG_TIMEOUT.
+//   * A selection warp drains the queue.  Lane r holds entry r of the piece's list, best first;
+//     a candidate is inserted with one ballot (its position) and one shuffle (the shift), and
+//     the k-th key is published in shared memory, where the consumers pick it up at their next
+//     stage.  No sorting network, no merge rounds.
+//   * tau starts from the piece's first stage: the consumer threads form 32 groups, each
+//     group's maximum is one distinct element, so the k-th largest group maximum (k <= 32) is a
+//     valid lower bound.  On input that defeats the threshold (an ascending row) every element
+//     goes through the queue: slow, never wrong; a full queue makes the consumers wait.
+//   * At the end of a piece the selection warp lets the consumers go on with the next one and
+//     only then writes the list to the workspace and counts the piece's blocks; the CTA that
+//     completes a sequence folds it in the same warp: the rows' pieces are merged by rank
+//     counting, the k logits become probabilities in float64, the acceptance test runs, row n's
+//     k pairs are written.  The counter's answer is looked at one piece later, so nobody waits
+//     for the round trip.
+//   * Every wait (mbarrier, queue, barrier hand-off) is bounded; a wait that runs out raises an
+//     error word in the workspace, the kernel runs to its end without faulting and every
+//     sequence folded after that carries DSSD_EDGE_FLAG_TIMEOUT.
 //
 // Device kernel: one warp per sequence, everything in registers and shuffles, sums strictly
 // sequential in float64 so that the draw is reproducible bit for bit.
@@ -61,20 +63,19 @@ namespace {
 #ifndef DSSD_TOPK_MIN_CTAS
 #define DSSD_TOPK_MIN_CTAS 2
 #endif
-#ifndef DSSD_TOPK_MERGE_AT
-#define DSSD_TOPK_MERGE_AT 24
-#endif
 constexpr int kConsWarps = DSSD_TOPK_CONS_WARPS;      // consumer warps per CTA (a power of two, 4..16)
 constexpr int kConsThreads = 32 * kConsWarps;
-constexpr int kTkThreads = kConsThreads + 32;        // + the producer warp
+constexpr int kTkThreads = kConsThreads + 64;        // + the producer warp and the selection warp
 constexpr int kStages = DSSD_TOPK_STAGES;            // ring stages per CTA
 constexpr int kStageBytes = DSSD_TOPK_STAGE_BYTES;   // logits bytes per stage (one bulk copy)
 constexpr int kStageVecs = kStageBytes / 16;         // 16-byte vectors per stage
 constexpr int kU = kStageVecs / kConsThreads;        // vectors per consumer thread per stage
 constexpr int kGroup = kConsThreads / 32;            // threads per group of the first threshold
 static_assert(kU >= 1 && kU * kConsThreads == kStageVecs && kGroup >= 4 && kGroup <= 16, "stage / consumer shape");
-constexpr int kCap = 512;                            // candidate buffer entries
-constexpr int kMergeAt = DSSD_TOPK_MERGE_AT;         // merge once this many candidates wait
+#ifndef DSSD_TOPK_QUEUE
+#define DSSD_TOPK_QUEUE 256
+#endif
+constexpr int kCap = DSSD_TOPK_QUEUE;                // candidate queue entries per channel (a power of two)
 constexpr unsigned kSpinLimit = 1u << 16;            // tries of a bounded wait (about 4 us each)
 constexpr unsigned kSpinLimitAborted = 8u;           // after a wait has run out
 constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
@@ -138,6 +139,13 @@ struct Vec<DSSD_F32> {
     {
         return __uint_as_float(j < 2 ? (j == 0 ? v.x : v.y) : (j == 2 ? v.z : v.w));
     }
+    // a vector whose element 0 is the element at `row[i]`
+    __device__ static __forceinline__ uint4 single(const void *row, int64_t i)
+    {
+        uint4 v = fill();
+        v.x = reinterpret_cast<const uint32_t *>(row)[i];
+        return v;
+    }
 };
 template <>
 struct Vec<DSSD_BF16> {
@@ -163,79 +171,116 @@ struct Vec<DSSD_BF16> {
         const uint32_t w = j < 4 ? (j < 2 ? v.x : v.y) : (j < 6 ? v.z : v.w);
         return (j & 1) ? bf16_hi(w) : bf16_lo(w);
     }
+    __device__ static __forceinline__ uint4 single(const void *row, int64_t i)
+    {
+        uint4 v = fill();
+        v.x = 0xff800000u | (uint32_t)reinterpret_cast<const unsigned short *>(row)[i];
+        return v;
+    }
+};
+
+// What the consumers and the selection warp share for one piece.  There are two of them, used
+// by even and odd pieces, so that the consumers can scan a piece while the selection warp is
+// still finishing the one before.
+struct Channel {
+    unsigned long long queue[kCap];     // candidate keys on their way to the selection warp; 0 = free slot
+    unsigned long long taukey;          // the selection warp's current k-th key (0: list not full yet)
+    unsigned q_head;                    // slots reserved by the consumers (counts up for the kernel's life)
+    unsigned q_tail;                    // slots the selection warp has taken
+    unsigned done;                      // consumer warps that have finished the piece
+    int bad;                            // the piece holds a NaN or +inf
 };
 
 struct Smem {
-    unsigned long long full[kStages];  // mbarriers: stage filled by the copy engine
-    unsigned long long empty[kStages]; // mbarriers: stage read by all consumer warps
-    unsigned long long list[2][32];    // the piece's current top-k, best first; two buffers, swapped by each merge
-    unsigned long long cand[kCap + 8]; // candidates since the last merge (a vector reserved below kCap may end past it)
-    float grp[32];                     // group maxima of the piece's first stage
-    int n[2];                          // candidate slots reserved (runs past kCap on overflow)
-    int nvalid[2];                     // first slot of the first refused reservation (INT_MAX: none)
-    int bad;                           // the piece holds a NaN or +inf
-    int fold_b;                        // sequence that this CTA completed and now folds (-1: none)
-    int abort;                         // a bounded wait ran out
-    int first_reject;                  // fold: first rejected position
-    unsigned fl;                       // fold: flags of the sequence
-    unsigned long long fold_keys[kConsWarps][kTopkMergeKeys];  // fold: one row's pieces, per warp
-    unsigned long long fold_top[kConsWarps][32];               // fold: the row's top-k, best first
+    unsigned long long full[kStages];   // mbarriers: stage filled by the copy engine
+    unsigned long long empty[kStages];  // mbarriers: stage read by all consumer warps
+    Channel ch[2];
+    float grp[2][32];                   // group maxima of a piece's first stage (by piece parity)
+    int abort;                          // a bounded wait ran out
+    unsigned long long fold_keys[kTopkMergeKeys];  // fold: one row's pieces
+    unsigned long long fold_top[32];               // fold: the row's top-k, best first
 };
 
-// barrier among the consumer warps only (the producer warp never joins)
-__device__ __forceinline__ void cons_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads) : "memory"); }
-
-// the same barrier, returning to every consumer the number of them that passed a true predicate
-__device__ __forceinline__ int cons_sync_count(bool pred)
+// Piece boundary (one named barrier per piece parity): before scanning piece j the consumers
+// wait here for each other and for the selection warp to have finished piece j - 2, which used
+// the same channel; the selection warp only arrives and goes on.
+__device__ __forceinline__ void boundary_sync(int parity)
 {
-    unsigned r;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.popc.u32 %0, 1, %2, p;\n\t}"
-        : "=r"(r)
-        : "r"((unsigned)pred), "n"(kConsThreads)
-        : "memory");
-    return (int)r;
+    if (parity) asm volatile("bar.sync 2, %0;" ::"n"(kConsThreads + 32) : "memory");
+    else asm volatile("bar.sync 1, %0;" ::"n"(kConsThreads + 32) : "memory");
+}
+__device__ __forceinline__ void boundary_arrive(int parity)
+{
+    if (parity) asm volatile("bar.arrive 2, %0;" ::"n"(kConsThreads + 32) : "memory");
+    else asm volatile("bar.arrive 1, %0;" ::"n"(kConsThreads + 32) : "memory");
 }
 
-constexpr int kNone = 0x7fffffff;
+// acquire-release fences (the sequentially consistent ones that __threadfence*() emit cost a
+// pipeline drain each, which the selection warp cannot afford once per batch)
+__device__ __forceinline__ void fence_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 
-// One element of a piece's ragged ends (called before the first scan, when the buffer is empty)
-__device__ __forceinline__ void offer(Smem &S, int nbuf, float f, int idx, unsigned long long taukey)
+__device__ __forceinline__ unsigned ld_shared_volatile_u32(const unsigned *p) { return *reinterpret_cast<const volatile unsigned *>(p); }
+__device__ __forceinline__ unsigned long long ld_shared_volatile_u64(const unsigned long long *p)
+{
+    return *reinterpret_cast<const volatile unsigned long long *>(p);
+}
+
+__device__ __forceinline__ void raise_abort(const TopkParams &P, Smem &S)
+{
+    *reinterpret_cast<volatile int *>(&S.abort) = 1;
+    atomicExch(P.error, 1u);
+}
+
+// Writes a key into its reserved queue position once the selection warp has freed the slot (it
+// is at most kCap positions behind).  Bounded; a key that cannot be delivered is dropped and
+// the error word is raised.
+__device__ __forceinline__ void deliver(const TopkParams &P, Smem &S, Channel &C, unsigned pos, unsigned long long key)
+{
+    unsigned it = 0;
+    while (pos - ld_shared_volatile_u32(&C.q_tail) >= (unsigned)kCap) {
+        if (++it > kSpinLimit * 64u || *reinterpret_cast<volatile int *>(&S.abort)) {
+            raise_abort(P, S);
+            return;
+        }
+        __nanosleep(64);
+    }
+    *reinterpret_cast<volatile unsigned long long *>(&C.queue[pos % kCap]) = key;
+}
+
+// One element of a piece's ragged ends
+__device__ __forceinline__ void offer(const TopkParams &P, Smem &S, Channel &C, float f, int idx, unsigned long long taukey)
 {
     if (f != f || f == INFINITY) {
-        S.bad = 1;
+        C.bad = 1;
         return;
     }
     const unsigned long long key = make_key(f, idx);
-    if (key > taukey) S.cand[atomicAdd(&S.n[nbuf], 1)] = key;
+    if (key > taukey) deliver(P, S, C, atomicAdd(&C.q_head, 1u), key);
 }
 
-// Where a warp stopped when the candidate buffer was full
-struct Resume {
-    int u;          // vector of the iteration (kU: the warp is done)
-    unsigned hot;   // lanes of that vector still to be taken apart
-};
-
-// Scans the warp's kU x 32 vectors.  A vector whose maximum reaches tau is taken apart by the
-// whole warp: its 16 bytes are broadcast and lane j judges element j, so a hit costs a few
-// instructions instead of a divergent per-element loop; the slots of a vector are reserved with
-// one shared-memory atomic.  Returns false when a reservation was refused (buffer full): `r`
-// then tells where to resume after the merge.  `asked` grows by the slots the warp asked for.  vi0 = this lane's first vector within the
-// piece's vector body, idx0 = vocabulary index of the body's first element.
+// Scans the warp's kU x 32 vectors of one stage.  One vote settles the common case that nothing
+// reaches tau.  Otherwise a vector whose maximum (NaN-propagating) reaches tau is taken apart
+// by the whole warp: its 16 bytes are broadcast and lane j judges element j; the queue slots of
+// a vector are reserved with one shared-memory atomic.  vi0 = this lane's first vector within
+// the piece's vector body, idx0 = vocabulary index of the body's first element.
 template <int DT>
-__device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resuming, int vi0, int nvec, int idx0,
-                                     float tau, unsigned long long taukey, Smem &S, int nbuf, int &asked)
+__device__ __forceinline__ void scan(const TopkParams &P, const uint4 (&a)[kU], int vi0, int nvec, int idx0, float tau,
+                                     unsigned long long taukey, Smem &S, Channel &C)
 {
     constexpr int E = Vec<DT>::E;
     const int lane = threadIdx.x & 31;
+    float vm[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) vm[u] = Vec<DT>::vmax(a[u]);
+    float top = vm[0];
+#pragma unroll
+    for (int u = 1; u < kU; ++u) top = max_nan(top, vm[u]);
+    if (!__any_sync(kFullMask, !(top < tau))) return;
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-        if (u < r.u) continue;
         const int vi = vi0 + u * kConsThreads;
-        unsigned hot = __ballot_sync(kFullMask, vi < nvec && !(Vec<DT>::vmax(a[u]) < tau));
-        if (resuming && u == r.u) hot = r.hot;
+        unsigned hot = __ballot_sync(kFullMask, vi < nvec && !(vm[u] < tau));
         while (hot) {
             const int src = __ffs(hot) - 1;
             uint4 v;
@@ -248,7 +293,7 @@ __device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resum
             unsigned long long key = 0ull;
             if (lane < E && !(f < tau)) {
                 if (f != f || f == INFINITY) {
-                    S.bad = 1;
+                    C.bad = 1;
                 } else {
                     key = make_key(f, idx0 + (vi - lane + src) * E + lane);
                     want = key > taukey;
@@ -256,91 +301,13 @@ __device__ __forceinline__ bool scan(const uint4 (&a)[kU], Resume &r, bool resum
             }
             const unsigned wm = __ballot_sync(kFullMask, want);
             if (wm) {
-                asked += __popc(wm);
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&S.n[nbuf], __popc(wm));
+                unsigned base = 0u;
+                if (lane == 0) base = atomicAdd(&C.q_head, (unsigned)__popc(wm));
                 base = __shfl_sync(kFullMask, base, 0);
-                if (base >= kCap) {
-                    if (lane == 0) atomicMin(&S.nvalid[nbuf], base);
-                    r.u = u;
-                    r.hot = hot;
-                    return false;
-                }
-                if (want) S.cand[base + __popc(wm & ((1u << lane) - 1u))] = key;
+                if (want) deliver(P, S, C, base + (unsigned)__popc(wm & ((1u << lane) - 1u)), key);
             }
             hot &= hot - 1u;
         }
-    }
-    r.u = kU;
-    return true;
-}
-
-// Merges n candidates with the current list by rank counting; the new list lands in the other
-// buffer.  All keys involved are distinct.  One warp per key: the lanes compare 32 keys at a time
-// with it and a ballot counts the larger ones, so there is no chain of dependent loads.  Called
-// by all consumers; ends with their barrier.
-__device__ __forceinline__ void merge(Smem &S, int cur, int nbuf, int n, int k)
-{
-    const int m = k + n, lane = threadIdx.x & 31;
-    const unsigned long long *top = S.list[cur];
-    unsigned long long *out = S.list[cur ^ 1];
-    if (threadIdx.x == 0) {
-        S.n[nbuf ^ 1] = 0;
-        S.nvalid[nbuf ^ 1] = kNone;
-    }
-    for (int i = threadIdx.x >> 5; i < m; i += kConsWarps) {
-        const unsigned long long x = i < k ? top[i] : S.cand[i - k];
-        int rank = 0;
-        for (int j0 = 0; j0 < m; j0 += 32) {
-            const int j = j0 + lane;
-            const unsigned long long y = j < k ? top[j] : (j < m ? S.cand[j - k] : 0ull);
-            rank += __popc(__ballot_sync(kFullMask, y > x));
-        }
-        if (lane == 0 && rank < k) out[rank] = x;
-    }
-    cons_sync();
-}
-
-// State of a piece's scan that the iterations share
-struct PieceState {
-    int cur, nbuf;              // list / counter buffers in use
-    float tau;                  // value of the threshold key
-    unsigned long long taukey;  // a key must exceed this to be a candidate
-    int pending;                // slots asked for since the last merge (the same in every consumer)
-};
-
-// One stage: scan the registers, meet, merge when worthwhile; repeats while the buffer overflows.
-// Every decision that the consumers must take alike comes out of the barrier itself (the count
-// of slots asked for, capped at 32 per warp, summed by the barrier) or is read from shared
-// memory at a point where no consumer can be writing it, so that a fast warp that has moved on
-// to the next stage never changes what a slow warp sees.  A refused reservation implies that
-// at least kCap slots were asked for since the last merge, so it always falls in a merge round.
-template <int DT>
-__device__ __forceinline__ void iteration(const uint4 (&a)[kU], int vi0, int nvec, int idx0, bool last_it, int k,
-                                          PieceState &st, Smem &S)
-{
-    const int lane = threadIdx.x & 31;
-    Resume r;
-    r.u = 0;
-    r.hot = 0u;
-    bool resuming = false;
-    for (;;) {
-        int asked = 0;
-        resuming = !scan<DT>(a, r, resuming, vi0, nvec, idx0, st.tau, st.taukey, S, st.nbuf, asked);
-        st.pending += cons_sync_count(lane < asked);
-        if (st.pending < kMergeAt && !last_it) break;
-        const int n_raw = S.n[st.nbuf], n_ok = S.nvalid[st.nbuf];
-        const bool overflow = n_ok != kNone;
-        merge(S, st.cur, st.nbuf, overflow ? n_ok : n_raw, k);
-        st.cur ^= 1;
-        st.nbuf ^= 1;
-        st.pending = 0;
-        const unsigned long long kth = S.list[st.cur][k - 1];
-        if (kth > st.taukey) {
-            st.taukey = kth;
-            st.tau = key_value(kth);
-        }
-        if (!overflow) break;
     }
 }
 
@@ -381,10 +348,7 @@ __device__ __forceinline__ Piece piece_at(const TopkParams &P, unsigned long lon
 __device__ __forceinline__ void ring_wait(const TopkParams &P, Smem &S, unsigned long long *bar, uint32_t parity)
 {
     const unsigned limit = *reinterpret_cast<volatile int *>(&S.abort) ? kSpinLimitAborted : kSpinLimit;
-    if (!mbar_wait(smem_addr(bar), parity, limit)) {
-        *reinterpret_cast<volatile int *>(&S.abort) = 1;
-        atomicExch(P.error, 1u);
-    }
+    if (!mbar_wait(smem_addr(bar), parity, limit)) raise_abort(P, S);
 }
 
 // The producer thread: streams the CTA's span, stage by stage, in the order the consumers read it.
@@ -406,79 +370,82 @@ __device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, unsigned l
     }
 }
 
-// Top-k of one piece into S.list[returned buffer]; S.bad tells whether the piece held a NaN or
-// +inf.  Called by all consumers, which have met at their barrier since they last touched S.
-// `q` counts the stages consumed so far (the ring position), as the producer counts them.
+// The consumers' part of one piece.  `q` counts the stages consumed so far (the ring position),
+// as the producer counts them; `parity` is the piece's parity within this CTA.
 template <int DT>
-__device__ int piece_topk(const TopkParams &P, const Piece &pc, int k, Smem &S, uint32_t ring, unsigned &q)
+__device__ void consume_piece(const TopkParams &P, const Piece &pc, int k, int parity, Smem &S, uint32_t ring, unsigned &q)
 {
     const int tid = threadIdx.x, lane = tid & 31;
-    // empty slots hold distinct small keys (k - r in slot r), below every real key
-    if (tid < 32) S.list[0][tid] = tid < k ? (unsigned long long)(k - tid) : 0ull;
-    if (tid == 0) {
-        S.n[0] = 0;
-        S.n[1] = 0;
-        S.nvalid[0] = kNone;
-        S.nvalid[1] = kNone;
-        S.bad = 0;
-    }
-    PieceState st;
-    st.cur = 0;
-    st.nbuf = 0;
-    st.pending = 0;
-    st.tau = -INFINITY;
-    for (int s = 0; s < pc.stages; ++s, ++q) {
-        const unsigned slot = q % kStages, pass = q / kStages;
-        ring_wait(P, S, &S.full[slot], pass & 1u);
-        uint4 a[kU];
-        const int vi0 = s * kStageVecs + tid;
-        const uint32_t src = ring + slot * (uint32_t)kStageBytes + (uint32_t)tid * 16u;
+    Channel &C = S.ch[parity];
+    uint4 a[kU];
+    unsigned slot = 0;
+    const uint32_t lane_off = (uint32_t)tid * 16u;
+    if (pc.stages > 0) {
+        slot = q % kStages;
+        ring_wait(P, S, &S.full[slot], (q / kStages) & 1u);
 #pragma unroll
         for (int u = 0; u < kU; ++u)
-            a[u] = vi0 + u * kConsThreads < pc.nvec ? lds16(src + (uint32_t)u * kConsThreads * 16u) : Vec<DT>::fill();
-        if (s == 0) {
-            // tau from the first stage: k-th largest of the 32 group maxima
-            float tm = -INFINITY;
+            a[u] = tid + u * kConsThreads < pc.nvec ? lds16(ring + slot * (uint32_t)kStageBytes + lane_off + (uint32_t)u * kConsThreads * 16u)
+                                                    : Vec<DT>::fill();
+    } else {
 #pragma unroll
-            for (int u = 0; u < kU; ++u) {
-                const float v = Vec<DT>::vmax(a[u]);
-                tm = fmaxf(tm, v == v ? v : -INFINITY);
-            }
+        for (int u = 0; u < kU; ++u) a[u] = Vec<DT>::fill();
+    }
+    // tau from the first stage: k-th largest of the 32 group maxima
+    float tm = -INFINITY;
 #pragma unroll
-            for (int o = 1; o < kGroup; o <<= 1) tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, o));
-            if ((tid & (kGroup - 1)) == 0) S.grp[tid / kGroup] = tm;
-            cons_sync();
-            const float g = S.grp[lane];
-            int rank = 0;
+    for (int u = 0; u < kU; ++u) {
+        const float v = Vec<DT>::vmax(a[u]);
+        tm = fmaxf(tm, v == v ? v : -INFINITY);
+    }
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float o = __shfl_sync(kFullMask, g, j);
-                rank += (o > g) || (o == g && j < lane);
-            }
-            const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
-            st.tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
-            st.taukey = (unsigned long long)ord(st.tau) << 32;
-            // the ragged ends of the piece, one element per thread
-            if (tid < pc.head) offer(S, 0, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, st.taukey);
-            if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
-                offer(S, 0, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, st.taukey);
+    for (int o = 1; o < kGroup; o <<= 1) tm = fmaxf(tm, __shfl_xor_sync(kFullMask, tm, o));
+    if ((tid & (kGroup - 1)) == 0) S.grp[parity][tid / kGroup] = tm;
+    boundary_sync(parity);  // the channel is free: the selection warp has finished the piece before the last
+    float tau;
+    {
+        const float g = S.grp[parity][lane];
+        int rank = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float o = __shfl_sync(kFullMask, g, j);
+            rank += (o > g) || (o == g && j < lane);
         }
-        iteration<DT>(a, vi0, pc.nvec, pc.idx0, s + 1 == pc.stages, k, st, S);
+        const unsigned hit = __ballot_sync(kFullMask, rank == k - 1);
+        tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
+    }
+    unsigned long long taukey = (unsigned long long)ord(tau) << 32;
+    // the ragged ends of the piece, one element per thread
+    if (tid < pc.head) offer(P, S, C, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, taukey);
+    if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
+        offer(P, S, C, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, taukey);
+    for (int s = 0; s < pc.stages; ++s, ++q) {
+        if (s > 0) {
+            slot = q % kStages;
+            ring_wait(P, S, &S.full[slot], (q / kStages) & 1u);
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+                a[u] = s * kStageVecs + tid + u * kConsThreads < pc.nvec
+                           ? lds16(ring + slot * (uint32_t)kStageBytes + lane_off + (uint32_t)u * kConsThreads * 16u)
+                           : Vec<DT>::fill();
+            // the selection warp's k-th key, once it beats what this warp filters with
+            const unsigned long long pub = ld_shared_volatile_u64(&C.taukey);
+            if (pub > taukey) {
+                taukey = pub;
+                tau = key_value(pub);
+            }
+        }
+        scan<DT>(P, a, s * kStageVecs + tid, pc.nvec, pc.idx0, tau, taukey, S, C);
         // the stage has been consumed from registers: hand the buffer back to the producer
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_addr(&S.empty[slot]));
     }
-    if (pc.stages == 0) {  // only ragged elements
-        cons_sync();
-        st.taukey = 0ull;
-        if (tid < pc.head) offer(S, 0, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, st.taukey);
-        if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
-            offer(S, 0, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, st.taukey);
-        cons_sync();
-        merge(S, st.cur, st.nbuf, S.n[st.nbuf], k);
-        st.cur ^= 1;
+    // this warp's candidates of the piece are all in the queue
+    __syncwarp();
+    if (lane == 0) {
+        fence_cta();
+        atomicAdd(&C.done, 1u);
     }
-    return st.cur;
 }
 
 // CTA that owns block `blk` when `total` blocks are divided over `grid` CTAs
@@ -493,47 +460,25 @@ struct RowDist {   // per lane r < k: entry r of the row's support, best first
     bool bad;      // the row has no distribution (warp-uniform)
 };
 
-// One warp: merges the pieces of `row`, then turns the k logits into probabilities (float64,
-// summed in rank order).
-__device__ RowDist row_dist(const TopkParams &P, int64_t row, unsigned long long *keys, unsigned long long *top)
+// pieces that share `row`
+__device__ __forceinline__ int pieces_of(const TopkParams &P, int64_t row)
+{
+    const unsigned long long first_blk = (unsigned long long)row * (unsigned long long)P.nb;
+    return (int)(owner_of(first_blk + P.nb - 1, P.grid, P.total_blocks) - owner_of(first_blk, P.grid, P.total_blocks)) + 1;
+}
+
+// One warp: lane r < k holds key r of a row's support (best first; kBadList in lane 0 marks a
+// row with a NaN or +inf).  Turns the k logits into probabilities in float64, summed in rank order.
+__device__ __forceinline__ RowDist dist_from_keys(const TopkParams &P, unsigned long long key)
 {
     const int lane = threadIdx.x & 31, k = P.k;
-    const unsigned long long first_blk = (unsigned long long)row * (unsigned long long)P.nb;
-    const int pieces = (int)(owner_of(first_blk + P.nb - 1, P.grid, P.total_blocks) - owner_of(first_blk, P.grid, P.total_blocks)) + 1;
-    const int m = pieces * k;
-    const unsigned long long *src = P.lists + (size_t)row * P.max_pieces * k;
-    bool bad = false;
-    for (int i = lane; i < m; i += 32) {
-        const unsigned long long x = __ldcg(src + i);
-        bad |= (x == kBadList);
-        keys[i] = x;
-    }
-    bad = __any_sync(kFullMask, bad);
-    __syncwarp();
     RowDist d;
     d.idx = -1;
     d.prob = NAN;
-    d.bad = bad;
-    if (bad) return d;
-    if (pieces == 1) {
-        if (lane < k) top[lane] = keys[lane];
-    } else {
-        for (int i = lane; i < m; i += 32) {
-            const unsigned long long x = keys[i];
-            int rank = 0;
-            for (int j = 0; j < m; ++j) rank += keys[j] > x;
-            if (rank < k) top[rank] = x;  // keys below rank k include every empty slot
-        }
-    }
-    __syncwarp();
-    const unsigned long long key = lane < k ? top[lane] : 0ull;
-    __syncwarp();
     const float val = key_value(key);
     const float best = __shfl_sync(kFullMask, val, 0);
-    if (!(best > -INFINITY)) {  // nothing above -inf
-        d.bad = true;
-        return d;
-    }
+    d.bad = __shfl_sync(kFullMask, key, 0) == kBadList || !(best > -INFINITY);  // nothing above -inf
+    if (d.bad) return d;
     const double T = (double)P.temperature;
     const double z = (double)val / T;
     const double mx = __shfl_sync(kFullMask, z, 0);
@@ -545,56 +490,225 @@ __device__ RowDist row_dist(const TopkParams &P, int64_t row, unsigned long long
     return d;
 }
 
-// The CTA that scanned a sequence's last block: acceptance tests, first rejection, row n's pairs.
-// Called by all consumers.
+// One warp: merges the `pieces` lists of `row` by rank counting; returns key r in lane r.
+__device__ unsigned long long merged_keys(const TopkParams &P, int64_t row, int pieces, unsigned long long *keys,
+                                          unsigned long long *top)
+{
+    const int lane = threadIdx.x & 31, k = P.k;
+    const int m = pieces * k;
+    const unsigned long long *src = P.lists + (size_t)row * P.max_pieces * k;
+    bool bad = false;
+    __syncwarp();
+    for (int i = lane; i < m; i += 32) {
+        const unsigned long long x = __ldcg(src + i);
+        bad |= (x == kBadList);
+        keys[i] = x;
+    }
+    bad = __any_sync(kFullMask, bad);
+    __syncwarp();
+    if (bad) return lane == 0 ? kBadList : 0ull;
+    for (int i = lane; i < m; i += 32) {
+        const unsigned long long x = keys[i];
+        int rank = 0;
+        for (int j = 0; j < m; ++j) rank += keys[j] > x;
+        if (rank < k) top[rank] = x;  // keys below rank k include every empty slot
+    }
+    __syncwarp();
+    return lane < k ? top[lane] : 0ull;
+}
+
+// The acceptance test of one position, as the oracle states it (float64 throughout)
+__device__ __forceinline__ bool judge(const TopkParams &P, const RowDist &d, int x, double u, double q, unsigned &fl,
+                                      double &p)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned holds = __ballot_sync(kFullMask, lane < P.k && !d.bad && d.idx == x);
+    const double p_in = __shfl_sync(kFullMask, d.prob, holds ? __ffs(holds) - 1 : 0);
+    if (x < 0 || x >= P.V) {
+        fl |= DSSD_EDGE_FLAG_BAD_TOKEN;
+        p = NAN;
+        return false;
+    }
+    p = d.bad ? NAN : (holds ? p_in : 0.0);
+    double ratio;
+    if (q != q || p != p) ratio = NAN;
+    else if (q <= 0.0) ratio = p > 0.0 ? INFINITY : 0.0;
+    else ratio = p / q;
+    return (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+}
+
+// The selection warp of the CTA that scanned a sequence's last block: acceptance tests, first
+// rejection, row n's pairs.  Rows are taken eight at a time: their lists and their drafts are
+// all requested before the first is used, so that a group costs one trip to the L2, not eight.
 __device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int kBatch = 8;
+    const int lane = threadIdx.x & 31;
     const int gamma = P.gamma, k = P.k;
-    if (tid == 0) {
-        S.first_reject = gamma;
-        S.fl = ld_relaxed_u32(P.error) ? DSSD_EDGE_FLAG_TIMEOUT : 0u;
-    }
-    cons_sync();
-    for (int j = warp; j <= gamma; j += kConsWarps) {
-        const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + j, S.fold_keys[warp], S.fold_top[warp]);
-        if (d.bad && lane == 0) atomicOr(&S.fl, DSSD_EDGE_FLAG_NONFINITE);
-        if (j == gamma) continue;
-        const size_t o = (size_t)b * gamma + j;
-        const int x = __ldg(P.draft_tokens + o);
-        const unsigned holds = __ballot_sync(kFullMask, lane < k && !d.bad && d.idx == x);
-        const double p_in = __shfl_sync(kFullMask, d.prob, holds ? __ffs(holds) - 1 : 0);
-        if (lane == 0) {
-            const double u = (double)__ldg(P.uniforms + o), q = (double)__ldg(P.draft_q_tok + o);
-            double p;
-            bool accept = false;
-            if (x < 0 || x >= P.V) {
-                atomicOr(&S.fl, DSSD_EDGE_FLAG_BAD_TOKEN);
-                p = NAN;
-            } else {
-                p = d.bad ? NAN : (holds ? p_in : 0.0);
-                double ratio;
-                if (q != q || p != p) ratio = NAN;
-                else if (q <= 0.0) ratio = p > 0.0 ? INFINITY : 0.0;
-                else ratio = p / q;
-                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+    unsigned fl = ld_relaxed_u32(P.error) ? DSSD_EDGE_FLAG_TIMEOUT : 0u;
+    int n = gamma;
+    unsigned long long key_n = 0ull;   // row n's keys: the first rejected row's, else the bonus row's
+    const int64_t row0 = (int64_t)b * (gamma + 1);
+    for (int base = 0; base <= gamma; base += kBatch) {
+        const int nrow = min(kBatch, gamma + 1 - base);
+        // lane r looks after row base + r: its number of pieces and its draft
+        int my_pieces = 1, my_x = 0;
+        float my_u = 0.f, my_q = 0.f;
+        if (lane < nrow) {
+            my_pieces = pieces_of(P, row0 + base + lane);
+            if (base + lane < gamma) {
+                const size_t o = (size_t)b * gamma + base + lane;
+                my_x = __ldg(P.draft_tokens + o);
+                my_u = __ldg(P.uniforms + o);
+                my_q = __ldg(P.draft_q_tok + o);
             }
-            if (P.p_tok) P.p_tok[o] = (float)p;
-            if (!accept) atomicMin(&S.first_reject, j);
+        }
+        unsigned long long kk[kBatch];
+#pragma unroll
+        for (int r = 0; r < kBatch; ++r) {
+            const int pcs = __shfl_sync(kFullMask, my_pieces, r);
+            kk[r] = 0ull;
+            if (r < nrow && pcs == 1 && lane < k) kk[r] = __ldcg(P.lists + (size_t)(row0 + base + r) * P.max_pieces * k + lane);
+        }
+#pragma unroll
+        for (int r = 0; r < kBatch; ++r) {
+            if (r >= nrow) break;
+            const int j = base + r;
+            const int pcs = __shfl_sync(kFullMask, my_pieces, r);
+            const unsigned long long key = pcs == 1 ? kk[r] : merged_keys(P, row0 + j, pcs, S.fold_keys, S.fold_top);
+            const RowDist d = dist_from_keys(P, key);
+            if (d.bad) fl |= DSSD_EDGE_FLAG_NONFINITE;
+            if (j == gamma) {
+                if (n == gamma) key_n = key;
+                break;
+            }
+            const int x = __shfl_sync(kFullMask, my_x, r);
+            const double u = (double)__shfl_sync(kFullMask, my_u, r), q = (double)__shfl_sync(kFullMask, my_q, r);
+            double p;
+            const bool accept = judge(P, d, x, u, q, fl, p);
+            if (lane == 0 && P.p_tok) P.p_tok[(size_t)b * gamma + j] = (float)p;
+            if (!accept && j < n) {
+                n = j;
+                key_n = key;
+            }
         }
     }
-    cons_sync();
-    const int n = S.first_reject;
-    if (warp == 0) {
-        const RowDist d = row_dist(P, (int64_t)b * (gamma + 1) + n, S.fold_keys[0], S.fold_top[0]);
-        if (lane < k) {
-            P.p_idx[(size_t)b * k + lane] = d.bad ? -1 : d.idx;
-            P.p_val[(size_t)b * k + lane] = d.bad ? NAN : (float)d.prob;
+    const RowDist d = dist_from_keys(P, key_n);
+    if (lane < k) {
+        P.p_idx[(size_t)b * k + lane] = d.bad ? -1 : d.idx;
+        P.p_val[(size_t)b * k + lane] = d.bad ? NAN : (float)d.prob;
+    }
+    if (lane == 0) {
+        P.accept_len[b] = n;
+        if (P.flags) P.flags[b] = fl;
+    }
+}
+
+// The selection warp.  Lane r holds entry r of the current piece's list, best first; candidates
+// arrive through the piece's queue in shared memory and are inserted by a ballot and a shuffle;
+// the k-th key is published for the consumers to filter with.  At the end of a piece the warp
+// frees the channel (boundary_arrive) before it writes the list out, counts the piece's
+// blocks and, when that completes a sequence, folds it; the other channel's queue buffers the
+// next piece's candidates meanwhile.
+template <int DT>
+__device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long blk, unsigned long long blk_end)
+{
+    const int lane = threadIdx.x & 31, k = P.k;
+    const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
+    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
+    unsigned tails[2] = {0u, 0u};  // queue positions taken so far, per channel
+    // the sequence counter's answer is not waited for: it is looked at one piece later
+    unsigned long long prev_sum = 0ull;
+    int prev_b = -1;
+    boundary_arrive(0);  // both channels start free
+    boundary_arrive(1);
+    int parity = 0;
+    while (blk < blk_end) {
+        const Piece pc = piece_at<DT>(P, blk, blk_end);
+        Channel &C = S.ch[parity];
+        unsigned tail = parity ? tails[1] : tails[0];
+        // empty slots hold distinct small keys (k - r in slot r), below every real key
+        unsigned long long key = lane < k ? (unsigned long long)(k - lane) : 0ull;
+        unsigned long long tkey = 0ull;
+        unsigned idle = 0;
+        for (;;) {
+            const unsigned long long v = ld_shared_volatile_u64(&C.queue[(tail + lane) % kCap]);
+            const unsigned valid = __ballot_sync(kFullMask, v != 0ull);
+            const int nv = valid == kFullMask ? 32 : __ffs(~valid) - 1;  // leading filled slots
+            if (nv == 0) {
+                if (ld_shared_volatile_u32(&C.done) == (unsigned)kConsWarps && tail == ld_shared_volatile_u32(&C.q_head))
+                    break;
+                if (++idle > kSpinLimit * 256u) {  // a reserved slot that is never filled
+                    raise_abort(P, S);
+                    break;
+                }
+                continue;
+            }
+            idle = 0;
+            if (lane < nv) *reinterpret_cast<volatile unsigned long long *>(&C.queue[(tail + lane) % kCap]) = 0ull;
+            fence_cta();
+            tail += (unsigned)nv;
+            if (lane == 0) *reinterpret_cast<volatile unsigned *>(&C.q_tail) = tail;
+            // insert the candidates that beat the k-th key as it stood when the batch was taken; one
+            // that has been overtaken within the batch lands beyond lane k - 1 and is never read
+            unsigned want = __ballot_sync(kFullMask, lane < nv && v > tkey);
+            while (want) {
+                const int src = __ffs(want) - 1;
+                want &= want - 1u;
+                const unsigned long long x = __shfl_sync(kFullMask, v, src);
+                const unsigned long long up = __shfl_up_sync(kFullMask, key, 1);
+                const int pos = __popc(__ballot_sync(kFullMask, key > x));  // keys above x form a prefix
+                key = lane == pos ? x : (lane > pos ? up : key);
+            }
+            const unsigned long long kth = __shfl_sync(kFullMask, key, k - 1);
+            if (kth > (unsigned long long)k && kth != tkey) {  // the list is full of real keys
+                tkey = kth;
+                if (lane == 0) *reinterpret_cast<volatile unsigned long long *>(&C.taukey) = tkey;
+            }
         }
+        if (parity) tails[1] = tail;
+        else tails[0] = tail;
+        // the piece is complete: take what the consumers left, reset the channel and free it
+        const int bad = *reinterpret_cast<volatile int *>(&C.bad);
+        __syncwarp();
         if (lane == 0) {
-            P.accept_len[b] = n;
-            if (P.flags) P.flags[b] = S.fl;
+            *reinterpret_cast<volatile int *>(&C.bad) = 0;
+            *reinterpret_cast<volatile unsigned *>(&C.done) = 0u;
+            *reinterpret_cast<volatile unsigned long long *>(&C.taukey) = 0ull;
+            fence_cta();
         }
+        __syncwarp();
+        boundary_arrive(parity);
+        // publish the list, then count the piece's blocks
+        const int slot = (int)(c - owner_of((unsigned long long)pc.row * P.nb, G, TB));
+        if (lane < k) {
+            unsigned long long out = key;
+            if (bad) out = lane == 0 ? kBadList : 0ull;
+            __stcg(P.lists + ((size_t)pc.row * P.max_pieces + slot) * k + lane, out);
+        }
+        fence_gpu();
+        __syncwarp();
+        const int b = (int)(pc.row / (P.gamma + 1));
+        int fold_b = -1;
+        if (lane == 0) {
+            fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
+            const unsigned long long done = (unsigned long long)(pc.lb - pc.fb);
+            prev_sum = atomicAdd(P.seq_done + b, done) + done;
+            prev_b = b;
+        }
+        fold_b = __shfl_sync(kFullMask, fold_b, 0);
+        if (fold_b >= 0) {
+            fence_gpu();
+            fold_sequence(P, fold_b, S);
+        }
+        blk += (unsigned long long)(pc.lb - pc.fb);
+        parity ^= 1;
+    }
+    int fold_b = (lane == 0 && prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
+    fold_b = __shfl_sync(kFullMask, fold_b, 0);
+    if (fold_b >= 0) {
+        fence_gpu();
+        fold_sequence(P, fold_b, S);
     }
 }
 
@@ -604,11 +718,19 @@ __global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_ke
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem &S = *reinterpret_cast<Smem *>(smem_raw + (size_t)kStages * kStageBytes);
     const uint32_t ring = smem_addr(smem_raw);
-    const int tid = threadIdx.x, k = P.k;
+    const int tid = threadIdx.x;
+    for (int i = tid; i < 2 * kCap; i += kTkThreads) S.ch[i / kCap].queue[i % kCap] = 0ull;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_addr(&S.full[s]), 1u);
             mbar_init(smem_addr(&S.empty[s]), (uint32_t)kConsWarps);
+        }
+        for (int h = 0; h < 2; ++h) {
+            S.ch[h].taukey = 0ull;
+            S.ch[h].q_head = 0u;
+            S.ch[h].q_tail = 0u;
+            S.ch[h].done = 0u;
+            S.ch[h].bad = 0;
         }
         S.abort = 0;
         mbar_init_fence();
@@ -617,50 +739,21 @@ __global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_ke
     const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
     const unsigned long long blk_end = (c + 1ull) * TB / G;
     unsigned long long blk = c * TB / G;
+    if (tid >= kConsThreads + 32) {
+        selection_warp<DT>(P, S, blk, blk_end);
+        return;
+    }
     if (tid >= kConsThreads) {
         if (tid == kConsThreads) producer<DT>(P, S, ring, blk, blk_end);
         return;
     }
-    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
     unsigned q = 0;
-    // The sequence counter's answer is not waited for: thread 0 looks at it one piece later.
-    unsigned long long prev_sum = 0ull;  // thread 0: counter value after the previous piece's blocks
-    int prev_b = -1;
+    int parity = 0;
     while (blk < blk_end) {
         const Piece pc = piece_at<DT>(P, blk, blk_end);
-        const int cur = piece_topk<DT>(P, pc, k, S, ring, q);
-        const int b = (int)(pc.row / (P.gamma + 1));
-        if (tid < 32) {
-            // warp 0 publishes the piece: list, fence, then the blocks are counted
-            const int slot = (int)(c - owner_of((unsigned long long)pc.row * P.nb, G, TB));
-            if (tid < k) {
-                unsigned long long key = S.list[cur][tid];
-                if (S.bad) key = tid == 0 ? kBadList : 0ull;
-                __stcg(P.lists + ((size_t)pc.row * P.max_pieces + slot) * k + tid, key);
-            }
-            __threadfence();
-            __syncwarp();
-            if (tid == 0) {
-                S.fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
-                const unsigned long long done = (unsigned long long)(pc.lb - pc.fb);
-                prev_sum = atomicAdd(P.seq_done + b, done) + done;
-                prev_b = b;
-            }
-        }
-        cons_sync();
-        const int fb = S.fold_b;
-        if (fb >= 0) {
-            __threadfence();
-            fold_sequence(P, fb, S);
-            cons_sync();
-        }
+        consume_piece<DT>(P, pc, P.k, parity, S, ring, q);
+        parity ^= 1;
         blk += (unsigned long long)(pc.lb - pc.fb);
-    }
-    if (tid == 0) S.fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
-    cons_sync();
-    if (S.fold_b >= 0) {
-        __threadfence();
-        fold_sequence(P, S.fold_b, S);
     }
 }
 
