@@ -73,9 +73,9 @@ constexpr int kU = kStageVecs / kConsThreads;        // vectors per consumer thr
 constexpr int kGroup = kConsThreads / 32;            // threads per group of the first threshold
 static_assert(kU >= 1 && kU * kConsThreads == kStageVecs && kGroup >= 4 && kGroup <= 16, "stage / consumer shape");
 #ifndef DSSD_TOPK_QUEUE
-#define DSSD_TOPK_QUEUE 256
+#define DSSD_TOPK_QUEUE 32
 #endif
-constexpr int kCap = DSSD_TOPK_QUEUE;                // candidate queue entries per channel (a power of two)
+constexpr int kCap = DSSD_TOPK_QUEUE;                // candidate keys per consumer warp and channel (32: one batch of the selection warp)
 constexpr unsigned kSpinLimit = 1u << 16;            // tries of a bounded wait (about 4 us each)
 constexpr unsigned kSpinLimitAborted = 8u;           // after a wait has run out
 constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
@@ -183,10 +183,10 @@ struct Vec<DSSD_BF16> {
 // by even and odd pieces, so that the consumers can scan a piece while the selection warp is
 // still finishing the one before.
 struct Channel {
-    unsigned long long queue[kCap];     // candidate keys on their way to the selection warp; 0 = free slot
+    unsigned long long keys[kConsWarps][kCap];  // candidate keys of consumer warp w on their way to the selection warp
+    unsigned head[kConsWarps];          // keys warp w has written (counts up for the kernel's life)
+    unsigned tail[kConsWarps];          // keys the selection warp has taken from warp w
     unsigned long long taukey;          // the selection warp's current k-th key (0: list not full yet)
-    unsigned q_head;                    // slots reserved by the consumers (counts up for the kernel's life)
-    unsigned q_tail;                    // slots the selection warp has taken
     unsigned done;                      // consumer warps that have finished the piece
     int bad;                            // the piece holds a NaN or +inf
 };
@@ -232,41 +232,69 @@ __device__ __forceinline__ void raise_abort(const TopkParams &P, Smem &S)
     atomicExch(P.error, 1u);
 }
 
-// Writes a key into its reserved queue position once the selection warp has freed the slot (it
-// is at most kCap positions behind).  Bounded; a key that cannot be delivered is dropped and
-// the error word is raised.
-__device__ __forceinline__ void deliver(const TopkParams &P, Smem &S, Channel &C, unsigned pos, unsigned long long key)
+// A consumer warp's end of its key ring (the same values in all lanes)
+struct Outbox {
+    unsigned head;   // keys written so far
+    unsigned tail;   // the selection warp's progress as last read
+};
+
+// Hands the keys of the lanes in `wm` (at most kCap of them) to the selection warp through the
+// warp's own ring: no atomic, no other consumer warp involved.  Waits, bounded, while the ring
+// is full; keys that cannot be delivered are dropped and the error word is raised.
+__device__ __forceinline__ void push_keys(const TopkParams &P, Smem &S, Channel &C, int warp, Outbox &ob, unsigned wm,
+                                          unsigned long long key)
 {
+    const int lane = threadIdx.x & 31;
+    const unsigned n = (unsigned)__popc(wm);
     unsigned it = 0;
-    while (pos - ld_shared_volatile_u32(&C.q_tail) >= (unsigned)kCap) {
+    while (ob.head + n - ob.tail > (unsigned)kCap) {
+        ob.tail = ld_shared_volatile_u32(&C.tail[warp]);
+        if (ob.head + n - ob.tail <= (unsigned)kCap) break;
         if (++it > kSpinLimit * 64u || *reinterpret_cast<volatile int *>(&S.abort)) {
             raise_abort(P, S);
             return;
         }
-        __nanosleep(64);
+        __nanosleep(32);
     }
-    *reinterpret_cast<volatile unsigned long long *>(&C.queue[pos % kCap]) = key;
+    if ((wm >> lane) & 1u)
+        *reinterpret_cast<volatile unsigned long long *>(&C.keys[warp][(ob.head + (unsigned)__popc(wm & ((1u << lane) - 1u))) % kCap]) = key;
+    ob.head += n;
+    __syncwarp();
+    if (lane == 0) {
+        fence_cta();
+        *reinterpret_cast<volatile unsigned *>(&C.head[warp]) = ob.head;
+    }
 }
 
-// One element of a piece's ragged ends
-__device__ __forceinline__ void offer(const TopkParams &P, Smem &S, Channel &C, float f, int idx, unsigned long long taukey)
+// The ragged ends of a piece: lane e < count judges element first + e
+template <int DT>
+__device__ __forceinline__ void offer_ragged(const TopkParams &P, Smem &S, Channel &C, int warp, Outbox &ob, const char *rowp,
+                                             int first, int count, unsigned long long taukey)
 {
-    if (f != f || f == INFINITY) {
-        C.bad = 1;
-        return;
+    const int lane = threadIdx.x & 31;
+    bool want = false;
+    unsigned long long key = 0ull;
+    if (lane < count) {
+        const float f = Vec<DT>::load(rowp, first + lane);
+        if (f != f || f == INFINITY) {
+            C.bad = 1;
+        } else {
+            key = make_key(f, first + lane);
+            want = key > taukey;
+        }
     }
-    const unsigned long long key = make_key(f, idx);
-    if (key > taukey) deliver(P, S, C, atomicAdd(&C.q_head, 1u), key);
+    const unsigned wm = __ballot_sync(kFullMask, want);
+    if (wm) push_keys(P, S, C, warp, ob, wm, key);
 }
 
 // Scans the warp's kU x 32 vectors of one stage.  One vote settles the common case that nothing
 // reaches tau.  Otherwise a vector whose maximum (NaN-propagating) reaches tau is taken apart
-// by the whole warp: its 16 bytes are broadcast and lane j judges element j; the queue slots of
-// a vector are reserved with one shared-memory atomic.  vi0 = this lane's first vector within
+// by the whole warp: its 16 bytes are broadcast and lane j judges element j; the keys that pass
+// go into the warp's own ring.  vi0 = this lane's first vector within
 // the piece's vector body, idx0 = vocabulary index of the body's first element.
 template <int DT>
 __device__ __forceinline__ void scan(const TopkParams &P, const uint4 (&a)[kU], int vi0, int nvec, int idx0, float tau,
-                                     unsigned long long taukey, Smem &S, Channel &C)
+                                     unsigned long long taukey, Smem &S, Channel &C, int warp, Outbox &ob)
 {
     constexpr int E = Vec<DT>::E;
     const int lane = threadIdx.x & 31;
@@ -300,12 +328,7 @@ __device__ __forceinline__ void scan(const TopkParams &P, const uint4 (&a)[kU], 
                 }
             }
             const unsigned wm = __ballot_sync(kFullMask, want);
-            if (wm) {
-                unsigned base = 0u;
-                if (lane == 0) base = atomicAdd(&C.q_head, (unsigned)__popc(wm));
-                base = __shfl_sync(kFullMask, base, 0);
-                if (want) deliver(P, S, C, base + (unsigned)__popc(wm & ((1u << lane) - 1u)), key);
-            }
+            if (wm) push_keys(P, S, C, warp, ob, wm, key);
             hot &= hot - 1u;
         }
     }
@@ -375,7 +398,7 @@ __device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, unsigned l
 template <int DT>
 __device__ void consume_piece(const TopkParams &P, const Piece &pc, int k, int parity, Smem &S, uint32_t ring, unsigned &q)
 {
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     Channel &C = S.ch[parity];
     uint4 a[kU];
     unsigned slot = 0;
@@ -415,10 +438,12 @@ __device__ void consume_piece(const TopkParams &P, const Piece &pc, int k, int p
         tau = __shfl_sync(kFullMask, g, __ffs(hit) - 1);
     }
     unsigned long long taukey = (unsigned long long)ord(tau) << 32;
-    // the ragged ends of the piece, one element per thread
-    if (tid < pc.head) offer(P, S, C, Vec<DT>::load(pc.rowp, pc.e0 + tid), pc.e0 + tid, taukey);
-    if (tid >= 32 && tid - 32 < pc.e1 - pc.tail0)
-        offer(P, S, C, Vec<DT>::load(pc.rowp, pc.tail0 + tid - 32), pc.tail0 + tid - 32, taukey);
+    Outbox ob;
+    ob.head = C.head[warp];  // only this warp writes it
+    ob.tail = ob.head;       // the ring is empty: the selection warp finished with this channel
+    // the ragged ends of the piece (warp 0: before the first whole vector, warp 1: after the last)
+    if (warp == 0 && pc.head > 0) offer_ragged<DT>(P, S, C, warp, ob, pc.rowp, pc.e0, pc.head, taukey);
+    if (warp == 1 % kConsWarps && pc.e1 > pc.tail0) offer_ragged<DT>(P, S, C, warp, ob, pc.rowp, pc.tail0, pc.e1 - pc.tail0, taukey);
     for (int s = 0; s < pc.stages; ++s, ++q) {
         if (s > 0) {
             slot = q % kStages;
@@ -435,7 +460,7 @@ __device__ void consume_piece(const TopkParams &P, const Piece &pc, int k, int p
                 tau = key_value(pub);
             }
         }
-        scan<DT>(P, a, s * kStageVecs + tid, pc.nvec, pc.idx0, tau, taukey, S, C);
+        scan<DT>(P, a, s * kStageVecs + tid, pc.nvec, pc.idx0, tau, taukey, S, C, warp, ob);
         // the stage has been consumed from registers: hand the buffer back to the producer
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_addr(&S.empty[slot]));
@@ -616,7 +641,7 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
     const int lane = threadIdx.x & 31, k = P.k;
     const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
     const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
-    unsigned tails[2] = {0u, 0u};  // queue positions taken so far, per channel
+    unsigned tails[2] = {0u, 0u};  // lane w < kConsWarps: keys taken from warp w's ring, per channel
     // the sequence counter's answer is not waited for: it is looked at one piece later
     unsigned long long prev_sum = 0ull;
     int prev_b = -1;
@@ -626,39 +651,47 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
     while (blk < blk_end) {
         const Piece pc = piece_at<DT>(P, blk, blk_end);
         Channel &C = S.ch[parity];
-        unsigned tail = parity ? tails[1] : tails[0];
+        unsigned tl = parity ? tails[1] : tails[0];
         // empty slots hold distinct small keys (k - r in slot r), below every real key
         unsigned long long key = lane < k ? (unsigned long long)(k - lane) : 0ull;
         unsigned long long tkey = 0ull;
         unsigned idle = 0;
         for (;;) {
-            const unsigned long long v = ld_shared_volatile_u64(&C.queue[(tail + lane) % kCap]);
-            const unsigned valid = __ballot_sync(kFullMask, v != 0ull);
-            const int nv = valid == kFullMask ? 32 : __ffs(~valid) - 1;  // leading filled slots
-            if (nv == 0) {
-                if (ld_shared_volatile_u32(&C.done) == (unsigned)kConsWarps && tail == ld_shared_volatile_u32(&C.q_head))
-                    break;
-                if (++idle > kSpinLimit * 256u) {  // a reserved slot that is never filled
+            const bool last_look = ld_shared_volatile_u32(&C.done) == (unsigned)kConsWarps;  // read before the heads
+            const unsigned h = lane < kConsWarps ? ld_shared_volatile_u32(&C.head[lane]) : 0u;
+            unsigned pend = __ballot_sync(kFullMask, lane < kConsWarps && h != tl);
+            if (!pend) {
+                if (last_look) break;
+                if (++idle > kSpinLimit * 256u) {
                     raise_abort(P, S);
                     break;
                 }
                 continue;
             }
             idle = 0;
-            if (lane < nv) *reinterpret_cast<volatile unsigned long long *>(&C.queue[(tail + lane) % kCap]) = 0ull;
-            fence_cta();
-            tail += (unsigned)nv;
-            if (lane == 0) *reinterpret_cast<volatile unsigned *>(&C.q_tail) = tail;
-            // insert the candidates that beat the k-th key as it stood when the batch was taken; one
-            // that has been overtaken within the batch lands beyond lane k - 1 and is never read
-            unsigned want = __ballot_sync(kFullMask, lane < nv && v > tkey);
-            while (want) {
-                const int src = __ffs(want) - 1;
-                want &= want - 1u;
-                const unsigned long long x = __shfl_sync(kFullMask, v, src);
-                const unsigned long long up = __shfl_up_sync(kFullMask, key, 1);
-                const int pos = __popc(__ballot_sync(kFullMask, key > x));  // keys above x form a prefix
-                key = lane == pos ? x : (lane > pos ? up : key);
+            while (pend) {
+                const int w = __ffs(pend) - 1;
+                pend &= pend - 1u;
+                const unsigned hw = __shfl_sync(kFullMask, h, w), tw = __shfl_sync(kFullMask, tl, w);
+                const unsigned long long v =
+                    (unsigned)lane < hw - tw ? ld_shared_volatile_u64(&C.keys[w][(tw + (unsigned)lane) % kCap]) : 0ull;
+                // insert the candidates that beat the k-th key as it stood when the batch was taken; one
+                // that has been overtaken within the batch lands beyond lane k - 1 and is never read
+                unsigned want = __ballot_sync(kFullMask, v > tkey);
+                // the keys are in registers: give the slots back
+                if (lane == w) {
+                    tl = hw;
+                    fence_cta();
+                    *reinterpret_cast<volatile unsigned *>(&C.tail[w]) = hw;
+                }
+                while (want) {
+                    const int src = __ffs(want) - 1;
+                    want &= want - 1u;
+                    const unsigned long long x = __shfl_sync(kFullMask, v, src);
+                    const unsigned long long up = __shfl_up_sync(kFullMask, key, 1);
+                    const int pos = __popc(__ballot_sync(kFullMask, key > x));  // keys above x form a prefix
+                    key = lane == pos ? x : (lane > pos ? up : key);
+                }
             }
             const unsigned long long kth = __shfl_sync(kFullMask, key, k - 1);
             if (kth > (unsigned long long)k && kth != tkey) {  // the list is full of real keys
@@ -666,8 +699,8 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
                 if (lane == 0) *reinterpret_cast<volatile unsigned long long *>(&C.taukey) = tkey;
             }
         }
-        if (parity) tails[1] = tail;
-        else tails[0] = tail;
+        if (parity) tails[1] = tl;
+        else tails[0] = tl;
         // the piece is complete: take what the consumers left, reset the channel and free it
         const int bad = *reinterpret_cast<volatile int *>(&C.bad);
         __syncwarp();
@@ -719,7 +752,6 @@ __global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_ke
     Smem &S = *reinterpret_cast<Smem *>(smem_raw + (size_t)kStages * kStageBytes);
     const uint32_t ring = smem_addr(smem_raw);
     const int tid = threadIdx.x;
-    for (int i = tid; i < 2 * kCap; i += kTkThreads) S.ch[i / kCap].queue[i % kCap] = 0ull;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_addr(&S.full[s]), 1u);
@@ -727,10 +759,12 @@ __global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_ke
         }
         for (int h = 0; h < 2; ++h) {
             S.ch[h].taukey = 0ull;
-            S.ch[h].q_head = 0u;
-            S.ch[h].q_tail = 0u;
             S.ch[h].done = 0u;
             S.ch[h].bad = 0;
+            for (int w = 0; w < kConsWarps; ++w) {
+                S.ch[h].head[w] = 0u;
+                S.ch[h].tail[w] = 0u;
+            }
         }
         S.abort = 0;
         mbar_init_fence();
