@@ -12,31 +12,34 @@
 //     kStages shared-memory stages with bulk asynchronous copies (TMA, untiled) that complete
 //     on "full" mbarriers; the consumer warps read a stage into registers (kU vectors of 16
 //     bytes per thread), scan them and release the stage through an "empty" mbarrier.  Memory
-//     latency is hidden by the rings, not by the consumers; several CTAs share an SM so that
-//     one CTA's barriers and merges overlap with the others' streaming.
+//     latency is hidden by the rings, not by the consumers; several small CTAs share an SM so
+//     that one CTA's selection work overlaps with the others' streaming.
 //   * Each vector is reduced to its maximum with NaN-propagating max instructions and compared
 //     with the warp's threshold tau, a lower bound on the piece's k-th largest logit.  A vector
 //     that reaches tau is taken apart by the whole warp: its 16 bytes are broadcast and lane j
-//     judges element j; the elements that beat the threshold key go into a queue in shared
-//     memory (one atomic per vector).  The consumers never meet at a barrier within a piece.
+//     judges element j; the elements that beat the threshold key go into the warp's own ring of
+//     keys in shared memory (no atomics).  One vote per stage settles the common case that
+//     nothing reaches tau.  The consumers never meet at a barrier within a piece.
 //   * A key is 64 bits: the logit mapped to an unsigned integer that sorts like the float
 //     (with -0 folded into +0), then the complemented index - larger key = earlier in the order
 //     (logit descending, index ascending), and all keys of a row are distinct.
-//   * A selection warp drains the queue.  Lane r holds entry r of the piece's list, best first;
+//   * A selection warp drains the rings.  Lane r holds entry r of the piece's list, best first;
 //     a candidate is inserted with one ballot (its position) and one shuffle (the shift), and
 //     the k-th key is published in shared memory, where the consumers pick it up at their next
 //     stage.  No sorting network, no merge rounds.
 //   * tau starts from the piece's first stage: the consumer threads form 32 groups, each
 //     group's maximum is one distinct element, so the k-th largest group maximum (k <= 32) is a
 //     valid lower bound.  On input that defeats the threshold (an ascending row) every element
-//     goes through the queue: slow, never wrong; a full queue makes the consumers wait.
-//   * At the end of a piece the selection warp lets the consumers go on with the next one and
-//     only then writes the list to the workspace and counts the piece's blocks; the CTA that
+//     goes through the rings: slow, never wrong; a full ring makes its warp wait.
+//   * Pieces alternate between two channels (rings, threshold, counters), so the consumers
+//     scan a piece while the selection warp still finishes the one before.  At the end of a
+//     piece the selection warp frees its channel and only then writes the list to the
+//     workspace and counts the piece's blocks; the CTA that
 //     completes a sequence folds it in the same warp: the rows' pieces are merged by rank
 //     counting, the k logits become probabilities in float64, the acceptance test runs, row n's
 //     k pairs are written.  The counter's answer is looked at one piece later, so nobody waits
 //     for the round trip.
-//   * Every wait (mbarrier, queue, barrier hand-off) is bounded; a wait that runs out raises an
+//   * Every wait (mbarrier, ring, channel hand-off) is bounded; a wait that runs out raises an
 //     error word in the workspace, the kernel runs to its end without faulting and every
 //     sequence folded after that carries DSSD_EDGE_FLAG_TIMEOUT.
 //
@@ -52,16 +55,16 @@ namespace dssd {
 namespace {
 
 #ifndef DSSD_TOPK_CONS_WARPS
-#define DSSD_TOPK_CONS_WARPS 8
+#define DSSD_TOPK_CONS_WARPS 4
 #endif
 #ifndef DSSD_TOPK_STAGE_BYTES
-#define DSSD_TOPK_STAGE_BYTES 32768
+#define DSSD_TOPK_STAGE_BYTES 16384
 #endif
 #ifndef DSSD_TOPK_STAGES
 #define DSSD_TOPK_STAGES 3
 #endif
 #ifndef DSSD_TOPK_MIN_CTAS
-#define DSSD_TOPK_MIN_CTAS 2
+#define DSSD_TOPK_MIN_CTAS 4
 #endif
 constexpr int kConsWarps = DSSD_TOPK_CONS_WARPS;      // consumer warps per CTA (a power of two, 4..16)
 constexpr int kConsThreads = 32 * kConsWarps;
@@ -139,13 +142,6 @@ struct Vec<DSSD_F32> {
     {
         return __uint_as_float(j < 2 ? (j == 0 ? v.x : v.y) : (j == 2 ? v.z : v.w));
     }
-    // a vector whose element 0 is the element at `row[i]`
-    __device__ static __forceinline__ uint4 single(const void *row, int64_t i)
-    {
-        uint4 v = fill();
-        v.x = reinterpret_cast<const uint32_t *>(row)[i];
-        return v;
-    }
 };
 template <>
 struct Vec<DSSD_BF16> {
@@ -170,12 +166,6 @@ struct Vec<DSSD_BF16> {
     {
         const uint32_t w = j < 4 ? (j < 2 ? v.x : v.y) : (j < 6 ? v.z : v.w);
         return (j & 1) ? bf16_hi(w) : bf16_lo(w);
-    }
-    __device__ static __forceinline__ uint4 single(const void *row, int64_t i)
-    {
-        uint4 v = fill();
-        v.x = 0xff800000u | (uint32_t)reinterpret_cast<const unsigned short *>(row)[i];
-        return v;
     }
 };
 
@@ -220,6 +210,19 @@ __device__ __forceinline__ void boundary_arrive(int parity)
 __device__ __forceinline__ void fence_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 
+// release / acquire on a shared-memory word at CTA scope: what the hand-offs between the
+// consumer warps and the selection warp are built from
+__device__ __forceinline__ void st_release_shared(unsigned *p, unsigned v)
+{
+    asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_addr(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire_shared(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_addr(p)) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ unsigned ld_shared_volatile_u32(const unsigned *p) { return *reinterpret_cast<const volatile unsigned *>(p); }
 __device__ __forceinline__ unsigned long long ld_shared_volatile_u64(const unsigned long long *p)
 {
@@ -248,7 +251,7 @@ __device__ __forceinline__ void push_keys(const TopkParams &P, Smem &S, Channel 
     const unsigned n = (unsigned)__popc(wm);
     unsigned it = 0;
     while (ob.head + n - ob.tail > (unsigned)kCap) {
-        ob.tail = ld_shared_volatile_u32(&C.tail[warp]);
+        ob.tail = ld_acquire_shared(&C.tail[warp]);
         if (ob.head + n - ob.tail <= (unsigned)kCap) break;
         if (++it > kSpinLimit * 64u || *reinterpret_cast<volatile int *>(&S.abort)) {
             raise_abort(P, S);
@@ -260,10 +263,7 @@ __device__ __forceinline__ void push_keys(const TopkParams &P, Smem &S, Channel 
         *reinterpret_cast<volatile unsigned long long *>(&C.keys[warp][(ob.head + (unsigned)__popc(wm & ((1u << lane) - 1u))) % kCap]) = key;
     ob.head += n;
     __syncwarp();
-    if (lane == 0) {
-        fence_cta();
-        *reinterpret_cast<volatile unsigned *>(&C.head[warp]) = ob.head;
-    }
+    if (lane == 0) st_release_shared(&C.head[warp], ob.head);
 }
 
 // The ragged ends of a piece: lane e < count judges element first + e
@@ -465,7 +465,7 @@ __device__ void consume_piece(const TopkParams &P, const Piece &pc, int k, int p
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_addr(&S.empty[slot]));
     }
-    // this warp's candidates of the piece are all in the queue
+    // this warp's candidates of the piece are all in its ring
     __syncwarp();
     if (lane == 0) {
         fence_cta();
@@ -630,10 +630,10 @@ __device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
 }
 
 // The selection warp.  Lane r holds entry r of the current piece's list, best first; candidates
-// arrive through the piece's queue in shared memory and are inserted by a ballot and a shuffle;
+// arrive through the consumer warps' rings in shared memory and are inserted by a ballot and a shuffle;
 // the k-th key is published for the consumers to filter with.  At the end of a piece the warp
 // frees the channel (boundary_arrive) before it writes the list out, counts the piece's
-// blocks and, when that completes a sequence, folds it; the other channel's queue buffers the
+// blocks and, when that completes a sequence, folds it; the other channel's rings buffer the
 // next piece's candidates meanwhile.
 template <int DT>
 __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long blk, unsigned long long blk_end)
@@ -658,7 +658,7 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
         unsigned idle = 0;
         for (;;) {
             const bool last_look = ld_shared_volatile_u32(&C.done) == (unsigned)kConsWarps;  // read before the heads
-            const unsigned h = lane < kConsWarps ? ld_shared_volatile_u32(&C.head[lane]) : 0u;
+            const unsigned h = lane < kConsWarps ? ld_acquire_shared(&C.head[lane]) : 0u;
             unsigned pend = __ballot_sync(kFullMask, lane < kConsWarps && h != tl);
             if (!pend) {
                 if (last_look) break;
@@ -681,8 +681,7 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
                 // the keys are in registers: give the slots back
                 if (lane == w) {
                     tl = hw;
-                    fence_cta();
-                    *reinterpret_cast<volatile unsigned *>(&C.tail[w]) = hw;
+                    st_release_shared(&C.tail[w], hw);
                 }
                 while (want) {
                     const int src = __ffs(want) - 1;
