@@ -10,6 +10,8 @@ The metric is verified rows per second, rows = B * (gamma + 1).
 With N > 1 (launched through torch.distributed.run) every rank verifies its own batch of the
 same shape (sequences are independent: no data-path collective); time is the maximum over ranks.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+`--sampler topk [--k 10]` runs the same round on distributions truncated to their k most likely
+tokens (dssd_edge_verify_topk, dssd_device_resample_topk), the sampler of the paper's experiments.
 """
 from __future__ import annotations
 
@@ -41,6 +43,18 @@ NCU_TRAFFIC = {
     # profiles/edge_verify_kernel_c4.md: 445.8 MB read + 98.0 MB written
     "c4": {"bytes": 543830016, "kernel_hash": "e57acd19c795ee01"},
 }
+
+
+# the same for topk_verify_kernel (k = 10)
+NCU_TRAFFIC_TOPK = {}
+
+
+def _kernel_hash_topk() -> str:
+    h = hashlib.sha256()
+    for f in ("topk_verify.cu", "topk_verify.h", "dssd_device.cuh"):
+        with open(os.path.join(ROOT, "paper_2507_12000_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
 
 
 def _kernel_hash() -> str:
@@ -362,6 +376,204 @@ def run_ours(args, w: di.Workload):
         dist.destroy_process_group()
 
 
+def topk_algorithmic_bytes(w: di.Workload) -> int:
+    """Bytes dssd_edge_verify_topk must move: every logit once (its outputs are k pairs per sequence)."""
+    return w.rows * w.V * w.logit_bytes
+
+
+def _config_topk(w: di.Workload, args):
+    c = _config(w, args)
+    c["workload"] = c["workload"].replace(f"{w.name}:", f"{w.name} with top-k sampling, k={args.k}:")
+    c["k"] = args.k
+    return c
+
+
+def run_reference_topk(args, w: di.Workload):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import oracle as O
+
+    O.build()
+    cores = os.cpu_count() or 1
+    n_seq = min(w.B, args.ref_sequences)
+    d = di.generate_topk(w, args.k, 0, n_seq, threads=cores)
+    for _ in range(args.warmup):
+        O.verify_round_topk(d, w.temperature, args.k, threads=cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.verify_round_topk(d, w.temperature, args.k, threads=cores)
+    dt = time.perf_counter() - t0
+    value = args.steps * n_seq * (w.gamma + 1) / dt
+    sample = f"first {n_seq} of {w.B} sequences of {w.name} per step, k={args.k}, both halves, float64"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config_topk(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours_topk(args, w: di.Workload):
+    import torch
+    import torch.distributed as dist
+
+    from oracle import oracle as O
+
+    O.build()  # before the first CUDA call
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cores = os.cpu_count() or 1
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2507_12000_b200 import binding as B
+
+    k = args.k
+    wr = rank_workload(w, rank)
+    d = di.generate_topk(wr, k, threads=max(1, cores // max(1, min(world, 8))))
+    logit_bytes = d["target_logits"].nbytes
+    copies = 1 if logit_bytes > 200e6 else int(min(64, 300e6 // max(logit_bytes, 1) + 1))
+    sets = [_torch_inputs(d, dev) for _ in range(copies)]
+    gamma, Bn, V = w.gamma, w.B, w.V
+    ws = torch.empty(B.dssd_edge_verify_topk_workspace_bytes(Bn, gamma, V, k), dtype=torch.uint8, device=dev)
+    ev_out = None
+    rs_out = None
+
+    def step(g):
+        nonlocal ev_out, rs_out
+        ev_out = B.dssd_edge_verify_topk(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                         w.temperature, k, out=ev_out, workspace=ws)
+        rs_out = B.dssd_device_resample_topk(ev_out["p_idx"], ev_out["p_val"], g["q_idx"], g["q_val"],
+                                             ev_out["accept_len"], g["uniforms_rs"], gamma, out=rs_out)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % copies])
+    torch.cuda.synchronize()
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.perf_counter()
+    for i in range(K):
+        g = sets[i % copies]
+        ev[i][0].record()
+        ev_out = B.dssd_edge_verify_topk(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                         w.temperature, k, out=ev_out, workspace=ws)
+        ev[i][1].record()
+        rs_out = B.dssd_device_resample_topk(ev_out["p_idx"], ev_out["p_val"], g["q_idx"], g["q_val"],
+                                             ev_out["accept_len"], g["uniforms_rs"], gamma, out=rs_out)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    t_host1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
+    edge_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    rs_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    if world > 1:
+        total_ms = max_over_ranks(total_ms, dist, dev)
+    sampler.stop_flag = True
+    sampler.join(timeout=1.0)
+    clocks = sampler.summary(t_host0, t_host1)
+    n_gpu = ev_out["accept_len"].cpu().numpy()
+    tok_gpu = rs_out["token"].cpu().numpy()
+
+    # ---- end to end: inputs start in pinned host memory, the tokens end there; copies are timed ----
+    host = _torch_inputs(d, pin=True)
+    names = ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "q_idx", "q_val", "uniforms_rs")
+    stage = {n: torch.empty_like(sets[0][n]) for n in names}
+    h_n = torch.empty(Bn, dtype=torch.int32).pin_memory()
+    h_tok = torch.empty(Bn, dtype=torch.int32).pin_memory()
+
+    def e2e_step():
+        for n in names:
+            stage[n].copy_(host[n], non_blocking=True)
+        step(stage)
+        h_n.copy_(ev_out["accept_len"], non_blocking=True)
+        h_tok.copy_(rs_out["token"], non_blocking=True)
+
+    e2e_steps = max(3, min(K, args.e2e_steps))
+    for _ in range(2):
+        e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = 2 * Bn * 4
+    assert (h_n.numpy() == n_gpu).all() and (h_tok.numpy() == tok_gpu).all()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    rows = w.rows
+    ms_per_step = total_ms / K
+    peak, peak_kind = _peaks()
+    edge_avg_ms = sum(edge_ms) / K
+    edge_bytes = topk_algorithmic_bytes(w)
+    achieved = edge_bytes / (edge_avg_ms * 1e-3) / 1e9
+    cpu = None
+    parity = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_seq = min(Bn, args.ref_sequences)
+        sub = {kk: v[:n_seq] for kk, v in d.items()}
+        passes, t0 = 0, time.perf_counter()
+        while True:
+            ref = O.verify_round_topk(sub, w.temperature, k, threads=cores)
+            passes += 1
+            dt = time.perf_counter() - t0
+            if dt >= 1.5 or passes >= 64:
+                break
+        cpu = {"value": passes * n_seq * (gamma + 1) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {n_seq} of {Bn} sequences of {w.name}, k={k}, both halves, {passes} passes in "
+                         f"{dt:.2f} s wall on {cores} threads"}
+        edge = ref["margin_acc"] < 1e-12
+        parity = {"sequences_checked": n_seq,
+                  "accept_len_mismatch": int(((n_gpu[:n_seq] != ref["accept_len"]) & ~edge).sum()),
+                  "support_mismatch": int((ev_out["p_idx"].cpu().numpy()[:n_seq] != ref["p_idx"]).any(axis=1).sum()),
+                  "token_mismatch": int((tok_gpu[:n_seq] != ref["token"]).sum()),
+                  "accept_rate": float(ref["accept_len"].mean() / max(gamma, 1))}
+    line = {
+        "metric": METRIC, "value": world * rows / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": _config_topk(w, args),
+        "roofline": {"bound": "hbm", "kernel": "topk_verify_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": edge_bytes, "avg_launch_ms": edge_avg_ms,
+                     "min_launch_ms": min(edge_ms), "traffic": NCU_TRAFFIC_TOPK.get(w.name, {}).get("bytes")
+                     if NCU_TRAFFIC_TOPK.get(w.name, {}).get("kernel_hash") == _kernel_hash_topk() else None},
+        "resample": {"avg_launch_ms": sum(rs_ms) / K},
+        "edge_rows_per_s": world * rows / (edge_avg_ms * 1e-3),
+        "cpu_baseline": cpu,
+        "parity": parity,
+        "e2e": {"value": world * rows / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 2 * K,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -372,11 +584,15 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-sequences", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sampler", default="full", choices=["full", "topk"])
+    ap.add_argument("--k", type=int, default=10)
     args = ap.parse_args()
     w = di.get_workload(args.workload)
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 2000
-    if args.impl == "reference":
+    if args.sampler == "topk":
+        (run_reference_topk if args.impl == "reference" else run_ours_topk)(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

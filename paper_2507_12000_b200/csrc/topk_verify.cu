@@ -921,7 +921,10 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
     P.total_blocks = rows * (unsigned long long)P.nb;
     // every span must hold at least ceil(nb / (max_pieces - 1)) blocks, so that no row is shared
     // by more than max_pieces CTAs
-    const unsigned long long wmin = ((unsigned long long)P.nb + P.max_pieces - 2) / (unsigned long long)(P.max_pieces - 1);
+    unsigned long long wmin = ((unsigned long long)P.nb + P.max_pieces - 2) / (unsigned long long)(P.max_pieces - 1);
+    // a span below about 32 KB is not worth a CTA of its own: small launches get fewer, larger pieces
+    const unsigned long long worth = 32768ull / ((unsigned long long)kTopkBlock * (dtype == DSSD_BF16 ? 2u : 4u));
+    if (wmin < worth) wmin = worth;
     unsigned long long grid = P.total_blocks / wmin;
     if (grid > (unsigned long long)ctas) grid = (unsigned long long)ctas;
     if (grid < 1) grid = 1;
