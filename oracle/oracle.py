@@ -161,12 +161,25 @@ def device_resample(p_row: np.ndarray, draft_q: Optional[np.ndarray], accept_len
     return out
 
 
-def verify_round(inputs: Dict[str, np.ndarray], temperature: float, threads: int = 1) -> Dict[str, np.ndarray]:
-    """Both halves on one generated batch: the device half consumes the float32 row
-    that the edge half emitted, as it would after the downlink."""
+def to_payload16(p_row64: np.ndarray) -> np.ndarray:
+    """The downlink row at b_prob = 16 bits (Section 2.2 allows 16 or 32): every probability
+    rounded once, from float64, to IEEE binary16 (nearest, ties to even; values below 2**-25
+    become 0, those below 2**-14 lose precision as subnormals).  Returns float16."""
+    return np.asarray(p_row64, dtype=np.float64).astype(np.float16)
+
+
+def verify_round(inputs: Dict[str, np.ndarray], temperature: float, threads: int = 1,
+                 payload: str = "f32") -> Dict[str, np.ndarray]:
+    """Both halves on one generated batch: the device half consumes the row that the edge half
+    emitted, as it would after the downlink: float32, or with payload="f16" the 16-bit row
+    (widened exactly to float32 for the draw)."""
     ev = edge_verify(inputs["target_logits"], inputs["draft_tokens"], inputs["draft_q_tok"],
-                     inputs["uniforms"], temperature, threads=threads)
+                     inputs["uniforms"], temperature, want_p_row64=(payload == "f16"), threads=threads)
     gamma = inputs["target_logits"].shape[1] - 1
+    if payload == "f16":
+        ev["p_row16"] = to_payload16(ev["p_row64"])
+        ev["p_row"] = ev["p_row16"].astype(np.float32)
+        ev["p_row64"] = None
     rs = device_resample(ev["p_row"], inputs["draft_q"], ev["accept_len"], inputs["uniforms_rs"],
                          gamma, threads=threads)
     out = dict(ev)

@@ -420,3 +420,39 @@ def test_degenerate_inputs(oracle_mod):
     ev = oracle_mod.edge_verify(lg, np.array([[0]], np.int32), np.array([[0.5]], np.float32),
                                 np.array([[0.0]], np.float32), 1.0)
     assert ev["accept_len"][0] == 0
+
+
+def test_p7_sixteen_bit_payload(oracle_mod):
+    """The b_prob = 16 row: one rounding to IEEE binary16, nearest-even, checked against bit
+    patterns worked out by hand; the draw then runs on the widened row unchanged."""
+    cases = [
+        (1.0, 0x3C00), (0.5, 0x3800), (1.0 / 3.0, 0x3555), (0.1, 0x2E66), (2.0 ** -14, 0x0400),
+        (2.0 ** -24, 0x0001),                      # smallest subnormal
+        (2.0 ** -25, 0x0000),                      # exactly half of it: ties to even, i.e. zero
+        (2.0 ** -25 * (1 + 2.0 ** -40), 0x0001),   # just above the tie
+        (1.0 + 2.0 ** -11, 0x3C00),                # tie between 1 and 1 + 2^-10: even mantissa wins
+        (1.0 + 3 * 2.0 ** -11, 0x3C02),            # tie between 1 + 2^-10 and 1 + 2^-9
+        (0.0, 0x0000), (3e-9, 0x0000),
+        # a value whose float32 rounding would sit on a binary16 tie, while the float64 value does not
+        (1.0 + 2.0 ** -11 + 2.0 ** -30, 0x3C01),
+    ]
+    got = oracle_mod.to_payload16(np.array([c[0] for c in cases], np.float64)).view(np.uint16)
+    assert got.tolist() == [c[1] for c in cases]
+    w = di.custom(B=12, gamma=3, V=3000, dtype="bf16", temperature=0.9, seed=21)
+    d = di.generate(w)
+    full = oracle_mod.verify_round(d, w.temperature)
+    half = oracle_mod.verify_round(d, w.temperature, payload="f16")
+    assert half["p_row16"].dtype == np.float16 and (half["accept_len"] == full["accept_len"]).all()
+    p16 = half["p_row16"].astype(np.float64)
+    p32 = full["p_row"].astype(np.float64)
+    normal = p32 >= 2.0 ** -14
+    assert (np.abs(p16 - p32)[normal] <= 2.0 ** -11 * p32[normal] * (1 + 1e-6)).all()
+    assert (np.abs(p16 - p32)[~normal] <= 2.0 ** -25 * (1 + 1e-6)).all()
+    assert (np.abs(p16.sum(axis=1) - 1.0) < 2e-3).all()
+    order = np.argsort(p32, axis=1, kind="stable")
+    assert (np.diff(np.take_along_axis(p16, order, axis=1), axis=1) >= 0).all()  # rounding keeps the order
+    # the draw on the 16-bit row is the dense draw on its widened values
+    again = oracle_mod.device_resample(half["p_row16"].astype(np.float32), d["draft_q"], half["accept_len"],
+                                       d["uniforms_rs"], w.gamma)
+    assert (again["token"] == half["token"]).all()
+    assert (half["token"] == full["token"]).mean() > 0.7  # most draws do not sit within 2^-11 of a CDF step
