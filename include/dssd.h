@@ -12,7 +12,9 @@
  *   dssd_round_host       both halves on host buffers, with the copies to and from the GPU;
  *   dssd_edge_verify_topk, dssd_device_resample_topk
  *                         the same round on distributions truncated to their k most likely
- *                         tokens, the sampler of the paper's experiments (Section 4).
+ *                         tokens, the sampler of the paper's experiments (Section 4);
+ *   dssd_edge_verify_p16, dssd_device_resample_p16
+ *                         the round with the downlink row in 16 bits per value (Section 2.2).
  *
  * Notation follows the paper: gamma draft tokens x_1..x_gamma with draft probabilities
  * q_i(x_i), target distributions P_1..P_{gamma+1} over a vocabulary of V entries, uniforms
@@ -270,6 +272,43 @@ dssd_status dssd_device_resample_topk(const int32_t *p_idx, const float *p_val,
                                       const int32_t *accept_len, const float *uniforms, int B,
                                       int gamma, int k, int32_t *token, uint32_t *flags,
                                       void *cuda_stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------
+ * 16-bit downlink payload (Section 2.2: a probability value takes b_prob = 32 or 16 bits; the
+ * payload |V| * b_prob of Section 3.1 halves).
+ *
+ * Reading of "16 bits": IEEE binary16, each probability rounded once to nearest-even.  Values
+ * below 2^-25 become 0 and those below 2^-14 are subnormal, so the far tail of a row loses its
+ * mass; the relative error of a normal value is at most 2^-11.
+ * ---------------------------------------------------------------------------------------------
+ */
+
+/*
+ * dssd_edge_verify with the row P_n(.) written as binary16 bit patterns.  Everything else -
+ * inputs, decisions, accept_len, p_tok, lse, flags, workspace - is as in dssd_edge_verify; the
+ * kernel writes half the bytes.  The probabilities are computed in float32 as there and rounded
+ * once more, so a value may differ from the float64 value's rounding by one unit in the last
+ * place of binary16.
+ *
+ * p_row16  [B, V] uint16 out: binary16 bit patterns of P_n(.), 2-byte aligned (8-byte aligned rows
+ *          take the fast path)
+ */
+dssd_status dssd_edge_verify_p16(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                 const int32_t *draft_tokens, const float *draft_q_tok,
+                                 const float *uniforms, float temperature, int B, int gamma, int V,
+                                 int32_t *accept_len, uint16_t *p_row16, float *p_tok, float *lse,
+                                 uint32_t *flags, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream);
+
+/*
+ * dssd_device_resample on a binary16 row: every p_v is widened exactly to float32 and the draw
+ * is the one of dssd_device_resample (same sums in float64, same flags, same workspace size).
+ */
+dssd_status dssd_device_resample_p16(const uint16_t *p_row16, const float *draft_q,
+                                     const int32_t *accept_len, const float *uniforms, int B,
+                                     int gamma, int V, int32_t *token, uint32_t *flags,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 #ifdef __cplusplus
 }

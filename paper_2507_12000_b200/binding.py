@@ -81,6 +81,10 @@ def _load() -> ctypes.CDLL:
     L.dssd_device_resample_topk.argtypes = [
         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
         c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p]
+    L.dssd_edge_verify_p16.restype = c.c_int
+    L.dssd_edge_verify_p16.argtypes = L.dssd_edge_verify.argtypes
+    L.dssd_device_resample_p16.restype = c.c_int
+    L.dssd_device_resample_p16.argtypes = L.dssd_device_resample.argtypes
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -129,10 +133,11 @@ def dssd_round_host_arena_bytes(B: int, gamma: int, V: int, dtype: int) -> int:
 def dssd_edge_verify(target_logits: torch.Tensor, draft_tokens: torch.Tensor, draft_q_tok: torch.Tensor,
                      uniforms: torch.Tensor, temperature: float, *, out: Optional[Dict[str, torch.Tensor]] = None,
                      want_p_tok: bool = True, want_lse: bool = True, workspace: Optional[torch.Tensor] = None,
-                     stream=None) -> Dict[str, torch.Tensor]:
+                     stream=None, payload: str = "f32") -> Dict[str, torch.Tensor]:
     """Edge half of one round.  target_logits: CUDA tensor [B, gamma+1, V], float32 or bfloat16,
     unit stride along V and a common stride between rows.  Returns accept_len, p_row, flags and,
-    if asked, p_tok and lse.  Pass `out` (a previous result) and `workspace` to allocate nothing."""
+    if asked, p_tok and lse.  Pass `out` (a previous result) and `workspace` to allocate nothing.
+    payload="f16" writes p_row as float16 (dssd_edge_verify_p16)."""
     assert target_logits.is_cuda and target_logits.dim() == 3
     B, g1, V = target_logits.shape
     gamma = g1 - 1
@@ -144,15 +149,17 @@ def dssd_edge_verify(target_logits: torch.Tensor, draft_tokens: torch.Tensor, dr
     if out is None:
         out = {
             "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
-            "p_row": torch.empty(B, V, dtype=torch.float32, device=dev),
+            "p_row": torch.empty(B, V, dtype=torch.float16 if payload == "f16" else torch.float32, device=dev),
             "flags": torch.empty(B, dtype=torch.int32, device=dev),
             "p_tok": torch.empty(B, gamma, dtype=torch.float32, device=dev) if want_p_tok else None,
             "lse": torch.empty(B, g1, dtype=torch.float32, device=dev) if want_lse else None,
         }
+    assert out["p_row"].dtype == (torch.float16 if payload == "f16" else torch.float32)
     need = dssd_edge_verify_workspace_bytes(B, gamma, V)
     if workspace is None:
         workspace = _workspace(need, dev)
-    st = lib.dssd_edge_verify(
+    fn = lib.dssd_edge_verify_p16 if payload == "f16" else lib.dssd_edge_verify
+    st = fn(
         target_logits.data_ptr(), _dtype_code(target_logits), row_stride,
         _ptr(draft_tokens), _ptr(draft_q_tok), _ptr(uniforms), ctypes.c_float(temperature), B, gamma, V,
         out["accept_len"].data_ptr(), out["p_row"].data_ptr(), _ptr(out.get("p_tok")), _ptr(out.get("lse")),
@@ -165,8 +172,9 @@ def dssd_edge_verify(target_logits: torch.Tensor, draft_tokens: torch.Tensor, dr
 def dssd_device_resample(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], accept_len: torch.Tensor,
                          uniforms_rs: torch.Tensor, gamma: int, *, out: Optional[Dict[str, torch.Tensor]] = None,
                          workspace: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
-    """Device half of one round.  p_row [B, V] float32, draft_q [B, gamma, V] float32 (contiguous)."""
-    assert p_row.is_cuda and p_row.dim() == 2 and p_row.is_contiguous() and p_row.dtype == torch.float32
+    """Device half of one round.  p_row [B, V] float32 (or float16: dssd_device_resample_p16),
+    draft_q [B, gamma, V] float32 (contiguous)."""
+    assert p_row.is_cuda and p_row.dim() == 2 and p_row.is_contiguous() and p_row.dtype in (torch.float32, torch.float16)
     B, V = p_row.shape
     if gamma > 0:
         assert draft_q.is_contiguous() and draft_q.dtype == torch.float32 and draft_q.numel() == B * gamma * V
@@ -177,7 +185,8 @@ def dssd_device_resample(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], a
     need = dssd_device_resample_workspace_bytes(B, gamma, V)
     if workspace is None:
         workspace = _workspace(need, dev)
-    st = lib.dssd_device_resample(
+    fn = lib.dssd_device_resample_p16 if p_row.dtype == torch.float16 else lib.dssd_device_resample
+    st = fn(
         p_row.data_ptr(), _ptr(draft_q) if gamma > 0 else None, accept_len.data_ptr(), uniforms_rs.data_ptr(),
         B, gamma, V, out["token"].data_ptr(), _ptr(out.get("flags")), workspace.data_ptr(), workspace.numel(),
         _stream(stream))

@@ -59,23 +59,24 @@ size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V)
     return dssd::edge_workspace_layout(B, gamma, dssd::edge_max_runs_per_row(V), nullptr, nullptr);
 }
 
-dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
-                             const int32_t *draft_tokens, const float *draft_q_tok,
-                             const float *uniforms, float temperature, int B, int gamma, int V,
-                             int32_t *accept_len, float *p_row, float *p_tok, float *lse,
-                             uint32_t *flags, void *workspace, size_t workspace_bytes,
-                             void *cuda_stream)
+namespace {
+dssd_status edge_verify_any(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                            const int32_t *draft_tokens, const float *draft_q_tok, const float *uniforms,
+                            float temperature, int B, int gamma, int V, int32_t *accept_len, float *p_row,
+                            uint16_t *p_row16, float *p_tok, float *lse, uint32_t *flags, void *workspace,
+                            size_t workspace_bytes, void *cuda_stream)
 {
     t_last_cuda_error = 0;
     dssd_status st = check_sizes(B, gamma, V);
     if (st != DSSD_OK) return st;
     if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
-    if (!target_logits || !accept_len || !p_row) return DSSD_ERR_INVALID_ARG;
+    if (!target_logits || !accept_len || (!p_row && !p_row16)) return DSSD_ERR_INVALID_ARG;
     if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms)) return DSSD_ERR_INVALID_ARG;
     if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
     if (row_stride < (int64_t)V) return DSSD_ERR_INVALID_ARG;
     const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
-    if ((reinterpret_cast<uintptr_t>(target_logits) % esz) || (reinterpret_cast<uintptr_t>(p_row) % 4))
+    if ((reinterpret_cast<uintptr_t>(target_logits) % esz) || (reinterpret_cast<uintptr_t>(p_row) % 4) ||
+        (reinterpret_cast<uintptr_t>(p_row16) % 2))
         return DSSD_ERR_INVALID_ARG;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < dssd_edge_verify_workspace_bytes(B, gamma, V))
@@ -93,11 +94,37 @@ dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_
     P.V = V;
     P.accept_len = accept_len;
     P.p_row = p_row;
+    P.p_row16 = p_row16;
     P.p_tok = p_tok;
     P.lse = lse;
     P.flags = flags;
     cudaError_t e = dssd::edge_verify_launch(P, (int)dtype, workspace, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+}  // namespace
+
+dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                             const int32_t *draft_tokens, const float *draft_q_tok,
+                             const float *uniforms, float temperature, int B, int gamma, int V,
+                             int32_t *accept_len, float *p_row, float *p_tok, float *lse,
+                             uint32_t *flags, void *workspace, size_t workspace_bytes,
+                             void *cuda_stream)
+{
+    if (!p_row) return DSSD_ERR_INVALID_ARG;
+    return edge_verify_any(target_logits, dtype, row_stride, draft_tokens, draft_q_tok, uniforms, temperature, B, gamma,
+                           V, accept_len, p_row, nullptr, p_tok, lse, flags, workspace, workspace_bytes, cuda_stream);
+}
+
+dssd_status dssd_edge_verify_p16(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                 const int32_t *draft_tokens, const float *draft_q_tok,
+                                 const float *uniforms, float temperature, int B, int gamma, int V,
+                                 int32_t *accept_len, uint16_t *p_row16, float *p_tok, float *lse,
+                                 uint32_t *flags, void *workspace, size_t workspace_bytes,
+                                 void *cuda_stream)
+{
+    if (!p_row16) return DSSD_ERR_INVALID_ARG;
+    return edge_verify_any(target_logits, dtype, row_stride, draft_tokens, draft_q_tok, uniforms, temperature, B, gamma,
+                           V, accept_len, nullptr, p_row16, p_tok, lse, flags, workspace, workspace_bytes, cuda_stream);
 }
 
 size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V)
@@ -106,17 +133,17 @@ size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V)
     return dssd::resample_workspace_layout(B, V, nullptr, nullptr);
 }
 
-dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
-                                 const int32_t *accept_len, const float *uniforms, int B,
-                                 int gamma, int V, int32_t *token, uint32_t *flags,
-                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+namespace {
+dssd_status device_resample_any(const void *p_row, int p_half, const float *draft_q, const int32_t *accept_len,
+                                const float *uniforms, int B, int gamma, int V, int32_t *token, uint32_t *flags,
+                                void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
     t_last_cuda_error = 0;
     dssd_status st = check_sizes(B, gamma, V);
     if (st != DSSD_OK) return st;
     if (!p_row || !accept_len || !uniforms || !token) return DSSD_ERR_INVALID_ARG;
     if (gamma > 0 && !draft_q) return DSSD_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(p_row) % 4) || (reinterpret_cast<uintptr_t>(draft_q) % 4))
+    if ((reinterpret_cast<uintptr_t>(p_row) % (p_half ? 2 : 4)) || (reinterpret_cast<uintptr_t>(draft_q) % 4))
         return DSSD_ERR_INVALID_ARG;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
         workspace_bytes < dssd_device_resample_workspace_bytes(B, gamma, V))
@@ -124,6 +151,7 @@ dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
 
     dssd::ResampleParams P{};
     P.p_row = p_row;
+    P.p_half = p_half;
     P.draft_q = draft_q;
     P.accept_len = accept_len;
     P.uniforms = uniforms;
@@ -134,6 +162,25 @@ dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
     P.flags = flags;
     cudaError_t e = dssd::resample_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+}  // namespace
+
+dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
+                                 const int32_t *accept_len, const float *uniforms, int B,
+                                 int gamma, int V, int32_t *token, uint32_t *flags,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return device_resample_any(p_row, 0, draft_q, accept_len, uniforms, B, gamma, V, token, flags, workspace,
+                               workspace_bytes, cuda_stream);
+}
+
+dssd_status dssd_device_resample_p16(const uint16_t *p_row16, const float *draft_q,
+                                     const int32_t *accept_len, const float *uniforms, int B,
+                                     int gamma, int V, int32_t *token, uint32_t *flags,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return device_resample_any(p_row16, 1, draft_q, accept_len, uniforms, B, gamma, V, token, flags, workspace,
+                               workspace_bytes, cuda_stream);
 }
 
 size_t dssd_edge_verify_topk_workspace_bytes(int B, int gamma, int V, int k)

@@ -34,57 +34,106 @@ __device__ __forceinline__ float4 as_f4(const uint4 &v)
     return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
 }
 
-// per-thread part of sum_{e in [e0,e1)} r_e ; q == nullptr means r = p
-__device__ __forceinline__ double chunk_mass(const float *p, const float *q, int e0, int e1)
+// The row p comes as float32 or, for the 16-bit payload, as IEEE binary16 bit patterns; the
+// kernel is written once over these accessors.  A "quad" is four consecutive entries.
+__device__ __forceinline__ float half_bits_to_float(unsigned short h) { return __half2float(__ushort_as_half(h)); }
+__device__ __forceinline__ float4 half_quad(uint2 v)
 {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&v.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+template <typename PT>
+struct PAcc;
+template <>
+struct PAcc<float> {
+    typedef uint4 Raw;
+    static constexpr unsigned kAlignMask = 15u;  // a quad is loaded with one 16-byte access
+    __device__ static __forceinline__ float ld(const float *p, int64_t e) { return __ldg(p + e); }
+    __device__ static __forceinline__ Raw ld_quad_stream(const float *p, int64_t quad)
+    {
+        return ld_stream16(reinterpret_cast<const uint4 *>(p) + quad);
+    }
+    __device__ static __forceinline__ float4 quad(const Raw &v) { return as_f4(v); }
+    __device__ static __forceinline__ float4 ld_quad(const float *p, int64_t quad)
+    {
+        return __ldg(reinterpret_cast<const float4 *>(p) + quad);
+    }
+};
+template <>
+struct PAcc<uint16_t> {
+    typedef uint2 Raw;
+    static constexpr unsigned kAlignMask = 7u;  // a quad is loaded with one 8-byte access
+    __device__ static __forceinline__ float ld(const uint16_t *p, int64_t e) { return half_bits_to_float(__ldg(p + e)); }
+    __device__ static __forceinline__ Raw ld_quad_stream(const uint16_t *p, int64_t quad)
+    {
+        uint2 v;
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
+                     : "=r"(v.x), "=r"(v.y)
+                     : "l"(reinterpret_cast<const uint2 *>(p) + quad));
+        return v;
+    }
+    __device__ static __forceinline__ float4 quad(const Raw &v) { return half_quad(v); }
+    __device__ static __forceinline__ float4 ld_quad(const uint16_t *p, int64_t quad)
+    {
+        return half_quad(__ldg(reinterpret_cast<const uint2 *>(p) + quad));
+    }
+};
+
+// per-thread part of sum_{e in [e0,e1)} r_e ; q == nullptr means r = p
+template <typename PT>
+__device__ __forceinline__ double chunk_mass(const PT *p, const float *q, int e0, int e1)
+{
+    typedef PAcc<PT> A;
     const int tid = threadIdx.x;
     double acc = 0.0;
     int done = e0;
-    const bool aligned =
-        ((reinterpret_cast<uintptr_t>(p + e0) | (q ? reinterpret_cast<uintptr_t>(q + e0) : 0)) & 15u) == 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(p + e0) & A::kAlignMask) == 0 &&
+                         (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0);
     if (aligned) {
         const int nvec = (e1 - e0) / 4;
-        const uint4 *p4 = reinterpret_cast<const uint4 *>(p + e0);
+        const PT *p4 = p + e0;  // quads are counted from here
         if (q) {
             const uint4 *q4 = reinterpret_cast<const uint4 *>(q + e0);
             int i = tid;
             for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                uint4 a[4], b[4];
+                typename A::Raw a[4];
+                uint4 b[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    a[u] = ld_stream16(p4 + i + u * kThreads);
+                    a[u] = A::ld_quad_stream(p4, i + u * kThreads);
                     b[u] = ld_stream16(q4 + i + u * kThreads);
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float4 x = as_f4(a[u]), y = as_f4(b[u]);
+                    const float4 x = A::quad(a[u]), y = as_f4(b[u]);
                     acc += (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
                 }
             }
             for (; i < nvec; i += kThreads) {
-                const float4 x = as_f4(ld_stream16(p4 + i)), y = as_f4(ld_stream16(q4 + i));
+                const float4 x = A::quad(A::ld_quad_stream(p4, i)), y = as_f4(ld_stream16(q4 + i));
                 acc += (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
             }
         } else {
             int i = tid;
             for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                uint4 a[4];
+                typename A::Raw a[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) a[u] = ld_stream16(p4 + i + u * kThreads);
+                for (int u = 0; u < 4; ++u) a[u] = A::ld_quad_stream(p4, i + u * kThreads);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float4 x = as_f4(a[u]);
+                    const float4 x = A::quad(a[u]);
                     acc += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
                 }
             }
             for (; i < nvec; i += kThreads) {
-                const float4 x = as_f4(ld_stream16(p4 + i));
+                const float4 x = A::quad(A::ld_quad_stream(p4, i));
                 acc += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
             }
         }
         done = e0 + nvec * 4;
     }
-    for (int e = done + tid; e < e1; e += kThreads) acc += q ? res(__ldg(p + e), __ldg(q + e)) : (double)__ldg(p + e);
+    for (int e = done + tid; e < e1; e += kThreads) acc += q ? res(A::ld(p, e), __ldg(q + e)) : (double)A::ld(p, e);
     return acc;
 }
 
@@ -165,7 +214,8 @@ __device__ __forceinline__ double block_scan(double x, double *s_scan, double &t
 }
 
 // pass B for sequence b; q == nullptr means r = p
-__device__ void draw(const ResampleParams &P, int64_t b, const float *p, const float *q, unsigned fl,
+template <typename PT>
+__device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const float *q, unsigned fl,
                      double *s_w, Pick *s_pick, int *s_i)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -288,15 +338,15 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
     int last_pos = -1;
     // The run's 16 entries are all requested before the first is used (one round trip for the
     // run, not one per entry); entries past the row's end read as 0.
-    const bool vec = (r1 - r0 == kRun) &&
-                     (((reinterpret_cast<uintptr_t>(p + r0) | (q ? reinterpret_cast<uintptr_t>(q + r0) : 0)) & 15u) == 0);
+    const bool vec = (r1 - r0 == kRun) && (reinterpret_cast<uintptr_t>(p + r0) & PAcc<PT>::kAlignMask) == 0 &&
+                     (!q || (reinterpret_cast<uintptr_t>(q + r0) & 15u) == 0);
 #pragma unroll
     for (int g = 0; g < kRun; g += 16) {
         float pv[16], qv[16];
         if (vec) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float4 a = __ldg(reinterpret_cast<const float4 *>(p + r0 + g) + j);
+                const float4 a = PAcc<PT>::ld_quad(p + r0 + g, j);
                 pv[4 * j] = a.x, pv[4 * j + 1] = a.y, pv[4 * j + 2] = a.z, pv[4 * j + 3] = a.w;
                 float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (q) c = __ldg(reinterpret_cast<const float4 *>(q + r0 + g) + j);
@@ -306,7 +356,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const int e = r0 + g + j;
-                pv[j] = e < r1 ? __ldg(p + e) : 0.f;
+                pv[j] = e < r1 ? PAcc<PT>::ld(p, e) : 0.f;
                 qv[j] = (q && e < r1) ? __ldg(q + e) : 0.f;
             }
         }
@@ -347,7 +397,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
         double C = before;
         int tok = last_pos;
         for (int e = r0; e < r1; ++e) {
-            C += q ? res(__ldg(p + e), __ldg(q + e)) : (double)__ldg(p + e);
+            C += q ? res(PAcc<PT>::ld(p, e), __ldg(q + e)) : (double)PAcc<PT>::ld(p, e);
             if (C > pk.target) { tok = e; break; }
         }
         P.token[b] = tok >= 0 ? tok : s_i[1];
@@ -355,6 +405,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const float *p, const f
     }
 }
 
+template <typename PT>
 __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ ResampleParams P)
 {
     __shared__ double s_w[2][kWarps][2];
@@ -379,7 +430,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         const int n = __ldg(P.accept_len + b);
         double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
         if (n >= 0 && n <= P.gamma) {
-            const float *p = P.p_row + (size_t)b * P.V;
+            const PT *p = reinterpret_cast<const PT *>(P.p_row) + (size_t)b * P.V;
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
             const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
             acc0 = chunk_mass(p, q, e0, e1);
@@ -434,9 +485,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
                 if (P.flags) P.flags[b] = DSSD_RS_FLAG_INVALID;
             }
         } else {
-            const float *p = P.p_row + (size_t)b * P.V;
+            const PT *p = reinterpret_cast<const PT *>(P.p_row) + (size_t)b * P.V;
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-            draw(P, b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
+            draw<PT>(P, b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
         }
         __syncthreads();
         d = s_ticket[buf];
@@ -477,14 +528,18 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     int dev = 0, sms = 0, occ = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-    if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, resample_kernel, kThreads, 0)) != cudaSuccess) return err;
+    int occ16 = 0;
+    if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, resample_kernel<float>, kThreads, 0)) != cudaSuccess) return err;
+    if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ16, resample_kernel<uint16_t>, kThreads, 0)) != cudaSuccess) return err;
+    if (occ16 < occ) occ = occ16;
     if (occ < 1) occ = 1;
     resample_workspace_layout(P.B, P.V, &P, static_cast<char *>(workspace));
     P.spin_limit = 1u << 20;
     if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long resident = (unsigned long long)sms * (unsigned long long)occ;
     const unsigned grid = (unsigned)(P.total_tickets < resident ? P.total_tickets : resident);
-    resample_kernel<<<grid, kThreads, 0, stream>>>(P);
+    if (P.p_half) resample_kernel<uint16_t><<<grid, kThreads, 0, stream>>>(P);
+    else resample_kernel<float><<<grid, kThreads, 0, stream>>>(P);
     return cudaGetLastError();
 }
 

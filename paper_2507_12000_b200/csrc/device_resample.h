@@ -10,7 +10,8 @@ namespace dssd {
 constexpr int kResampleChunk = 8192;  // vocabulary entries per ticket
 
 struct ResampleParams {
-    const float *p_row;
+    const void *p_row;   // float32 entries, or IEEE binary16 bit patterns when p_half is set
+    int p_half;
     const float *draft_q;
     const int32_t *accept_len;
     const float *uniforms;

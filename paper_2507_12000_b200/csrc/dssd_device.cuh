@@ -1,6 +1,7 @@
 // Device-side helpers shared by the verification kernels (sm_100a).
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -22,6 +23,21 @@ __device__ __forceinline__ uint4 ld_stream16(const void *p)
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
     return v;
+}
+
+// two floats rounded to IEEE binary16 (nearest even), low half = first
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
+{
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+__device__ __forceinline__ unsigned short to_half_bits(float x) { return __half_as_ushort(__float2half_rn(x)); }
+
+// 8-byte streaming store (evict-first)
+__device__ __forceinline__ void st_stream8(void *p, uint32_t a, uint32_t b)
+{
+    asm volatile("st.global.cs.v2.b32 [%0], {%1,%2};" ::"l"(p), "r"(a), "r"(b) : "memory");
 }
 
 // 16-byte streaming store (evict-first): output that this kernel never reads back.

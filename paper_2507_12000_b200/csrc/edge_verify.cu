@@ -322,6 +322,58 @@ __device__ __forceinline__ void emit_consume(uint32_t stage, int nbytes, float *
     }
 }
 
+// The same for the 16-bit payload: four probabilities rounded to IEEE binary16, one 8-byte store
+__device__ __forceinline__ void emit_quad16(uint16_t *out, float z0, float z1, float z2, float z3, f32x2 cc, f32x2 nn, f32x2 ss)
+{
+    float a, b, c, d;
+    unpack2(fma2(pack2(z0, z1), cc, nn), a, b);
+    unpack2(fma2(pack2(z2, z3), cc, nn), c, d);
+    unpack2(mul2(pack2(ex2(a), ex2(b)), ss), a, b);
+    unpack2(mul2(pack2(ex2(c), ex2(d)), ss), c, d);
+    st_stream8(out, pack_half2(a, b), pack_half2(c, d));
+}
+
+template <int DT>
+__device__ __forceinline__ void emit_consume16(uint32_t stage, int nbytes, uint16_t *body, float c1, float nref, float invS)
+{
+    using E = Elem<DT>;
+    const int lane = threadIdx.x & 31;
+    const int nelem = nbytes / E::kBytes;
+    const f32x2 cc = pack2(c1, c1), nn = pack2(nref, nref), ss = pack2(invS, invS);
+    if ((reinterpret_cast<uintptr_t>(body) & 7u) == 0) {
+        const int nquad = nelem >> 2;
+        if (DT == DSSD_BF16) {
+            const uint32_t base = stage + (uint32_t)lane * 8u;
+#pragma unroll 4
+            for (int i = lane; i < nquad; i += 32) {
+                const uint2 w = lds8(base + (uint32_t)(i - lane) * 8u);
+                emit_quad16(body + (size_t)i * 4, bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y), cc, nn, ss);
+            }
+        } else {
+            const uint32_t base = stage + (uint32_t)lane * 16u;
+#pragma unroll 4
+            for (int i = lane; i < nquad; i += 32) {
+                const uint4 w = lds16(base + (uint32_t)(i - lane) * 16u);
+                emit_quad16(body + (size_t)i * 4, __uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z),
+                            __uint_as_float(w.w), cc, nn, ss);
+            }
+        }
+    } else {
+        // output not 8-byte aligned here: coalesced 2-byte stores
+        for (int i = lane; i < nelem; i += 32) {
+            float z;
+            if (DT == DSSD_BF16) {
+                unsigned short h;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(stage + (uint32_t)i * 2u));
+                z = __uint_as_float((uint32_t)h << 16);
+            } else {
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(z) : "r"(stage + (uint32_t)i * 4u));
+            }
+            body[i] = to_half_bits(ex2(fmaf(z, c1, nref)) * invS);
+        }
+    }
+}
+
 // ---- the fold warp -------------------------------------------------------------------------
 
 // v * 2^d for an integer d <= 0 and a normal, positive v of float32 range: exponent arithmetic,
@@ -673,14 +725,23 @@ __device__ __forceinline__ void consumer_warp(const EdgeParams &P, Shared *sh, u
                 for_ragged<DT>(P, lt.head, k, [&](int64_t e) { online_add(o, E::load(rowp, e), c1); });
             }
         } else if (et.out_off >= 0) {
-            float *outp = P.p_row + et.out_off;
             const float nref = -et.ref2, invS = et.invS;
-            if (v1 > v0)
-                emit_consume<DT>(stage + (uint32_t)v0 * 16u, (v1 - v0) * 16,
-                                 outp + (et.head + (long long)k * kS + (long long)v0 * 16) / E::kBytes, c1, nref, invS);
-            if ((meta & kMetaRagged) && w == 0) {
-                const char *rowp = row_ptr<DT>(P, et.row);
-                for_ragged<DT>(P, et.head, k, [&](int64_t e) { outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS; });
+            const long long first = (et.head + (long long)k * kS + (long long)v0 * 16) / E::kBytes;
+            if (P.p_row16) {
+                uint16_t *outp = P.p_row16 + et.out_off;
+                if (v1 > v0) emit_consume16<DT>(stage + (uint32_t)v0 * 16u, (v1 - v0) * 16, outp + first, c1, nref, invS);
+                if ((meta & kMetaRagged) && w == 0) {
+                    const char *rowp = row_ptr<DT>(P, et.row);
+                    for_ragged<DT>(P, et.head, k,
+                                   [&](int64_t e) { outp[e] = to_half_bits(ex2(fmaf(E::load(rowp, e), c1, nref)) * invS); });
+                }
+            } else {
+                float *outp = P.p_row + et.out_off;
+                if (v1 > v0) emit_consume<DT>(stage + (uint32_t)v0 * 16u, (v1 - v0) * 16, outp + first, c1, nref, invS);
+                if ((meta & kMetaRagged) && w == 0) {
+                    const char *rowp = row_ptr<DT>(P, et.row);
+                    for_ragged<DT>(P, et.head, k, [&](int64_t e) { outp[e] = ex2(fmaf(E::load(rowp, e), c1, nref)) * invS; });
+                }
             }
         }
         // release the stage: the arrival orders this warp's reads before the producer's next copy
@@ -1111,12 +1172,36 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         const long long body = rowbytes - head;
         const int nvec = (int)(body >> 4);
         const uint4 *v4 = reinterpret_cast<const uint4 *>(rowp + head);
-        float *outp = P.p_row + (size_t)b * P.V;
-        float *bodyp = outp + head / E::kBytes;
         const float nref = -ref2;
         const f32x2 cc = pack2(c1, c1), nn = pack2(nref, nref), ss = pack2(invS, invS);
-        const bool vec_out = (reinterpret_cast<uintptr_t>(bodyp) & 15u) == 0;
         const int vbeg = (int)((long long)nvec * crank / csize), vend = (int)((long long)nvec * (crank + 1) / csize);
+        if (P.p_row16) {
+            uint16_t *outp = P.p_row16 + (size_t)b * P.V;
+            uint16_t *bodyp = outp + head / E::kBytes;
+            const bool vec_out = (reinterpret_cast<uintptr_t>(bodyp) & 7u) == 0;
+            for (int j = vbeg + tid; j < vend; j += kSmallThreads) {
+                float f[E::kVec];
+                E::unpack(ld_stream16(v4 + j), f);
+                uint16_t *o = bodyp + (size_t)j * E::kVec;
+                if (vec_out) {
+#pragma unroll
+                    for (int q = 0; q < E::kVec; q += 4) emit_quad16(o + q, f[q], f[q + 1], f[q + 2], f[q + 3], cc, nn, ss);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < E::kVec; ++q) o[q] = to_half_bits(ex2(fmaf(f[q], c1, nref)) * invS);
+                }
+            }
+            if (warp == 0 && crank == 0) {
+                if (lane < head / E::kBytes) outp[lane] = to_half_bits(ex2(fmaf(E::load(rowp, lane), c1, nref)) * invS);
+                const int tail = (int)((body - ((long long)nvec << 4)) / E::kBytes);
+                const int64_t e = (int64_t)((head + ((long long)nvec << 4)) / E::kBytes) + lane;
+                if (lane < tail) outp[e] = to_half_bits(ex2(fmaf(E::load(rowp, e), c1, nref)) * invS);
+            }
+            return;
+        }
+        float *outp = P.p_row + (size_t)b * P.V;
+        float *bodyp = outp + head / E::kBytes;
+        const bool vec_out = (reinterpret_cast<uintptr_t>(bodyp) & 15u) == 0;
         for (int j = vbeg + tid; j < vend; j += kSmallThreads) {
             float f[E::kVec];
             E::unpack(ld_stream16(v4 + j), f);

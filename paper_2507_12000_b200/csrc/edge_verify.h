@@ -54,7 +54,8 @@ struct EdgeParams {
     float c1;  // log2(e) / T, rounded to float32; the kernel's temperature scaling throughout
     int B, gamma, V;
     int32_t *accept_len;
-    float *p_row;
+    float *p_row;          // float32 payload, or
+    uint16_t *p_row16;     // IEEE binary16 payload (exactly one of the two is set)
     float *p_tok;
     float *lse;
     uint32_t *flags;
