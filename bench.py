@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 445.8 MB read + 98.0 MB written
-    "c4": {"bytes": 543830016, "kernel_hash": "e57acd19c795ee01"},
+    # profiles/edge_verify_kernel_c4.md: 448.5 MB read + 99.3 MB written
+    "c4": {"bytes": 547835136, "kernel_hash": "74f7d348e60bbe49"},
 }
 
 
@@ -76,14 +76,14 @@ def _peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-def edge_algorithmic_bytes(w: di.Workload) -> int:
-    """Bytes dssd_edge_verify must move: every logit once, plus the float32 row it emits."""
-    return w.B * w.V * ((w.gamma + 1) * w.logit_bytes + 4)
+def edge_algorithmic_bytes(w: di.Workload, payload_bytes: int = 4) -> int:
+    """Bytes dssd_edge_verify must move: every logit once, plus the row it emits (4 or 2 bytes per value)."""
+    return w.B * w.V * ((w.gamma + 1) * w.logit_bytes + payload_bytes)
 
 
-def resample_algorithmic_bytes(w: di.Workload, n_bonus: int) -> int:
+def resample_algorithmic_bytes(w: di.Workload, n_bonus: int, payload_bytes: int = 4) -> int:
     """p row for every sequence, q row for the rejected ones, one token each."""
-    return w.V * 4 * (2 * w.B - n_bonus) + 4 * w.B
+    return w.V * (payload_bytes * w.B + 4 * (w.B - n_bonus)) + 4 * w.B
 
 
 class ClockSampler(threading.Thread):
@@ -152,7 +152,7 @@ def _torch_inputs(d, device=None, pin=False):
     return out
 
 
-def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float = 1.5):
+def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float = 1.5, payload: str = "f32"):
     """rows/s of the CPU oracle (both halves) on the first n_seq sequences: whole passes are
     repeated until about `min_seconds` of wall time (some 10-30 s of CPU work on all cores) have gone."""
     from oracle import oracle as O
@@ -161,7 +161,7 @@ def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float 
     passes = 0
     t0 = time.perf_counter()
     while True:
-        O.verify_round(sub, w.temperature, threads=threads)
+        O.verify_round(sub, w.temperature, threads=threads, payload=payload)
         passes += 1
         dt = time.perf_counter() - t0
         if dt >= min_seconds or passes >= 64:
@@ -204,7 +204,8 @@ def _config(w: di.Workload, args):
             "B": w.B, "gamma": w.gamma, "V": w.V, "logits_dtype": w.dtype, "temperature": w.temperature,
             "l2": "inputs larger than L2, no flush" if w.rows * w.V * w.logit_bytes > 200e6 else
                   "inputs rotate through copies larger than L2",
-            "parallelism": f"batch-sharded x{args.gpus}, no collective"}
+            "parallelism": f"batch-sharded x{args.gpus}, no collective",
+            "payload": getattr(args, "payload", "f32")}
 
 
 def rank_workload(w: di.Workload, rank: int) -> di.Workload:
@@ -251,10 +252,12 @@ def run_ours(args, w: di.Workload):
     rs_out = None
 
     def step(i):
+        step_on(sets[i % copies])
+
+    def step_on(g):
         nonlocal ev_out, rs_out
-        g = sets[i % copies]
         ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
-                                    w.temperature, out=ev_out, workspace=ws_e)
+                                    w.temperature, out=ev_out, workspace=ws_e, payload=args.payload)
         rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
                                         gamma, out=rs_out, workspace=ws_r)
 
@@ -273,7 +276,7 @@ def run_ours(args, w: di.Workload):
         g = sets[i % copies]
         ev[i][0].record()
         ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
-                                    w.temperature, out=ev_out, workspace=ws_e)
+                                    w.temperature, out=ev_out, workspace=ws_e, payload=args.payload)
         ev[i][1].record()
         rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
                                         gamma, out=rs_out, workspace=ws_r)
@@ -295,19 +298,38 @@ def run_ours(args, w: di.Workload):
 
     # ---- end to end through the host-buffer entry point: copies inside the timed region ----
     host = _torch_inputs(d, pin=True)
-    arena = torch.empty(B.dssd_round_host_arena_bytes(Bn, gamma, V, B.DSSD_BF16 if w.dtype == "bf16" else B.DSSD_F32),
-                        dtype=torch.uint8, device=dev)
-    h_out = None
     e2e_steps = max(3, min(K, args.e2e_steps))
+    if args.payload == "f32":
+        arena = torch.empty(B.dssd_round_host_arena_bytes(Bn, gamma, V, B.DSSD_BF16 if w.dtype == "bf16" else B.DSSD_F32),
+                            dtype=torch.uint8, device=dev)
+        h_out = None
+
+        def e2e_step():
+            nonlocal h_out
+            h_out = B.dssd_round_host(host, w.temperature, arena, out=h_out)
+    else:
+        # the host-buffer entry point carries the float32 row only: copy, call, copy back by hand
+        names = ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs")
+        stage = {n: torch.empty_like(sets[0][n]) for n in names}
+        h_out = {"accept_len": torch.empty(Bn, dtype=torch.int32).pin_memory(),
+                 "token": torch.empty(Bn, dtype=torch.int32).pin_memory()}
+
+        def e2e_step():
+            for n in names:
+                stage[n].copy_(host[n], non_blocking=True)
+            step_on(stage)
+            h_out["accept_len"].copy_(ev_out["accept_len"], non_blocking=True)
+            h_out["token"].copy_(rs_out["token"], non_blocking=True)
+
     for _ in range(2):
-        h_out = B.dssd_round_host(host, w.temperature, arena, out=h_out)
+        e2e_step()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
-        h_out = B.dssd_round_host(host, w.temperature, arena, out=h_out)
+        e2e_step()
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
@@ -315,7 +337,7 @@ def run_ours(args, w: di.Workload):
         e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = sum(host[k].numel() * host[k].element_size() for k in
               ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs"))
-    d2h = 4 * Bn * 4
+    d2h = (4 if args.payload == "f32" else 2) * Bn * 4
     assert (h_out["accept_len"].numpy() == n_gpu).all()
 
     if rank != 0:
@@ -327,23 +349,24 @@ def run_ours(args, w: di.Workload):
     value = world * rows / (ms_per_step * 1e-3)
     peak, peak_kind = _peaks()
     edge_avg_ms = sum(edge_ms) / K
-    edge_bytes = edge_algorithmic_bytes(w)
+    pbytes = 4 if args.payload == "f32" else 2
+    edge_bytes = edge_algorithmic_bytes(w, pbytes)
     achieved = edge_bytes / (edge_avg_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC.get(w.name)
+    traffic = NCU_TRAFFIC.get(w.name) if args.payload == "f32" else None
     if traffic is not None and traffic.get("kernel_hash") != _kernel_hash():
         traffic = None
     rs_avg_ms = sum(rs_ms) / K
-    rs_bytes = resample_algorithmic_bytes(w, n_bonus)
+    rs_bytes = resample_algorithmic_bytes(w, n_bonus, pbytes)
 
     # ---- CPU baseline: the oracle as it stands, on this machine's host cores, rank 0, N = 1 ----
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         n_seq = min(Bn, args.ref_sequences)
-        rate, secs, passes = oracle_rate(w, d, n_seq, cores)
+        rate, secs, passes = oracle_rate(w, d, n_seq, cores, payload=args.payload)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"first {n_seq} of {Bn} sequences of {w.name}, both halves, {passes} passes in {secs:.2f} s "
                          f"wall on {cores} threads"}
-        ref = O.verify_round({k: v[:n_seq] for k, v in d.items()}, w.temperature, threads=cores)
+        ref = O.verify_round({k: v[:n_seq] for k, v in d.items()}, w.temperature, threads=cores, payload=args.payload)
         near = ref["margin_acc"] < 1e-6
         parity = {"sequences_checked": n_seq,
                   "accept_len_mismatch": int(((n_gpu[:n_seq] != ref["accept_len"]) & ~near).sum()),
@@ -589,6 +612,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sampler", default="full", choices=["full", "topk"])
     ap.add_argument("--k", type=int, default=10)
+    ap.add_argument("--payload", default="f32", choices=["f32", "f16"], help="width of the emitted row P_n (full sampler only)")
     args = ap.parse_args()
     w = di.get_workload(args.workload)
     if args.steps is None:
