@@ -131,11 +131,6 @@ struct Vec<DSSD_F32> {
         return max_nan(max_nan(__uint_as_float(v.x), __uint_as_float(v.y)),
                        max_nan(__uint_as_float(v.z), __uint_as_float(v.w)));
     }
-    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
-    {
-        f[0] = __uint_as_float(v.x), f[1] = __uint_as_float(v.y);
-        f[2] = __uint_as_float(v.z), f[3] = __uint_as_float(v.w);
-    }
     __device__ static __forceinline__ float load(const void *row, int64_t i) { return reinterpret_cast<const float *>(row)[i]; }
     // element j of the vector (j < E)
     __device__ static __forceinline__ float elem(const uint4 &v, int j)
@@ -152,11 +147,6 @@ struct Vec<DSSD_BF16> {
     {
         const uint32_t w = max_nan_bf16x2(max_nan_bf16x2(v.x, v.y), max_nan_bf16x2(v.z, v.w));
         return max_nan(bf16_lo(w), bf16_hi(w));
-    }
-    __device__ static __forceinline__ void unpack(const uint4 &v, float *f)
-    {
-        f[0] = bf16_lo(v.x), f[1] = bf16_hi(v.x), f[2] = bf16_lo(v.y), f[3] = bf16_hi(v.y);
-        f[4] = bf16_lo(v.z), f[5] = bf16_hi(v.z), f[6] = bf16_lo(v.w), f[7] = bf16_hi(v.w);
     }
     __device__ static __forceinline__ float load(const void *row, int64_t i)
     {

@@ -29,13 +29,22 @@ def _rank_main(rank, world, port, out_dir):
     mine = torch.from_numpy(np.stack([ref["accept_len"], ref["token"]]).astype(np.int64))
     gathered = [torch.zeros_like(mine) for _ in range(world)]
     dist.all_gather(gathered, mine)                          # only to check: the path itself needs no collective
+    # the truncated-support round shards the same way
+    dk = di.generate_topk(w, 5, rank * per, (rank + 1) * per)
+    refk = O.verify_round_topk(dk, w.temperature, 5)
+    mine_k = torch.from_numpy(np.stack([refk["accept_len"], refk["token"]]).astype(np.int64))
+    gathered_k = [torch.zeros_like(mine_k) for _ in range(world)]
+    dist.all_gather(gathered_k, mine_k)
     slowest = bench.max_over_ranks(10.0 + rank, dist, torch.device("cpu"))
     seeds = [bench.rank_workload(w, r).seed for r in range(world)]
     if rank == 0:
         whole = O.verify_round(di.generate(w), w.temperature)
         got = torch.cat(gathered, dim=1).numpy()
+        whole_k = O.verify_round_topk(di.generate_topk(w, 5), w.temperature, 5)
+        got_k = torch.cat(gathered_k, dim=1).numpy()
         np.save(os.path.join(out_dir, "ok.npy"),
-                np.array([int((got[0] == whole["accept_len"]).all() and (got[1] == whole["token"]).all()),
+                np.array([int((got[0] == whole["accept_len"]).all() and (got[1] == whole["token"]).all() and
+                              (got_k[0] == whole_k["accept_len"]).all() and (got_k[1] == whole_k["token"]).all()),
                           int(slowest == 10.0 + world - 1), int(len(set(seeds)) == world)]))
     dist.barrier()
     dist.destroy_process_group()
