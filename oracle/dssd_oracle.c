@@ -452,3 +452,114 @@ int dssd_oracle_device_resample_topk(const int32_t *p_idx, const float *p_val,
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Algorithm 1 (DSD): the verification that the paper's split scheme is compared with.  The
+ * edge holds the full draft rows Q_i(.) (they were uploaded), so it tests every position with
+ * q_i(x_i) read from the row, and on the first rejection resamples from
+ * norm(max(0, P_n - Q_n)) itself; when all drafts pass it samples the bonus token from
+ * P_{gamma+1}.  No row is transmitted, so nothing is rounded to a payload format: the residual
+ * is formed from the float64 target probabilities.
+ *
+ * target_logits [B, gamma+1, V] (row_stride elements between rows), draft_q [B, gamma, V] float32,
+ * draft_tokens [B, gamma], uniforms [B, gamma] (acceptance), uniforms_rs [B] (the draw).
+ * outputs: accept_len [B], token [B], flags [B] (edge flags, may be NULL), rs_flags [B] (may be
+ * NULL), margin_acc [B], margin_cdf [B] (may be NULL) as in the split functions.
+ * ------------------------------------------------------------------------------------------ */
+int dssd_oracle_dsd_verify(const void *target_logits, int dtype, int64_t row_stride,
+                           const float *draft_q, const int32_t *draft_tokens,
+                           const float *uniforms, const float *uniforms_rs, float temperature,
+                           int B, int gamma, int V,
+                           int32_t *accept_len, int32_t *token, uint32_t *flags, uint32_t *rs_flags,
+                           double *margin_acc, double *margin_cdf)
+{
+    const double T = (double)temperature;
+    const size_t esz = (dtype == ORACLE_BF16) ? 2 : 4;
+    if (B < 1 || gamma < 0 || V < 1 || !(T > 0.0) || row_stride < V) return 1;
+    for (int b = 0; b < B; ++b) {
+        uint32_t fl = 0, rfl = 0;
+        int n = gamma, flag_open = 1;
+        double margin = INFINITY;
+        for (int i = 0; i <= gamma; ++i) {
+            const char *row = (const char *)target_logits +
+                              ((size_t)b * (size_t)(gamma + 1) + (size_t)i) * (size_t)row_stride * esz;
+            int ok;
+            double l = row_lse(row, dtype, V, T, &ok);
+            if (!ok) fl |= FLAG_NONFINITE;
+            if (i == gamma) break;
+            int32_t x = draft_tokens[(size_t)b * gamma + i];
+            double u = (double)uniforms[(size_t)b * gamma + i];
+            double ratio;
+            int accept;
+            if (x < 0 || x >= V) {
+                fl |= FLAG_BAD_TOKEN;
+                accept = 0;
+                ratio = NAN;
+            } else {
+                double q = (double)draft_q[((size_t)b * gamma + i) * (size_t)V + x];
+                double p = exp(load_logit(row, dtype, x) / T - l);
+                if (q != q) ratio = NAN;
+                else if (q <= 0.0) ratio = (p > 0.0) ? INFINITY : 0.0;
+                else ratio = p / q;
+                accept = (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
+            }
+            if (flag_open) {
+                if (ratio == ratio) {
+                    double d = fabs(u - (ratio < 1.0 ? ratio : 1.0));
+                    if (d < margin) margin = d;
+                }
+                if (!accept) { n = i; flag_open = 0; }
+            }
+        }
+        accept_len[b] = n;
+        /* the draw at position n: residual against Q_n, or the bonus row itself */
+        {
+            const char *row = (const char *)target_logits +
+                              ((size_t)b * (size_t)(gamma + 1) + (size_t)n) * (size_t)row_stride * esz;
+            const float *q = n < gamma ? draft_q + ((size_t)b * gamma + n) * (size_t)V : NULL;
+            int ok;
+            double l = row_lse(row, dtype, V, T, &ok);
+            double u = (double)uniforms_rs[b];
+            int32_t tok = -1;
+            double mg = 0.0;
+            if (n == gamma) rfl |= RS_FLAG_BONUS;
+            for (int pass = 0; pass < 2 && tok < 0; ++pass) {
+                /* pass 0: the residual (or the bonus row); pass 1: fall back to P_n when it has no mass */
+                const float *qq = pass == 0 ? q : NULL;
+                double Z = 0.0;
+                if (pass == 1) {
+                    if (!q) break;
+                    rfl |= RS_FLAG_FALLBACK;
+                }
+                for (int v = 0; v < V; ++v) {
+                    double p = exp(load_logit(row, dtype, v) / T - l);
+                    Z += qq ? fmax(0.0, p - (double)qq[v]) : p;
+                }
+                if (!(Z > 0.0) || !(Z < INFINITY)) continue;
+                double t = u * Z, C = 0.0, Cprev;
+                int32_t last_pos = -1;
+                for (int v = 0; v < V; ++v) {
+                    double p = exp(load_logit(row, dtype, v) / T - l);
+                    double r = qq ? fmax(0.0, p - (double)qq[v]) : p;
+                    Cprev = C;
+                    C += r;
+                    if (r > 0.0) last_pos = v;
+                    if (C > t) {
+                        double lo = t - Cprev, hi = C - t;
+                        mg = (lo < hi ? lo : hi) / Z;
+                        tok = v;
+                        break;
+                    }
+                }
+                if (tok < 0) { tok = last_pos; mg = 0.0; }
+            }
+            if (tok < 0) { rfl |= RS_FLAG_INVALID; mg = 0.0; }
+            token[b] = tok;
+            if (margin_cdf) margin_cdf[b] = mg;
+        }
+        if (flags) flags[b] = fl;
+        if (rs_flags) rs_flags[b] = rfl;
+        if (margin_acc) margin_acc[b] = margin;
+    }
+    return 0;
+}

@@ -57,6 +57,10 @@ def _load():
         lib.dssd_oracle_device_resample.argtypes = [
             c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int,
             c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+        lib.dssd_oracle_dsd_verify.restype = c.c_int
+        lib.dssd_oracle_dsd_verify.argtypes = [
+            c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+            c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
         lib.dssd_oracle_edge_verify_topk.restype = c.c_int
         lib.dssd_oracle_edge_verify_topk.argtypes = [
             c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -278,4 +282,43 @@ def verify_round_topk(inputs: Dict[str, np.ndarray], temperature: float, k: int,
     out["rs_flags"] = rs["flags"]
     out["margin_cdf"] = rs["margin_cdf"]
     out["Z"] = rs["Z"]
+    return out
+
+
+def dsd_verify(inputs: Dict[str, np.ndarray], temperature: float, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Algorithm 1 (DSD) on one generated batch: the edge holds the full draft rows, tests with
+    q_i(x_i) read from them, and draws the corrected or bonus token itself."""
+    lib = _load()
+    tl = np.ascontiguousarray(inputs["target_logits"])
+    assert tl.ndim == 3 and tl.dtype in (np.float32, np.uint16)
+    dtype = BF16 if tl.dtype == np.uint16 else F32
+    B, g1, V = tl.shape
+    gamma = g1 - 1
+    q = (np.ascontiguousarray(inputs["draft_q"], dtype=np.float32).reshape(B, gamma, V) if gamma > 0
+         else np.zeros((B, 0, V), np.float32))
+    tok = np.ascontiguousarray(inputs["draft_tokens"], dtype=np.int32).reshape(B, gamma)
+    u = np.ascontiguousarray(inputs["uniforms"], dtype=np.float32).reshape(B, gamma)
+    urs = np.ascontiguousarray(inputs["uniforms_rs"], dtype=np.float32).reshape(B)
+    out = {
+        "accept_len": np.zeros(B, np.int32), "token": np.zeros(B, np.int32),
+        "flags": np.zeros(B, np.uint32), "rs_flags": np.zeros(B, np.uint32),
+        "margin_acc": np.zeros(B, np.float64), "margin_cdf": np.zeros(B, np.float64),
+    }
+
+    def run(rng):
+        b0, b1 = rng
+        rc = lib.dssd_oracle_dsd_verify(
+            _ptr(tl[b0:b1]), dtype, V, _ptr(q[b0:b1]) if gamma > 0 else None, _ptr(tok[b0:b1]), _ptr(u[b0:b1]),
+            _ptr(urs[b0:b1]), ctypes.c_float(temperature), b1 - b0, gamma, V,
+            _ptr(out["accept_len"][b0:b1]), _ptr(out["token"][b0:b1]), _ptr(out["flags"][b0:b1]),
+            _ptr(out["rs_flags"][b0:b1]), _ptr(out["margin_acc"][b0:b1]), _ptr(out["margin_cdf"][b0:b1]))
+        if rc != 0:
+            raise ValueError("dssd_oracle_dsd_verify: invalid arguments")
+
+    parts = _chunks(B, threads)
+    if len(parts) == 1:
+        run(parts[0])
+    else:
+        with ThreadPoolExecutor(len(parts)) as ex:
+            list(ex.map(run, parts))
     return out
