@@ -14,7 +14,8 @@
  *                         the same round on distributions truncated to their k most likely
  *                         tokens, the sampler of the paper's experiments (Section 4);
  *   dssd_edge_verify_p16, dssd_device_resample_p16
- *                         the round with the downlink row in 16 bits per value (Section 2.2).
+ *                         the round with the downlink row in 16 bits per value (Section 2.2);
+ *   dssd_dsd_verify       the fused verification of Algorithm 1 (no row is transmitted).
  *
  * Notation follows the paper: gamma draft tokens x_1..x_gamma with draft probabilities
  * q_i(x_i), target distributions P_1..P_{gamma+1} over a vocabulary of V entries, uniforms
@@ -309,6 +310,37 @@ dssd_status dssd_device_resample_p16(const uint16_t *p_row16, const float *draft
                                      const int32_t *accept_len, const float *uniforms, int B,
                                      int gamma, int V, int32_t *token, uint32_t *flags,
                                      void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------
+ * Fused verification of Algorithm 1 (DSD, the scheme the paper's split round is measured against):
+ * the edge holds the uploaded draft rows Q_i(.), so it tests every position with q_i(x_i) read
+ * from the row and draws the corrected token from norm(max(0, P_n - Q_n)), or the bonus token from
+ * P_{gamma+1}, itself.  No row P_n is written or read back: the draw forms p_v from row n's
+ * logits on the fly with the log-sum-exp the first pass left behind.
+ * ---------------------------------------------------------------------------------------------
+ */
+
+/* Bytes of scratch that dssd_dsd_verify needs (0 if the sizes are invalid). */
+size_t dssd_dsd_verify_workspace_bytes(int B, int gamma, int V);
+
+/*
+ * Acceptance rule, first-rejection scan, flags: as dssd_edge_verify.  Draw: as dssd_device_resample,
+ * with p_v = the float32 value dssd_edge_verify would have emitted, so that the token equals the one
+ * the two split calls give on the same inputs.
+ *
+ * target_logits [B, gamma+1, V] as in dssd_edge_verify;  draft_q [B, gamma, V] float32, contiguous
+ * draft_tokens, uniforms [B, gamma];  uniforms_rs [B]      (draft_* and uniforms may be NULL iff gamma == 0)
+ * accept_len [B] int32 out;  token [B] int32 out
+ * edge_flags [B] uint32 out, optional: DSSD_EDGE_FLAG_*;  rs_flags [B] uint32 out, optional: DSSD_RS_FLAG_*
+ * workspace  >= dssd_dsd_verify_workspace_bytes(B, gamma, V) bytes, 256-byte aligned
+ */
+dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                            const float *draft_q, const int32_t *draft_tokens, const float *uniforms,
+                            const float *uniforms_rs, float temperature, int B, int gamma, int V,
+                            int32_t *accept_len, int32_t *token, uint32_t *edge_flags,
+                            uint32_t *rs_flags, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -85,6 +85,12 @@ def _load() -> ctypes.CDLL:
     L.dssd_edge_verify_p16.argtypes = L.dssd_edge_verify.argtypes
     L.dssd_device_resample_p16.restype = c.c_int
     L.dssd_device_resample_p16.argtypes = L.dssd_device_resample.argtypes
+    L.dssd_dsd_verify_workspace_bytes.restype = c.c_size_t
+    L.dssd_dsd_verify_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int]
+    L.dssd_dsd_verify.restype = c.c_int
+    L.dssd_dsd_verify.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -278,6 +284,40 @@ def dssd_device_resample_topk(p_idx: torch.Tensor, p_val: torch.Tensor, q_idx: O
         out["token"].data_ptr(), _ptr(out.get("flags")), _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_device_resample_topk")
+    return out
+
+
+def dssd_dsd_verify_workspace_bytes(B: int, gamma: int, V: int) -> int:
+    return int(lib.dssd_dsd_verify_workspace_bytes(B, gamma, V))
+
+
+def dssd_dsd_verify(target_logits: torch.Tensor, draft_q: Optional[torch.Tensor], draft_tokens: torch.Tensor,
+                    uniforms: torch.Tensor, uniforms_rs: torch.Tensor, temperature: float, *,
+                    out: Optional[Dict[str, torch.Tensor]] = None, workspace: Optional[torch.Tensor] = None,
+                    stream=None) -> Dict[str, torch.Tensor]:
+    """Fused verification of Algorithm 1: acceptance tests with q_i(x_i) read from the draft rows and
+    the corrected / bonus draw, without any row P_n in memory.  Returns accept_len, token, edge_flags, rs_flags."""
+    assert target_logits.is_cuda and target_logits.dim() == 3
+    B, g1, V = target_logits.shape
+    gamma = g1 - 1
+    assert target_logits.stride(2) == 1 or V == 1
+    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
+    if B > 1 and target_logits.stride(0) != g1 * row_stride:
+        raise ValueError("rows of target_logits must be equally spaced")
+    if gamma > 0:
+        assert draft_q.is_contiguous() and draft_q.dtype == torch.float32 and draft_q.numel() == B * gamma * V
+    dev = target_logits.device
+    if out is None:
+        out = {k: torch.empty(B, dtype=torch.int32, device=dev) for k in ("accept_len", "token", "edge_flags", "rs_flags")}
+    if workspace is None:
+        workspace = _workspace(dssd_dsd_verify_workspace_bytes(B, gamma, V), dev)
+    st = lib.dssd_dsd_verify(
+        target_logits.data_ptr(), _dtype_code(target_logits), row_stride, _ptr(draft_q) if gamma > 0 else None,
+        _ptr(draft_tokens), _ptr(uniforms), uniforms_rs.data_ptr(), ctypes.c_float(temperature), B, gamma, V,
+        out["accept_len"].data_ptr(), out["token"].data_ptr(), _ptr(out.get("edge_flags")), _ptr(out.get("rs_flags")),
+        workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_dsd_verify")
     return out
 
 

@@ -28,6 +28,16 @@ dssd_status check_sizes(int B, int gamma, int V)
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// q_i(x_i) read out of the draft rows (fused verification); a token id outside the vocabulary
+// gets NaN - the edge kernel rejects and flags that position by the id itself
+__global__ void gather_q_tok(const float *draft_q, const int32_t *tokens, float *q_tok, long long n, int V)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int x = tokens[i];
+    q_tok[i] = (x >= 0 && x < V) ? draft_q[(size_t)i * (size_t)V + (size_t)x] : __int_as_float(0x7fc00000);
+}
+
 }  // namespace
 
 namespace dssd {
@@ -181,6 +191,79 @@ dssd_status dssd_device_resample_p16(const uint16_t *p_row16, const float *draft
 {
     return device_resample_any(p_row16, 1, draft_q, accept_len, uniforms, B, gamma, V, token, flags, workspace,
                                workspace_bytes, cuda_stream);
+}
+
+size_t dssd_dsd_verify_workspace_bytes(int B, int gamma, int V)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    return align256(dssd_edge_verify_workspace_bytes(B, gamma, V)) +
+           align256(dssd_device_resample_workspace_bytes(B, gamma, V)) + align256((size_t)B * (size_t)gamma * 4 + 4);
+}
+
+dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                            const float *draft_q, const int32_t *draft_tokens, const float *uniforms,
+                            const float *uniforms_rs, float temperature, int B, int gamma, int V,
+                            int32_t *accept_len, int32_t *token, uint32_t *edge_flags,
+                            uint32_t *rs_flags, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !uniforms_rs || !accept_len || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_q || !draft_tokens || !uniforms)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(target_logits) % esz) || (reinterpret_cast<uintptr_t>(draft_q) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_dsd_verify_workspace_bytes(B, gamma, V))
+        return DSSD_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    char *ws_edge = static_cast<char *>(workspace);
+    char *ws_rs = ws_edge + align256(dssd_edge_verify_workspace_bytes(B, gamma, V));
+    float *q_tok = reinterpret_cast<float *>(ws_rs + align256(dssd_device_resample_workspace_bytes(B, gamma, V)));
+
+    // q_i(x_i) out of the uploaded rows
+    if (gamma > 0) {
+        const long long n = (long long)B * gamma;
+        gather_q_tok<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(draft_q, draft_tokens, q_tok, n, V);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    dssd::EdgeParams E{};
+    E.logits = target_logits;
+    E.row_stride = row_stride;
+    E.draft_tokens = draft_tokens;
+    E.draft_q_tok = q_tok;
+    E.uniforms = uniforms;
+    E.temperature = temperature;
+    E.B = B;
+    E.gamma = gamma;
+    E.V = V;
+    E.accept_len = accept_len;
+    E.flags = edge_flags;  // no row: nothing is emitted
+    cudaError_t e = dssd::edge_verify_launch(E, (int)dtype, ws_edge, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    dssd::ResampleParams R{};
+    R.logits = target_logits;
+    R.row_stride = row_stride;
+    R.logits_dtype = (int)dtype;
+    R.c1 = E.c1;
+    R.ready = E.ready;
+    R.draft_q = draft_q;
+    R.accept_len = accept_len;
+    R.uniforms = uniforms_rs;
+    R.B = B;
+    R.gamma = gamma;
+    R.V = V;
+    R.token = token;
+    R.flags = rs_flags;
+    e = dssd::resample_launch(R, ws_rs, s);
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
 }
 
 size_t dssd_edge_verify_topk_workspace_bytes(int B, int gamma, int V, int k)

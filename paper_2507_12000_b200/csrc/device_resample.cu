@@ -12,6 +12,7 @@
 // All sums are float64, so the token differs from an index-order float64 scan only when u' * Z
 // lies within rounding (about 1e-13 relative) of a CDF step.
 #include "device_resample.h"
+#include "edge_verify.h"
 
 #include <mutex>
 
@@ -34,8 +35,11 @@ __device__ __forceinline__ float4 as_f4(const uint4 &v)
     return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
 }
 
-// The row p comes as float32 or, for the 16-bit payload, as IEEE binary16 bit patterns; the
-// kernel is written once over these accessors.  A "quad" is four consecutive entries.
+// The row p comes as float32, as IEEE binary16 bit patterns (the 16-bit payload), or - for the
+// fused verification of Algorithm 1, where no row is ever written - as the target logits of row n
+// together with the row's reference exponent and 1 / sum, from which p_v = 2^(l_v c1 - ref2) / S is
+// formed on the fly exactly as the edge kernel forms it when it emits a row.  The kernel is
+// written once over these views.  A "quad" is four consecutive entries.
 __device__ __forceinline__ float half_bits_to_float(unsigned short h) { return __half2float(__ushort_as_half(h)); }
 __device__ __forceinline__ float4 half_quad(uint2 v)
 {
@@ -43,97 +47,161 @@ __device__ __forceinline__ float4 half_quad(uint2 v)
     const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&v.y));
     return make_float4(a.x, a.y, b.x, b.y);
 }
-template <typename PT>
-struct PAcc;
-template <>
-struct PAcc<float> {
+__device__ __forceinline__ uint2 ld_stream8(const void *p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+struct RowF32 {  // p_row as float32
     typedef uint4 Raw;
-    static constexpr unsigned kAlignMask = 15u;  // a quad is loaded with one 16-byte access
-    __device__ static __forceinline__ float ld(const float *p, int64_t e) { return __ldg(p + e); }
-    __device__ static __forceinline__ Raw ld_quad_stream(const float *p, int64_t quad)
+    const float *p;
+    __device__ static __forceinline__ RowF32 make(const ResampleParams &P, int64_t b, int)
     {
-        return ld_stream16(reinterpret_cast<const uint4 *>(p) + quad);
+        RowF32 r;
+        r.p = reinterpret_cast<const float *>(P.p_row) + (size_t)b * P.V;
+        return r;
     }
-    __device__ static __forceinline__ float4 quad(const Raw &v) { return as_f4(v); }
-    __device__ static __forceinline__ float4 ld_quad(const float *p, int64_t quad)
+    __device__ __forceinline__ bool aligned(int e) const { return (reinterpret_cast<uintptr_t>(p + e) & 15u) == 0; }
+    __device__ __forceinline__ float ld(int64_t e) const { return __ldg(p + e); }
+    __device__ __forceinline__ Raw ld_quad_stream(int e0, int64_t quad) const
     {
-        return __ldg(reinterpret_cast<const float4 *>(p) + quad);
+        return ld_stream16(reinterpret_cast<const uint4 *>(p + e0) + quad);
     }
-};
-template <>
-struct PAcc<uint16_t> {
-    typedef uint2 Raw;
-    static constexpr unsigned kAlignMask = 7u;  // a quad is loaded with one 8-byte access
-    __device__ static __forceinline__ float ld(const uint16_t *p, int64_t e) { return half_bits_to_float(__ldg(p + e)); }
-    __device__ static __forceinline__ Raw ld_quad_stream(const uint16_t *p, int64_t quad)
+    __device__ __forceinline__ float4 quad(const Raw &v) const { return as_f4(v); }
+    __device__ __forceinline__ float4 ld_quad(int e0, int64_t quad) const
     {
-        uint2 v;
-        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
-                     : "=r"(v.x), "=r"(v.y)
-                     : "l"(reinterpret_cast<const uint2 *>(p) + quad));
-        return v;
-    }
-    __device__ static __forceinline__ float4 quad(const Raw &v) { return half_quad(v); }
-    __device__ static __forceinline__ float4 ld_quad(const uint16_t *p, int64_t quad)
-    {
-        return half_quad(__ldg(reinterpret_cast<const uint2 *>(p) + quad));
+        return __ldg(reinterpret_cast<const float4 *>(p + e0) + quad);
     }
 };
 
+struct RowF16 {  // p_row as binary16 bit patterns
+    typedef uint2 Raw;
+    const uint16_t *p;
+    __device__ static __forceinline__ RowF16 make(const ResampleParams &P, int64_t b, int)
+    {
+        RowF16 r;
+        r.p = reinterpret_cast<const uint16_t *>(P.p_row) + (size_t)b * P.V;
+        return r;
+    }
+    __device__ __forceinline__ bool aligned(int e) const { return (reinterpret_cast<uintptr_t>(p + e) & 7u) == 0; }
+    __device__ __forceinline__ float ld(int64_t e) const { return half_bits_to_float(__ldg(p + e)); }
+    __device__ __forceinline__ Raw ld_quad_stream(int e0, int64_t quad) const
+    {
+        return ld_stream8(reinterpret_cast<const uint2 *>(p + e0) + quad);
+    }
+    __device__ __forceinline__ float4 quad(const Raw &v) const { return half_quad(v); }
+    __device__ __forceinline__ float4 ld_quad(int e0, int64_t quad) const
+    {
+        return half_quad(__ldg(reinterpret_cast<const uint2 *>(p + e0) + quad));
+    }
+};
+
+// four consecutive logits: how they are loaded and widened
+template <int DT>
+struct LogitQuad;
+template <>
+struct LogitQuad<DSSD_F32> {
+    typedef uint4 Raw;
+    __device__ static __forceinline__ Raw ld_stream(const void *p) { return ld_stream16(p); }
+    __device__ static __forceinline__ float4 widen(const Raw &v) { return as_f4(v); }
+};
+template <>
+struct LogitQuad<DSSD_BF16> {
+    typedef uint2 Raw;
+    __device__ static __forceinline__ Raw ld_stream(const void *p) { return ld_stream8(p); }
+    __device__ static __forceinline__ float4 widen(const Raw &v)
+    {
+        return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    }
+};
+
+template <int DT>
+struct RowLogits {  // row n of the target logits, turned into probabilities on the fly
+    typedef typename LogitQuad<DT>::Raw Raw;
+    const char *row;
+    float c1, nref, invS;
+    __device__ static __forceinline__ RowLogits make(const ResampleParams &P, int64_t b, int n)
+    {
+        RowLogits r;
+        r.row = reinterpret_cast<const char *>(P.logits) +
+                ((size_t)b * (size_t)(P.gamma + 1) + (size_t)n) * (size_t)P.row_stride * Elem<DT>::kBytes;
+        const ReadySlot s = reinterpret_cast<const ReadySlot *>(P.ready)[b];
+        r.c1 = P.c1;
+        r.nref = -s.ref2;
+        r.invS = s.invS;
+        return r;
+    }
+    __device__ __forceinline__ float prob(float l) const { return ex2(fmaf(l, c1, nref)) * invS; }
+    __device__ __forceinline__ bool aligned(int e) const
+    {
+        return (reinterpret_cast<uintptr_t>(row + (size_t)e * Elem<DT>::kBytes) & (4u * Elem<DT>::kBytes - 1u)) == 0;
+    }
+    __device__ __forceinline__ float ld(int64_t e) const { return prob(Elem<DT>::load(row, e)); }
+    __device__ __forceinline__ Raw ld_quad_stream(int e0, int64_t quad) const
+    {
+        return LogitQuad<DT>::ld_stream(row + ((size_t)e0 + 4 * (size_t)quad) * Elem<DT>::kBytes);
+    }
+    __device__ __forceinline__ float4 quad(const Raw &v) const
+    {
+        const float4 l = LogitQuad<DT>::widen(v);
+        return make_float4(prob(l.x), prob(l.y), prob(l.z), prob(l.w));
+    }
+    __device__ __forceinline__ float4 ld_quad(int e0, int64_t quad) const { return this->quad(ld_quad_stream(e0, quad)); }
+};
+
 // per-thread part of sum_{e in [e0,e1)} r_e ; q == nullptr means r = p
-template <typename PT>
-__device__ __forceinline__ double chunk_mass(const PT *p, const float *q, int e0, int e1)
+template <typename RV>
+__device__ __forceinline__ double chunk_mass(const RV &row, const float *q, int e0, int e1)
 {
-    typedef PAcc<PT> A;
     const int tid = threadIdx.x;
     double acc = 0.0;
     int done = e0;
-    const bool aligned = (reinterpret_cast<uintptr_t>(p + e0) & A::kAlignMask) == 0 &&
-                         (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0);
+    const bool aligned = row.aligned(e0) && (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0);
     if (aligned) {
         const int nvec = (e1 - e0) / 4;
-        const PT *p4 = p + e0;  // quads are counted from here
         if (q) {
             const uint4 *q4 = reinterpret_cast<const uint4 *>(q + e0);
             int i = tid;
             for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                typename A::Raw a[4];
+                typename RV::Raw a[4];
                 uint4 b[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    a[u] = A::ld_quad_stream(p4, i + u * kThreads);
+                    a[u] = row.ld_quad_stream(e0, i + u * kThreads);
                     b[u] = ld_stream16(q4 + i + u * kThreads);
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float4 x = A::quad(a[u]), y = as_f4(b[u]);
+                    const float4 x = row.quad(a[u]), y = as_f4(b[u]);
                     acc += (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
                 }
             }
             for (; i < nvec; i += kThreads) {
-                const float4 x = A::quad(A::ld_quad_stream(p4, i)), y = as_f4(ld_stream16(q4 + i));
+                const float4 x = row.quad(row.ld_quad_stream(e0, i)), y = as_f4(ld_stream16(q4 + i));
                 acc += (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
             }
         } else {
             int i = tid;
             for (; i + 3 * kThreads < nvec; i += 4 * kThreads) {
-                typename A::Raw a[4];
+                typename RV::Raw a[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) a[u] = A::ld_quad_stream(p4, i + u * kThreads);
+                for (int u = 0; u < 4; ++u) a[u] = row.ld_quad_stream(e0, i + u * kThreads);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float4 x = A::quad(a[u]);
+                    const float4 x = row.quad(a[u]);
                     acc += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
                 }
             }
             for (; i < nvec; i += kThreads) {
-                const float4 x = A::quad(A::ld_quad_stream(p4, i));
+                const float4 x = row.quad(row.ld_quad_stream(e0, i));
                 acc += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
             }
         }
         done = e0 + nvec * 4;
     }
-    for (int e = done + tid; e < e1; e += kThreads) acc += q ? res(A::ld(p, e), __ldg(q + e)) : (double)A::ld(p, e);
+    for (int e = done + tid; e < e1; e += kThreads) acc += q ? res(row.ld(e), __ldg(q + e)) : (double)row.ld(e);
     return acc;
 }
 
@@ -214,8 +282,8 @@ __device__ __forceinline__ double block_scan(double x, double *s_scan, double &t
 }
 
 // pass B for sequence b; q == nullptr means r = p
-template <typename PT>
-__device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const float *q, unsigned fl,
+template <typename RV>
+__device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const float *q, unsigned fl,
                      double *s_w, Pick *s_pick, int *s_i)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -326,7 +394,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const floa
         fl |= DSSD_RS_FLAG_FALLBACK;
         for (int c = 0; c < P.n_sub; ++c) {
             const int e0 = c * kSub, e1 = min(P.V, e0 + kSub);
-            const double tot = block_sum(chunk_mass(p, nullptr, e0, e1), s_w);
+            const double tot = block_sum(chunk_mass(row, nullptr, e0, e1), s_w);
             if (tid == 0) st_relaxed_u64(cs + c, (unsigned long long)__double_as_longlong(tot));
         }
         __syncthreads();
@@ -338,15 +406,14 @@ __device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const floa
     int last_pos = -1;
     // The run's 16 entries are all requested before the first is used (one round trip for the
     // run, not one per entry); entries past the row's end read as 0.
-    const bool vec = (r1 - r0 == kRun) && (reinterpret_cast<uintptr_t>(p + r0) & PAcc<PT>::kAlignMask) == 0 &&
-                     (!q || (reinterpret_cast<uintptr_t>(q + r0) & 15u) == 0);
+    const bool vec = (r1 - r0 == kRun) && row.aligned(r0) && (!q || (reinterpret_cast<uintptr_t>(q + r0) & 15u) == 0);
 #pragma unroll
     for (int g = 0; g < kRun; g += 16) {
         float pv[16], qv[16];
         if (vec) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float4 a = PAcc<PT>::ld_quad(p + r0 + g, j);
+                const float4 a = row.ld_quad(r0 + g, j);
                 pv[4 * j] = a.x, pv[4 * j + 1] = a.y, pv[4 * j + 2] = a.z, pv[4 * j + 3] = a.w;
                 float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (q) c = __ldg(reinterpret_cast<const float4 *>(q + r0 + g) + j);
@@ -356,7 +423,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const floa
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 const int e = r0 + g + j;
-                pv[j] = e < r1 ? PAcc<PT>::ld(p, e) : 0.f;
+                pv[j] = e < r1 ? row.ld(e) : 0.f;
                 qv[j] = (q && e < r1) ? __ldg(q + e) : 0.f;
             }
         }
@@ -397,7 +464,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const floa
         double C = before;
         int tok = last_pos;
         for (int e = r0; e < r1; ++e) {
-            C += q ? res(PAcc<PT>::ld(p, e), __ldg(q + e)) : (double)PAcc<PT>::ld(p, e);
+            C += q ? res(row.ld(e), __ldg(q + e)) : (double)row.ld(e);
             if (C > pk.target) { tok = e; break; }
         }
         P.token[b] = tok >= 0 ? tok : s_i[1];
@@ -405,7 +472,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const PT *p, const floa
     }
 }
 
-template <typename PT>
+template <typename RV>
 __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ ResampleParams P)
 {
     __shared__ double s_w[2][kWarps][2];
@@ -430,11 +497,11 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         const int n = __ldg(P.accept_len + b);
         double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
         if (n >= 0 && n <= P.gamma) {
-            const PT *p = reinterpret_cast<const PT *>(P.p_row) + (size_t)b * P.V;
+            const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
             const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
-            acc0 = chunk_mass(p, q, e0, e1);
-            if (e2 > e1) acc1 = chunk_mass(p, q, e1, e2);
+            acc0 = chunk_mass(row, q, e0, e1);
+            if (e2 > e1) acc1 = chunk_mass(row, q, e1, e2);
         }
         acc0 = warp_sum(acc0);
         acc1 = warp_sum(acc1);
@@ -485,9 +552,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
                 if (P.flags) P.flags[b] = DSSD_RS_FLAG_INVALID;
             }
         } else {
-            const PT *p = reinterpret_cast<const PT *>(P.p_row) + (size_t)b * P.V;
+            const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-            draw<PT>(P, b, p, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
+            draw<RV>(P, b, row, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
         }
         __syncthreads();
         d = s_ticket[buf];
@@ -528,18 +595,29 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     int dev = 0, sms = 0, occ = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-    int occ16 = 0;
-    if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, resample_kernel<float>, kThreads, 0)) != cudaSuccess) return err;
-    if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ16, resample_kernel<uint16_t>, kThreads, 0)) != cudaSuccess) return err;
-    if (occ16 < occ) occ = occ16;
+    {
+        int o[4] = {0, 0, 0, 0};
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[0], resample_kernel<RowF32>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[1], resample_kernel<RowF16>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[2], resample_kernel<RowLogits<DSSD_F32>>, kThreads, 0)) != cudaSuccess) return err;
+        if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[3], resample_kernel<RowLogits<DSSD_BF16>>, kThreads, 0)) != cudaSuccess) return err;
+        occ = o[0];
+        for (int i = 1; i < 4; ++i) occ = o[i] < occ ? o[i] : occ;
+    }
     if (occ < 1) occ = 1;
     resample_workspace_layout(P.B, P.V, &P, static_cast<char *>(workspace));
     P.spin_limit = 1u << 20;
     if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long resident = (unsigned long long)sms * (unsigned long long)occ;
     const unsigned grid = (unsigned)(P.total_tickets < resident ? P.total_tickets : resident);
-    if (P.p_half) resample_kernel<uint16_t><<<grid, kThreads, 0, stream>>>(P);
-    else resample_kernel<float><<<grid, kThreads, 0, stream>>>(P);
+    if (P.logits) {
+        if (P.logits_dtype == DSSD_BF16) resample_kernel<RowLogits<DSSD_BF16>><<<grid, kThreads, 0, stream>>>(P);
+        else resample_kernel<RowLogits<DSSD_F32>><<<grid, kThreads, 0, stream>>>(P);
+    } else if (P.p_half) {
+        resample_kernel<RowF16><<<grid, kThreads, 0, stream>>>(P);
+    } else {
+        resample_kernel<RowF32><<<grid, kThreads, 0, stream>>>(P);
+    }
     return cudaGetLastError();
 }
 

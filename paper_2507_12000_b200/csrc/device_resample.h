@@ -12,6 +12,13 @@ constexpr int kResampleChunk = 8192;  // vocabulary entries per ticket
 struct ResampleParams {
     const void *p_row;   // float32 entries, or IEEE binary16 bit patterns when p_half is set
     int p_half;
+    // instead of p_row (fused verification): the target logits, from which row n's probabilities are
+    // formed on the fly with the (ref2, 1/S) that the edge kernel left in its workspace
+    const void *logits;  // nullptr: read p_row
+    int64_t row_stride;
+    int logits_dtype;
+    float c1;            // log2(e) / T, as the edge kernel used it
+    const void *ready;   // [B] ReadySlot
     const float *draft_q;
     const int32_t *accept_len;
     const float *uniforms;

@@ -1313,8 +1313,11 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     }
     const int esz = dtype == DSSD_BF16 ? 2 : 4;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
+    // Without an output row (the fused verification of Algorithm 1) nothing is emitted: there are no
+    // EMIT tickets, and what the draw needs about row n stays in the workspace (`ready`).
+    const bool no_emit = !P.p_row && !P.p_row16;
     // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
-    {
+    if (!no_emit) {
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;
@@ -1354,7 +1357,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
     P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
     P.total_lse = R * (unsigned long long)P.n_lse_runs;
-    P.total_emit = (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
+    P.total_emit = no_emit ? 0ull : (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
     // t / d == mulhi64(t, ceil(2^64 / d)) for every t with t * d * d < 2^64
     auto magic = [](unsigned long long total, int d) -> unsigned long long {
         if (d < 2 || d > (1 << 15) || total > (1ull << 33)) return 0ull;

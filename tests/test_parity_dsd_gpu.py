@@ -1,0 +1,118 @@
+"""Parity of the fused verification of Algorithm 1 (dssd_dsd_verify) with its oracle, and with
+the two split calls, whose arithmetic it shares."""
+import numpy as np
+import pytest
+import torch
+
+import dssd_inputs as di
+from gpu_util import NEAR, RTOL, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2507_12000_b200 import binding
+
+    assert torch.cuda.is_available()
+    return binding
+
+
+def compare_dsd(B, O, d, T, logits_view=None, threads=4):
+    ref = O.dsd_verify(d, T, threads=threads)
+    g = to_device(d)
+    tl = g["target_logits"] if logits_view is None else logits_view(g["target_logits"])
+    out = B.dssd_dsd_verify(tl, g.get("draft_q"), g["draft_tokens"], g["uniforms"], g["uniforms_rs"], T)
+    torch.cuda.synchronize()
+    n = out["accept_len"].cpu().numpy()
+    tok = out["token"].cpu().numpy()
+    assert (out["edge_flags"].cpu().numpy().astype(np.uint32) == ref["flags"]).all()
+    near = ref["margin_acc"] < NEAR
+    assert ((n == ref["accept_len"]) | near).all()
+    same = n == ref["accept_len"]
+    # the kernel's p is a float32 (relative error RTOL): a CDF step may move by about RTOL / Z relative to Z
+    Z_floor = 1e-3
+    slack = np.maximum(NEAR, 2 * RTOL / Z_floor)
+    bad = (tok != ref["token"]) & same & ~(ref["margin_cdf"] < slack)
+    assert not bad.any(), (np.nonzero(bad)[0][:8], tok[bad][:8], ref["token"][bad][:8], ref["margin_cdf"][bad][:8])
+    assert (out["rs_flags"].cpu().numpy().astype(np.uint32)[same] == ref["rs_flags"][same]).all()
+    return n, tok, g, tl
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_vocabularies(B, oracle_mod, dtype):
+    seed = 700
+    for V in (1, 3, 7, 33, 1000, 1025, 16389):
+        for gamma in (0, 3):
+            for Bn in (2, 150):
+                seed += 1
+                w = di.custom(B=Bn, gamma=gamma, V=V, dtype=dtype, temperature=0.9, sigma_d=1.0, zipf=V > 8, seed=seed)
+                compare_dsd(B, oracle_mod, di.generate(w, threads=4), w.temperature)
+
+
+@pytest.mark.parametrize("dtype,V,gamma,Bn", [
+    ("f32", 50272, 2, 6), ("bf16", 40003, 3, 5), ("bf16", 128256, 8, 4), ("f32", 20001, 16, 3),
+    ("bf16", 151936, 4, 9), ("f32", 16385, 1, 40),
+])
+def test_several_slices_and_ragged_tails(B, oracle_mod, dtype, V, gamma, Bn):
+    w = di.custom(B=Bn, gamma=gamma, V=V, dtype=dtype, temperature=0.8, sigma_d=0.8, seed=V + gamma)
+    compare_dsd(B, oracle_mod, di.generate(w, threads=4), w.temperature)
+
+
+def test_strided_and_unaligned_rows(B, oracle_mod):
+    for dtype, V, off, Bn in (("f32", 1000, 1, 3), ("bf16", 4097, 3, 151), ("bf16", 20001, 1, 3), ("f32", 9001, 2, 151)):
+        w = di.custom(B=Bn, gamma=2, V=V, dtype=dtype, seed=V)
+        d = di.generate(w)
+        stride = V + 5
+
+        def view(t, stride=stride, off=off, Bn=Bn, V=V):
+            buf = torch.zeros(Bn * 3 * stride + 16, dtype=t.dtype, device="cuda")
+            v = buf[off:off + Bn * 3 * stride].view(Bn, 3, stride)[:, :, :V]
+            v.copy_(t)
+            assert v.data_ptr() % 16 != 0
+            return v
+
+        compare_dsd(B, oracle_mod, d, w.temperature, logits_view=view)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_same_tokens_as_the_split_calls(B, oracle_mod, dtype):
+    """More sequences than SMs, so that the split edge call takes the streaming kernel too: the
+    fused call then forms bit-identical probabilities and must return identical results."""
+    w = di.custom(B=300, gamma=4, V=30011, dtype=dtype, temperature=0.7, sigma_d=0.5, seed=12)
+    d = di.generate(w, threads=4)
+    n, tok, g, tl = compare_dsd(B, oracle_mod, d, w.temperature)
+    ev = B.dssd_edge_verify(tl, g["draft_tokens"], g["draft_q_tok"], g["uniforms"], w.temperature)
+    rs = B.dssd_device_resample(ev["p_row"], g["draft_q"], ev["accept_len"], g["uniforms_rs"], w.gamma)
+    torch.cuda.synchronize()
+    assert (ev["accept_len"].cpu().numpy() == n).all()
+    assert (rs["token"].cpu().numpy() == tok).all()
+
+
+def test_anomalies_are_flagged_not_faulted(B, oracle_mod):
+    V, gamma, Bn = 3000, 3, 8
+    w = di.custom(B=Bn, gamma=gamma, V=V, dtype="f32", seed=5)
+    d = di.generate(w)
+    tl = d["target_logits"]
+    tl[0, 1, 17] = np.nan
+    tl[1, 0, 5] = np.inf
+    tl[2, 2, :] = -np.inf
+    tl[3, 1, ::2] = -np.inf
+    d["draft_tokens"][4, 0] = -1
+    d["draft_tokens"][5, 2] = V
+    d["uniforms"][7, :] = 0.0
+    ref = oracle_mod.dsd_verify(d, 1.0)
+    g = to_device(d)
+    out = B.dssd_dsd_verify(g["target_logits"], g["draft_q"], g["draft_tokens"], g["uniforms"], g["uniforms_rs"], 1.0)
+    torch.cuda.synchronize()
+    assert (out["edge_flags"].cpu().numpy().astype(np.uint32) == ref["flags"]).all()
+    assert (out["accept_len"].cpu().numpy() == ref["accept_len"]).all()
+    clean = ref["flags"] == 0
+    assert (out["token"].cpu().numpy()[clean] == ref["token"][clean]).all()
+    assert (out["rs_flags"].cpu().numpy().astype(np.uint32) == ref["rs_flags"]).all()
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4"])
+def test_named_configs(B, oracle_mod, name):
+    w = di.get_workload(name)
+    compare_dsd(B, oracle_mod, di.generate(w, threads=8), w.temperature, threads=8)
