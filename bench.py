@@ -600,6 +600,149 @@ def run_ours_topk(args, w: di.Workload):
         dist.destroy_process_group()
 
 
+def run_ours_fused(args, w: di.Workload):
+    """One step = one dssd_dsd_verify call (Algorithm 1: acceptance tests and the draw at the edge,
+    no row P_n in memory)."""
+    import torch
+    import torch.distributed as dist
+
+    from oracle import oracle as O
+
+    O.build()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cores = os.cpu_count() or 1
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2507_12000_b200 import binding as B
+
+    wr = rank_workload(w, rank)
+    d = di.generate(wr, threads=max(1, cores // max(1, min(world, 8))))
+    logit_bytes = d["target_logits"].nbytes
+    copies = 1 if logit_bytes > 200e6 else int(min(64, 300e6 // max(logit_bytes, 1) + 1))
+    sets = [_torch_inputs(d, dev) for _ in range(copies)]
+    gamma, Bn, V = w.gamma, w.B, w.V
+    ws = torch.empty(B.dssd_dsd_verify_workspace_bytes(Bn, gamma, V), dtype=torch.uint8, device=dev)
+    out = None
+
+    def step(g):
+        nonlocal out
+        out = B.dssd_dsd_verify(g["target_logits"], g["draft_q"], g["draft_tokens"], g["uniforms"], g["uniforms_rs"],
+                                w.temperature, out=out, workspace=ws)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % copies])
+    torch.cuda.synchronize()
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_host0 = time.perf_counter()
+    ev[0].record()
+    for i in range(K):
+        step(sets[i % copies])
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    t_host1 = time.perf_counter()
+    if world > 1:
+        dist.barrier()
+    total_ms = ev[0].elapsed_time(ev[K])
+    call_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(K)]
+    if world > 1:
+        total_ms = max_over_ranks(total_ms, dist, dev)
+    sampler.stop_flag = True
+    sampler.join(timeout=1.0)
+    clocks = sampler.summary(t_host0, t_host1)
+    n_gpu = out["accept_len"].cpu().numpy()
+    tok_gpu = out["token"].cpu().numpy()
+    n_bonus = int((n_gpu == gamma).sum())
+
+    host = _torch_inputs(d, pin=True)
+    names = ("target_logits", "draft_tokens", "uniforms", "draft_q", "uniforms_rs")
+    stage = {n: torch.empty_like(sets[0][n]) for n in names}
+    h_n = torch.empty(Bn, dtype=torch.int32).pin_memory()
+    h_tok = torch.empty(Bn, dtype=torch.int32).pin_memory()
+
+    def e2e_step():
+        for n in names:
+            stage[n].copy_(host[n], non_blocking=True)
+        step(stage)
+        h_n.copy_(out["accept_len"], non_blocking=True)
+        h_tok.copy_(out["token"], non_blocking=True)
+
+    e2e_steps = max(3, min(K, args.e2e_steps))
+    for _ in range(2):
+        e2e_step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    assert (h_n.numpy() == n_gpu).all() and (h_tok.numpy() == tok_gpu).all()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    rows = w.rows
+    ms_per_step = total_ms / K
+    peak, peak_kind = _peaks()
+    # every logit once, row n of every sequence once more, the draft row of every rejected sequence
+    call_bytes = rows * V * w.logit_bytes + Bn * V * w.logit_bytes + 4 * V * (Bn - n_bonus)
+    avg_ms = sum(call_ms) / K
+    achieved = call_bytes / (avg_ms * 1e-3) / 1e9
+    cpu = None
+    parity = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_seq = min(Bn, args.ref_sequences)
+        sub = {kk: v[:n_seq] for kk, v in d.items()}
+        passes, t0 = 0, time.perf_counter()
+        while True:
+            ref = O.dsd_verify(sub, w.temperature, threads=cores)
+            passes += 1
+            dt = time.perf_counter() - t0
+            if dt >= 1.5 or passes >= 64:
+                break
+        cpu = {"value": passes * n_seq * (gamma + 1) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {n_seq} of {Bn} sequences of {w.name}, Algorithm 1, {passes} passes in {dt:.2f} s wall "
+                         f"on {cores} threads"}
+        near = ref["margin_acc"] < 1e-6
+        parity = {"sequences_checked": n_seq,
+                  "accept_len_mismatch": int(((n_gpu[:n_seq] != ref["accept_len"]) & ~near).sum()),
+                  "token_mismatch": int((tok_gpu[:n_seq] != ref["token"]).sum()),
+                  "accept_rate": float(ref["accept_len"].mean() / max(gamma, 1))}
+    cfg = _config(w, args)
+    cfg["workload"] = cfg["workload"].replace(f"{w.name}:", f"{w.name}, fused verification of Algorithm 1:")
+    print(json.dumps({
+        "metric": METRIC, "value": world * rows / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg,
+        "roofline": {"bound": "hbm", "kernel": "edge_verify_kernel + resample_kernel (one call)", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "algorithmic_bytes_per_launch": call_bytes,
+                     "avg_launch_ms": avg_ms, "min_launch_ms": min(call_ms), "traffic": None},
+        "cpu_baseline": cpu, "parity": parity,
+        "e2e": {"value": world * rows / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": 2 * Bn * 4, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": 3 * K, "clocks": clocks,
+    }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -611,13 +754,16 @@ def main():
     ap.add_argument("--ref-sequences", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sampler", default="full", choices=["full", "topk"])
+    ap.add_argument("--fused", action="store_true", help="Algorithm 1 in one call (dssd_dsd_verify) instead of the split round")
     ap.add_argument("--k", type=int, default=10)
     ap.add_argument("--payload", default="f32", choices=["f32", "f16"], help="width of the emitted row P_n (full sampler only)")
     args = ap.parse_args()
     w = di.get_workload(args.workload)
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 2000
-    if args.sampler == "topk":
+    if args.fused and args.impl == "ours":
+        run_ours_fused(args, w)
+    elif args.sampler == "topk":
         (run_reference_topk if args.impl == "reference" else run_ours_topk)(args, w)
     elif args.impl == "reference":
         run_reference(args, w)

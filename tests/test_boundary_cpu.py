@@ -52,6 +52,8 @@ def test_workspace_sizes(B):
     assert B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 0) == 0
     assert B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 33) == 0
     assert B.dssd_edge_verify_topk_workspace_bytes(1, 0, 8, 9) == 0
+    fused = B.dssd_dsd_verify_workspace_bytes(256, 4, 151936)
+    assert fused >= b + r and fused % 256 == 0 and B.dssd_dsd_verify_workspace_bytes(0, 4, 100) == 0
     t = B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 10)
     assert 0 < t < 4 << 20 and t % 256 == 0
     assert B.dssd_round_host_arena_bytes(8, 4, 32000, B.DSSD_BF16) > 8 * 5 * 32000 * 2 + 8 * 4 * 32000 * 4
@@ -126,6 +128,30 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
     assert rsk(Bn=0) == B.DSSD_ERR_INVALID_ARG
     assert rsk(k=0) == B.DSSD_ERR_INVALID_ARG
     assert rsk(k=33) == B.DSSD_ERR_UNSUPPORTED
+
+    def p16(prow=p, **kw):
+        return L.dssd_edge_verify_p16(p, 0, 16, p, p, p, f(1.0), 1, 2, 16, p, prow, None, None, None, p, kw.get("wsb", ok_ws),
+                                      None)
+
+    assert p16(prow=None) == B.DSSD_ERR_INVALID_ARG
+    assert p16(prow=p + 1) == B.DSSD_ERR_INVALID_ARG
+    assert p16(wsb=16) == B.DSSD_ERR_WORKSPACE
+    assert L.dssd_device_resample_p16(None, p, p, p, 1, 2, 16, p, None, p, ok_ws, None) == B.DSSD_ERR_INVALID_ARG
+    assert L.dssd_device_resample_p16(p + 1, p, p, p, 1, 2, 16, p, None, p, ok_ws, None) == B.DSSD_ERR_INVALID_ARG
+
+    def dsd(logits=p, dtype=0, stride=16, q=p, tok=p, u=p, urs=p, T=1.0, Bn=1, g=2, V=16, n=p, token=p, ws=p,
+            wsb=ok_ws):
+        return L.dssd_dsd_verify(logits, dtype, stride, q, tok, u, urs, f(T), Bn, g, V, n, token, None, None, ws, wsb, None)
+
+    assert dsd(logits=None) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(q=None) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(urs=None) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(token=None) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(T=0.0) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(stride=15) == B.DSSD_ERR_INVALID_ARG
+    assert dsd(dtype=3) == B.DSSD_ERR_UNSUPPORTED
+    assert dsd(ws=None) == B.DSSD_ERR_WORKSPACE
+    assert dsd(wsb=64) == B.DSSD_ERR_WORKSPACE
 
     assert L.dssd_round_host(None, 0, p, p, p, p, p, f(1.0), 1, 2, 16, p, p, None, None, None, p, ok_ws, None) \
         == B.DSSD_ERR_INVALID_ARG
