@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 448.5 MB read + 99.3 MB written
-    "c4": {"bytes": 547835136, "kernel_hash": "74f7d348e60bbe49"},
+    # profiles/edge_verify_kernel_c4.md: 447.7 MB read + 99.6 MB written
+    "c4": {"bytes": 547327744, "kernel_hash": "b4750696c257446f"},
 }
 
 
