@@ -152,7 +152,8 @@ def _torch_inputs(d, device=None, pin=False):
     return out
 
 
-def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float = 1.5, payload: str = "f32"):
+def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float = 1.5, payload: str = "f32",
+                bonus: str = "device"):
     """rows/s of the CPU oracle (both halves) on the first n_seq sequences: whole passes are
     repeated until about `min_seconds` of wall time (some 10-30 s of CPU work on all cores) have gone."""
     from oracle import oracle as O
@@ -161,7 +162,10 @@ def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float 
     passes = 0
     t0 = time.perf_counter()
     while True:
-        O.verify_round(sub, w.temperature, threads=threads, payload=payload)
+        if bonus == "edge":
+            O.verify_round_bonus_at_edge(sub, w.temperature, threads=threads)
+        else:
+            O.verify_round(sub, w.temperature, threads=threads, payload=payload)
         passes += 1
         dt = time.perf_counter() - t0
         if dt >= min_seconds or passes >= 64:
@@ -250,16 +254,36 @@ def run_ours(args, w: di.Workload):
     ws_r = torch.empty(B.dssd_device_resample_workspace_bytes(Bn, gamma, V), dtype=torch.uint8, device=dev)
     ev_out = None
     rs_out = None
+    bonus_edge = args.bonus == "edge"  # Algorithm 2 as printed: the edge draws the bonus token, rows go down after rejections only
+    if bonus_edge:
+        assert args.payload == "f32", "--bonus edge carries the float32 row"
+        ws_e = torch.empty(B.dssd_edge_verify_bonus_workspace_bytes(Bn, gamma, V), dtype=torch.uint8, device=dev)
+
+    def edge_call(g):
+        nonlocal ev_out
+        if bonus_edge:
+            ev_out = B.dssd_edge_verify_bonus(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                              g["uniforms_rs"], w.temperature, out=ev_out, workspace=ws_e)
+        else:
+            ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                        w.temperature, out=ev_out, workspace=ws_e, payload=args.payload)
+
+    def device_call(g):
+        nonlocal rs_out
+        if bonus_edge:
+            rs_out = B.dssd_device_resample_rejected(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
+                                                     gamma, out={"token": ev_out["token"], "flags": ev_out["token_flags"]},
+                                                     workspace=ws_r)
+        else:
+            rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
+                                            gamma, out=rs_out, workspace=ws_r)
 
     def step(i):
         step_on(sets[i % copies])
 
     def step_on(g):
-        nonlocal ev_out, rs_out
-        ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
-                                    w.temperature, out=ev_out, workspace=ws_e, payload=args.payload)
-        rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
-                                        gamma, out=rs_out, workspace=ws_r)
+        edge_call(g)
+        device_call(g)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -275,11 +299,9 @@ def run_ours(args, w: di.Workload):
     for i in range(K):
         g = sets[i % copies]
         ev[i][0].record()
-        ev_out = B.dssd_edge_verify(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
-                                    w.temperature, out=ev_out, workspace=ws_e, payload=args.payload)
+        edge_call(g)
         ev[i][1].record()
-        rs_out = B.dssd_device_resample(ev_out["p_row"], g["draft_q"], ev_out["accept_len"], g["uniforms_rs"],
-                                        gamma, out=rs_out, workspace=ws_r)
+        device_call(g)
         ev[i][2].record()
     torch.cuda.synchronize()
     t_host1 = time.perf_counter()
@@ -299,7 +321,7 @@ def run_ours(args, w: di.Workload):
     # ---- end to end through the host-buffer entry point: copies inside the timed region ----
     host = _torch_inputs(d, pin=True)
     e2e_steps = max(3, min(K, args.e2e_steps))
-    if args.payload == "f32":
+    if args.payload == "f32" and not bonus_edge:
         arena = torch.empty(B.dssd_round_host_arena_bytes(Bn, gamma, V, B.DSSD_BF16 if w.dtype == "bf16" else B.DSSD_F32),
                             dtype=torch.uint8, device=dev)
         h_out = None
@@ -337,7 +359,7 @@ def run_ours(args, w: di.Workload):
         e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = sum(host[k].numel() * host[k].element_size() for k in
               ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs"))
-    d2h = (4 if args.payload == "f32" else 2) * Bn * 4
+    d2h = (4 if args.payload == "f32" and not bonus_edge else 2) * Bn * 4
     assert (h_out["accept_len"].numpy() == n_gpu).all()
 
     if rank != 0:
@@ -351,22 +373,28 @@ def run_ours(args, w: di.Workload):
     edge_avg_ms = sum(edge_ms) / K
     pbytes = 4 if args.payload == "f32" else 2
     edge_bytes = edge_algorithmic_bytes(w, pbytes)
+    if bonus_edge:  # every logit once, a row written per rejected sequence; row gamma's second read is not counted
+        edge_bytes = w.rows * V * w.logit_bytes + (Bn - n_bonus) * V * 4
     achieved = edge_bytes / (edge_avg_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC.get(w.name) if args.payload == "f32" else None
+    traffic = NCU_TRAFFIC.get(w.name) if args.payload == "f32" and not bonus_edge else None
     if traffic is not None and traffic.get("kernel_hash") != _kernel_hash():
         traffic = None
     rs_avg_ms = sum(rs_ms) / K
     rs_bytes = resample_algorithmic_bytes(w, n_bonus, pbytes)
+    if bonus_edge:  # p and q rows of the rejected sequences only
+        rs_bytes = (Bn - n_bonus) * (8 * V + 4)
 
     # ---- CPU baseline: the oracle as it stands, on this machine's host cores, rank 0, N = 1 ----
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         n_seq = min(Bn, args.ref_sequences)
-        rate, secs, passes = oracle_rate(w, d, n_seq, cores, payload=args.payload)
+        rate, secs, passes = oracle_rate(w, d, n_seq, cores, payload=args.payload, bonus=args.bonus)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"first {n_seq} of {Bn} sequences of {w.name}, both halves, {passes} passes in {secs:.2f} s "
                          f"wall on {cores} threads"}
-        ref = O.verify_round({k: v[:n_seq] for k, v in d.items()}, w.temperature, threads=cores, payload=args.payload)
+        sub = {k: v[:n_seq] for k, v in d.items()}
+        ref = (O.verify_round_bonus_at_edge(sub, w.temperature, threads=cores) if bonus_edge else
+               O.verify_round(sub, w.temperature, threads=cores, payload=args.payload))
         near = ref["margin_acc"] < 1e-6
         parity = {"sequences_checked": n_seq,
                   "accept_len_mismatch": int(((n_gpu[:n_seq] != ref["accept_len"]) & ~near).sum()),
@@ -394,9 +422,14 @@ def run_ours(args, w: di.Workload):
         "parity": parity,
         "e2e": {"value": world * rows / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
-        "gpu_launches": 2 * K,
+        "gpu_launches": (3 if bonus_edge else 2) * K,
         "clocks": clocks,
     }
+    if bonus_edge:
+        line["config"]["workload"] = line["config"]["workload"].replace(
+            f"{w.name}:", f"{w.name}, bonus token drawn at the edge (Algorithm 2 as printed):")
+        line["config"]["fully_accepted_sequences"] = n_bonus
+        line["roofline"]["kernel"] = "edge_verify_kernel + resample_kernel<RowLogits> (dssd_edge_verify_bonus)"
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -755,6 +788,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sampler", default="full", choices=["full", "topk"])
     ap.add_argument("--fused", action="store_true", help="Algorithm 1 in one call (dssd_dsd_verify) instead of the split round")
+    ap.add_argument("--bonus", default="device", choices=["device", "edge"],
+                    help="who draws the bonus token of a fully accepted sequence: the device from the emitted row "
+                         "(dssd_edge_verify), or the edge itself with no row emitted (dssd_edge_verify_bonus)")
     ap.add_argument("--k", type=int, default=10)
     ap.add_argument("--payload", default="f32", choices=["f32", "f16"], help="width of the emitted row P_n (full sampler only)")
     args = ap.parse_args()

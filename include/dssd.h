@@ -342,6 +342,57 @@ dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t
                             uint32_t *rs_flags, void *workspace, size_t workspace_bytes,
                             void *cuda_stream);
 
+/*
+ * ---------------------------------------------------------------------------------------------
+ * The bonus token drawn at the edge (Algorithm 2, "if j = gamma + 1: sample x_{gamma+1} ~
+ * P_{gamma+1}" inside the edge's verification loop; Section 3, "Downlink Transmission": after a
+ * round without rejection the downlink carries a token, not a row, which is the a = 0 term of the
+ * latency model of Section 3.1).  dssd_edge_verify hands the bonus row to the device instead; the
+ * two calls below follow the printed algorithm: a row P_n(.) is emitted only for sequences with a
+ * rejection, and a fully accepted sequence gets its token at the edge, drawn straight from row
+ * gamma's logits (no row is written for it, none is read back).
+ * ---------------------------------------------------------------------------------------------
+ */
+
+/* Bytes of scratch that dssd_edge_verify_bonus needs (0 if the sizes are invalid). */
+size_t dssd_edge_verify_bonus_workspace_bytes(int B, int gamma, int V);
+
+/*
+ * dssd_edge_verify plus the bonus draw.  Decisions, accept_len, p_tok, lse, flags as there.
+ *
+ * uniforms_bonus [B] float32  u' in [0,1): read for fully accepted sequences only
+ * p_row          [B, V] float32 out: row b is written iff accept_len[b] < gamma; the rows of
+ *                fully accepted sequences keep their previous contents
+ * token          [B] int32 out: the bonus token min{k : sum_{v<=k} p_v > u' * sum_v p_v} where
+ *                accept_len[b] == gamma (p_v the float32 value dssd_edge_verify would have
+ *                emitted, sums in float64), -1 elsewhere
+ * token_flags    [B] uint32 out, optional (NULL ok): DSSD_RS_FLAG_BONUS (| _INVALID for a row
+ *                without mass) where accept_len[b] == gamma, 0 elsewhere
+ * workspace      >= dssd_edge_verify_bonus_workspace_bytes(B, gamma, V) bytes, 256-byte aligned;
+ *                contents need not be initialised and are garbage afterwards
+ * Passing `token` and `token_flags` on to dssd_device_resample_rejected completes the round.
+ */
+dssd_status dssd_edge_verify_bonus(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                   const int32_t *draft_tokens, const float *draft_q_tok,
+                                   const float *uniforms, const float *uniforms_bonus,
+                                   float temperature, int B, int gamma, int V, int32_t *accept_len,
+                                   float *p_row, int32_t *token, float *p_tok, float *lse,
+                                   uint32_t *flags, uint32_t *token_flags, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * dssd_device_resample for the rejected sequences only (Algorithm 2, "Resample"): where
+ * accept_len[b] < gamma the residual draw is made and token[b], flags[b] are written; where
+ * accept_len[b] == gamma nothing is read of row b and token[b], flags[b] are left as they are
+ * (the bonus token arrived with the downlink).  accept_len outside [0, gamma]: token -1,
+ * DSSD_RS_FLAG_INVALID.  Arguments and workspace size as dssd_device_resample.
+ */
+dssd_status dssd_device_resample_rejected(const float *p_row, const float *draft_q,
+                                          const int32_t *accept_len, const float *uniforms, int B,
+                                          int gamma, int V, int32_t *token, uint32_t *flags,
+                                          void *workspace, size_t workspace_bytes,
+                                          void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -194,6 +194,56 @@ def verify_round(inputs: Dict[str, np.ndarray], temperature: float, threads: int
     return out
 
 
+RS_FLAG_BONUS, RS_FLAG_FALLBACK, RS_FLAG_INVALID = 1, 2, 4
+
+
+def bonus_draw(p_row64: np.ndarray, u: float):
+    """x_{gamma+1} ~ P_{gamma+1} at the edge (Algorithm 2, the branch j = gamma + 1): inverse CDF in
+    index order on the float64 row, token = min{k : sum_{v<=k} p_v > u * sum_v p_v}, clamped to the
+    last entry with mass.  Returns (token, flags, margin relative to the row's sum)."""
+    p = np.asarray(p_row64, dtype=np.float64)
+    C = np.cumsum(p)  # sequential, in index order
+    Z = C[-1]
+    if not (np.isfinite(Z) and Z > 0.0):
+        return -1, RS_FLAG_BONUS | RS_FLAG_INVALID, 0.0
+    t = float(np.float64(np.float32(u))) * Z
+    k = int(np.searchsorted(C, t, side="right"))
+    if k >= p.size:
+        k = int(np.nonzero(p > 0.0)[0][-1])
+        return k, RS_FLAG_BONUS, 0.0
+    below = C[k - 1] if k > 0 else 0.0
+    return k, RS_FLAG_BONUS, float(min(t - below, C[k] - t) / Z)
+
+
+def verify_round_bonus_at_edge(inputs: Dict[str, np.ndarray], temperature: float,
+                               threads: int = 1) -> Dict[str, np.ndarray]:
+    """One round as Algorithm 2 prints it: after gamma acceptances the edge itself draws the bonus
+    token from P_{gamma+1} (in float64: nothing is rounded for a transmission that does not take
+    place) and the downlink carries that token (Section 3, "Downlink Transmission"; a = 0 in Section
+    3.1); after a rejection the float32 row P_n goes down and the device draws from the residual.
+    `bonus_token` is what the edge sends (-1 for rejected sequences), `token` the round's result."""
+    ev = edge_verify(inputs["target_logits"], inputs["draft_tokens"], inputs["draft_q_tok"],
+                     inputs["uniforms"], temperature, want_p_row64=True, threads=threads)
+    gamma = inputs["target_logits"].shape[1] - 1
+    n = ev["accept_len"]
+    rs = device_resample(ev["p_row"], inputs["draft_q"], n, inputs["uniforms_rs"], gamma, threads=threads)
+    B = n.shape[0]
+    out = dict(ev)
+    out["token"] = rs["token"].copy()
+    out["rs_flags"] = rs["flags"].copy()
+    out["margin_cdf"] = rs["margin_cdf"].copy()
+    out["Z"] = rs["Z"].copy()
+    out["bonus_token"] = np.full(B, -1, np.int32)
+    out["bonus_flags"] = np.zeros(B, np.uint32)
+    for b in np.nonzero(n == gamma)[0]:
+        tok, fl, margin = bonus_draw(ev["p_row64"][b], inputs["uniforms_rs"][b])
+        out["bonus_token"][b] = out["token"][b] = tok
+        out["bonus_flags"][b] = out["rs_flags"][b] = fl
+        out["margin_cdf"][b] = margin
+    out["p_row64"] = None
+    return out
+
+
 TOPK_MAX = 32
 
 

@@ -91,6 +91,15 @@ def _load() -> ctypes.CDLL:
     L.dssd_dsd_verify.argtypes = [
         c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
         c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_edge_verify_bonus_workspace_bytes.restype = c.c_size_t
+    L.dssd_edge_verify_bonus_workspace_bytes.argtypes = [c.c_int, c.c_int, c.c_int]
+    L.dssd_edge_verify_bonus.restype = c.c_int
+    L.dssd_edge_verify_bonus.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_device_resample_rejected.restype = c.c_int
+    L.dssd_device_resample_rejected.argtypes = L.dssd_device_resample.argtypes
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -318,6 +327,70 @@ def dssd_dsd_verify(target_logits: torch.Tensor, draft_q: Optional[torch.Tensor]
         workspace.data_ptr(), workspace.numel(), _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_dsd_verify")
+    return out
+
+
+def dssd_edge_verify_bonus_workspace_bytes(B: int, gamma: int, V: int) -> int:
+    return int(lib.dssd_edge_verify_bonus_workspace_bytes(B, gamma, V))
+
+
+def dssd_edge_verify_bonus(target_logits: torch.Tensor, draft_tokens: torch.Tensor, draft_q_tok: torch.Tensor,
+                           uniforms: torch.Tensor, uniforms_bonus: torch.Tensor, temperature: float, *,
+                           out: Optional[Dict[str, torch.Tensor]] = None, want_p_tok: bool = True,
+                           want_lse: bool = True, workspace: Optional[torch.Tensor] = None,
+                           stream=None) -> Dict[str, torch.Tensor]:
+    """Edge half with the bonus token drawn at the edge (Algorithm 2 as printed): p_row is written only
+    for sequences with a rejection; `token` holds the bonus token of fully accepted sequences (-1
+    elsewhere) and `token_flags` its flags.  Returns accept_len, p_row, token, token_flags, flags and,
+    if asked, p_tok and lse.  A fresh p_row starts out as zeros so that unwritten rows are defined."""
+    assert target_logits.is_cuda and target_logits.dim() == 3
+    B, g1, V = target_logits.shape
+    gamma = g1 - 1
+    assert target_logits.stride(2) == 1 or V == 1
+    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
+    if B > 1 and target_logits.stride(0) != g1 * row_stride:
+        raise ValueError("rows of target_logits must be equally spaced")
+    dev = target_logits.device
+    if out is None:
+        out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_row": torch.zeros(B, V, dtype=torch.float32, device=dev),
+            "token": torch.empty(B, dtype=torch.int32, device=dev),
+            "token_flags": torch.empty(B, dtype=torch.int32, device=dev),
+            "flags": torch.empty(B, dtype=torch.int32, device=dev),
+            "p_tok": torch.empty(B, gamma, dtype=torch.float32, device=dev) if want_p_tok else None,
+            "lse": torch.empty(B, g1, dtype=torch.float32, device=dev) if want_lse else None,
+        }
+    if workspace is None:
+        workspace = _workspace(dssd_edge_verify_bonus_workspace_bytes(B, gamma, V), dev)
+    st = lib.dssd_edge_verify_bonus(
+        target_logits.data_ptr(), _dtype_code(target_logits), row_stride,
+        _ptr(draft_tokens), _ptr(draft_q_tok), _ptr(uniforms), uniforms_bonus.data_ptr(), ctypes.c_float(temperature),
+        B, gamma, V, out["accept_len"].data_ptr(), out["p_row"].data_ptr(), out["token"].data_ptr(),
+        _ptr(out.get("p_tok")), _ptr(out.get("lse")), _ptr(out.get("flags")), _ptr(out.get("token_flags")),
+        workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_verify_bonus")
+    return out
+
+
+def dssd_device_resample_rejected(p_row: torch.Tensor, draft_q: Optional[torch.Tensor], accept_len: torch.Tensor,
+                                  uniforms_rs: torch.Tensor, gamma: int, *, out: Dict[str, torch.Tensor],
+                                  workspace: Optional[torch.Tensor] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """Device half for the rejected sequences only: out["token"] / out["flags"] (int32 [B], as
+    dssd_edge_verify_bonus left them) are written where accept_len < gamma and kept elsewhere."""
+    assert p_row.is_cuda and p_row.dim() == 2 and p_row.is_contiguous() and p_row.dtype == torch.float32
+    B, V = p_row.shape
+    if gamma > 0:
+        assert draft_q.is_contiguous() and draft_q.dtype == torch.float32 and draft_q.numel() == B * gamma * V
+    if workspace is None:
+        workspace = _workspace(dssd_device_resample_workspace_bytes(B, gamma, V), p_row.device)
+    st = lib.dssd_device_resample_rejected(
+        p_row.data_ptr(), _ptr(draft_q) if gamma > 0 else None, accept_len.data_ptr(), uniforms_rs.data_ptr(),
+        B, gamma, V, out["token"].data_ptr(), _ptr(out.get("flags")), workspace.data_ptr(), workspace.numel(),
+        _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_device_resample_rejected")
     return out
 
 

@@ -146,7 +146,7 @@ size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V)
 namespace {
 dssd_status device_resample_any(const void *p_row, int p_half, const float *draft_q, const int32_t *accept_len,
                                 const float *uniforms, int B, int gamma, int V, int32_t *token, uint32_t *flags,
-                                void *workspace, size_t workspace_bytes, void *cuda_stream)
+                                void *workspace, size_t workspace_bytes, void *cuda_stream, int select = 0)
 {
     t_last_cuda_error = 0;
     dssd_status st = check_sizes(B, gamma, V);
@@ -168,6 +168,7 @@ dssd_status device_resample_any(const void *p_row, int p_half, const float *draf
     P.B = B;
     P.gamma = gamma;
     P.V = V;
+    P.select = select;
     P.token = token;
     P.flags = flags;
     cudaError_t e = dssd::resample_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
@@ -264,6 +265,85 @@ dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t
     R.flags = rs_flags;
     e = dssd::resample_launch(R, ws_rs, s);
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+size_t dssd_edge_verify_bonus_workspace_bytes(int B, int gamma, int V)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    return align256(dssd_edge_verify_workspace_bytes(B, gamma, V)) + align256(dssd_device_resample_workspace_bytes(B, gamma, V));
+}
+
+dssd_status dssd_edge_verify_bonus(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
+                                   const int32_t *draft_tokens, const float *draft_q_tok,
+                                   const float *uniforms, const float *uniforms_bonus,
+                                   float temperature, int B, int gamma, int V, int32_t *accept_len,
+                                   float *p_row, int32_t *token, float *p_tok, float *lse,
+                                   uint32_t *flags, uint32_t *token_flags, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !accept_len || !p_row || !token || !uniforms_bonus) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(target_logits) % esz) || (reinterpret_cast<uintptr_t>(p_row) % 4)) return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_edge_verify_bonus_workspace_bytes(B, gamma, V))
+        return DSSD_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    char *ws_edge = static_cast<char *>(workspace);
+    char *ws_rs = ws_edge + align256(dssd_edge_verify_workspace_bytes(B, gamma, V));
+
+    dssd::EdgeParams E{};
+    E.logits = target_logits;
+    E.row_stride = row_stride;
+    E.draft_tokens = draft_tokens;
+    E.draft_q_tok = draft_q_tok;
+    E.uniforms = uniforms;
+    E.temperature = temperature;
+    E.B = B;
+    E.gamma = gamma;
+    E.V = V;
+    E.accept_len = accept_len;
+    E.p_row = p_row;
+    E.p_tok = p_tok;
+    E.lse = lse;
+    E.flags = flags;
+    E.skip_bonus_row = 1;  // rows of fully accepted sequences are not emitted
+    cudaError_t e = dssd::edge_verify_launch(E, (int)dtype, ws_edge, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    // the bonus draws, from row gamma's logits and what the edge kernel left about that row
+    dssd::ResampleParams R{};
+    R.logits = target_logits;
+    R.row_stride = row_stride;
+    R.logits_dtype = (int)dtype;
+    R.c1 = E.c1;
+    R.ready = E.ready;
+    R.accept_len = accept_len;
+    R.uniforms = uniforms_bonus;
+    R.B = B;
+    R.gamma = gamma;
+    R.V = V;
+    R.select = 1;
+    R.token = token;
+    R.flags = token_flags;
+    e = dssd::resample_launch(R, ws_rs, s);
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+dssd_status dssd_device_resample_rejected(const float *p_row, const float *draft_q,
+                                          const int32_t *accept_len, const float *uniforms, int B,
+                                          int gamma, int V, int32_t *token, uint32_t *flags,
+                                          void *workspace, size_t workspace_bytes,
+                                          void *cuda_stream)
+{
+    return device_resample_any(p_row, 0, draft_q, accept_len, uniforms, B, gamma, V, token, flags, workspace,
+                               workspace_bytes, cuda_stream, 2);
 }
 
 size_t dssd_edge_verify_topk_workspace_bytes(int B, int gamma, int V, int k)

@@ -230,6 +230,12 @@ struct Pick {  // what thread 0 hands to the CTA for pass B
 
 constexpr unsigned long long kFill64 = ~0ull;
 
+// is a sequence with accepted length n (0 <= n <= gamma) one this launch draws for?
+__device__ __forceinline__ bool selected(const ResampleParams &P, int n)
+{
+    return P.select == 0 || (P.select == 1 ? n == P.gamma : n < P.gamma);
+}
+
 __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
 
 // chunk sum (b, c); a sum whose store has not landed yet still shows the fill pattern and is
@@ -496,7 +502,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         const int c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
         const int n = __ldg(P.accept_len + b);
         double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
-        if (n >= 0 && n <= P.gamma) {
+        if (n >= 0 && n <= P.gamma && selected(P, n)) {
             const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
             const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
@@ -550,6 +556,11 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
             if (tid == 0) {
                 P.token[b] = -1;
                 if (P.flags) P.flags[b] = DSSD_RS_FLAG_INVALID;
+            }
+        } else if (!selected(P, n)) {
+            if (P.select == 1 && tid == 0) {  // a rejected sequence: its token comes from the device half
+                P.token[b] = -1;
+                if (P.flags) P.flags[b] = 0u;
             }
         } else {
             const RV row = RV::make(P, b, n);

@@ -23,6 +23,10 @@ struct ResampleParams {
     const int32_t *accept_len;
     const float *uniforms;
     int B, gamma, V;
+    // which sequences are drawn for: 0 all; 1 only fully accepted ones (n == gamma: the bonus token
+    // drawn at the edge; the others get token -1 and flags 0); 2 only rejected ones (n < gamma; the
+    // entries of fully accepted sequences are left as they are)
+    int select;
     int32_t *token;
     uint32_t *flags;
     int n_chunks;   // tickets per sequence (kResampleChunk entries each)

@@ -857,6 +857,11 @@ __device__ __forceinline__ bool claim_step(const EdgeParams &P, Claim &c, Ticket
     unsigned long long b;
     split_ticket(c.ticket, P.n_emit_runs, P.emit_magic, b, t.run);
     const int n = (int)(unsigned)(c.w0 >> 32);
+    if (P.skip_bonus_row && n == P.gamma) {  // the bonus token is drawn from the logits: no row to emit
+        c.state = kWatch;
+        claim_watch(P, c);
+        return false;
+    }
     t.ref2 = __uint_as_float((unsigned)c.w1);
     t.invS = __uint_as_float((unsigned)(c.w1 >> 32));
     t.seq = (long long)b;
@@ -1317,7 +1322,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     // EMIT tickets, and what the draw needs about row n stays in the workspace (`ready`).
     const bool no_emit = !P.p_row && !P.p_row16;
     // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
-    if (!no_emit) {
+    if (!no_emit && !P.skip_bonus_row) {
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;

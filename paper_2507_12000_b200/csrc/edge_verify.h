@@ -59,6 +59,7 @@ struct EdgeParams {
     float *p_tok;
     float *lse;
     uint32_t *flags;
+    int skip_bonus_row;    // 1: no row is emitted for fully accepted sequences (n == gamma)
     // ticket geometry
     int n_slices;                  // stages per row
     int lse_run, emit_run;         // stages per LSE / EMIT ticket

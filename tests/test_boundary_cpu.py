@@ -54,6 +54,8 @@ def test_workspace_sizes(B):
     assert B.dssd_edge_verify_topk_workspace_bytes(1, 0, 8, 9) == 0
     fused = B.dssd_dsd_verify_workspace_bytes(256, 4, 151936)
     assert fused >= b + r and fused % 256 == 0 and B.dssd_dsd_verify_workspace_bytes(0, 4, 100) == 0
+    eb = B.dssd_edge_verify_bonus_workspace_bytes(256, 4, 151936)
+    assert eb >= b + r and eb % 256 == 0 and B.dssd_edge_verify_bonus_workspace_bytes(1, 4, 0) == 0
     t = B.dssd_edge_verify_topk_workspace_bytes(256, 4, 151936, 10)
     assert 0 < t < 4 << 20 and t % 256 == 0
     assert B.dssd_round_host_arena_bytes(8, 4, 32000, B.DSSD_BF16) > 8 * 5 * 32000 * 2 + 8 * 4 * 32000 * 4
@@ -152,6 +154,25 @@ def test_bad_arguments_are_rejected_before_any_launch(B):
     assert dsd(dtype=3) == B.DSSD_ERR_UNSUPPORTED
     assert dsd(ws=None) == B.DSSD_ERR_WORKSPACE
     assert dsd(wsb=64) == B.DSSD_ERR_WORKSPACE
+
+    def evb(logits=p, dtype=0, stride=16, tok=p, qt=p, u=p, ub=p, T=1.0, Bn=1, g=2, V=16, n=p, prow=p, token=p, ws=p,
+            wsb=ok_ws):
+        return L.dssd_edge_verify_bonus(logits, dtype, stride, tok, qt, u, ub, f(T), Bn, g, V, n, prow, token, None, None,
+                                        None, None, ws, wsb, None)
+
+    assert evb(logits=None) == B.DSSD_ERR_INVALID_ARG
+    assert evb(ub=None) == B.DSSD_ERR_INVALID_ARG
+    assert evb(token=None) == B.DSSD_ERR_INVALID_ARG
+    assert evb(prow=None) == B.DSSD_ERR_INVALID_ARG
+    assert evb(qt=None) == B.DSSD_ERR_INVALID_ARG
+    assert evb(T=0.0) == B.DSSD_ERR_INVALID_ARG
+    assert evb(stride=15) == B.DSSD_ERR_INVALID_ARG
+    assert evb(dtype=3) == B.DSSD_ERR_UNSUPPORTED
+    assert evb(ws=None) == B.DSSD_ERR_WORKSPACE
+    assert evb(wsb=B.dssd_edge_verify_workspace_bytes(1, 2, 16)) == B.DSSD_ERR_WORKSPACE  # the draw's scratch is missing
+    assert L.dssd_device_resample_rejected(None, p, p, p, 1, 2, 16, p, None, p, ok_ws, None) == B.DSSD_ERR_INVALID_ARG
+    assert L.dssd_device_resample_rejected(p, p, p, p, 1, 2, 16, None, None, p, ok_ws, None) == B.DSSD_ERR_INVALID_ARG
+    assert L.dssd_device_resample_rejected(p, p, p, p, 1, 2, 16, p, None, p, 8, None) == B.DSSD_ERR_WORKSPACE
 
     assert L.dssd_round_host(None, 0, p, p, p, p, p, f(1.0), 1, 2, 16, p, p, None, None, None, p, ok_ws, None) \
         == B.DSSD_ERR_INVALID_ARG
