@@ -1,7 +1,7 @@
 // Device half of the verification round: residual (or bonus) inverse-CDF draw.
 //
 // Pass A, ticket (b, c): stream chunk c of p_row[b] and of Q_n[b], form r = max(0, p - q) (or
-// r = p for the bonus draw) and add it up in float64 -> two chunk sums, 8-byte slots that are
+// r = p for the bonus draw) and add it up in float64 -> one or two chunk sums, 8-byte slots that are
 // valid once they differ from the all-ones pattern the workspace is filled with.  A ticket costs
 // one barrier and waits for no round trip.
 // Pass B, ticket b, taken by a CTA once no chunk is left for it: a block-wide float64 prefix over
@@ -24,7 +24,7 @@ namespace dssd {
 
 namespace {
 
-constexpr int kSub = kResampleChunk / 2;  // entries per chunk sum: a ticket covers two of them
+constexpr int kSub = kResampleSub;         // entries per chunk sum: a ticket covers P.subs of them
 constexpr int kRun = kSub / kThreads;      // contiguous entries per thread in pass B
 static_assert(kRun == 16, "pass B fetches a run as one group of 16 entries");
 
@@ -501,11 +501,11 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         const int64_t b = (int64_t)(t / (unsigned)P.n_chunks);
         const int c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
         const int n = __ldg(P.accept_len + b);
-        double acc0 = 0.0, acc1 = 0.0;  // the ticket's two chunk sums
+        double acc0 = 0.0, acc1 = 0.0;  // the ticket's chunk sums
         if (n >= 0 && n <= P.gamma && selected(P, n)) {
             const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-            const int e0 = c * kResampleChunk, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + kResampleChunk);
+            const int e0 = c * P.subs * kSub, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + P.subs * kSub);
             acc0 = chunk_mass(row, q, e0, e1);
             if (e2 > e1) acc1 = chunk_mass(row, q, e1, e2);
         }
@@ -527,9 +527,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
                 tot0 += s_w[buf][w][0];
                 tot1 += s_w[buf][w][1];
             }
-            unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub + 2 * c;
+            unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub + P.subs * c;
             st_relaxed_u64(cs, (unsigned long long)__double_as_longlong(tot0));
-            if (2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
+            if (P.subs == 2 && 2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
         }
         t = s_ticket[buf];
     }
@@ -578,7 +578,6 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
 {
     // all of it is filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
     // and the chunk sums read "not yet"
-    const int n_chunks = (V + kResampleChunk - 1) / kResampleChunk;
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t o = off;
@@ -586,16 +585,17 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
         return o;
     };
     const size_t o_ticket = take(256);  // the two ticket counters, on separate 128-byte lines
-    const int n_sub = (V + kResampleChunk / 2 - 1) / (kResampleChunk / 2);
+    const int n_sub = (V + kResampleSub - 1) / kResampleSub;
     const size_t o_sum = take((size_t)B * (size_t)n_sub * sizeof(double));
     if (P) {
         P->ticket = reinterpret_cast<unsigned long long *>(base + o_ticket);
         P->draw_ticket = reinterpret_cast<unsigned long long *>(base + o_ticket + 128);
         P->chunk_sum = reinterpret_cast<double *>(base + o_sum);
         P->fill_bytes = off;
-        P->n_chunks = n_chunks;
+        if (P->subs != 1) P->subs = 2;
+        P->n_chunks = (n_sub + P->subs - 1) / P->subs;
         P->n_sub = n_sub;
-        P->total_tickets = (unsigned long long)B * (unsigned long long)n_chunks;
+        P->total_tickets = (unsigned long long)B * (unsigned long long)P->n_chunks;
     }
     return off;
 }
@@ -616,6 +616,12 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
         for (int i = 1; i < 4; ++i) occ = o[i] < occ ? o[i] : occ;
     }
     if (occ < 1) occ = 1;
+    // two chunk sums per ticket halve the barriers; one per ticket evens out the CTAs' shares when
+    // there are only a few tickets for each
+    {
+        const unsigned long long pairs = (unsigned long long)P.B * (unsigned long long)(((P.V + kResampleSub - 1) / kResampleSub + 1) / 2);
+        P.subs = pairs < 4ull * (unsigned long long)sms * (unsigned long long)occ ? 1 : 2;
+    }
     resample_workspace_layout(P.B, P.V, &P, static_cast<char *>(workspace));
     P.spin_limit = 1u << 20;
     if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;

@@ -7,7 +7,7 @@
 
 namespace dssd {
 
-constexpr int kResampleChunk = 8192;  // vocabulary entries per ticket
+constexpr int kResampleSub = 4096;  // vocabulary entries per chunk sum; a ticket covers one or two of them
 
 struct ResampleParams {
     const void *p_row;   // float32 entries, or IEEE binary16 bit patterns when p_half is set
@@ -29,8 +29,9 @@ struct ResampleParams {
     int select;
     int32_t *token;
     uint32_t *flags;
-    int n_chunks;   // tickets per sequence (kResampleChunk entries each)
-    int n_sub;      // chunk sums per sequence (two per ticket)
+    int subs;       // chunk sums per ticket: 2, or 1 when there are few tickets per resident CTA
+    int n_chunks;   // tickets per sequence (subs * kResampleSub entries each)
+    int n_sub;      // chunk sums per sequence
     unsigned long long total_tickets;
     // scratch
     unsigned long long *ticket;       // next chunk ticket
@@ -40,6 +41,7 @@ struct ResampleParams {
     unsigned spin_limit;
 };
 
+// Carves the scratch (its size does not depend on P->subs, which the caller sets before: 1 or 2).
 size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base);
 
 cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream);
