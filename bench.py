@@ -359,6 +359,10 @@ def run_ours(args, w: di.Workload):
         e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = sum(host[k].numel() * host[k].element_size() for k in
               ("target_logits", "draft_tokens", "draft_q_tok", "uniforms", "draft_q", "uniforms_rs"))
+    if args.payload == "f32" and not bonus_edge:
+        # dssd_round_host uploads of draft_q only the rows Q_n of the sequences with a rejection
+        h2d -= host["draft_q"].numel() * 4
+        h2d += int((n_gpu < gamma).sum()) * V * 4
     d2h = (4 if args.payload == "f32" and not bonus_edge else 2) * Bn * 4
     assert (h_out["accept_len"].numpy() == n_gpu).all()
 

@@ -191,6 +191,12 @@ size_t dssd_round_host_arena_bytes(int B, int gamma, int V, dssd_dtype dtype);
  * `cuda_stream`.  The host buffers must stay valid until the stream has finished; use pinned
  * memory for the copies to be asynchronous.
  *
+ * Of the draft distributions only the rows the device half reads cross the bus: the call waits
+ * on the host for the accepted lengths (one cudaStreamSynchronize in the middle; accept_len is
+ * final when the call returns) and then uploads row Q_n of every sequence with a rejection,
+ * B * V * 4 bytes at most instead of B * gamma * V * 4.  Because of that wait the call cannot be
+ * made while the stream is being captured (DSSD_ERR_CUDA then).
+ *
  * host inputs:  target_logits [B, gamma+1, V] contiguous, draft_tokens, draft_q_tok, uniforms
  *               [B, gamma], draft_q [B, gamma, V], uniforms_rs [B]
  * host outputs: accept_len [B], token [B], edge_flags [B] (NULL ok), rs_flags [B] (NULL ok),

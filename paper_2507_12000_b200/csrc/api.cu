@@ -493,17 +493,25 @@ dssd_status dssd_round_host(const void *target_logits, dssd_dtype dtype,
         DSSD_TRY(cudaMemcpyAsync(d_tok_in, draft_tokens, Bz * g * 4, cudaMemcpyHostToDevice, s));
         DSSD_TRY(cudaMemcpyAsync(d_qtok, draft_q_tok, Bz * g * 4, cudaMemcpyHostToDevice, s));
         DSSD_TRY(cudaMemcpyAsync(d_u, uniforms, Bz * g * 4, cudaMemcpyHostToDevice, s));
-        DSSD_TRY(cudaMemcpyAsync(d_q, draft_q, Bz * g * Vz * 4, cudaMemcpyHostToDevice, s));
     }
     DSSD_TRY(cudaMemcpyAsync(d_urs, uniforms_rs, Bz * 4, cudaMemcpyHostToDevice, s));
     st = dssd_edge_verify(d_logits, dtype, (int64_t)V, gamma ? d_tok_in : nullptr, gamma ? d_qtok : nullptr,
                           gamma ? d_u : nullptr, temperature, B, gamma, V, d_n, d_prow, nullptr, nullptr,
                           d_ef, d_ws_e, ws_e, cuda_stream);
     if (st != DSSD_OK) return st;
+    // The device half reads row Q_n only: wait for the accepted lengths, then upload those rows
+    // (each to its place in the [B, gamma, V] array, the rest of which is never read).
+    DSSD_TRY(cudaMemcpyAsync(accept_len, d_n, Bz * 4, cudaMemcpyDeviceToHost, s));
+    DSSD_TRY(cudaStreamSynchronize(s));
+    for (size_t b = 0; b < Bz; ++b) {
+        const int n = accept_len[b];
+        if (n < 0 || n >= gamma) continue;  // bonus draw (no Q row), or no draw at all
+        const size_t off = (b * g + (size_t)n) * Vz;
+        DSSD_TRY(cudaMemcpyAsync(d_q + off, draft_q + off, Vz * 4, cudaMemcpyHostToDevice, s));
+    }
     st = dssd_device_resample(d_prow, gamma ? d_q : nullptr, d_n, d_urs, B, gamma, V, d_token, d_rf, d_ws_r,
                               ws_r, cuda_stream);
     if (st != DSSD_OK) return st;
-    DSSD_TRY(cudaMemcpyAsync(accept_len, d_n, Bz * 4, cudaMemcpyDeviceToHost, s));
     DSSD_TRY(cudaMemcpyAsync(token, d_token, Bz * 4, cudaMemcpyDeviceToHost, s));
     if (edge_flags) DSSD_TRY(cudaMemcpyAsync(edge_flags, d_ef, Bz * 4, cudaMemcpyDeviceToHost, s));
     if (rs_flags) DSSD_TRY(cudaMemcpyAsync(rs_flags, d_rf, Bz * 4, cudaMemcpyDeviceToHost, s));

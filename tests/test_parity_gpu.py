@@ -217,3 +217,25 @@ def test_round_on_host_buffers(B, oracle_mod):
     assert (out["token"].numpy() == ref["token"]).all()
     assert (out["rs_flags"].numpy().astype(np.uint32) == ref["rs_flags"]).all()
     assert prob_close(out["p_row"].numpy(), ref["p_row"]).all()
+
+
+@pytest.mark.parametrize("gamma", [0, 3])
+def test_round_on_host_buffers_uploads_only_the_rows_it_reads(B, oracle_mod, gamma):
+    """Every row of draft_q except Q_n of the sequences with a rejection is poisoned on the host:
+    the results must not change (those rows neither cross the bus nor are read)."""
+    w = di.custom(B=24, gamma=gamma, V=20000, dtype="f32", temperature=0.9, sigma_d=0.5, seed=41 + gamma)
+    d = di.generate(w)
+    ref = oracle_mod.verify_round(d, w.temperature)
+    assert gamma == 0 or (0 < (ref["accept_len"] == gamma).sum() < w.B)
+    if gamma:
+        keep = np.zeros((w.B, gamma), bool)
+        rej = ref["accept_len"] < gamma
+        keep[np.nonzero(rej)[0], ref["accept_len"][rej]] = True
+        d["draft_q"][~keep] = np.nan
+    host = {k: torch.from_numpy(v).pin_memory() for k, v in d.items()}
+    arena = torch.full((B.dssd_round_host_arena_bytes(w.B, w.gamma, w.V, B.DSSD_F32),), 0xFF, dtype=torch.uint8, device="cuda")
+    out = B.dssd_round_host(host, w.temperature, arena)
+    torch.cuda.synchronize()
+    assert (out["accept_len"].numpy() == ref["accept_len"]).all()
+    assert (out["token"].numpy() == ref["token"]).all()
+    assert (out["rs_flags"].numpy().astype(np.uint32) == ref["rs_flags"]).all()
