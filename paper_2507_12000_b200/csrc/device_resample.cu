@@ -16,6 +16,7 @@
 
 #include <mutex>
 
+#include <limits.h>
 #include <math.h>
 
 #include "dssd_device.cuh"
@@ -289,7 +290,7 @@ __device__ __forceinline__ double block_scan(double x, double *s_scan, double &t
 
 // pass B for sequence b; q == nullptr means r = p
 template <typename RV>
-__device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const float *q, unsigned fl,
+__device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const float *q, unsigned fl, float u,
                      double *s_w, Pick *s_pick, int *s_i)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -304,7 +305,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
             const double incl = block_scan(m, s_w, Z);
             ok = (Z > 0.0) && (Z < INFINITY);
             if (ok) {
-                const double target = (double)__ldg(P.uniforms + b) * Z;
+                const double target = (double)u * Z;
                 if (tid == 0) {
                     s_i[0] = 0x7fffffff;
                     s_i[1] = -1;
@@ -346,7 +347,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
         ok = (Z > 0.0) && (Z < INFINITY);
         if (ok) {
             // the first chunk whose inclusive prefix exceeds the target, else the last chunk with mass
-            const double target = (double)__ldg(P.uniforms + b) * Z;
+            const double target = (double)u * Z;
             if (tid == 0) {
                 s_i[0] = 0x7fffffff;
                 s_i[1] = -1;
@@ -486,13 +487,24 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     __shared__ Pick s_pick;
     __shared__ int s_i[2];
     __shared__ unsigned long long s_ticket[2];
+    __shared__ float s_first_u;
+    __shared__ int s_first_n;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // ---- pass A: chunk sums.  One barrier per ticket, no round trip waited for. ----
     unsigned long long next_raw = 0;  // thread 0: the ticket after the next one, drawn early
+    // thread 0: when there is at most one draw per CTA, this CTA's draw ticket is taken now, so that
+    // neither the ticket nor the sequence's accepted length and uniform are waited for when the
+    // draws begin (with more draws than CTAs the first ticket is taken when the draws begin, by
+    // whoever gets there first)
+    const bool early = (unsigned long long)P.B <= (unsigned long long)gridDim.x;
+    unsigned long long draw_raw = 0;
+    int first_n = INT_MIN;  // not loaded
+    float first_u = 0.f;
     if (tid == 0) {
         s_ticket[1] = logical(atomicAdd(P.ticket, 1ull));
         next_raw = atomicAdd(P.ticket, 1ull);
+        if (early) draw_raw = atomicAdd(P.draw_ticket, 1ull);
     }
     __syncthreads();
     unsigned long long t = s_ticket[1];
@@ -518,6 +530,10 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         if (tid == 0) {
             s_ticket[buf] = logical(next_raw);
             next_raw = atomicAdd(P.ticket, 1ull);
+            if (it == 0 && early && logical(draw_raw) < (unsigned long long)P.B) {
+                first_n = __ldg(P.accept_len + logical(draw_raw));
+                first_u = __ldg(P.uniforms + logical(draw_raw));
+            }
         }
         __syncthreads();
         if (tid == 0) {
@@ -539,11 +555,15 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     // short; a chunk sum that has not landed yet is polled for (its CTA is still running). ----
     __syncthreads();
     if (tid == 0) {
-        s_ticket[0] = logical(atomicAdd(P.draw_ticket, 1ull));
+        if (!early) draw_raw = atomicAdd(P.draw_ticket, 1ull);
+        s_ticket[0] = logical(draw_raw);
+        s_first_n = first_n;
+        s_first_u = first_u;
         next_raw = atomicAdd(P.draw_ticket, 1ull);
     }
     __syncthreads();
     unsigned long long d = s_ticket[0];
+    const bool prefetched = s_first_n != INT_MIN;
     for (int it = 1; d < (unsigned long long)P.B; ++it) {
         const int buf = it & 1;
         if (tid == 0) {
@@ -551,7 +571,8 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
             next_raw = atomicAdd(P.draw_ticket, 1ull);
         }
         const int64_t b = (int64_t)d;
-        const int n = __ldg(P.accept_len + b);
+        const int n = (it == 1 && prefetched) ? s_first_n : __ldg(P.accept_len + b);
+        const float u = (it == 1 && prefetched) ? s_first_u : __ldg(P.uniforms + b);
         if (n < 0 || n > P.gamma) {
             if (tid == 0) {
                 P.token[b] = -1;
@@ -565,7 +586,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         } else {
             const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
-            draw<RV>(P, b, row, q, q ? 0u : DSSD_RS_FLAG_BONUS, s_scan, &s_pick, s_i);
+            draw<RV>(P, b, row, q, q ? 0u : DSSD_RS_FLAG_BONUS, u, s_scan, &s_pick, s_i);
         }
         __syncthreads();
         d = s_ticket[buf];
