@@ -28,16 +28,6 @@ dssd_status check_sizes(int B, int gamma, int V)
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// q_i(x_i) read out of the draft rows (fused verification); a token id outside the vocabulary
-// gets NaN - the edge kernel rejects and flags that position by the id itself
-__global__ void gather_q_tok(const float *draft_q, const int32_t *tokens, float *q_tok, long long n, int V)
-{
-    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    const int x = tokens[i];
-    q_tok[i] = (x >= 0 && x < V) ? draft_q[(size_t)i * (size_t)V + (size_t)x] : __int_as_float(0x7fc00000);
-}
-
 }  // namespace
 
 namespace dssd {
@@ -197,8 +187,7 @@ dssd_status dssd_device_resample_p16(const uint16_t *p_row16, const float *draft
 size_t dssd_dsd_verify_workspace_bytes(int B, int gamma, int V)
 {
     if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
-    return align256(dssd_edge_verify_workspace_bytes(B, gamma, V)) +
-           align256(dssd_device_resample_workspace_bytes(B, gamma, V)) + align256((size_t)B * (size_t)gamma * 4 + 4);
+    return align256(dssd_edge_verify_workspace_bytes(B, gamma, V)) + align256(dssd_device_resample_workspace_bytes(B, gamma, V));
 }
 
 dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
@@ -225,20 +214,12 @@ dssd_status dssd_dsd_verify(const void *target_logits, dssd_dtype dtype, int64_t
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     char *ws_edge = static_cast<char *>(workspace);
     char *ws_rs = ws_edge + align256(dssd_edge_verify_workspace_bytes(B, gamma, V));
-    float *q_tok = reinterpret_cast<float *>(ws_rs + align256(dssd_device_resample_workspace_bytes(B, gamma, V)));
 
-    // q_i(x_i) out of the uploaded rows
-    if (gamma > 0) {
-        const long long n = (long long)B * gamma;
-        gather_q_tok<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(draft_q, draft_tokens, q_tok, n, V);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
     dssd::EdgeParams E{};
     E.logits = target_logits;
     E.row_stride = row_stride;
     E.draft_tokens = draft_tokens;
-    E.draft_q_tok = q_tok;
+    E.draft_q_rows = draft_q;  // q_i(x_i) is read out of the uploaded rows where a sequence is folded
     E.uniforms = uniforms;
     E.temperature = temperature;
     E.B = B;

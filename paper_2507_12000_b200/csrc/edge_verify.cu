@@ -477,8 +477,13 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
         if (live && i < P.gamma) {
             const size_t di = (size_t)b * P.gamma + i;
             x = P.draft_tokens[di];
-            qx = P.draft_q_tok[di];
             ux = P.uniforms[di];
+            if (P.draft_q_rows) {
+                // a token id outside the vocabulary has no q: NaN (the id itself gets the position rejected and flagged)
+                qx = (x >= 0 && x < P.V) ? __ldg(P.draft_q_rows + di * (size_t)P.V + (size_t)x) : __int_as_float(0x7fc00000);
+            } else {
+                qx = P.draft_q_tok[di];
+            }
             if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
         }
         // The sequence's arrival counter says every ticket has been counted; a partial whose
@@ -1322,7 +1327,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     // EMIT tickets, and what the draw needs about row n stays in the workspace (`ready`).
     const bool no_emit = !P.p_row && !P.p_row16;
     // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
-    if (!no_emit && !P.skip_bonus_row) {
+    if (!no_emit && !P.skip_bonus_row && !P.draft_q_rows) {
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;

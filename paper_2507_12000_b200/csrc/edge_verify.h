@@ -49,6 +49,7 @@ struct EdgeParams {
     int64_t row_stride;
     const int32_t *draft_tokens;
     const float *draft_q_tok;
+    const float *draft_q_rows;  // instead of draft_q_tok: the full rows [B, gamma, V]; q_i(x_i) is read out of them
     const float *uniforms;
     float temperature;
     float c1;  // log2(e) / T, rounded to float32; the kernel's temperature scaling throughout
