@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 448.0 MB read + 98.5 MB written
-    "c4": {"bytes": 546438144, "kernel_hash": "809612bdfcaa8d78"},
+    # profiles/edge_verify_kernel_c4.md: 449.0 MB read + 97.5 MB written
+    "c4": {"bytes": 546554880, "kernel_hash": "f3f74a0a3781e65c"},
 }
 
 
