@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 449.0 MB read + 97.5 MB written
-    "c4": {"bytes": 546554880, "kernel_hash": "f3f74a0a3781e65c"},
+    # profiles/edge_verify_kernel_c4.md: 451.6 MB read + 96.4 MB written
+    "c4": {"bytes": 548060928, "kernel_hash": "42fad7757195ce25"},
 }
 
 

@@ -916,6 +916,10 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     claim_watch(P, c);
     unsigned long long lse_raw = atomicAdd(P.lse_ticket, 1ull);  // the LSE ticket in hand, drawn one ticket early
     bool lse_left = true;
+    // Towards the end of the launch no new EMIT ticket is claimed while LSE work is left: the last
+    // waves of LSE tickets then finish sooner (their sequences complete sooner) and the rows held
+    // back fill the time in which the final sequences complete, on all CTAs, in short tickets.
+    bool endgame = false;
     Run lr, er;  // the LSE and the EMIT run in progress; an EMIT run goes first
     lr.kind = er.kind = kEnd;
     unsigned st = 0, par = 1;  // a fresh barrier passes a wait on parity 1: the ring starts out empty
@@ -924,9 +928,11 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     for (;;) {
         Ticket t;
         int k_begin = 0, k_end = 0;
-        if (er.kind == kEnd && claim_step(P, c, t, k_begin, k_end, !lse_left && lr.kind == kEnd)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
+        const bool hold = endgame && (lse_left || lr.kind != kEnd) && c.state == kWatch;
+        if (er.kind == kEnd && !hold && claim_step(P, c, t, k_begin, k_end, !lse_left && lr.kind == kEnd)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
         if (er.kind == kEnd && lr.kind == kEnd && lse_left) {
             const unsigned long long no = logical(lse_raw);
+            endgame = no + P.endgame_tickets >= P.total_lse;
             if (no < P.total_lse) {
                 unsigned long long row;
                 split_ticket(no, P.n_lse_runs, P.lse_magic, row, t.run);
@@ -1367,6 +1373,16 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     P.n_lse_runs = (P.n_slices + P.lse_run - 1) / P.lse_run;
     P.n_emit_runs = (P.n_slices + P.emit_run - 1) / P.emit_run;
     P.total_lse = R * (unsigned long long)P.n_lse_runs;
+    {
+        // the last kEdgeEndgameWaves waves of LSE tickets; in long launches with many positions per
+        // sequence (the rows to emit are a small share of the bytes, and a stream of reads alone runs
+        // faster than one with writes mixed in) all but the first eighth of the waves
+        const unsigned long long waves = (P.total_lse + resident_ctas - 1) / resident_ctas;
+        unsigned long long hold = (unsigned long long)kEdgeEndgameWaves;
+        if (waves >= (unsigned long long)kEdgeEndgameLongWaves && P.gamma + 1 >= kEdgeEndgameLongRows)
+            hold = waves * (unsigned long long)kEdgeEndgameLongEighths / 8;
+        P.endgame_tickets = hold * resident_ctas;
+    }
     P.total_emit = no_emit ? 0ull : (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
     // t / d == mulhi64(t, ceil(2^64 / d)) for every t with t * d * d < 2^64
     auto magic = [](unsigned long long total, int d) -> unsigned long long {

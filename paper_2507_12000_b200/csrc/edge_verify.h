@@ -26,6 +26,19 @@ namespace dssd {
 #define DSSD_EDGE_TICKETS_PER_CTA 2
 #endif
 
+#ifndef DSSD_EDGE_ENDGAME_WAVES
+#define DSSD_EDGE_ENDGAME_WAVES 3
+#endif
+#ifndef DSSD_EDGE_ENDGAME_LONG_WAVES
+#define DSSD_EDGE_ENDGAME_LONG_WAVES 32
+#endif
+#ifndef DSSD_EDGE_ENDGAME_LONG_EIGHTHS
+#define DSSD_EDGE_ENDGAME_LONG_EIGHTHS 7
+#endif
+constexpr int kEdgeEndgameWaves = DSSD_EDGE_ENDGAME_WAVES;  // EMIT claims are held back during the last so many waves of LSE tickets
+constexpr int kEdgeEndgameLongRows = 8;                                  // ... with at least so many positions per sequence ...
+constexpr int kEdgeEndgameLongWaves = DSSD_EDGE_ENDGAME_LONG_WAVES;      // launches of at least so many waves ...
+constexpr int kEdgeEndgameLongEighths = DSSD_EDGE_ENDGAME_LONG_EIGHTHS;  // ... hold them back during the last so many eighths of the waves
 constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
 constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 2);  // + the producer warp and the fold warp
 constexpr int kEdgeStageBytes = DSSD_EDGE_STAGE_BYTES;   // logits bytes per ring stage (one bulk copy)
@@ -67,6 +80,7 @@ struct EdgeParams {
     int n_lse_runs, n_emit_runs;   // tickets per row
     unsigned long long total_lse;  // rows * n_lse_runs
     unsigned long long total_emit; // B * n_emit_runs
+    unsigned long long endgame_tickets;  // EMIT claims are held back once so few LSE tickets are left
     unsigned long long lse_magic, emit_magic;  // ceil(2^64 / n_*_runs) when multiply-high division is exact, else 0
     unsigned spin_limit;
     // workspace, filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
