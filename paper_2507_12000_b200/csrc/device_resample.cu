@@ -621,13 +621,19 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
     return off;
 }
 
+// resident CTAs per device, looked up on the first launch made with that device current (the
+// occupancy depends on the compiled kernels only); 0: not looked up yet
+static int g_resample_resident[64];
+static int g_resample_sms[64];
+
 cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream)
 {
     cudaError_t err;
     int dev = 0, sms = 0, occ = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
-    if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-    {
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (g_resample_resident[dev] == 0) {
+        if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
         int o[4] = {0, 0, 0, 0};
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[0], resample_kernel<RowF32>, kThreads, 0)) != cudaSuccess) return err;
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[1], resample_kernel<RowF16>, kThreads, 0)) != cudaSuccess) return err;
@@ -635,7 +641,12 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[3], resample_kernel<RowLogits<DSSD_BF16>>, kThreads, 0)) != cudaSuccess) return err;
         occ = o[0];
         for (int i = 1; i < 4; ++i) occ = o[i] < occ ? o[i] : occ;
+        if (occ < 1) occ = 1;
+        g_resample_sms[dev] = sms;
+        g_resample_resident[dev] = occ;  // written last: a concurrent first call finds either 0 or the final pair
     }
+    sms = g_resample_sms[dev];
+    occ = g_resample_resident[dev];
     if (occ < 1) occ = 1;
     // two chunk sums per ticket halve the barriers; one per ticket evens out the CTAs' shares when
     // there are only a few tickets for each
