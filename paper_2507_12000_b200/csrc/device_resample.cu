@@ -25,6 +25,12 @@ namespace dssd {
 
 namespace {
 
+#ifndef DSSD_RS_WIDE
+#define DSSD_RS_WIDE 1  // whole tickets request all their loads at once (ticket_mass2)
+#endif
+#ifndef DSSD_RS_CTAS
+#define DSSD_RS_CTAS 4
+#endif
 constexpr int kSub = kResampleSub;         // entries per chunk sum: a ticket covers P.subs of them
 constexpr int kRun = kSub / kThreads;      // contiguous entries per thread in pass B
 static_assert(kRun == 16, "pass B fetches a run as one group of 16 entries");
@@ -204,6 +210,40 @@ __device__ __forceinline__ double chunk_mass(const RV &row, const float *q, int 
     }
     for (int e = done + tid; e < e1; e += kThreads) acc += q ? res(row.ld(e), __ldg(q + e)) : (double)row.ld(e);
     return acc;
+}
+
+// A whole ticket of two full chunk sums whose rows are 16-byte aligned: all of a thread's loads
+// (eight quads of p and of q) are requested before the first is used.  Quads u < 4 of a thread
+// belong to the first chunk sum, the others to the second; the order of addition within each is
+// the one chunk_mass uses, so both give the same bits.
+template <typename RV>
+__device__ __forceinline__ void ticket_mass2(const RV &row, const float *q, int e0, double &acc0, double &acc1)
+{
+    const int tid = threadIdx.x;
+    typename RV::Raw a[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) a[u] = row.ld_quad_stream(e0, tid + u * kThreads);
+    if (q) {
+        const uint4 *q4 = reinterpret_cast<const uint4 *>(q + e0);
+        uint4 b[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) b[u] = ld_stream16(q4 + tid + u * kThreads);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float4 x = row.quad(a[u]), y = as_f4(b[u]);
+            const double t = (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
+            if (u < 4) acc0 += t;
+            else acc1 += t;
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float4 x = row.quad(a[u]);
+            const double t = ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
+            if (u < 4) acc0 += t;
+            else acc1 += t;
+        }
+    }
 }
 
 // CTA-wide sum in a fixed order; result valid in thread 0
@@ -480,7 +520,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
 }
 
 template <typename RV>
-__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ ResampleParams P)
+__global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const __grid_constant__ ResampleParams P)
 {
     __shared__ double s_w[2][kWarps][2];
     __shared__ double s_scan[kWarps];
@@ -518,8 +558,13 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
             const RV row = RV::make(P, b, n);
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
             const int e0 = c * P.subs * kSub, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + P.subs * kSub);
-            acc0 = chunk_mass(row, q, e0, e1);
-            if (e2 > e1) acc1 = chunk_mass(row, q, e1, e2);
+            static_assert(kSub == 4 * 4 * kThreads, "a thread's four quads per chunk sum");
+            if (DSSD_RS_WIDE && e2 - e0 == 2 * kSub && row.aligned(e0) && (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0)) {
+                ticket_mass2(row, q, e0, acc0, acc1);
+            } else {
+                acc0 = chunk_mass(row, q, e0, e1);
+                if (e2 > e1) acc1 = chunk_mass(row, q, e1, e2);
+            }
         }
         acc0 = warp_sum(acc0);
         acc1 = warp_sum(acc1);
