@@ -194,3 +194,29 @@ def test_garbage_workspace_and_cuda_graph(B):
     torch.cuda.synchronize()
     for k in ("accept_len", "token", "token_flags", "flags"):
         assert torch.equal(out[k], ref[k]), k
+
+
+def test_rejected_only_draw_leaves_other_entries_alone(B, oracle_mod):
+    """dssd_device_resample_rejected on hand-made accepted lengths: n < gamma is drawn for, n == gamma
+    keeps what the arrays held, n outside [0, gamma] gives token -1 and DSSD_RS_FLAG_INVALID."""
+    V, gamma = 9000, 3
+    rng = np.random.default_rng(3)
+    p = rng.random((6, V)).astype(np.float32)
+    p /= p.sum(axis=1, keepdims=True)
+    q = rng.random((6, gamma, V)).astype(np.float32)
+    q /= q.sum(axis=2, keepdims=True)
+    n = np.array([0, gamma, -1, gamma + 1, 2, gamma], np.int32)
+    u = rng.random(6).astype(np.float32)
+    ref = oracle_mod.device_resample(p, q, n, u, gamma)
+    tok = torch.full((6,), -77, dtype=torch.int32, device="cuda")
+    fl = torch.full((6,), -77, dtype=torch.int32, device="cuda")
+    B.dssd_device_resample_rejected(torch.from_numpy(p).cuda(), torch.from_numpy(q).cuda(), torch.from_numpy(n).cuda(),
+                                    torch.from_numpy(u).cuda(), gamma, out={"token": tok, "flags": fl})
+    torch.cuda.synchronize()
+    tok, fl = tok.cpu().numpy(), fl.cpu().numpy()
+    for b in (0, 4):
+        assert tok[b] == ref["token"][b] and np.uint32(fl[b]) == ref["flags"][b]
+    for b in (1, 5):
+        assert tok[b] == -77 and fl[b] == -77
+    for b in (2, 3):
+        assert tok[b] == -1 and np.uint32(fl[b]) == ref["flags"][b] == oracle_mod.RS_FLAG_INVALID
