@@ -464,14 +464,15 @@ int dssd_oracle_device_resample_topk(const int32_t *p_idx, const float *p_val,
  * target_logits [B, gamma+1, V] (row_stride elements between rows), draft_q [B, gamma, V] float32,
  * draft_tokens [B, gamma], uniforms [B, gamma] (acceptance), uniforms_rs [B] (the draw).
  * outputs: accept_len [B], token [B], flags [B] (edge flags, may be NULL), rs_flags [B] (may be
- * NULL), margin_acc [B], margin_cdf [B] (may be NULL) as in the split functions.
+ * NULL), margin_acc [B], margin_cdf [B] (may be NULL) as in the split functions, Z_out [B] (may be
+ * NULL): the mass sum_v r_v that the returned token was drawn from (0 when there was none).
  * ------------------------------------------------------------------------------------------ */
 int dssd_oracle_dsd_verify(const void *target_logits, int dtype, int64_t row_stride,
                            const float *draft_q, const int32_t *draft_tokens,
                            const float *uniforms, const float *uniforms_rs, float temperature,
                            int B, int gamma, int V,
                            int32_t *accept_len, int32_t *token, uint32_t *flags, uint32_t *rs_flags,
-                           double *margin_acc, double *margin_cdf)
+                           double *margin_acc, double *margin_cdf, double *Z_out)
 {
     const double T = (double)temperature;
     const size_t esz = (dtype == ORACLE_BF16) ? 2 : 4;
@@ -521,7 +522,7 @@ int dssd_oracle_dsd_verify(const void *target_logits, int dtype, int64_t row_str
             double l = row_lse(row, dtype, V, T, &ok);
             double u = (double)uniforms_rs[b];
             int32_t tok = -1;
-            double mg = 0.0;
+            double mg = 0.0, Z_used = 0.0;
             if (n == gamma) rfl |= RS_FLAG_BONUS;
             for (int pass = 0; pass < 2 && tok < 0; ++pass) {
                 /* pass 0: the residual (or the bonus row); pass 1: fall back to P_n when it has no mass */
@@ -536,6 +537,7 @@ int dssd_oracle_dsd_verify(const void *target_logits, int dtype, int64_t row_str
                     Z += qq ? fmax(0.0, p - (double)qq[v]) : p;
                 }
                 if (!(Z > 0.0) || !(Z < INFINITY)) continue;
+                Z_used = Z;
                 double t = u * Z, C = 0.0, Cprev;
                 int32_t last_pos = -1;
                 for (int v = 0; v < V; ++v) {
@@ -556,6 +558,7 @@ int dssd_oracle_dsd_verify(const void *target_logits, int dtype, int64_t row_str
             if (tok < 0) { rfl |= RS_FLAG_INVALID; mg = 0.0; }
             token[b] = tok;
             if (margin_cdf) margin_cdf[b] = mg;
+            if (Z_out) Z_out[b] = tok < 0 ? 0.0 : Z_used;
         }
         if (flags) flags[b] = fl;
         if (rs_flags) rs_flags[b] = rfl;

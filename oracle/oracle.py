@@ -60,7 +60,8 @@ def _load():
         lib.dssd_oracle_dsd_verify.restype = c.c_int
         lib.dssd_oracle_dsd_verify.argtypes = [
             c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
-            c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+            c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+            c.c_void_p]
         lib.dssd_oracle_edge_verify_topk.restype = c.c_int
         lib.dssd_oracle_edge_verify_topk.argtypes = [
             c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -353,6 +354,7 @@ def dsd_verify(inputs: Dict[str, np.ndarray], temperature: float, threads: int =
         "accept_len": np.zeros(B, np.int32), "token": np.zeros(B, np.int32),
         "flags": np.zeros(B, np.uint32), "rs_flags": np.zeros(B, np.uint32),
         "margin_acc": np.zeros(B, np.float64), "margin_cdf": np.zeros(B, np.float64),
+        "Z": np.zeros(B, np.float64),
     }
 
     def run(rng):
@@ -361,7 +363,8 @@ def dsd_verify(inputs: Dict[str, np.ndarray], temperature: float, threads: int =
             _ptr(tl[b0:b1]), dtype, V, _ptr(q[b0:b1]) if gamma > 0 else None, _ptr(tok[b0:b1]), _ptr(u[b0:b1]),
             _ptr(urs[b0:b1]), ctypes.c_float(temperature), b1 - b0, gamma, V,
             _ptr(out["accept_len"][b0:b1]), _ptr(out["token"][b0:b1]), _ptr(out["flags"][b0:b1]),
-            _ptr(out["rs_flags"][b0:b1]), _ptr(out["margin_acc"][b0:b1]), _ptr(out["margin_cdf"][b0:b1]))
+            _ptr(out["rs_flags"][b0:b1]), _ptr(out["margin_acc"][b0:b1]), _ptr(out["margin_cdf"][b0:b1]),
+            _ptr(out["Z"][b0:b1]))
         if rc != 0:
             raise ValueError("dssd_oracle_dsd_verify: invalid arguments")
 

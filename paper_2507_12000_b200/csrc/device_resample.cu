@@ -14,6 +14,7 @@
 #include "device_resample.h"
 #include "edge_verify.h"
 
+#include <atomic>
 #include <mutex>
 
 #include <limits.h>
@@ -668,8 +669,8 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
 
 // resident CTAs per device, looked up on the first launch made with that device current (the
 // occupancy depends on the compiled kernels only); 0: not looked up yet
-static int g_resample_resident[64];
-static int g_resample_sms[64];
+static std::atomic<int> g_resample_resident[64];  // published last (release), read first (acquire)
+static std::atomic<int> g_resample_sms[64];
 
 cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream)
 {
@@ -677,7 +678,8 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     int dev = 0, sms = 0, occ = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (g_resample_resident[dev] == 0) {
+    occ = g_resample_resident[dev].load(std::memory_order_acquire);
+    if (occ == 0) {
         if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
         int o[4] = {0, 0, 0, 0};
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[0], resample_kernel<RowF32>, kThreads, 0)) != cudaSuccess) return err;
@@ -687,12 +689,10 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
         occ = o[0];
         for (int i = 1; i < 4; ++i) occ = o[i] < occ ? o[i] : occ;
         if (occ < 1) occ = 1;
-        g_resample_sms[dev] = sms;
-        g_resample_resident[dev] = occ;  // written last: a concurrent first call finds either 0 or the final pair
+        g_resample_sms[dev].store(sms, std::memory_order_relaxed);
+        g_resample_resident[dev].store(occ, std::memory_order_release);  // a concurrent first call finds either 0 or the final pair
     }
-    sms = g_resample_sms[dev];
-    occ = g_resample_resident[dev];
-    if (occ < 1) occ = 1;
+    sms = g_resample_sms[dev].load(std::memory_order_relaxed);
     // two chunk sums per ticket halve the barriers; one per ticket evens out the CTAs' shares when
     // there are only a few tickets for each
     {
@@ -756,7 +756,9 @@ extern "C" dssd_status dssd_device_resample_static(const float *p_row, const flo
         std::lock_guard<std::mutex> lock(g_static_mutex);
         if (!g_static_ptr[dev]) {
             void *ptr = nullptr;
-            if ((e = cudaGetSymbolAddress(&ptr, g_static_scratch)) != cudaSuccess || !ptr) {
+            e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e == cudaSuccess && !ptr) e = cudaErrorInvalidSymbol;  // a look-up that gives no address is a failed one
+            if (e != cudaSuccess) {
                 dssd::set_last_cuda_error((int)e);
                 return DSSD_ERR_CUDA;
             }

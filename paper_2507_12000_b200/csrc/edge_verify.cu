@@ -35,6 +35,8 @@
 
 #include <math.h>
 
+#include <atomic>
+
 #include <cooperative_groups.h>
 
 #include "dssd_device.cuh"
@@ -1048,6 +1050,10 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
     const long long b = blockIdx.x / csize;
     const float c1 = P.c1;
     const long long rowbytes = (long long)P.V * E::kBytes;
+    // A CTA's shared memory may be written by its peers only once it is known to have started:
+    // every CTA announces itself here, and the matching wait stands before the first remote
+    // store (the streaming loop lies between the two, so the wait costs nothing).
+    if (csize > 1) (void)cluster.barrier_arrive();
     // Every CTA of the cluster takes a contiguous 1/csize of each row's 16-byte vectors.
     // The rows are streamed side by side, a group of `wpr` warps per row, so that the loads of
     // all rows are in flight together; the first lane of each group also fetches the row's
@@ -1104,6 +1110,7 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
         }
     }
     __syncthreads();
+    if (csize > 1) cluster.barrier_wait();  // every CTA of the cluster is running
     // each CTA's result per row goes to rank 0's shared memory (distributed shared memory)
     if (tid < rows) {
         float R = DSSD_NEG_INF;
@@ -1305,9 +1312,11 @@ size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, 
     return off;
 }
 
-// launch geometry per device, filled on first use (occupancy depends on the compiled kernel only)
-static int g_edge_ctas_per_sm[64][2];
-static int g_sm_count[64];
+// launch geometry per device, filled on first use (occupancy depends on the compiled kernel only).
+// g_sm_count is published last (release) and read first (acquire): a concurrent first call finds
+// either 0 and looks the constants up itself, or the complete set.
+static std::atomic<int> g_edge_ctas_per_sm[64][2];
+static std::atomic<int> g_sm_count[64];
 
 cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaStream_t stream)
 {
@@ -1315,7 +1324,8 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     int dev = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (g_sm_count[dev] == 0) {
+    int sm_count = g_sm_count[dev].load(std::memory_order_acquire);
+    if (sm_count == 0) {
         int sms = 0, occ0 = 0, occ1 = 0;
         if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
         if ((err = cudaFuncSetAttribute(edge_verify_kernel<DSSD_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEdgeSmemBytes)) != cudaSuccess) return err;
@@ -1323,10 +1333,12 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ0, edge_verify_kernel<DSSD_F32>, kEdgeThreads, kEdgeSmemBytes)) != cudaSuccess) return err;
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, edge_verify_kernel<DSSD_BF16>, kEdgeThreads, kEdgeSmemBytes)) != cudaSuccess) return err;
         if (occ0 < 1 || occ1 < 1) return cudaErrorLaunchOutOfResources;
-        g_edge_ctas_per_sm[dev][0] = occ0;
-        g_edge_ctas_per_sm[dev][1] = occ1;
-        g_sm_count[dev] = sms;
+        g_edge_ctas_per_sm[dev][0].store(occ0, std::memory_order_relaxed);
+        g_edge_ctas_per_sm[dev][1].store(occ1, std::memory_order_relaxed);
+        g_sm_count[dev].store(sms, std::memory_order_release);
+        sm_count = sms;
     }
+    const int ctas_per_sm = g_edge_ctas_per_sm[dev][dtype == DSSD_BF16].load(std::memory_order_relaxed);
     const int esz = dtype == DSSD_BF16 ? 2 : 4;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
     // Without an output row (the fused verification of Algorithm 1) nothing is emitted: there are no
@@ -1337,9 +1349,9 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;
-        while (csize > 1 && (long long)P.B * csize > g_sm_count[dev]) csize /= 2;
+        while (csize > 1 && (long long)P.B * csize > sm_count) csize /= 2;
         if (P.gamma + 1 <= kSmallMaxRows && seq_bytes / csize <= kSmallMaxCtaBytes &&
-            (long long)P.B * csize <= g_sm_count[dev]) {
+            (long long)P.B * csize <= sm_count) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3((unsigned)(P.B * csize));
             cfg.blockDim = dim3(kSmallThreads);
@@ -1359,7 +1371,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     const unsigned long long R = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);
     const long long n_slices = ((long long)P.V * esz + kS - 1) / kS;
     P.n_slices = (int)(n_slices < 1 ? 1 : n_slices);
-    const unsigned long long resident_ctas = (unsigned long long)g_sm_count[dev] * g_edge_ctas_per_sm[dev][dtype == DSSD_BF16];
+    const unsigned long long resident_ctas = (unsigned long long)sm_count * (unsigned long long)ctas_per_sm;
     // Stages per ticket: as long as every resident CTA still gets about kEdgeTicketsPerCta
     // tickets, at most kEdgeMaxRun, and then evened out so that a row splits into equal tickets.
     unsigned long long run = (R * (unsigned long long)P.n_slices) / (resident_ctas * kEdgeTicketsPerCta);

@@ -45,6 +45,7 @@
 //
 // Device kernel: one warp per sequence, everything in registers and shuffles, sums strictly
 // sequential in float64 so that the draw is reproducible bit for bit.
+#include <atomic>
 #include "topk_verify.h"
 
 #include <math.h>
@@ -884,7 +885,7 @@ size_t topk_workspace_layout(int B, int gamma, int k, TopkParams *P, char *base)
     return cnt + ((lists + 255) & ~(size_t)255);
 }
 
-static int g_topk_ctas[64];  // CTAs resident on the device at once (0 = not asked yet)
+static std::atomic<int> g_topk_ctas[64];  // CTAs resident on the device at once (0 = not asked yet)
 constexpr size_t kTopkSmemBytes = (size_t)kStages * kStageBytes + sizeof(Smem);
 
 cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaStream_t stream)
@@ -892,7 +893,7 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
     cudaError_t err;
     int dev = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
-    int ctas = (dev >= 0 && dev < 64) ? g_topk_ctas[dev] : 0;
+    int ctas = (dev >= 0 && dev < 64) ? g_topk_ctas[dev].load(std::memory_order_acquire) : 0;
     if (ctas == 0) {
         int sms = 0;
         if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
@@ -903,7 +904,7 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
         if ((err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ1, topk_verify_kernel<DSSD_BF16>, kTkThreads, kTopkSmemBytes)) != cudaSuccess) return err;
         const int occ = occ0 < occ1 ? occ0 : occ1;
         ctas = (sms < 1 ? 1 : sms) * (occ < 1 ? 1 : occ);
-        if (dev >= 0 && dev < 64) g_topk_ctas[dev] = ctas;
+        if (dev >= 0 && dev < 64) g_topk_ctas[dev].store(ctas, std::memory_order_release);
     }
     topk_workspace_layout(P.B, P.gamma, P.k, &P, static_cast<char *>(workspace));
     const unsigned long long rows = (unsigned long long)P.B * (unsigned long long)(P.gamma + 1);

@@ -53,6 +53,9 @@ def test_d2_agrees_with_the_split_round(oracle_mod, dtype):
     assert (fused["accept_len"] == split["accept_len"]).all()
     assert (fused["flags"] == split["flags"]).all() and (fused["rs_flags"] == split["rs_flags"]).all()
     np.testing.assert_allclose(fused["margin_acc"], split["margin_acc"], rtol=1e-12)
+    # the mass the token is drawn from: the split round forms it from the float32 row (each entry within
+    # 2^-24 relative of the float64 one, so the sums differ by at most 2^-24 * sum p = 6e-8)
+    np.testing.assert_allclose(fused["Z"], split["Z"], rtol=0, atol=1e-7)
     safe = split["margin_cdf"] > 1e-5
     assert safe.mean() > 0.95 and (fused["token"][safe] == split["token"][safe]).all()
     assert len(set(fused["accept_len"].tolist())) >= 3

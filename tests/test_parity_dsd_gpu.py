@@ -30,12 +30,15 @@ def compare_dsd(B, O, d, T, logits_view=None, threads=4):
     near = ref["margin_acc"] < NEAR
     assert ((n == ref["accept_len"]) | near).all()
     same = n == ref["accept_len"]
-    # the kernel's p is a float32 (relative error RTOL): a CDF step may move by about RTOL / Z relative to Z
-    Z_floor = 1e-3
-    slack = np.maximum(NEAR, 2 * RTOL / Z_floor)
-    bad = (tok != ref["token"]) & same & ~(ref["margin_cdf"] < slack)
+    # the kernel's p is a float32 (relative error RTOL): a CDF step may move by about RTOL / Z relative to
+    # Z, the mass the oracle drew from; only sequences closer than that to a step may differ
+    slack = np.maximum(NEAR, 2 * RTOL / np.maximum(ref["Z"], 1e-30))
+    excused = same & (ref["margin_cdf"] < slack)
+    bad = (tok != ref["token"]) & same & ~excused
     assert not bad.any(), (np.nonzero(bad)[0][:8], tok[bad][:8], ref["token"][bad][:8], ref["margin_cdf"][bad][:8])
     assert (out["rs_flags"].cpu().numpy().astype(np.uint32)[same] == ref["rs_flags"][same]).all()
+    compare_dsd.last = {"sequences": int(n.size), "near_accept": int(near.sum()), "near_cdf": int(excused.sum()),
+                        "token_differs": int(((tok != ref["token"]) & same).sum())}
     return n, tok, g, tl
 
 
@@ -116,3 +119,7 @@ def test_anomalies_are_flagged_not_faulted(B, oracle_mod):
 def test_named_configs(B, oracle_mod, name):
     w = di.get_workload(name)
     compare_dsd(B, oracle_mod, di.generate(w, threads=8), w.temperature, threads=8)
+    rep = compare_dsd.last
+    print(f"fused parity on {name}: {rep}")
+    # the draws excused as near a CDF step are a small minority, not the bulk of the batch
+    assert rep["near_cdf"] <= max(2, rep["sequences"] // 10), rep
