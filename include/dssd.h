@@ -15,7 +15,10 @@
  *                         tokens, the sampler of the paper's experiments (Section 4);
  *   dssd_edge_verify_p16, dssd_device_resample_p16
  *                         the round with the downlink row in 16 bits per value (Section 2.2);
- *   dssd_dsd_verify       the fused verification of Algorithm 1 (no row is transmitted).
+ *   dssd_dsd_verify       the fused verification of Algorithm 1 (no row is transmitted);
+ *   dssd_edge_partial, dssd_edge_combine, dssd_edge_emit_shard, dssd_resample_shard_mass,
+ *   dssd_resample_shard_draw
+ *                         the round for an edge whose vocabulary is sharded over several GPUs.
  *
  * Notation follows the paper: gamma draft tokens x_1..x_gamma with draft probabilities
  * q_i(x_i), target distributions P_1..P_{gamma+1} over a vocabulary of V entries, uniforms
@@ -398,6 +401,126 @@ dssd_status dssd_device_resample_rejected(const float *p_row, const float *draft
                                           int gamma, int V, int32_t *token, uint32_t *flags,
                                           void *workspace, size_t workspace_bytes,
                                           void *cuda_stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------
+ * Vocabulary-sharded round.  (The paper runs the target model on one GPU; this is Algorithm 2,
+ * "Verification Process" / "Downlink Transmission" / "Resample" of Section 3, unchanged, for an
+ * edge whose LM head is tensor-parallel: GPU g of G holds entries [v_g, v_{g+1}) of every logit
+ * row.  Only the sums over the vocabulary are formed shard by shard.)
+ *
+ *   1. every shard: dssd_edge_partial          per row, its slice's share of sum_v exp(l_v / T)
+ *   2. exchange:    all-gather of part_ref, part_sum [B, gamma+1] and tok_logit [B, gamma]
+ *                   (a few bytes per row; the caller's collective, e.g. NCCL)
+ *   3. every shard: dssd_edge_combine          log-sum-exp, acceptance test, first rejection n:
+ *                                              identical inputs give identical results everywhere
+ *   4. every shard: dssd_edge_emit_shard       its slice of the downlink row P_n
+ *   5. every shard: dssd_resample_shard_mass   its slice's residual mass and plain mass
+ *   6. exchange:    all-gather of mass [B, 2]
+ *   7. every shard: dssd_resample_shard_draw   the shard that holds u' Z returns the token, the
+ *                                              others -1 (a max over shards completes the round)
+ * Steps 5-7 are the device half for a device that holds the rows sharded the same way; a device
+ * that receives whole rows calls dssd_device_resample on the assembled row instead.
+ * The library makes no collective call itself and never reads another GPU's memory.
+ * ---------------------------------------------------------------------------------------------
+ */
+
+/* Bytes of scratch that dssd_edge_partial needs (0 if the sizes are invalid). */
+size_t dssd_edge_partial_workspace_bytes(int B, int gamma, int V_shard);
+
+/*
+ * One shard's share of every row's log-sum-exp (Section 3, "Verification Process").
+ *
+ * logits_shard  this shard's slice of the target logits: row (b, i) starts at element
+ *               (b*(gamma+1)+i)*row_stride and holds V_shard entries, vocabulary ids
+ *               v_begin .. v_begin + V_shard - 1 (a view into whole rows works: row_stride >= V_shard)
+ * draft_tokens  [B, gamma] int32  x_i, ids in the whole vocabulary (may be NULL iff gamma == 0)
+ * part_ref      [B, gamma+1] float32 out, integer-valued, and
+ * part_sum      [B, gamma+1] float64 out:  sum_{v in slice} 2^(l_v * c1) = part_sum * 2^part_ref with
+ *               c1 = float32(log2(e) / T); (0, 0) for a slice of -inf only; part_sum is NaN for a
+ *               slice that holds a NaN or +inf
+ * tok_logit     [B, gamma] float32 out: l_{x_i} where v_begin <= x_i < v_begin + V_shard, NaN
+ *               elsewhere (may be NULL iff gamma == 0)
+ * workspace     >= dssd_edge_partial_workspace_bytes(B, gamma, V_shard) bytes, 256-byte aligned;
+ *               contents need not be initialised and are garbage afterwards
+ */
+dssd_status dssd_edge_partial(const void *logits_shard, dssd_dtype dtype, int64_t row_stride,
+                              const int32_t *draft_tokens, int v_begin, float temperature, int B,
+                              int gamma, int V_shard, float *part_ref, double *part_sum,
+                              float *tok_logit, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream);
+
+/*
+ * The shards' partial sums -> log-sum-exp of every row, p_i(x_i), the acceptance test
+ * u_i < min(1, p_i(x_i) / q_i(x_i)) and the first rejection n (Algorithm 2, "Verification
+ * Process"), evaluated exactly as dssd_edge_verify evaluates them.
+ *
+ * part_ref, part_sum  [G, B, gamma+1], tok_logit [G, B, gamma]: the outputs of the G calls of
+ *               dssd_edge_partial, shard-major (the layout an all-gather leaves)
+ * temperature   the T the partial sums were formed with
+ * V             size of the whole vocabulary (ids outside [0, V) are rejected and flagged)
+ * accept_len    [B] int32 out;  p_tok [B, gamma], lse [B, gamma+1], flags [B] out, optional
+ * row_scale     [B, 2] float32 out: row n's reference exponent and 1 / sum, which
+ *               dssd_edge_emit_shard turns logits into probabilities with
+ */
+dssd_status dssd_edge_combine(const float *part_ref, const double *part_sum, const float *tok_logit,
+                              int G, const int32_t *draft_tokens, const float *draft_q_tok,
+                              const float *uniforms, float temperature, int B, int gamma, int V,
+                              int32_t *accept_len, float *row_scale, float *p_tok, float *lse,
+                              uint32_t *flags, void *cuda_stream);
+
+/*
+ * This shard's slice of the downlink row (Section 3, "Downlink Transmission"; b_prob = 32):
+ * p_row_shard[b, v] = P_n(v_begin + v) for the slice's V_shard entries, the float32 values that
+ * dssd_edge_verify would have written there.  p_stride: elements between consecutive rows of
+ * p_row_shard (>= V_shard; the slices of all shards may interleave into whole rows).  Rows of
+ * sequences with accept_len outside [0, gamma] are left untouched.
+ */
+dssd_status dssd_edge_emit_shard(const void *logits_shard, dssd_dtype dtype, int64_t row_stride,
+                                 const int32_t *accept_len, const float *row_scale,
+                                 float temperature, int B, int gamma, int V_shard,
+                                 float *p_row_shard, int64_t p_stride, void *cuda_stream);
+
+/* Bytes of scratch shared by dssd_resample_shard_mass and dssd_resample_shard_draw. */
+size_t dssd_resample_shard_workspace_bytes(int B, int gamma, int V_shard);
+
+/*
+ * One shard's masses for the draw (Section 3, "Resample"): mass[b, 0] = sum over the slice of
+ * max(0, p_v - q_{n,v}) (of p_v when n == gamma: the bonus draw), mass[b, 1] = sum over the slice
+ * of p_v (what the draw falls back to when no shard has residual mass); float64, NaN for a
+ * sequence with n outside [0, gamma].
+ *
+ * p_row_shard   [B, V_shard] float32, p_stride elements between rows
+ * draft_q_shard [B, gamma, V_shard] float32: row (b, i) starts at element (b*gamma+i)*q_stride
+ *               (may be NULL iff gamma == 0); only row n of each sequence is read
+ * mass          [B, 2] float64 out
+ * workspace     >= dssd_resample_shard_workspace_bytes(...) bytes, 256-byte aligned; it keeps the
+ *               per-chunk sums that dssd_resample_shard_draw needs: pass the same, untouched
+ *               buffer to that call
+ */
+dssd_status dssd_resample_shard_mass(const float *p_row_shard, int64_t p_stride,
+                                     const float *draft_q_shard, int64_t q_stride,
+                                     const int32_t *accept_len, int B, int gamma, int V_shard,
+                                     double *mass, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream);
+
+/*
+ * The draw as shard g sees it.  masses [G, B, 2] are the G outputs of dssd_resample_shard_mass,
+ * shard-major.  Z = sum_g masses[g, b, 0] (in shard order); if Z <= 0 for a rejected sequence the
+ * draw falls back to the plain masses (DSSD_RS_FLAG_FALLBACK); t = u' * Z; the owner is the first
+ * shard whose running total exceeds t (the last shard with mass if rounding leaves none).  On the
+ * owner token[b] = v_begin + min{k : c_k > t - (mass before the shard)} over its slice, as in
+ * dssd_device_resample; on every other shard token[b] = -1.  flags[b] are the sequence's
+ * DSSD_RS_FLAG_* and are the same on every shard.  The other arguments as for the mass call,
+ * with the same rows and the workspace that call left.
+ */
+dssd_status dssd_resample_shard_draw(const double *masses, int G, int g, int v_begin,
+                                     const float *p_row_shard, int64_t p_stride,
+                                     const float *draft_q_shard, int64_t q_stride,
+                                     const int32_t *accept_len, const float *uniforms, int B,
+                                     int gamma, int V_shard, int32_t *token, uint32_t *flags,
+                                     const void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream);
 
 #ifdef __cplusplus
 }

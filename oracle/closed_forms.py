@@ -30,3 +30,25 @@ def expected_accept_len(alpha: float, gamma: int) -> float:
 def t_comm_ms(alpha: float, gamma: int, t_ntt_ms: float, payload_ms: float) -> float:
     """Expected DSSD communication time (Section 3.1), payload_ms = |V| b_prob / R_down."""
     return prob_rejection(alpha, gamma) * payload_ms + t_ntt_ms
+
+
+def batch_acceptance_rate(target_logits: np.ndarray, draft_q: np.ndarray, temperature: float, n_seq: int = 32) -> float:
+    """Mean over the first n_seq sequences and their gamma draft positions of alpha = sum_v min(p_v, q_v)
+    (Section 3.1's alpha), p = softmax(l / T) in float64.  Logits are float32, or uint16 holding bfloat16."""
+    tl = target_logits[:n_seq]
+    if tl.dtype == np.uint16:
+        tl = (tl.astype(np.uint32) << 16).view(np.float32)
+    gamma = tl.shape[1] - 1
+    if gamma == 0:
+        return float("nan")
+    T = float(np.float32(temperature))
+    total, count = 0.0, 0
+    for b in range(tl.shape[0]):
+        z = tl[b, :gamma].astype(np.float64) / T
+        z -= z.max(axis=1, keepdims=True)
+        p = np.exp(z)
+        p /= p.sum(axis=1, keepdims=True)
+        for i in range(gamma):
+            total += acceptance_rate(p[i], draft_q[b, i])
+            count += 1
+    return total / count

@@ -168,9 +168,10 @@ def edge_emit_shard(logits_shard: np.ndarray, accept_len: np.ndarray, lse: np.nd
 
 
 def _residual(p_row_shard: np.ndarray, q_shard: Optional[np.ndarray], n: int, gamma: int, b: int) -> np.ndarray:
+    # max(0, p - q) as C's fmax forms it in the dense oracle: a NaN difference counts as no mass
     p = p_row_shard[b].astype(np.float64)
     if n < gamma:
-        return np.maximum(0.0, p - q_shard[b, n].astype(np.float64))
+        return np.fmax(0.0, p - q_shard[b, n].astype(np.float64))
     return p
 
 
@@ -248,7 +249,7 @@ def resample_shard_draw(masses: np.ndarray, g: int, v_begin: int, p_row_shard: n
         if own != g:
             continue
         p = p_row_shard[b].astype(np.float64)
-        r = np.maximum(0.0, p - draft_q_shard[b, n].astype(np.float64)) if use_q else p
+        r = np.fmax(0.0, p - draft_q_shard[b, n].astype(np.float64)) if use_q else p
         c = np.cumsum(r)
         pos = np.nonzero(r > 0.0)[0]
         k = r.size if beyond else int(np.searchsorted(c, t - before, side="right"))

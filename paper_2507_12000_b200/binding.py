@@ -13,8 +13,7 @@ from typing import Dict, Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-# DSSD_LIBRARY overrides the in-tree library (e.g. a build with other tuning constants)
-LIB_PATH = os.environ.get("DSSD_LIBRARY") or os.path.join(_PKG, "libdssd.so")
+LIB_PATH = os.path.join(_PKG, "libdssd.so")
 
 DSSD_OK = 0
 DSSD_ERR_INVALID_ARG = 1
@@ -41,13 +40,13 @@ class DssdError(RuntimeError):
         super().__init__(f"{where}: {name}{extra}")
 
 
-def _load() -> ctypes.CDLL:
-    if not os.path.exists(LIB_PATH):
+def _load(path: str = LIB_PATH) -> ctypes.CDLL:
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2507_12000_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2507_12000_b200.build` "
             "(needs nvcc); this package has no CPU fallback")
     c = ctypes
-    L = c.CDLL(LIB_PATH)
+    L = c.CDLL(path)
     L.dssd_status_string.restype = c.c_char_p
     L.dssd_status_string.argtypes = [c.c_int]
     L.dssd_version.restype = c.c_int
@@ -100,6 +99,30 @@ def _load() -> ctypes.CDLL:
         c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
     L.dssd_device_resample_rejected.restype = c.c_int
     L.dssd_device_resample_rejected.argtypes = L.dssd_device_resample.argtypes
+    for f in (L.dssd_edge_partial_workspace_bytes, L.dssd_resample_shard_workspace_bytes):
+        f.restype = c.c_size_t
+        f.argtypes = [c.c_int, c.c_int, c.c_int]
+    L.dssd_edge_partial.restype = c.c_int
+    L.dssd_edge_partial.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_int, c.c_float, c.c_int, c.c_int, c.c_int,
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_edge_combine.restype = c.c_int
+    L.dssd_edge_combine.argtypes = [
+        c.c_void_p, c.c_void_p, c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+    L.dssd_edge_emit_shard.restype = c.c_int
+    L.dssd_edge_emit_shard.argtypes = [
+        c.c_void_p, c.c_int, c.c_int64, c.c_void_p, c.c_void_p, c.c_float, c.c_int, c.c_int, c.c_int,
+        c.c_void_p, c.c_int64, c.c_void_p]
+    L.dssd_resample_shard_mass.restype = c.c_int
+    L.dssd_resample_shard_mass.argtypes = [
+        c.c_void_p, c.c_int64, c.c_void_p, c.c_int64, c.c_void_p, c.c_int, c.c_int, c.c_int,
+        c.c_void_p, c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_resample_shard_draw.restype = c.c_int
+    L.dssd_resample_shard_draw.argtypes = [
+        c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_int64, c.c_void_p, c.c_int64,
+        c.c_void_p, c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_size_t, c.c_void_p]
     L.dssd_round_host.restype = c.c_int
     L.dssd_round_host.argtypes = [
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
@@ -129,6 +152,16 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"target_logits must be float32 or bfloat16, got {t.dtype}")
 
 
+def _row_stride(target_logits: torch.Tensor) -> int:
+    """Elements between consecutive rows of a [B, gamma+1, V] tensor with unit stride along V."""
+    B, g1, V = target_logits.shape
+    assert target_logits.stride(2) == 1 or V == 1
+    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
+    if B > 1 and target_logits.stride(0) != g1 * row_stride:
+        raise ValueError("rows of target_logits must be equally spaced")
+    return row_stride
+
+
 def _workspace(nbytes: int, device) -> torch.Tensor:
     return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
 
@@ -156,10 +189,7 @@ def dssd_edge_verify(target_logits: torch.Tensor, draft_tokens: torch.Tensor, dr
     assert target_logits.is_cuda and target_logits.dim() == 3
     B, g1, V = target_logits.shape
     gamma = g1 - 1
-    assert target_logits.stride(2) == 1 or V == 1
-    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
-    if B > 1 and target_logits.stride(0) != g1 * row_stride:
-        raise ValueError("rows of target_logits must be equally spaced")
+    row_stride = _row_stride(target_logits)
     dev = target_logits.device
     if out is None:
         out = {
@@ -246,10 +276,7 @@ def dssd_edge_verify_topk(target_logits: torch.Tensor, draft_tokens: torch.Tenso
     assert target_logits.is_cuda and target_logits.dim() == 3
     B, g1, V = target_logits.shape
     gamma = g1 - 1
-    assert target_logits.stride(2) == 1 or V == 1
-    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
-    if B > 1 and target_logits.stride(0) != g1 * row_stride:
-        raise ValueError("rows of target_logits must be equally spaced")
+    row_stride = _row_stride(target_logits)
     dev = target_logits.device
     if out is None:
         kk = max(0, min(k, TOPK_MAX))
@@ -309,10 +336,7 @@ def dssd_dsd_verify(target_logits: torch.Tensor, draft_q: Optional[torch.Tensor]
     assert target_logits.is_cuda and target_logits.dim() == 3
     B, g1, V = target_logits.shape
     gamma = g1 - 1
-    assert target_logits.stride(2) == 1 or V == 1
-    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
-    if B > 1 and target_logits.stride(0) != g1 * row_stride:
-        raise ValueError("rows of target_logits must be equally spaced")
+    row_stride = _row_stride(target_logits)
     if gamma > 0:
         assert draft_q.is_contiguous() and draft_q.dtype == torch.float32 and draft_q.numel() == B * gamma * V
     dev = target_logits.device
@@ -346,10 +370,7 @@ def dssd_edge_verify_bonus(target_logits: torch.Tensor, draft_tokens: torch.Tens
     assert target_logits.is_cuda and target_logits.dim() == 3
     B, g1, V = target_logits.shape
     gamma = g1 - 1
-    assert target_logits.stride(2) == 1 or V == 1
-    row_stride = target_logits.stride(1) if g1 > 1 else max(V, target_logits.stride(0))
-    if B > 1 and target_logits.stride(0) != g1 * row_stride:
-        raise ValueError("rows of target_logits must be equally spaced")
+    row_stride = _row_stride(target_logits)
     dev = target_logits.device
     if out is None:
         out = {
@@ -416,4 +437,146 @@ def dssd_round_host(host: Dict[str, torch.Tensor], temperature: float, arena: to
         arena.data_ptr(), arena.numel(), _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_round_host")
+    return out
+
+
+# ---- the vocabulary-sharded round: five calls per shard, two small exchanges between them ----
+
+
+def dssd_edge_partial_workspace_bytes(B: int, gamma: int, V_shard: int) -> int:
+    return int(lib.dssd_edge_partial_workspace_bytes(B, gamma, V_shard))
+
+
+def dssd_resample_shard_workspace_bytes(B: int, gamma: int, V_shard: int) -> int:
+    return int(lib.dssd_resample_shard_workspace_bytes(B, gamma, V_shard))
+
+
+def dssd_edge_partial(logits_shard: torch.Tensor, draft_tokens: torch.Tensor, v_begin: int, temperature: float, *,
+                      out: Optional[Dict[str, torch.Tensor]] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> Dict[str, torch.Tensor]:
+    """One shard's partial sums.  logits_shard [B, gamma+1, V_shard]: this shard's slice of every row (a
+    view into whole rows works), vocabulary ids v_begin .. v_begin + V_shard - 1.  Returns part_ref
+    [B, gamma+1] float32, part_sum [B, gamma+1] float64, tok_logit [B, gamma] float32."""
+    assert logits_shard.is_cuda and logits_shard.dim() == 3
+    B, g1, Vs = logits_shard.shape
+    gamma = g1 - 1
+    row_stride = _row_stride(logits_shard)
+    dev = logits_shard.device
+    if out is None:
+        out = {"part_ref": torch.empty(B, g1, dtype=torch.float32, device=dev),
+               "part_sum": torch.empty(B, g1, dtype=torch.float64, device=dev),
+               "tok_logit": torch.empty(B, gamma, dtype=torch.float32, device=dev)}
+    if workspace is None:
+        workspace = _workspace(dssd_edge_partial_workspace_bytes(B, gamma, Vs), dev)
+    st = lib.dssd_edge_partial(
+        logits_shard.data_ptr(), _dtype_code(logits_shard), row_stride, _ptr(draft_tokens), v_begin,
+        ctypes.c_float(temperature), B, gamma, Vs, out["part_ref"].data_ptr(), out["part_sum"].data_ptr(),
+        _ptr(out["tok_logit"]), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_partial")
+    return out
+
+
+def dssd_edge_combine(part_ref: torch.Tensor, part_sum: torch.Tensor, tok_logit: torch.Tensor,
+                      draft_tokens: torch.Tensor, draft_q_tok: torch.Tensor, uniforms: torch.Tensor,
+                      temperature: float, V: int, *, out: Optional[Dict[str, torch.Tensor]] = None,
+                      stream=None) -> Dict[str, torch.Tensor]:
+    """part_ref, part_sum [G, B, gamma+1] and tok_logit [G, B, gamma], gathered from the G shards ->
+    accept_len [B], row_scale [B, 2], p_tok, lse, flags.  V is the size of the whole vocabulary."""
+    assert part_ref.is_cuda and part_ref.dim() == 3 and part_ref.is_contiguous() and part_ref.dtype == torch.float32
+    assert part_sum.shape == part_ref.shape and part_sum.is_contiguous() and part_sum.dtype == torch.float64
+    G, B, g1 = part_ref.shape
+    gamma = g1 - 1
+    assert tok_logit.is_contiguous() and tok_logit.dtype == torch.float32 and tok_logit.numel() == G * B * gamma
+    dev = part_ref.device
+    if out is None:
+        out = {"accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+               "row_scale": torch.empty(B, 2, dtype=torch.float32, device=dev),
+               "p_tok": torch.empty(B, gamma, dtype=torch.float32, device=dev),
+               "lse": torch.empty(B, g1, dtype=torch.float32, device=dev),
+               "flags": torch.empty(B, dtype=torch.int32, device=dev)}
+    st = lib.dssd_edge_combine(
+        part_ref.data_ptr(), part_sum.data_ptr(), _ptr(tok_logit), G, _ptr(draft_tokens), _ptr(draft_q_tok),
+        _ptr(uniforms), ctypes.c_float(temperature), B, gamma, V, out["accept_len"].data_ptr(),
+        out["row_scale"].data_ptr(), _ptr(out.get("p_tok")), _ptr(out.get("lse")), _ptr(out.get("flags")),
+        _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_combine")
+    return out
+
+
+def _rows_2d(t: torch.Tensor) -> int:
+    """Elements between consecutive rows of a [B, V] float32 tensor with unit stride along V."""
+    assert t.is_cuda and t.dim() == 2 and t.dtype == torch.float32 and (t.stride(1) == 1 or t.shape[1] == 1)
+    return max(t.shape[1], t.stride(0)) if t.shape[0] > 1 else t.shape[1]
+
+
+def dssd_edge_emit_shard(logits_shard: torch.Tensor, accept_len: torch.Tensor, row_scale: torch.Tensor,
+                         temperature: float, *, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """This shard's slice of the downlink row: [B, V_shard] float32 (`out` may be a view into whole rows)."""
+    assert logits_shard.is_cuda and logits_shard.dim() == 3
+    B, g1, Vs = logits_shard.shape
+    if out is None:
+        out = torch.empty(B, Vs, dtype=torch.float32, device=logits_shard.device)
+    assert out.shape == (B, Vs)
+    st = lib.dssd_edge_emit_shard(
+        logits_shard.data_ptr(), _dtype_code(logits_shard), _row_stride(logits_shard), accept_len.data_ptr(),
+        row_scale.data_ptr(), ctypes.c_float(temperature), B, g1 - 1, Vs, out.data_ptr(), _rows_2d(out),
+        _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_edge_emit_shard")
+    return out
+
+
+def _q_stride(draft_q_shard: Optional[torch.Tensor], B: int, gamma: int, Vs: int) -> int:
+    if gamma == 0 or draft_q_shard is None:
+        return Vs
+    q = draft_q_shard
+    assert q.is_cuda and q.dtype == torch.float32 and q.shape == (B, gamma, Vs) and (q.stride(2) == 1 or Vs == 1)
+    stride = q.stride(1) if gamma > 1 else max(Vs, q.stride(0))
+    if B > 1 and q.stride(0) != gamma * stride:
+        raise ValueError("rows of draft_q_shard must be equally spaced")
+    return stride
+
+
+def dssd_resample_shard_mass(p_row_shard: torch.Tensor, draft_q_shard: Optional[torch.Tensor],
+                             accept_len: torch.Tensor, gamma: int, *, out: Optional[torch.Tensor] = None,
+                             workspace: Optional[torch.Tensor] = None, stream=None):
+    """This shard's residual mass and plain mass per sequence: ([B, 2] float64, the workspace that
+    dssd_resample_shard_draw needs next)."""
+    B, Vs = p_row_shard.shape
+    dev = p_row_shard.device
+    if out is None:
+        out = torch.empty(B, 2, dtype=torch.float64, device=dev)
+    if workspace is None:
+        workspace = _workspace(dssd_resample_shard_workspace_bytes(B, gamma, Vs), dev)
+    st = lib.dssd_resample_shard_mass(
+        p_row_shard.data_ptr(), _rows_2d(p_row_shard), _ptr(draft_q_shard) if gamma > 0 else None,
+        _q_stride(draft_q_shard, B, gamma, Vs), accept_len.data_ptr(), B, gamma, Vs, out.data_ptr(),
+        workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_resample_shard_mass")
+    return out, workspace
+
+
+def dssd_resample_shard_draw(masses: torch.Tensor, g: int, v_begin: int, p_row_shard: torch.Tensor,
+                             draft_q_shard: Optional[torch.Tensor], accept_len: torch.Tensor,
+                             uniforms_rs: torch.Tensor, gamma: int, workspace: torch.Tensor, *,
+                             out: Optional[Dict[str, torch.Tensor]] = None, stream=None) -> Dict[str, torch.Tensor]:
+    """The draw as shard g sees it; masses [G, B, 2] float64 gathered from all shards.  token is the id
+    in the whole vocabulary on the owning shard and -1 on the others; flags are the sequence's."""
+    assert masses.is_cuda and masses.dim() == 3 and masses.is_contiguous() and masses.dtype == torch.float64
+    G = masses.shape[0]
+    B, Vs = p_row_shard.shape
+    dev = p_row_shard.device
+    if out is None:
+        out = {"token": torch.empty(B, dtype=torch.int32, device=dev),
+               "flags": torch.empty(B, dtype=torch.int32, device=dev)}
+    st = lib.dssd_resample_shard_draw(
+        masses.data_ptr(), G, g, v_begin, p_row_shard.data_ptr(), _rows_2d(p_row_shard),
+        _ptr(draft_q_shard) if gamma > 0 else None, _q_stride(draft_q_shard, B, gamma, Vs), accept_len.data_ptr(),
+        uniforms_rs.data_ptr(), B, gamma, Vs, out["token"].data_ptr(), _ptr(out.get("flags")),
+        workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_resample_shard_draw")
     return out

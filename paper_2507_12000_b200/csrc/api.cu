@@ -5,6 +5,7 @@
 #include "device_resample.h"
 #include "dssd.h"
 #include "edge_verify.h"
+#include "shard_verify.h"
 #include "topk_verify.h"
 
 namespace {
@@ -401,6 +402,202 @@ dssd_status dssd_device_resample_topk(const int32_t *p_idx, const float *p_val,
     P.token = token;
     P.flags = flags;
     cudaError_t e = dssd::topk_resample_launch(P, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+// ---- the vocabulary-sharded round ---------------------------------------------------------------
+
+size_t dssd_edge_partial_workspace_bytes(int B, int gamma, int V_shard)
+{
+    return dssd_edge_verify_workspace_bytes(B, gamma, V_shard);
+}
+
+dssd_status dssd_edge_partial(const void *logits_shard, dssd_dtype dtype, int64_t row_stride,
+                              const int32_t *draft_tokens, int v_begin, float temperature, int B,
+                              int gamma, int V_shard, float *part_ref, double *part_sum,
+                              float *tok_logit, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V_shard);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!logits_shard || !part_ref || !part_sum || v_begin < 0) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !tok_logit)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V_shard) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(logits_shard) % esz) || (reinterpret_cast<uintptr_t>(part_sum) % 8) ||
+        (reinterpret_cast<uintptr_t>(part_ref) % 4) || (reinterpret_cast<uintptr_t>(tok_logit) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_edge_partial_workspace_bytes(B, gamma, V_shard))
+        return DSSD_ERR_WORKSPACE;
+    dssd::EdgeParams P{};
+    P.logits = logits_shard;
+    P.row_stride = row_stride;
+    P.draft_tokens = draft_tokens;
+    P.temperature = temperature;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V_shard;
+    P.v_begin = v_begin;
+    P.shard_ref = part_ref;
+    P.shard_sum = part_sum;
+    P.shard_tok_logit = tok_logit;
+    cudaError_t e = dssd::edge_verify_launch(P, (int)dtype, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+dssd_status dssd_edge_combine(const float *part_ref, const double *part_sum, const float *tok_logit,
+                              int G, const int32_t *draft_tokens, const float *draft_q_tok,
+                              const float *uniforms, float temperature, int B, int gamma, int V,
+                              int32_t *accept_len, float *row_scale, float *p_tok, float *lse,
+                              uint32_t *flags, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (G < 1) return DSSD_ERR_INVALID_ARG;
+    if (G > dssd::kShardMax) return DSSD_ERR_UNSUPPORTED;
+    if (!part_ref || !part_sum || !accept_len || !row_scale) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!tok_logit || !draft_tokens || !draft_q_tok || !uniforms)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(part_sum) % 8) return DSSD_ERR_INVALID_ARG;
+    dssd::CombineParams P{};
+    P.part_ref = part_ref;
+    P.part_sum = part_sum;
+    P.tok_logit = tok_logit;
+    P.G = G;
+    P.draft_tokens = draft_tokens;
+    P.draft_q_tok = draft_q_tok;
+    P.uniforms = uniforms;
+    P.c1 = (float)(1.4426950408889634 / (double)temperature);
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V;
+    P.accept_len = accept_len;
+    P.row_scale = row_scale;
+    P.p_tok = p_tok;
+    P.lse = lse;
+    P.flags = flags;
+    cudaError_t e = dssd::shard_combine_launch(P, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+dssd_status dssd_edge_emit_shard(const void *logits_shard, dssd_dtype dtype, int64_t row_stride,
+                                 const int32_t *accept_len, const float *row_scale,
+                                 float temperature, int B, int gamma, int V_shard,
+                                 float *p_row_shard, int64_t p_stride, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V_shard);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (!logits_shard || !accept_len || !row_scale || !p_row_shard) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (row_stride < (int64_t)V_shard || p_stride < (int64_t)V_shard) return DSSD_ERR_INVALID_ARG;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(logits_shard) % esz) || (reinterpret_cast<uintptr_t>(p_row_shard) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    dssd::EmitShardParams P{};
+    P.logits = logits_shard;
+    P.row_stride = row_stride;
+    P.accept_len = accept_len;
+    P.row_scale = row_scale;
+    P.c1 = (float)(1.4426950408889634 / (double)temperature);
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V_shard;
+    P.p_row = p_row_shard;
+    P.p_stride = p_stride;
+    cudaError_t e = dssd::shard_emit_launch(P, (int)dtype, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+size_t dssd_resample_shard_workspace_bytes(int B, int gamma, int V_shard)
+{
+    if (check_sizes(B, gamma, V_shard) != DSSD_OK) return 0;
+    return dssd::shard_resample_workspace_bytes(B, V_shard);
+}
+
+namespace {
+dssd_status check_shard_rows(const float *p_row_shard, int64_t p_stride, const float *draft_q_shard, int64_t q_stride,
+                             const int32_t *accept_len, int B, int gamma, int V_shard, const void *workspace,
+                             size_t workspace_bytes)
+{
+    dssd_status st = check_sizes(B, gamma, V_shard);
+    if (st != DSSD_OK) return st;
+    if (!p_row_shard || !accept_len) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && !draft_q_shard) return DSSD_ERR_INVALID_ARG;
+    if (p_stride < (int64_t)V_shard || (gamma > 0 && q_stride < (int64_t)V_shard)) return DSSD_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(p_row_shard) % 4) || (reinterpret_cast<uintptr_t>(draft_q_shard) % 4))
+        return DSSD_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        workspace_bytes < dssd_resample_shard_workspace_bytes(B, gamma, V_shard))
+        return DSSD_ERR_WORKSPACE;
+    return DSSD_OK;
+}
+}  // namespace
+
+dssd_status dssd_resample_shard_mass(const float *p_row_shard, int64_t p_stride,
+                                     const float *draft_q_shard, int64_t q_stride,
+                                     const int32_t *accept_len, int B, int gamma, int V_shard,
+                                     double *mass, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_shard_rows(p_row_shard, p_stride, draft_q_shard, q_stride, accept_len, B, gamma, V_shard,
+                                      workspace, workspace_bytes);
+    if (st != DSSD_OK) return st;
+    if (!mass || (reinterpret_cast<uintptr_t>(mass) % 8)) return DSSD_ERR_INVALID_ARG;
+    dssd::ShardResampleParams P{};
+    P.p_row = p_row_shard;
+    P.p_stride = p_stride;
+    P.draft_q = draft_q_shard;
+    P.q_stride = q_stride;
+    P.accept_len = accept_len;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V_shard;
+    P.mass = mass;
+    cudaError_t e = dssd::shard_mass_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
+}
+
+dssd_status dssd_resample_shard_draw(const double *masses, int G, int g, int v_begin,
+                                     const float *p_row_shard, int64_t p_stride,
+                                     const float *draft_q_shard, int64_t q_stride,
+                                     const int32_t *accept_len, const float *uniforms, int B,
+                                     int gamma, int V_shard, int32_t *token, uint32_t *flags,
+                                     const void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_shard_rows(p_row_shard, p_stride, draft_q_shard, q_stride, accept_len, B, gamma, V_shard,
+                                      workspace, workspace_bytes);
+    if (st != DSSD_OK) return st;
+    if (!masses || (reinterpret_cast<uintptr_t>(masses) % 8) || !uniforms || !token) return DSSD_ERR_INVALID_ARG;
+    if (G < 1 || g < 0 || g >= G || v_begin < 0) return DSSD_ERR_INVALID_ARG;
+    if (G > dssd::kShardMax) return DSSD_ERR_UNSUPPORTED;
+    if ((long long)v_begin + (long long)V_shard > (long long)DSSD_MAX_V) return DSSD_ERR_UNSUPPORTED;
+    dssd::ShardResampleParams P{};
+    P.p_row = p_row_shard;
+    P.p_stride = p_stride;
+    P.draft_q = draft_q_shard;
+    P.q_stride = q_stride;
+    P.accept_len = accept_len;
+    P.B = B;
+    P.gamma = gamma;
+    P.V = V_shard;
+    P.masses = masses;
+    P.G = G;
+    P.g = g;
+    P.v_begin = v_begin;
+    P.uniforms = uniforms;
+    P.token = token;
+    P.flags = flags;
+    cudaError_t e = dssd::shard_draw_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
 }
 

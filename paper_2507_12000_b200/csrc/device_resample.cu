@@ -329,6 +329,88 @@ __device__ __forceinline__ double block_scan(double x, double *s_scan, double &t
     return before + incl;
 }
 
+// The draw inside the chunk that `pk` names: every thread fetches its run of the chunk, a prefix over
+// the CTA finds the thread whose run holds the target, and that thread walks its run.  The token
+// (its index in the row plus tok_base, or -1 when the chunk has no positive entry) and the flags
+// go to *token_out / *flags_out.  q == nullptr means r = p.
+template <typename RV>
+__device__ __forceinline__ void walk_chunk(const Pick &pk, int V, const RV &row, const float *q, unsigned fl, int tok_base,
+                                           int32_t *token_out, uint32_t *flags_out, double *s_w, int *s_i)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int e0 = pk.chunk * kSub, e1 = min(V, e0 + kSub);
+    const int r0 = min(e1, e0 + tid * kRun), r1 = min(e1, r0 + kRun);
+    double mine = 0.0;
+    int last_pos = -1;
+    // The run's 16 entries are all requested before the first is used (one round trip for the
+    // run, not one per entry); entries past the row's end read as 0.
+    const bool vec = (r1 - r0 == kRun) && row.aligned(r0) && (!q || (reinterpret_cast<uintptr_t>(q + r0) & 15u) == 0);
+#pragma unroll
+    for (int g = 0; g < kRun; g += 16) {
+        float pv[16], qv[16];
+        if (vec) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float4 a = row.ld_quad(r0 + g, j);
+                pv[4 * j] = a.x, pv[4 * j + 1] = a.y, pv[4 * j + 2] = a.z, pv[4 * j + 3] = a.w;
+                float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (q) c = __ldg(reinterpret_cast<const float4 *>(q + r0 + g) + j);
+                qv[4 * j] = c.x, qv[4 * j + 1] = c.y, qv[4 * j + 2] = c.z, qv[4 * j + 3] = c.w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int e = r0 + g + j;
+                pv[j] = e < r1 ? row.ld(e) : 0.f;
+                qv[j] = (q && e < r1) ? __ldg(q + e) : 0.f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const double r = q ? res(pv[j], qv[j]) : (double)pv[j];
+            mine += r;
+            if (r > 0.0) last_pos = r0 + g + j;
+        }
+    }
+    // exclusive prefix of the per-thread run sums across the CTA
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) s_w[warp] = incl;
+    __syncthreads();
+    double before = pk.base;
+    for (int w = 0; w < warp; ++w) before += s_w[w];
+    before += incl - mine;
+    const bool crosses = !pk.beyond && (before + mine > pk.target);
+    const unsigned bal = __ballot_sync(0xffffffffu, crosses);
+    if (tid == 0) { s_i[0] = 0x7fffffff; s_i[1] = -1; }
+    __syncthreads();
+    if (lane == 0 && bal) atomicMin(&s_i[0], warp * 32 + __ffs(bal) - 1);
+    if (last_pos >= 0) atomicMax(&s_i[1], last_pos);
+    __syncthreads();
+    const int first = s_i[0];
+    if (first == 0x7fffffff) {
+        if (tid == 0) {
+            *token_out = s_i[1] < 0 ? -1 : tok_base + s_i[1];
+            if (flags_out) *flags_out = fl | (s_i[1] < 0 ? DSSD_RS_FLAG_INVALID : 0u);
+        }
+    } else if (tid == first) {
+        double C = before;
+        int tok = last_pos;
+        for (int e = r0; e < r1; ++e) {
+            C += q ? res(row.ld(e), __ldg(q + e)) : (double)row.ld(e);
+            if (C > pk.target) { tok = e; break; }
+        }
+        tok = tok >= 0 ? tok : s_i[1];
+        *token_out = tok < 0 ? -1 : tok_base + tok;
+        if (flags_out) *flags_out = fl;
+    }
+}
+
 // pass B for sequence b; q == nullptr means r = p
 template <typename RV>
 __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const float *q, unsigned fl, float u,
@@ -448,76 +530,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
         __syncthreads();
     }
     const Pick pk = *s_pick;
-    const int e0 = pk.chunk * kSub, e1 = min(P.V, e0 + kSub);
-    const int r0 = min(e1, e0 + tid * kRun), r1 = min(e1, r0 + kRun);
-    double mine = 0.0;
-    int last_pos = -1;
-    // The run's 16 entries are all requested before the first is used (one round trip for the
-    // run, not one per entry); entries past the row's end read as 0.
-    const bool vec = (r1 - r0 == kRun) && row.aligned(r0) && (!q || (reinterpret_cast<uintptr_t>(q + r0) & 15u) == 0);
-#pragma unroll
-    for (int g = 0; g < kRun; g += 16) {
-        float pv[16], qv[16];
-        if (vec) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float4 a = row.ld_quad(r0 + g, j);
-                pv[4 * j] = a.x, pv[4 * j + 1] = a.y, pv[4 * j + 2] = a.z, pv[4 * j + 3] = a.w;
-                float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (q) c = __ldg(reinterpret_cast<const float4 *>(q + r0 + g) + j);
-                qv[4 * j] = c.x, qv[4 * j + 1] = c.y, qv[4 * j + 2] = c.z, qv[4 * j + 3] = c.w;
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int e = r0 + g + j;
-                pv[j] = e < r1 ? row.ld(e) : 0.f;
-                qv[j] = (q && e < r1) ? __ldg(q + e) : 0.f;
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const double r = q ? res(pv[j], qv[j]) : (double)pv[j];
-            mine += r;
-            if (r > 0.0) last_pos = r0 + g + j;
-        }
-    }
-    // exclusive prefix of the per-thread run sums across the CTA
-    double incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    __syncthreads();
-    if (lane == 31) s_w[warp] = incl;
-    __syncthreads();
-    double before = pk.base;
-    for (int w = 0; w < warp; ++w) before += s_w[w];
-    before += incl - mine;
-    const bool crosses = !pk.beyond && (before + mine > pk.target);
-    const unsigned bal = __ballot_sync(0xffffffffu, crosses);
-    if (tid == 0) { s_i[0] = 0x7fffffff; s_i[1] = -1; }
-    __syncthreads();
-    if (lane == 0 && bal) atomicMin(&s_i[0], warp * 32 + __ffs(bal) - 1);
-    if (last_pos >= 0) atomicMax(&s_i[1], last_pos);
-    __syncthreads();
-    const int first = s_i[0];
-    if (first == 0x7fffffff) {
-        if (tid == 0) {
-            P.token[b] = s_i[1];
-            if (P.flags) P.flags[b] = fl | (s_i[1] < 0 ? DSSD_RS_FLAG_INVALID : 0u);
-        }
-    } else if (tid == first) {
-        double C = before;
-        int tok = last_pos;
-        for (int e = r0; e < r1; ++e) {
-            C += q ? res(row.ld(e), __ldg(q + e)) : (double)row.ld(e);
-            if (C > pk.target) { tok = e; break; }
-        }
-        P.token[b] = tok >= 0 ? tok : s_i[1];
-        if (P.flags) P.flags[b] = fl;
-    }
+    walk_chunk<RV>(pk, P.V, row, q, fl, 0, P.token + b, P.flags ? P.flags + b : nullptr, s_w, s_i);
 }
 
 template <typename RV>
@@ -639,6 +652,234 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
     }
 }
 
+// ---- one shard of the vocabulary ---------------------------------------------------------------
+//
+// The draw over a row that is spread over G shards takes two steps with one small exchange
+// between them.  shard_mass_kernel streams this shard's slice of p_row and of Q_n once and leaves,
+// per chunk of kSub entries, the residual mass sum max(0, p - q) (sum p for a bonus draw) and the
+// plain mass sum p (needed if the residual turns out to have no mass anywhere);
+// shard_total_kernel adds a sequence's chunks up.  After the masses of all shards have been
+// gathered, shard_draw_kernel - one CTA per sequence - takes the same decisions on every shard
+// (Z, fall-back, the shard that holds u' Z) and the owning shard walks its slice exactly as the
+// dense kernel walks a row.  Plain stores and stream order connect the launches: no slot is read
+// before the launch that wrote it has ended, so the scratch needs no fill.
+
+template <typename RV>
+__device__ __forceinline__ void chunk_mass2(const RV &row, const float *q, int e0, int e1, double &acc_r, double &acc_p)
+{
+    const int tid = threadIdx.x;
+    int done = e0;
+    const bool aligned = row.aligned(e0) && (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0);
+    if (aligned) {
+        const int nvec = (e1 - e0) / 4;
+        const uint4 *q4 = reinterpret_cast<const uint4 *>(q + e0);
+        for (int i = tid; i < nvec; i += 4 * kThreads) {
+            typename RV::Raw a[4];
+            uint4 c[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool in = i + u * kThreads < nvec;
+                a[u] = in ? row.ld_quad_stream(e0, i + u * kThreads) : typename RV::Raw();
+                c[u] = (in && q) ? ld_stream16(q4 + i + u * kThreads) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i + u * kThreads >= nvec) continue;
+                const float4 x = row.quad(a[u]), y = as_f4(c[u]);
+                acc_p += ((double)x.x + (double)x.y) + ((double)x.z + (double)x.w);
+                if (q) acc_r += (res(x.x, y.x) + res(x.y, y.y)) + (res(x.z, y.z) + res(x.w, y.w));
+            }
+        }
+        done = e0 + nvec * 4;
+    }
+    for (int e = done + tid; e < e1; e += kThreads) {
+        const float pv = row.ld(e);
+        acc_p += (double)pv;
+        if (q) acc_r += res(pv, __ldg(q + e));
+    }
+    if (!q) acc_r = acc_p;
+}
+
+__device__ __forceinline__ RowF32 shard_row(const ShardResampleParams &P, int64_t b)
+{
+    RowF32 r;
+    r.p = P.p_row + (size_t)b * (size_t)P.p_stride;
+    return r;
+}
+
+__global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) shard_mass_kernel(const __grid_constant__ ShardResampleParams P)
+{
+    __shared__ double s_w[kWarps][2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long total = (long long)P.B * P.n_sub;
+    for (long long t = blockIdx.x; t < total; t += gridDim.x) {
+        const int64_t b = t / P.n_sub;
+        const int c = (int)(t - b * P.n_sub);
+        const int n = __ldg(P.accept_len + b);
+        double acc_r = 0.0, acc_p = 0.0;
+        const bool valid = n >= 0 && n <= P.gamma;
+        if (valid) {
+            const RowF32 row = shard_row(P, b);
+            const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.q_stride : nullptr;
+            const int e0 = c * kSub, e1 = min(P.V, e0 + kSub);
+            chunk_mass2(row, q, e0, e1, acc_r, acc_p);
+        }
+        acc_r = warp_sum(acc_r);
+        acc_p = warp_sum(acc_p);
+        __syncthreads();  // the previous ticket's sums have been read
+        if (lane == 0) {
+            s_w[warp][0] = acc_r;
+            s_w[warp][1] = acc_p;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double tr = 0.0, tp = 0.0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                tr += s_w[w][0];
+                tp += s_w[w][1];
+            }
+            const double nan = __longlong_as_double(0x7ff8000000000000ll);
+            double *cs = P.chunk_sum + ((size_t)b * P.n_sub + c) * 2;
+            cs[0] = valid ? tr : nan;
+            cs[1] = valid ? tp : nan;
+        }
+    }
+}
+
+// one warp per sequence: the chunk sums in a fixed order
+__global__ void __launch_bounds__(kThreads) shard_total_kernel(const __grid_constant__ ShardResampleParams P)
+{
+    const int lane = threadIdx.x & 31;
+    const long long b = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (b >= P.B) return;
+    const double *cs = P.chunk_sum + (size_t)b * P.n_sub * 2;
+    double r = 0.0, p = 0.0;
+    for (int c = lane; c < P.n_sub; c += 32) {
+        r += cs[2 * c];
+        p += cs[2 * c + 1];
+    }
+    r = warp_sum(r);
+    p = warp_sum(p);
+    if (lane == 0) {
+        P.mass[2 * b] = r;
+        P.mass[2 * b + 1] = p;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) shard_draw_kernel(const __grid_constant__ ShardResampleParams P)
+{
+    __shared__ double s_scan[kWarps];
+    __shared__ Pick s_pick;
+    __shared__ int s_i[2];
+    const int tid = threadIdx.x;
+    const int64_t b = blockIdx.x;
+    const int n = __ldg(P.accept_len + b);
+    int32_t *token_out = P.token + b;
+    uint32_t *flags_out = P.flags ? P.flags + b : nullptr;
+    if (n < 0 || n > P.gamma) {
+        if (tid == 0) {
+            *token_out = -1;
+            if (flags_out) *flags_out = DSSD_RS_FLAG_INVALID;
+        }
+        return;
+    }
+    // The verdict on the sequence, from all shards' masses: every thread of every shard takes the
+    // same steps in the same order.
+    unsigned fl = n == P.gamma ? DSSD_RS_FLAG_BONUS : 0u;
+    int col = 0;
+    double Z = 0.0;
+    for (int h = 0; h < P.G; ++h) Z += __ldg(P.masses + ((size_t)h * P.B + b) * 2);
+    bool ok = (Z > 0.0) && (Z < INFINITY);
+    if (!ok && n < P.gamma) {  // no residual mass anywhere: draw from p instead
+        fl |= DSSD_RS_FLAG_FALLBACK;
+        col = 1;
+        Z = 0.0;
+        for (int h = 0; h < P.G; ++h) Z += __ldg(P.masses + ((size_t)h * P.B + b) * 2 + 1);
+        ok = (Z > 0.0) && (Z < INFINITY);
+    }
+    if (!ok) {
+        if (tid == 0) {
+            *token_out = -1;
+            if (flags_out) *flags_out = fl | DSSD_RS_FLAG_INVALID;
+        }
+        return;
+    }
+    const double t = (double)__ldg(P.uniforms + b) * Z;
+    double C = 0.0, before = 0.0;
+    int owner = -1, last_mass = -1;
+    for (int h = 0; h < P.G; ++h) {
+        const double m = __ldg(P.masses + ((size_t)h * P.B + b) * 2 + col);
+        if (m > 0.0) last_mass = h;
+        if (owner < 0 && C + m > t) {
+            owner = h;
+            before = C;
+        }
+        C += m;
+    }
+    const bool beyond = owner < 0;  // rounding left no shard above t: the last shard with mass, its last positive entry
+    if (beyond) owner = last_mass;
+    if (owner != P.g) {
+        if (tid == 0) {
+            *token_out = -1;
+            if (flags_out) *flags_out = fl;
+        }
+        return;
+    }
+    // this shard holds the target: the chunk first, then the walk inside it
+    const double target = t - before;
+    const double *cs = P.chunk_sum + (size_t)b * P.n_sub * 2 + col;
+    if (tid == 0) {
+        s_i[0] = 0x7fffffff;
+        s_i[1] = -1;
+    }
+    __syncthreads();
+    double carry = 0.0, my_base_first = 0.0, my_base_last = 0.0;
+    int my_first = 0x7fffffff, my_last = -1;
+    for (int base = 0; base < P.n_sub; base += kThreads) {
+        const int c = base + tid;
+        const double m = c < P.n_sub ? cs[2 * c] : 0.0;
+        double tot;
+        const double incl = carry + block_scan(m, s_scan, tot);
+        if (!beyond && c < P.n_sub && incl > target && my_first == 0x7fffffff) {
+            my_first = c;
+            my_base_first = incl - m;
+        }
+        if (c < P.n_sub && m > 0.0) {
+            my_last = c;
+            my_base_last = incl - m;
+        }
+        carry += tot;
+        __syncthreads();
+    }
+    if (my_first != 0x7fffffff) atomicMin(&s_i[0], my_first);
+    if (my_last >= 0) atomicMax(&s_i[1], my_last);
+    __syncthreads();
+    const int first = s_i[0], last = s_i[1];
+    if (first == 0x7fffffff && last < 0) {  // cannot happen while this shard's mass is positive
+        if (tid == 0) {
+            *token_out = -1;
+            if (flags_out) *flags_out = fl | DSSD_RS_FLAG_INVALID;
+        }
+        return;
+    }
+    if (first != 0x7fffffff ? (my_first == first) : (my_last == last)) {
+        Pick pk;
+        pk.ok = 1;
+        pk.beyond = first == 0x7fffffff;
+        pk.chunk = pk.beyond ? last : first;
+        pk.base = pk.beyond ? my_base_last : my_base_first;
+        pk.target = target;
+        s_pick = pk;
+    }
+    __syncthreads();
+    const Pick pk = s_pick;
+    const RowF32 row = shard_row(P, b);
+    const float *q = (col == 0 && n < P.gamma) ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.q_stride : nullptr;
+    walk_chunk<RowF32>(pk, P.V, row, q, fl, P.v_begin, token_out, flags_out, s_scan, s_i);
+}
+
+
 }  // namespace
 
 size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
@@ -712,6 +953,36 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     } else {
         resample_kernel<RowF32><<<grid, kThreads, 0, stream>>>(P);
     }
+    return cudaGetLastError();
+}
+
+size_t shard_resample_workspace_bytes(int B, int V)
+{
+    const size_t n_sub = (size_t)((V + kResampleSub - 1) / kResampleSub);
+    return (((size_t)B * n_sub * 2 * sizeof(double)) + 255) & ~(size_t)255;
+}
+
+cudaError_t shard_mass_launch(ShardResampleParams &P, void *workspace, cudaStream_t stream)
+{
+    cudaError_t err;
+    int dev = 0, sms = 0;
+    if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
+    if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
+    P.n_sub = (P.V + kResampleSub - 1) / kResampleSub;
+    P.chunk_sum = static_cast<double *>(workspace);
+    const long long total = (long long)P.B * P.n_sub;
+    const long long resident = (long long)(sms < 1 ? 1 : sms) * DSSD_RS_CTAS;
+    shard_mass_kernel<<<(unsigned)(total < resident ? total : resident), kThreads, 0, stream>>>(P);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    shard_total_kernel<<<(unsigned)((P.B + kWarps - 1) / kWarps), kThreads, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+cudaError_t shard_draw_launch(ShardResampleParams &P, const void *workspace, cudaStream_t stream)
+{
+    P.n_sub = (P.V + kResampleSub - 1) / kResampleSub;
+    P.chunk_sum = const_cast<double *>(static_cast<const double *>(workspace));
+    shard_draw_kernel<<<(unsigned)P.B, kThreads, 0, stream>>>(P);
     return cudaGetLastError();
 }
 

@@ -46,6 +46,30 @@ size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base);
 
 cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t stream);
 
+// ---- one shard of the vocabulary (entries v_begin .. v_begin + V - 1 of every row) ----
+struct ShardResampleParams {
+    const float *p_row;     // [B, V] this shard's slice of row P_n, p_stride elements between rows
+    int64_t p_stride;
+    const float *draft_q;   // [B, gamma, V] this shard's slice of the device's rows, q_stride elements between rows
+    int64_t q_stride;
+    const int32_t *accept_len;
+    int B, gamma, V;
+    int n_sub;              // chunk sums per sequence
+    double *chunk_sum;      // scratch [B, n_sub, 2]: residual mass and plain mass of every chunk
+    // mass
+    double *mass;           // [B, 2] out: the slice's residual mass and plain mass
+    // draw
+    const double *masses;   // [G, B, 2] gathered from all shards
+    int G, g, v_begin;
+    const float *uniforms;
+    int32_t *token;
+    uint32_t *flags;
+};
+
+size_t shard_resample_workspace_bytes(int B, int V);
+cudaError_t shard_mass_launch(ShardResampleParams &P, void *workspace, cudaStream_t stream);
+cudaError_t shard_draw_launch(ShardResampleParams &P, const void *workspace, cudaStream_t stream);
+
 void set_last_cuda_error(int e);  // defined with the C ABI
 
 }  // namespace dssd

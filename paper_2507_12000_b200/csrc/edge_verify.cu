@@ -23,9 +23,11 @@
 // sequences have unclaimed tickets (or eagerly once they have no LSE work left); an EMIT ticket
 // goes before the next LSE stage, so the second read of row n follows the first as closely as
 // the fold allows.
-// Nothing on the global path waits on a fence: results travel through 8-byte slots that the
-// host pre-filled with all ones and that carry their own validity; a reader that sees the fill
-// pattern asks again (bounded) for a store that a running warp has already issued.  Values that
+// Nothing on the global path waits on a fence: results travel through 8-byte slots that carry
+// their own validity (the kernel itself sets the whole workspace to all ones before any CTA uses
+// it: one grid-wide barrier at the start of a cooperative launch, overlapped with the first
+// copies); a reader that sees the fill pattern asks again (bounded) for a store that a running
+// warp has already issued.  Values that
 // a thread will need later (ticket numbers, counters, `ready` entries) are requested one step
 // ahead and looked at one step later, so no round trip is waited for while streaming.
 // A producer only ever waits for work held by running CTAs, and never while its own CTA holds
@@ -36,10 +38,12 @@
 #include <math.h>
 
 #include <atomic>
+#include <utility>
 
 #include <cooperative_groups.h>
 
 #include "dssd_device.cuh"
+#include "edge_judge.cuh"
 
 namespace dssd {
 
@@ -55,12 +59,11 @@ constexpr int kComb = 16;  // ticket records; tickets in flight in a CTA <= kEdg
 static_assert(kComb >= kEdgeStages + 2 && kComb <= 16 && (kComb & (kComb - 1)) == 0, "ticket records");
 constexpr int kMeet = 4;   // meeting areas where the consumers leave an LSE ticket's per-lane results for the fold warp
 constexpr int kMail = 32;  // mailbox entries of the fold warp, a power of two
-constexpr unsigned kBitAccept = 1u, kBitBadToken = 2u, kBitNonFinite = 4u, kBitTimeout = 8u;
 
 enum Kind : unsigned { kEnd = 0, kIdle = 1, kLse = 2, kEmit = 3 };
 constexpr unsigned kMetaFirst = 4u, kMetaLast = 8u, kMetaRagged = 16u;  // first / last stage of its ticket; scalars outside the copy
 
-// counters start at all ones (the workspace fill pattern): logical value = raw + 1
+// counters start at all ones (the pattern the workspace is cleared to): logical value = raw + 1
 __device__ __forceinline__ unsigned logical(unsigned raw) { return raw + 1u; }
 __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { return raw + 1ull; }
 
@@ -101,6 +104,15 @@ struct __align__(16) Mail {
 };
 static_assert(sizeof(Mail) == 32, "Mail layout");
 
+// An EMIT ticket on its way from the scout to the producer.
+struct __align__(16) EmitWork {
+    Ticket t;
+    int k_begin, k_end;
+    int pad[2];
+};
+constexpr int kEmitQ = 2;  // powers of two
+constexpr int kLseQ = 2;
+
 struct Shared {  // carved from dynamic shared memory behind the ring
     Ticket ticket[kComb];
     StageDesc desc[kEdgeStages];
@@ -112,6 +124,14 @@ struct Shared {  // carved from dynamic shared memory behind the ring
     Mail mail[kMail];
     unsigned mail_tail;
     unsigned cons_done;
+    // the scout's hand-offs to the producer (single writer, single reader each)
+    EmitWork emit_q[kEmitQ];           // claimed EMIT tickets whose sequence is ready
+    unsigned emit_pushed, emit_popped;
+    unsigned long long lse_q[kLseQ];   // drawn LSE ticket numbers (one beyond the last ticket: no more)
+    unsigned lse_pushed, lse_popped;
+    unsigned lse_busy;                 // producer: it still has LSE stages to issue or LSE tickets to expect
+    unsigned scout_done;               // scout: nothing further will be pushed
+    unsigned abort;                    // producer: a wait ran out; everybody winds down
 };
 
 template <int DT>
@@ -378,76 +398,6 @@ __device__ __forceinline__ void emit_consume16(uint32_t stage, int nbytes, uint1
 
 // ---- the fold warp -------------------------------------------------------------------------
 
-// v * 2^d for an integer d <= 0 and a normal, positive v of float32 range: exponent arithmetic,
-// exact; anything below 2^-900 of v counts as nothing
-__device__ __forceinline__ double scale_pow2(double v, float d)
-{
-    if (!(d > -900.f)) return 0.0;
-    return __hiloint2double(__double2hiint(v) + ((int)d << 20), __double2loint(v));
-}
-
-// 2^x in float64 for x <= about 1 (relative error below 1e-11): x = n + f, |f| <= 1/2, and the
-// degree-9 Taylor polynomial of e^(f ln 2); 0 below 2^-1000, NaN for NaN
-__device__ __forceinline__ double exp2_small(double x)
-{
-    if (x != x) return x;
-    if (!(x > -1000.0)) return 0.0;
-    const int n = __double2int_rn(x);
-    const double y = (x - (double)n) * 0.6931471805599453;
-    double p = 2.7557319223985893e-6;
-    p = fma(p, y, 2.48015873015873e-5);
-    p = fma(p, y, 1.984126984126984e-4);
-    p = fma(p, y, 1.388888888888889e-3);
-    p = fma(p, y, 8.333333333333333e-3);
-    p = fma(p, y, 4.1666666666666664e-2);
-    p = fma(p, y, 1.6666666666666666e-1);
-    p = fma(p, y, 0.5);
-    p = fma(p, y, 1.0);
-    p = fma(p, y, 1.0);
-    return __hiloint2double(__double2hiint(p) + (n << 20), __double2loint(p));
-}
-
-// One position i of sequence b, given its row's sum_v 2^(l_v * c1) = S * 2^Rr (float64 S, integer
-// Rr): writes lse and p_i(x_i), evaluates the acceptance test and returns the position's bits;
-// Rs, invS are what the emission of this row would need.  A lane that is not live returns "accepted".
-__device__ __forceinline__ unsigned judge_position(const EdgeParams &P, long long b, int i, bool live, float Rr, double S,
-                                                   bool bad, bool timeout, int x, float zx, float qx, float ux,
-                                                   float &Rs, float &invS)
-{
-    const double c1 = (double)P.c1;
-    // the sum has a finite logarithm iff S is positive and finite
-    const bool finite = !timeout && !bad && (S > 0.0) && (S < INFINITY) && (Rr != DSSD_NEG_INF);
-    unsigned bits = live ? ((finite ? 0u : kBitNonFinite) | (timeout ? kBitTimeout : 0u)) : kBitAccept;
-    if (live && P.lse)
-        P.lse[b * (P.gamma + 1) + i] = finite ? (Rr + __log2f((float)S)) * 0.6931471805599453f : __int_as_float(0x7fc00000);
-    // 1 / S in float64: the float32 reciprocal refined by one Newton step
-    double invS_d = NAN;
-    if (finite) {
-        const double r0 = (double)(1.0f / (float)S);
-        invS_d = r0 * (2.0 - S * r0);
-    }
-    if (live && i < P.gamma) {
-        double p = NAN;
-        bool accept = false;
-        if (x < 0 || x >= P.V) {
-            bits |= kBitBadToken;
-        } else {
-            // u < min(1, p(x)/q(x)) in float64, as  u < 1  and  u * q < p  (u * q is exact)
-            p = finite ? exp2_small((double)zx * c1 - (double)Rr) * invS_d : NAN;
-            const double q = (double)qx;
-            const double u = (double)ux;
-            if (q != q || p != p) accept = false;
-            else if (q <= 0.0) accept = (p > 0.0) && (u < 1.0);
-            else accept = (u < 1.0) && (u * q < p);
-        }
-        if (P.p_tok) P.p_tok[(size_t)b * P.gamma + i] = (float)p;
-        bits |= accept ? kBitAccept : 0u;
-    }
-    invS = finite ? (float)invS_d : __int_as_float(0x7fc00000);
-    Rs = finite ? Rr : 0.f;
-    return bits;
-}
-
 // Run by the fold warp that brought the last partial of sequence b.  One lane per position
 // i = 0..gamma: the row's partials -> log-sum-exp (float64) -> acceptance test
 //   u_i < min(1, p_i(x_i) / q_i(x_i));
@@ -476,17 +426,23 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
         for (int k = 0; k < kAhead; ++k) pw[k] = (live && k < P.n_lse_runs) ? ld_relaxed_u64(part + k) : 0ull;
         int x = -1;
         float zx = 0.f, qx = 0.f, ux = 0.f;
+        bool owned = false;
         if (live && i < P.gamma) {
             const size_t di = (size_t)b * P.gamma + i;
             x = P.draft_tokens[di];
-            ux = P.uniforms[di];
-            if (P.draft_q_rows) {
+            if (P.uniforms) ux = P.uniforms[di];
+            if (P.shard_sum) {
+                // partial sums only: no test here
+            } else if (P.draft_q_rows) {
                 // a token id outside the vocabulary has no q: NaN (the id itself gets the position rejected and flagged)
                 qx = (x >= 0 && x < P.V) ? __ldg(P.draft_q_rows + di * (size_t)P.V + (size_t)x) : __int_as_float(0x7fc00000);
             } else {
                 qx = P.draft_q_tok[di];
             }
-            if (x >= 0 && x < P.V) zx = E::load(row_ptr<DT>(P, row), x);
+            // (a shard of the vocabulary holds entries v_begin .. v_begin + V - 1; v_begin is 0 otherwise)
+            const long long xl = (long long)x - (long long)P.v_begin;
+            owned = xl >= 0 && xl < (long long)P.V;
+            if (owned) zx = E::load(row_ptr<DT>(P, row), xl);
         }
         // The sequence's arrival counter says every ticket has been counted; a partial whose
         // store has not landed yet still shows the fill pattern and is polled for.
@@ -511,16 +467,19 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
                     timeout = true;
                     continue;
                 }
-                const float pr = __uint_as_float((unsigned)w), ps = __uint_as_float((unsigned)(w >> 32));
-                if (ps != ps) bad = true;
-                if (ps > 0.f) {  // S is kept relative to the largest reference seen so far
-                    if (pr > Rr) {
-                        S = (Rr == DSSD_NEG_INF || S == 0.0) ? 0.0 : scale_pow2(S, Rr - pr);
-                        Rr = pr;
-                    }
-                    S += scale_pow2((double)ps, pr - Rr);
-                }
+                add_partial(Rr, S, bad, __uint_as_float((unsigned)w), (double)__uint_as_float((unsigned)(w >> 32)));
             }
+        }
+        if (P.shard_sum) {
+            // one shard of the vocabulary: the row's partial sum and the drafted token's logit (where
+            // this shard holds it) go out as they are; the test is made once all shards' sums have met
+            if (live) {
+                P.shard_ref[row] = Rr == DSSD_NEG_INF ? 0.f : Rr;
+                P.shard_sum[row] = (bad || timeout) ? (double)__int_as_float(0x7fc00000) : S;
+                if (i < P.gamma) P.shard_tok_logit[(size_t)b * P.gamma + i] = owned ? zx : __int_as_float(0x7fc00000);
+            }
+            any_timeout = any_timeout || __any_sync(kFull, timeout);
+            continue;
         }
         float Rs, invS;
         const unsigned bits = judge_position(P, b, i, live, Rr, S, bad, timeout, x, zx, qx, ux, Rs, invS);
@@ -534,6 +493,10 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
             ref2_n = __shfl_sync(kFull, Rs, n - base);
             invS_n = __shfl_sync(kFull, invS, n - base);
         }
+    }
+    if (P.shard_sum) {
+        if (lane == 0 && any_timeout) *P.error = 1u;
+        return;
     }
     if (lane == 0) {
         P.accept_len[b] = any_timeout ? -1 : n;
@@ -907,60 +870,128 @@ __device__ __forceinline__ void start_run(const EdgeParams &P, Shared *sh, Run &
     r.remain = (long long)P.V * E::kBytes - t.head - (long long)k_begin * kS;
 }
 
+// The producer's position in the ring and in its tickets.  The first part of it is set up before
+// the grid-wide barrier (see producer_prologue), the rest by producer_thread.
+struct ProducerState {
+    Run lr;  // the LSE run in progress
+    unsigned st, par;
+    unsigned issued, tickets, lse_tickets;
+    bool lse_left;
+};
+
+// LSE ticket number `no` (< total_lse) -> its ticket record and stage range; starts the run
 template <int DT>
-__device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh, uint32_t ring)
+__device__ __forceinline__ void start_lse_ticket(const EdgeParams &P, Shared *sh, Run &lr, unsigned long long no,
+                                                 unsigned &tickets, unsigned &lse_tickets)
+{
+    Ticket t;
+    unsigned long long row;
+    split_ticket(no, P.n_lse_runs, P.lse_magic, row, t.run);
+    t.row = (long long)row;
+    t.seq = (row >> 32) == 0 ? (long long)((unsigned)row / (unsigned)(P.gamma + 1))
+                             : (long long)(row / (unsigned)(P.gamma + 1));
+    t.out_off = -1;
+    t.ref2 = t.invS = 0.f;
+    const int k_begin = t.run * P.lse_run;
+    const int k_end = min(P.n_slices, k_begin + P.lse_run);
+    start_run<DT>(P, sh, lr, kLse, t, k_begin, k_end, tickets, lse_tickets);
+}
+
+// Arms ring stage `st` with the next stage of run r and issues its copy.  The stage must be free.
+__device__ __forceinline__ void issue_stage(Shared *sh, uint32_t ring, Run &r, unsigned &st, unsigned &par,
+                                            unsigned &issued, uint64_t pol_emit)
+{
+    const unsigned len = r.remain <= 0 ? 0u : (r.remain >= kS ? (unsigned)kS : (unsigned)r.remain);
+    const unsigned bulk = len & ~15u;
+    const bool ragged = (r.k == 0 && r.head != 0) || (len & 15u);
+    const unsigned meta = r.kind | (r.k == r.k_begin ? kMetaFirst : 0u) | (r.k + 1 == r.k_end ? kMetaLast : 0u) |
+                          (ragged ? kMetaRagged : 0u) | (r.slot << kMetaSlotShift) | ((unsigned)r.k << kMetaKShift);
+    sh->desc[st] = make_uint2(meta, bulk);
+    const uint32_t bar = smem_addr(&sh->full[st]);
+    if (bulk) {
+        mbar_arrive_expect_tx(bar, bulk);
+        if (r.kind == kEmit) bulk_g2s_hint(ring + st * (uint32_t)kS, r.src, bulk, bar, pol_emit);
+        else bulk_g2s(ring + st * (uint32_t)kS, r.src, bulk, bar);
+    } else {
+        mbar_arrive(bar);
+    }
+    ++issued;
+    r.src += kS;
+    r.remain -= kS;
+    if (++r.k == r.k_end) r.kind = kEnd;
+    if (++st == (unsigned)kEdgeStages) {
+        st = 0;
+        par ^= 1u;
+    }
+}
+
+// Before the grid-wide barrier that follows the clearing of the workspace nothing of the workspace
+// may be touched, but the logits may be read: every CTA's first LSE ticket is its own number
+// (the ticket counter starts at the number of CTAs), and its first stages go out at once, into
+// the still empty ring, so that the copies are in flight while the barrier completes.
+template <int DT>
+__device__ __forceinline__ void producer_prologue(const EdgeParams &P, Shared *sh, uint32_t ring, ProducerState &s)
+{
+    s.lr.kind = kEnd;
+    s.st = 0;
+    s.par = 1;  // a fresh barrier passes a wait on parity 1: the ring starts out empty
+    s.issued = s.tickets = s.lse_tickets = 0;
+    s.lse_left = true;
+    const unsigned long long no = blockIdx.x;
+    if (no >= P.total_lse) {
+        s.lse_left = false;
+        return;
+    }
+    start_lse_ticket<DT>(P, sh, s.lr, no, s.tickets, s.lse_tickets);
+    for (int j = 0; j < kEdgeStages && s.lr.kind != kEnd; ++j) issue_stage(sh, ring, s.lr, s.st, s.par, s.issued, 0ull);
+}
+
+// The producer issues stages and nothing else: which ticket comes next it learns from two small
+// queues in shared memory that the scout fills, so no round trip to global memory ever stands
+// between a freed stage of the ring and the next copy.
+template <int DT>
+__device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh, uint32_t ring, ProducerState &s)
 {
     const uint64_t pol_emit = l2_policy_evict_first();
-    Claim c;
-    c.state = kWatch;
-    c.exhausted = false;
-    c.claim_raw = c.ticket = c.w0 = c.w1 = 0;
-    claim_watch(P, c);
-    unsigned long long lse_raw = atomicAdd(P.lse_ticket, 1ull);  // the LSE ticket in hand, drawn one ticket early
-    bool lse_left = true;
-    // Towards the end of the launch no new EMIT ticket is claimed while LSE work is left: the last
-    // waves of LSE tickets then finish sooner (their sequences complete sooner) and the rows held
-    // back fill the time in which the final sequences complete, on all CTAs, in short tickets.
-    bool endgame = false;
-    Run lr, er;  // the LSE and the EMIT run in progress; an EMIT run goes first
-    lr.kind = er.kind = kEnd;
-    unsigned st = 0, par = 1;  // a fresh barrier passes a wait on parity 1: the ring starts out empty
-    unsigned issued = 0, tickets = 0, lse_tickets = 0, idle = 0;
+    bool lse_left = s.lse_left;
+    Run lr = s.lr, er;  // the LSE and the EMIT run in progress; an EMIT run goes first
+    er.kind = kEnd;
+    unsigned st = s.st, par = s.par;
+    unsigned issued = s.issued, tickets = s.tickets, lse_tickets = s.lse_tickets, idle = 0;
+    unsigned emit_popped = 0, lse_popped = 0;
     bool failed = false;
+    volatile unsigned *emit_pushed = &sh->emit_pushed, *lse_pushed = &sh->lse_pushed, *scout_done = &sh->scout_done;
     for (;;) {
-        Ticket t;
-        int k_begin = 0, k_end = 0;
-        const bool hold = endgame && (lse_left || lr.kind != kEnd) && c.state == kWatch;
-        if (er.kind == kEnd && !hold && claim_step(P, c, t, k_begin, k_end, !lse_left && lr.kind == kEnd)) start_run<DT>(P, sh, er, kEmit, t, k_begin, k_end, tickets, lse_tickets);
-        if (er.kind == kEnd && lr.kind == kEnd && lse_left) {
-            const unsigned long long no = logical(lse_raw);
-            endgame = no + P.endgame_tickets >= P.total_lse;
-            if (no < P.total_lse) {
-                unsigned long long row;
-                split_ticket(no, P.n_lse_runs, P.lse_magic, row, t.run);
-                t.row = (long long)row;
-                t.seq = (row >> 32) == 0 ? (long long)((unsigned)row / (unsigned)(P.gamma + 1))
-                                         : (long long)(row / (unsigned)(P.gamma + 1));
-                t.out_off = -1;
-                t.ref2 = t.invS = 0.f;
-                k_begin = t.run * P.lse_run;
-                k_end = min(P.n_slices, k_begin + P.lse_run);
-                lse_raw = atomicAdd(P.lse_ticket, 1ull);
-                start_run<DT>(P, sh, lr, kLse, t, k_begin, k_end, tickets, lse_tickets);
-            } else {
-                lse_left = false;
-            }
+        if (er.kind == kEnd && *emit_pushed != emit_popped) {
+            __threadfence_block();
+            EmitWork w = sh->emit_q[emit_popped & (kEmitQ - 1)];
+            ++emit_popped;
+            __threadfence_block();
+            *(volatile unsigned *)&sh->emit_popped = emit_popped;
+            start_run<DT>(P, sh, er, kEmit, w.t, w.k_begin, w.k_end, tickets, lse_tickets);
+        }
+        if (er.kind == kEnd && lr.kind == kEnd && lse_left && *lse_pushed != lse_popped) {
+            __threadfence_block();
+            const unsigned long long no = sh->lse_q[lse_popped & (kLseQ - 1)];
+            ++lse_popped;
+            __threadfence_block();
+            *(volatile unsigned *)&sh->lse_popped = lse_popped;
+            if (no < P.total_lse) start_lse_ticket<DT>(P, sh, lr, no, tickets, lse_tickets);
+            else lse_left = false;
+        }
+        {
+            const unsigned busy = (lse_left || lr.kind != kEnd) ? 1u : 0u;
+            if (*(volatile unsigned *)&sh->lse_busy != busy) *(volatile unsigned *)&sh->lse_busy = busy;
         }
         Run &r = er.kind != kEnd ? er : lr;
         if (r.kind == kEnd) {
-            // nothing to issue: done once no LSE ticket is left, no claim is under way and every
-            // EMIT ticket has been claimed by someone
-            if (!lse_left && c.state == kWatch && (c.exhausted || logical(c.head_raw) >= P.total_emit)) break;
+            // nothing to issue: done once no LSE ticket is left and the scout has nothing more to hand over
+            if (!lse_left && *scout_done && *emit_pushed == emit_popped) break;
             if (++idle > P.spin_limit) {
                 failed = true;
                 break;
             }
-            __nanosleep(200);
+            __nanosleep(100);
             continue;
         }
         idle = 0;
@@ -968,28 +999,7 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
             failed = true;  // the consumers went silent
             break;
         }
-        const unsigned len = r.remain <= 0 ? 0u : (r.remain >= kS ? (unsigned)kS : (unsigned)r.remain);
-        const unsigned bulk = len & ~15u;
-        const bool ragged = (r.k == 0 && r.head != 0) || (len & 15u);
-        const unsigned meta = r.kind | (r.k == r.k_begin ? kMetaFirst : 0u) | (r.k + 1 == r.k_end ? kMetaLast : 0u) |
-                              (ragged ? kMetaRagged : 0u) | (r.slot << kMetaSlotShift) | ((unsigned)r.k << kMetaKShift);
-        sh->desc[st] = make_uint2(meta, bulk);
-        const uint32_t bar = smem_addr(&sh->full[st]);
-        if (bulk) {
-            mbar_arrive_expect_tx(bar, bulk);
-            if (r.kind == kEmit) bulk_g2s_hint(ring + st * (uint32_t)kS, r.src, bulk, bar, pol_emit);
-            else bulk_g2s(ring + st * (uint32_t)kS, r.src, bulk, bar);
-        } else {
-            mbar_arrive(bar);
-        }
-        ++issued;
-        r.src += kS;
-        r.remain -= kS;
-        if (++r.k == r.k_end) r.kind = kEnd;
-        if (++st == (unsigned)kEdgeStages) {
-            st = 0;
-            par ^= 1u;
-        }
+        issue_stage(sh, ring, r, st, par, issued, pol_emit);
     }
     if (!failed && mbar_wait(smem_addr(&sh->empty[st]), par, P.spin_limit)) {
         // tell the consumers that nothing follows
@@ -1001,6 +1011,7 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
     // flight into the ring; wait for them (bounded) before the CTA's shared memory can be handed
     // to another CTA.  The last min(issued, kEdgeStages) stages armed are st - 1, st - 2, ...
     *P.error = 1u;
+    *(volatile unsigned *)&sh->abort = 1u;
     unsigned s2 = st, p2 = par;
     for (unsigned j = 0; j < (unsigned)kEdgeStages && j < issued; ++j) {
         if (s2 == 0) {
@@ -1009,6 +1020,84 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
         }
         --s2;
         mbar_wait(smem_addr(&sh->full[s2]), p2 ^ 1u, P.spin_limit);  // armed in the pass whose empty parity was p2
+    }
+}
+
+
+// The scout (one thread) does everything that needs a round trip to global memory on the
+// producer's behalf: it draws the CTA's next LSE ticket (one ticket ahead) and runs the claim on
+// EMIT work - watch the counters, claim a ticket, look up its sequence's `ready` entry - and
+// pushes what it gets into the two queues.  Its loop runs at the pace of those round trips, which
+// no longer matters to the stream.
+template <int DT>
+__device__ __forceinline__ void scout_thread(const EdgeParams &P, Shared *sh)
+{
+    Claim c;
+    c.state = kWatch;
+    c.exhausted = false;
+    c.claim_raw = c.ticket = c.w0 = c.w1 = 0;
+    claim_watch(P, c);
+    bool more_lse = (unsigned long long)blockIdx.x < P.total_lse;  // else the CTA never had an LSE ticket
+    bool lse_pending = false;
+    unsigned long long lse_raw = 0;
+    // Towards the end of the launch no new EMIT ticket is claimed while LSE work is left: the last
+    // waves of LSE tickets then finish sooner (their sequences complete sooner) and the rows held
+    // back fill the time in which the final sequences complete, on all CTAs, in short tickets.
+    bool endgame = (unsigned long long)blockIdx.x + P.endgame_tickets >= P.total_lse;
+    unsigned emit_pushed = 0, lse_pushed = 0, idle = 0;
+    volatile unsigned *emit_popped = &sh->emit_popped, *lse_popped = &sh->lse_popped, *lse_busy = &sh->lse_busy,
+                      *abort = &sh->abort;
+    EmitWork w;
+    bool have = false;  // a claimed, ready EMIT ticket waiting for room in the queue
+    for (;;) {
+        if (*abort) return;
+        // the next LSE ticket: drawn as soon as the producer has taken the one before
+        if (more_lse && !lse_pending && lse_pushed == *lse_popped) {
+            lse_raw = atomicAdd(P.lse_ticket, 1ull);
+            lse_pending = true;
+        }
+        const bool busy = *lse_busy != 0u || more_lse;
+        if (have) {
+            if (emit_pushed - *emit_popped < (unsigned)kEmitQ) {
+                sh->emit_q[emit_pushed & (kEmitQ - 1)] = w;
+                __threadfence_block();
+                *(volatile unsigned *)&sh->emit_pushed = ++emit_pushed;
+                have = false;
+                idle = 0;
+            }
+        } else {
+            const bool hold = endgame && busy && c.state == kWatch;
+            if (!hold) {
+                const int before = c.state;
+                have = claim_step(P, c, w.t, w.k_begin, w.k_end, !busy);
+                if (have || c.state != before) idle = 0;
+            } else if (!lse_pending) {
+                __nanosleep(200);  // nothing to ask memory for: do not take issue slots from the working warps
+            }
+        }
+        if (lse_pending) {  // asked for at the top of this pass, or earlier: by now it is usually back
+            const unsigned long long no = logical(lse_raw);
+            lse_pending = false;
+            endgame = no + P.endgame_tickets >= P.total_lse;
+            if (no >= P.total_lse) more_lse = false;
+            sh->lse_q[lse_pushed & (kLseQ - 1)] = no;  // a number beyond the last ticket tells the producer that none is left
+            __threadfence_block();
+            *(volatile unsigned *)&sh->lse_pushed = ++lse_pushed;
+            idle = 0;
+        }
+        // done once no LSE ticket is left anywhere, no claim is under way, nothing waits here and every
+        // EMIT ticket has been claimed by someone
+        if (!more_lse && !have && c.state == kWatch && (c.exhausted || logical(c.head_raw) >= P.total_emit)) {
+            __threadfence_block();
+            *(volatile unsigned *)&sh->scout_done = 1u;
+            return;
+        }
+        if (++idle > P.spin_limit) {
+            *P.error = 1u;  // waited too long (for a sequence to become ready, or for the producer)
+            *(volatile unsigned *)&sh->scout_done = 1u;
+            return;
+        }
+        if (have || (c.state == kWatch && !busy)) __nanosleep(100);
     }
 }
 
@@ -1152,14 +1241,7 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
             if (live) {
                 for (int k = 0; k < csize; ++k) {
                     const float2 c = s_clu[i][k];
-                    if (c.y != c.y) bad = true;
-                    if (c.y > 0.f) {
-                        if (c.x > Rr) {
-                            S = (Rr == DSSD_NEG_INF || S == 0.0) ? 0.0 : scale_pow2(S, Rr - c.x);
-                            Rr = c.x;
-                        }
-                        S += scale_pow2((double)c.y, c.x - Rr);
-                    }
+                    add_partial(Rr, S, bad, c.x, (double)c.y);
                 }
             }
             float Rs, invS;
@@ -1248,10 +1330,33 @@ __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __gr
 
 constexpr size_t kEdgeSmemBytes = (size_t)kEdgeStages * kS + sizeof(Shared);
 
+// The workspace is cleared inside the kernel: every slot and counter to all ones, except the LSE
+// ticket counter, which starts at the number of CTAs (every CTA's first ticket is its own number).
+__device__ __forceinline__ void clear_workspace(const EdgeParams &P)
+{
+    uint4 *w = reinterpret_cast<uint4 *>(P.lse_ticket);  // the workspace starts with the counters
+    const size_t n = P.fill_bytes / 16;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        uint4 v = make_uint4(kFull, kFull, kFull, kFull);
+        if (i == 0) {  // raw value of the 64-bit counter: logical value - 1
+            v.x = gridDim.x - 1u;
+            v.y = 0u;
+        }
+        w[i] = v;
+    }
+}
+
+// Launched cooperatively (all CTAs resident), which is what allows the one grid-wide barrier
+// between the clearing of the workspace and its first use.  The barrier is split: every CTA
+// arrives once its share of the workspace is cleared, its producer sends the first copies on their
+// way, and only then does the CTA wait for the others; no CTA waits for anything before it has
+// arrived, so the barrier always completes.
 template <int DT>
 __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __grid_constant__ EdgeParams P)
 {
     extern __shared__ __align__(128) unsigned char smem[];
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t ring = smem_addr(smem);
     Shared *sh = reinterpret_cast<Shared *>(smem + (size_t)kEdgeStages * kS);
@@ -1265,15 +1370,24 @@ __global__ void __launch_bounds__(kEdgeThreads, 1) edge_verify_kernel(const __gr
         for (int i = 0; i < kMail; ++i) sh->mail[i].valid = 0;
         sh->mail_tail = 0;
         sh->cons_done = 0;
+        sh->emit_pushed = sh->emit_popped = sh->lse_pushed = sh->lse_popped = 0;
+        sh->lse_busy = 1;
+        sh->scout_done = sh->abort = 0;
         mbar_init_fence();
     }
-    __syncthreads();
+    clear_workspace(P);
+    auto arrived = grid.barrier_arrive();  // (a CTA-wide barrier is part of it)
+    ProducerState ps;
+    if (threadIdx.x == 0) producer_prologue<DT>(P, sh, ring, ps);
+    grid.barrier_wait(std::move(arrived));
     if (warp == 0) {
-        if (lane == 0) producer_thread<DT>(P, sh, ring);
+        if (lane == 0) producer_thread<DT>(P, sh, ring, ps);
     } else if (warp <= kNC) {
         consumer_warp<DT>(P, sh, ring, warp - 1);
-    } else {
+    } else if (warp == kNC + 1) {
         fold_warp<DT>(P, sh);
+    } else {
+        if (lane == 0) scout_thread<DT>(P, sh);
     }
 }
 
@@ -1287,7 +1401,7 @@ int edge_max_runs_per_row(int V)
 
 size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, char *base)
 {
-    // all of it is filled with 0xFF before the launch: counters then read "logical 0", slots "not yet"
+    // the kernel sets all of it to 0xFF before use: counters then read "logical 0", slots "not yet"
     const size_t R = (size_t)B * (size_t)(gamma + 1);
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -1345,7 +1459,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     // EMIT tickets, and what the draw needs about row n stays in the workspace (`ready`).
     const bool no_emit = !P.p_row && !P.p_row16;
     // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
-    if (!no_emit && !P.skip_bonus_row && !P.draft_q_rows) {
+    if (!no_emit && !P.skip_bonus_row && !P.draft_q_rows && !P.shard_sum) {
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;
@@ -1406,12 +1520,14 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     P.spin_limit = 1u << 20;
     P.c1 = (float)(1.4426950408889634 / (double)P.temperature);
     edge_workspace_layout(P.B, P.gamma, P.n_lse_runs, &P, static_cast<char *>(workspace));
-    if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long tickets = P.total_lse + P.total_emit;
     const unsigned grid = (unsigned)(tickets < resident_ctas ? tickets : resident_ctas);
-    if (dtype == DSSD_BF16) edge_verify_kernel<DSSD_BF16><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
-    else edge_verify_kernel<DSSD_F32><<<grid, kEdgeThreads, kEdgeSmemBytes, stream>>>(P);
-    return cudaGetLastError();
+    // a cooperative launch: all CTAs are resident at once (grid <= resident_ctas), which the kernel's
+    // grid-wide barrier after the clearing of the workspace relies on
+    void *args[] = {&P};
+    const void *fn = dtype == DSSD_BF16 ? reinterpret_cast<const void *>(edge_verify_kernel<DSSD_BF16>)
+                                        : reinterpret_cast<const void *>(edge_verify_kernel<DSSD_F32>);
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kEdgeThreads), args, kEdgeSmemBytes, stream);
 }
 
 }  // namespace dssd

@@ -40,7 +40,7 @@ constexpr int kEdgeEndgameLongRows = 8;                                  // ... 
 constexpr int kEdgeEndgameLongWaves = DSSD_EDGE_ENDGAME_LONG_WAVES;      // launches of at least so many waves ...
 constexpr int kEdgeEndgameLongEighths = DSSD_EDGE_ENDGAME_LONG_EIGHTHS;  // ... hold them back during the last so many eighths of the waves
 constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
-constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 2);  // + the producer warp and the fold warp
+constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 3);  // + the producer warp, the fold warp and the scout warp
 constexpr int kEdgeStageBytes = DSSD_EDGE_STAGE_BYTES;   // logits bytes per ring stage (one bulk copy)
 constexpr int kEdgeStages = DSSD_EDGE_STAGES;            // ring stages per CTA
 constexpr int kEdgeMaxRun = DSSD_EDGE_MAX_RUN;           // most consecutive stages of a row in one ticket
@@ -48,7 +48,7 @@ constexpr int kEdgeEmitRun = DSSD_EDGE_EMIT_RUN;        // most stages of row n 
 constexpr int kEdgeTicketsPerCta = DSSD_EDGE_TICKETS_PER_CTA;  // tickets aimed at per resident CTA
 
 // What the emission of row P_n needs to know about a folded sequence: two 8-byte slots, each
-// valid once it differs from the all-ones pattern the workspace is filled with before the launch.
+// valid once it differs from the all-ones pattern the kernel clears the workspace to.
 struct ReadySlot {
     int b;       // sequence (>= 0)
     int n;       // accepted length, or -1 if a wait ran out
@@ -74,6 +74,13 @@ struct EdgeParams {
     float *lse;
     uint32_t *flags;
     int skip_bonus_row;    // 1: no row is emitted for fully accepted sequences (n == gamma)
+    // one shard of the vocabulary (entries v_begin .. v_begin + V - 1 of every row): when shard_sum is
+    // set the kernel only forms each row's partial sum, sum_v 2^(l_v c1) = shard_sum * 2^shard_ref, and
+    // looks up the logits of the drafted tokens it holds; nothing is tested or emitted
+    float *shard_ref;         // [B, gamma+1]
+    double *shard_sum;        // [B, gamma+1]
+    float *shard_tok_logit;   // [B, gamma]; NaN where the token lies outside the shard
+    int v_begin;
     // ticket geometry
     int n_slices;                  // stages per row
     int lse_run, emit_run;         // stages per LSE / EMIT ticket
@@ -83,7 +90,7 @@ struct EdgeParams {
     unsigned long long endgame_tickets;  // EMIT claims are held back once so few LSE tickets are left
     unsigned long long lse_magic, emit_magic;  // ceil(2^64 / n_*_runs) when multiply-high division is exact, else 0
     unsigned spin_limit;
-    // workspace, filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
+    // workspace, set to 0xFF by the kernel before use: counters then read "logical 0" (raw + 1)
     // and 8-byte slots read "not yet" until their one store has landed
     unsigned long long *lse_ticket;  // next LSE ticket
     unsigned long long *emit_head;   // next EMIT ticket
@@ -102,7 +109,7 @@ int edge_max_runs_per_row(int V);
 // With P == nullptr only computes the size.
 size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, char *base);
 
-// Fills the geometry fields of P, clears the workspace and launches the kernel on `stream`.
+// Fills the geometry fields of P and launches the kernel (which clears the workspace itself) on `stream`.
 cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaStream_t stream);
 
 }  // namespace dssd

@@ -55,3 +55,51 @@ def test_two_ranks_shard_by_sequence(tmp_path, oracle_mod):
     mp.spawn(_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     ok = np.load(tmp_path / "ok.npy")
     assert ok.tolist() == [1, 1, 1]
+
+
+def _vocab_rank_main(rank, world, port, out_dir):
+    """Vocabulary sharding over two gloo ranks: every rank holds its slice of each row, computes the
+    oracle's per-shard quantities, and the two exchanges go through the package's own gather helper
+    (the one the CUDA ranks use)."""
+    sys.path.insert(0, ROOT)
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import dssd_inputs as di
+    from oracle import oracle as O
+    from oracle import shard_oracle as S
+    from paper_2507_12000_b200.sharded import all_gather_shards
+
+    w = di.custom(B=24, gamma=3, V=1001, dtype="bf16", temperature=0.8, sigma_d=0.9, seed=321)
+    d = di.generate(w)  # the per-sequence inputs are replicated; of the rows a rank looks at its slice only
+    a, b = S.shard_bounds(w.V, world)[rank]
+    tl, dq = d["target_logits"][:, :, a:b], d["draft_q"][:, :, a:b]
+    part = S.edge_partial(tl, d["draft_tokens"], a, w.temperature)
+    gathered = {k: all_gather_shards(torch.from_numpy(v)).numpy() for k, v in part.items()}
+    parts = [{k: gathered[k][g] for k in part} for g in range(world)]
+    ev = S.edge_combine(parts, d["draft_tokens"], d["draft_q_tok"], d["uniforms"], w.V)
+    row = S.edge_emit_shard(tl, ev["accept_len"], ev["lse"], w.temperature)
+    mass = S.resample_shard_mass(row, dq, ev["accept_len"], w.gamma)
+    masses = all_gather_shards(torch.from_numpy(mass)).numpy()
+    dr = S.resample_shard_draw(masses, rank, a, row, dq, ev["accept_len"], d["uniforms_rs"], w.gamma)
+    token = torch.from_numpy(dr["token"].astype(np.int64))
+    dist.all_reduce(token, op=dist.ReduceOp.MAX)
+    rows = all_gather_shards(torch.from_numpy(np.pad(row, ((0, 0), (0, (w.V + world - 1) // world - row.shape[1]))))).numpy()
+    if rank == 0:
+        ref = O.verify_round(d, w.temperature)
+        whole = np.concatenate([rows[g][:, :hi - lo] for g, (lo, hi) in enumerate(S.shard_bounds(w.V, world))], axis=1)
+        safe = ref["margin_cdf"] > 1e-9
+        np.save(os.path.join(out_dir, "ok.npy"),
+                np.array([int((ev["accept_len"] == ref["accept_len"]).all()),
+                          int(np.allclose(whole, ref["p_row"], rtol=1.2e-7, atol=0)),
+                          int((token.numpy()[safe] == ref["token"][safe]).all() and safe.mean() > 0.9),
+                          int((dr["flags"] == ref["rs_flags"]).all())]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_by_vocabulary(tmp_path, oracle_mod):
+    port = 31500 + (os.getpid() % 2000)
+    mp.spawn(_vocab_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    ok = np.load(tmp_path / "ok.npy")
+    assert ok.tolist() == [1, 1, 1, 1]
