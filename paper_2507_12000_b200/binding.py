@@ -40,7 +40,8 @@ class DssdError(RuntimeError):
         super().__init__(f"{where}: {name}{extra}")
 
 
-def _load(path: str = LIB_PATH) -> ctypes.CDLL:
+def _load(path: Optional[str] = None) -> ctypes.CDLL:
+    path = path or LIB_PATH
     if not os.path.exists(path):
         raise ImportError(
             f"{path} is missing: build it with `python -m paper_2507_12000_b200.build` "
