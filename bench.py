@@ -177,7 +177,7 @@ def oracle_rate(w: di.Workload, d, n_seq: int, threads: int, min_seconds: float 
 def run_reference(args, w: di.Workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
-        return
+        return  # the oracle runs on rank 0's host cores alone; the other ranks leave at once
     from oracle import oracle as O
 
     O.build()
@@ -1018,6 +1018,16 @@ def main():
     ap.add_argument("--also", default="c5max,c3",
                     help="workloads measured after the default one and reported as sub-records (empty: none)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand rather than by a launcher: become the launcher, one rank per GPU of this node
+        import socket
+
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:])
     w = di.get_workload(args.workload)
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 2000

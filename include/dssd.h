@@ -27,8 +27,13 @@
  *
  * General rules
  *   - Every pointer is a DEVICE pointer unless its comment says "host".
- *   - The caller owns every buffer.  The library allocates no memory, keeps no state between
- *     calls, enqueues its work on the given CUDA stream and returns without synchronising.
+ *   - The caller owns every buffer.  The library allocates no memory, enqueues its work on the
+ *     given CUDA stream and returns without synchronising.  It keeps no state between calls except
+ *     per-device launch constants (SM count, resident CTAs per kernel), which are looked up on the
+ *     first call made with a device current and cached, and the built-in scratch of
+ *     dssd_device_resample_static.
+ *   - The streaming kernels are launched cooperatively (every CTA resident at once): two calls
+ *     issued to different streams run one after the other on the GPU, not side by side.
  *   - Buffers need only their natural alignment; 16-byte aligned rows take the fast path.
  *   - A status other than DSSD_OK means nothing was enqueued (except DSSD_ERR_CUDA, after
  *     which the outputs are undefined).  Data-dependent anomalies never fault or trap: they
@@ -104,8 +109,15 @@ size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V);
  * dssd_device_resample can draw the bonus token; a caller that wants the paper's byte saving
  * simply does not transmit it.
  *
- * Comparison details: the test is evaluated in float64 from a float64 log-sum-exp; u == 1 never
- * accepts; q <= 0 accepts iff p > 0; a NaN q or an out-of-range token rejects.
+ * Arithmetic: with c1 = float32(log2(e) / T), every term 2^(l_v * c1 - ref) is formed in float32
+ * (one fused multiply-add, one ex2 of relative error 2^-22) and added up in float32 per lane, at
+ * most a few hundred terms per accumulator; the per-lane sums are combined in float64 by exact
+ * power-of-two scaling.  p_i(x_i) = 2^(l_x * c1 - ref) / S and the test u * q < p are evaluated in
+ * float64.  The result is within about 1e-6 relative of the exact softmax as long as
+ * |l| * log2(e) / T stays well inside the float32 range (the rounding of c1 alone contributes
+ * 6e-8 * |l_v / T - E_p[l / T]| to ln p); rows whose scaled logits overflow float32 are flagged
+ * DSSD_EDGE_FLAG_NONFINITE.  u == 1 never accepts; q <= 0 accepts iff p > 0; a NaN q or an
+ * out-of-range token rejects.
  *
  * target_logits  [B, gamma+1, V] of `dtype`, unit stride along V, `row_stride` elements between
  *                consecutive rows (>= V); row (b, i) starts at element (b*(gamma+1)+i)*row_stride
@@ -113,7 +125,7 @@ size_t dssd_edge_verify_workspace_bytes(int B, int gamma, int V);
  * draft_q_tok    [B, gamma] float32    q_i(x_i)     (may be NULL iff gamma == 0)
  * uniforms       [B, gamma] float32    u_i in [0,1) (may be NULL iff gamma == 0)
  * temperature    T > 0, finite
- * accept_len     [B] int32     out: n in [0, gamma]
+ * accept_len     [B] int32     out: n in [0, gamma]; -1 (with DSSD_EDGE_FLAG_TIMEOUT) if an internal wait ran out
  * p_row          [B, V] float32 out: P_n(.)
  * p_tok          [B, gamma] float32   out, optional (NULL ok): p_i(x_i)
  * lse            [B, gamma+1] float32 out, optional (NULL ok): ln sum_v exp(l_v / T)
@@ -169,11 +181,14 @@ dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
  * nothing.
  *
  * Same inputs, outputs and results as dssd_device_resample (the two share the kernel).
- *   - Sizes whose scratch need (dssd_device_resample_workspace_bytes) exceeds
- *     DSSD_STATIC_SCRATCH_BYTES are refused with DSSD_ERR_UNSUPPORTED before anything is enqueued;
- *     use dssd_device_resample for those.
+ *   - Sizes whose scratch need (dssd_device_resample_workspace_bytes: 256 bytes of counters plus
+ *     8 bytes per 4096 vocabulary entries per sequence) exceeds DSSD_STATIC_SCRATCH_BYTES, i.e.
+ *     B * ceil(V / 4096) > 131 040, are refused with DSSD_ERR_UNSUPPORTED before anything is
+ *     enqueued; use dssd_device_resample for those.
  *   - The first call made with a given device current looks up the array's device address (once
- *     per device).  Make that first call during set-up, before any stream capture is begun.
+ *     per device ordinal, for the context current at that moment: a process that creates a second
+ *     context on the same device must not use this entry point from it).  Make that first call
+ *     during set-up, before any stream capture is begun.
  *   - Every call on a device uses the same array.  Each call clears the counters it needs and
  *     overwrites the rest before reading it, so calls that follow one another on a stream are
  *     independent; two calls that run on the GPU at the same time (different streams, or

@@ -4,6 +4,7 @@
 
 #include "device_resample.h"
 #include "dssd.h"
+#include "dssd_test_hooks.h"
 #include "edge_verify.h"
 #include "shard_verify.h"
 #include "topk_verify.h"
@@ -65,7 +66,8 @@ dssd_status edge_verify_any(const void *target_logits, dssd_dtype dtype, int64_t
                             const int32_t *draft_tokens, const float *draft_q_tok, const float *uniforms,
                             float temperature, int B, int gamma, int V, int32_t *accept_len, float *p_row,
                             uint16_t *p_row16, float *p_tok, float *lse, uint32_t *flags, void *workspace,
-                            size_t workspace_bytes, void *cuda_stream)
+                            size_t workspace_bytes, void *cuda_stream, long long drop_row_plus1 = 0,
+                            unsigned poll_limit = 0)
 {
     t_last_cuda_error = 0;
     dssd_status st = check_sizes(B, gamma, V);
@@ -99,10 +101,28 @@ dssd_status edge_verify_any(const void *target_logits, dssd_dtype dtype, int64_t
     P.p_tok = p_tok;
     P.lse = lse;
     P.flags = flags;
+    P.test_drop_row_plus1 = drop_row_plus1;
+    P.test_poll_limit = poll_limit;
     cudaError_t e = dssd::edge_verify_launch(P, (int)dtype, workspace, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
 }
 }  // namespace
+
+dssd_status dssd_test_edge_verify_wait_runs_out(const void *target_logits, dssd_dtype dtype,
+                                                int64_t row_stride, const int32_t *draft_tokens,
+                                                const float *draft_q_tok, const float *uniforms,
+                                                float temperature, int B, int gamma, int V,
+                                                int32_t *accept_len, float *p_row, uint32_t *flags,
+                                                void *workspace, size_t workspace_bytes,
+                                                long long drop_row, unsigned poll_limit,
+                                                void *cuda_stream)
+{
+    if (!p_row) return DSSD_ERR_INVALID_ARG;
+    if (check_sizes(B, gamma, V) == DSSD_OK && (drop_row < 0 || drop_row >= (long long)B * (gamma + 1))) return DSSD_ERR_INVALID_ARG;
+    return edge_verify_any(target_logits, dtype, row_stride, draft_tokens, draft_q_tok, uniforms, temperature, B, gamma,
+                           V, accept_len, p_row, nullptr, nullptr, nullptr, flags, workspace, workspace_bytes, cuda_stream,
+                           drop_row + 1, poll_limit);
+}
 
 dssd_status dssd_edge_verify(const void *target_logits, dssd_dtype dtype, int64_t row_stride,
                              const int32_t *draft_tokens, const float *draft_q_tok,
@@ -137,7 +157,8 @@ size_t dssd_device_resample_workspace_bytes(int B, int gamma, int V)
 namespace {
 dssd_status device_resample_any(const void *p_row, int p_half, const float *draft_q, const int32_t *accept_len,
                                 const float *uniforms, int B, int gamma, int V, int32_t *token, uint32_t *flags,
-                                void *workspace, size_t workspace_bytes, void *cuda_stream, int select = 0)
+                                void *workspace, size_t workspace_bytes, void *cuda_stream, int select = 0,
+                                int drop_seq_plus1 = 0, unsigned poll_limit = 0)
 {
     t_last_cuda_error = 0;
     dssd_status st = check_sizes(B, gamma, V);
@@ -162,10 +183,25 @@ dssd_status device_resample_any(const void *p_row, int p_half, const float *draf
     P.select = select;
     P.token = token;
     P.flags = flags;
+    P.test_drop_seq_plus1 = drop_seq_plus1;
+    P.test_poll_limit = poll_limit;
     cudaError_t e = dssd::resample_launch(P, workspace, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? DSSD_OK : cuda_fail(e);
 }
 }  // namespace
+
+dssd_status dssd_test_device_resample_wait_runs_out(const float *p_row, const float *draft_q,
+                                                    const int32_t *accept_len,
+                                                    const float *uniforms, int B, int gamma, int V,
+                                                    int32_t *token, uint32_t *flags,
+                                                    void *workspace, size_t workspace_bytes,
+                                                    int drop_seq, unsigned poll_limit,
+                                                    void *cuda_stream)
+{
+    if (B >= 1 && (drop_seq < 0 || drop_seq >= B)) return DSSD_ERR_INVALID_ARG;
+    return device_resample_any(p_row, 0, draft_q, accept_len, uniforms, B, gamma, V, token, flags, workspace,
+                               workspace_bytes, cuda_stream, 0, drop_seq + 1, poll_limit);
+}
 
 dssd_status dssd_device_resample(const float *p_row, const float *draft_q,
                                  const int32_t *accept_len, const float *uniforms, int B,

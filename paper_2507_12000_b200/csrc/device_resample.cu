@@ -20,6 +20,10 @@
 #include <limits.h>
 #include <math.h>
 
+#include <utility>
+
+#include <cooperative_groups.h>
+
 #include "dssd_device.cuh"
 
 namespace dssd {
@@ -282,10 +286,10 @@ __device__ __forceinline__ unsigned long long logical(unsigned long long raw) { 
 
 // chunk sum (b, c); a sum whose store has not landed yet still shows the fill pattern and is
 // polled for (bounded); when the wait runs out the fill pattern itself comes back (see timed_out)
-__device__ __forceinline__ double load_chunk_sum(const ResampleParams &P, const unsigned long long *cs, int c)
+__device__ __forceinline__ double load_chunk_sum(const ResampleParams &P, const unsigned long long *cs, int c, unsigned polls)
 {
     unsigned long long w = ld_relaxed_u64(cs + c);
-    for (unsigned it = 0; w == kFill64 && it < P.spin_limit; ++it) {
+    for (unsigned it = 0; w == kFill64 && it < polls; ++it) {
         __nanosleep(32);
         w = ld_relaxed_u64(cs + c);
     }
@@ -418,11 +422,12 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub;
+    const unsigned polls = b + 1 == (int64_t)P.test_drop_seq_plus1 ? P.test_poll_limit : P.spin_limit;
     for (int attempt = 0; attempt < 2; ++attempt) {
         bool ok;
         if (P.n_sub <= kThreads) {
             // one chunk per thread: a single scan gives Z and every inclusive prefix
-            const double m = tid < P.n_sub ? load_chunk_sum(P, cs, tid) : 0.0;
+            const double m = tid < P.n_sub ? load_chunk_sum(P, cs, tid, polls) : 0.0;
             if (give_up(P, b, timed_out(m), fl)) return;
             double Z;
             const double incl = block_scan(m, s_w, Z);
@@ -459,7 +464,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
         bool late = false;
         for (int base = 0; base < P.n_sub; base += kThreads) {
             const int c = base + tid;
-            const double m = c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0;
+            const double m = c < P.n_sub ? load_chunk_sum(P, cs, c, polls) : 0.0;
             late |= timed_out(m);
             double tot;
             block_scan(m, s_w, tot);
@@ -481,7 +486,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
             int my_first = 0x7fffffff, my_last = -1;
             for (int base = 0; base < P.n_sub; base += kThreads) {
                 const int c = base + tid;
-                const double m = c < P.n_sub ? load_chunk_sum(P, cs, c) : 0.0;
+                const double m = c < P.n_sub ? load_chunk_sum(P, cs, c, polls) : 0.0;
                 double tot;
                 const double incl = carry + block_scan(m, s_w, tot);
                 if (c < P.n_sub && incl > target && my_first == 0x7fffffff) {
@@ -545,23 +550,45 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
     __shared__ int s_first_n;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    // ---- the scratch is cleared here, by the kernel itself: every chunk sum to the all-ones pattern,
+    // the ticket counter to twice the number of CTAs (every CTA's first two tickets are its own
+    // number and that plus the number of CTAs), the draw counter to the number of CTAs when every
+    // sequence has a CTA of its own.  One grid-wide barrier (a cooperative launch: all CTAs are
+    // resident) separates the clearing from the first use; it is split around the first ticket's
+    // loads, which need nothing of the scratch. ----
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    const bool early = (unsigned long long)P.B <= (unsigned long long)gridDim.x;
+    {
+        uint4 *w = reinterpret_cast<uint4 *>(P.ticket);  // the scratch starts with the counters
+        const size_t nw = P.fill_bytes / 16;
+        for (size_t i = (size_t)blockIdx.x * kThreads + tid; i < nw; i += (size_t)gridDim.x * kThreads) {
+            uint4 v = make_uint4(~0u, ~0u, ~0u, ~0u);
+            if (i == 0) {  // raw value of a 64-bit counter: logical value - 1
+                const unsigned long long raw = 2ull * gridDim.x - 1ull;
+                v.x = (unsigned)raw;
+                v.y = (unsigned)(raw >> 32);
+            }
+            if (i == 8 && early) {  // the draw counter, 128 bytes on
+                v.x = gridDim.x - 1u;
+                v.y = 0u;
+            }
+            w[i] = v;
+        }
+    }
+    auto arrived = grid.barrier_arrive();
+    bool waited = false;
+
     // ---- pass A: chunk sums.  One barrier per ticket, no round trip waited for. ----
     unsigned long long next_raw = 0;  // thread 0: the ticket after the next one, drawn early
-    // thread 0: when there is at most one draw per CTA, this CTA's draw ticket is taken now, so that
-    // neither the ticket nor the sequence's accepted length and uniform are waited for when the
+    // when there is at most one draw per CTA, a CTA's draw is the sequence of its own number, so
+    // that neither a ticket nor the sequence's accepted length and uniform are waited for when the
     // draws begin (with more draws than CTAs the first ticket is taken when the draws begin, by
     // whoever gets there first)
-    const bool early = (unsigned long long)P.B <= (unsigned long long)gridDim.x;
-    unsigned long long draw_raw = 0;
+    const unsigned long long my_draw = blockIdx.x;
     int first_n = INT_MIN;  // not loaded
     float first_u = 0.f;
-    if (tid == 0) {
-        s_ticket[1] = logical(atomicAdd(P.ticket, 1ull));
-        next_raw = atomicAdd(P.ticket, 1ull);
-        if (early) draw_raw = atomicAdd(P.draw_ticket, 1ull);
-    }
-    __syncthreads();
-    unsigned long long t = s_ticket[1];
+    unsigned long long t = blockIdx.x;
     for (int it = 0; t < P.total_tickets; ++it) {
         const int buf = it & 1;
         const int64_t b = (int64_t)(t / (unsigned)P.n_chunks);
@@ -586,12 +613,16 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
             s_w[buf][warp][0] = acc0;
             s_w[buf][warp][1] = acc1;
         }
+        if (it == 0) {  // the first ticket's loads are done: from here on the scratch is used
+            grid.barrier_wait(std::move(arrived));
+            waited = true;
+        }
         if (tid == 0) {
-            s_ticket[buf] = logical(next_raw);
+            s_ticket[buf] = it == 0 ? t + gridDim.x : logical(next_raw);
             next_raw = atomicAdd(P.ticket, 1ull);
-            if (it == 0 && early && logical(draw_raw) < (unsigned long long)P.B) {
-                first_n = __ldg(P.accept_len + logical(draw_raw));
-                first_u = __ldg(P.uniforms + logical(draw_raw));
+            if (it == 0 && early && my_draw < (unsigned long long)P.B) {
+                first_n = __ldg(P.accept_len + my_draw);
+                first_u = __ldg(P.uniforms + my_draw);
             }
         }
         __syncthreads();
@@ -603,8 +634,10 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
                 tot1 += s_w[buf][w][1];
             }
             unsigned long long *cs = reinterpret_cast<unsigned long long *>(P.chunk_sum) + (size_t)b * P.n_sub + P.subs * c;
-            st_relaxed_u64(cs, (unsigned long long)__double_as_longlong(tot0));
-            if (P.subs == 2 && 2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
+            if (b + 1 != (int64_t)P.test_drop_seq_plus1) {  // (the test hook withholds these stores)
+                st_relaxed_u64(cs, (unsigned long long)__double_as_longlong(tot0));
+                if (P.subs == 2 && 2 * c + 1 < P.n_sub) st_relaxed_u64(cs + 1, (unsigned long long)__double_as_longlong(tot1));
+            }
         }
         t = s_ticket[buf];
     }
@@ -612,10 +645,10 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
     // ---- pass B: the draws, one sequence per ticket, once this CTA has no chunk left.  By then
     // the memory system is no longer saturated by the streams, so a draw's two round trips are
     // short; a chunk sum that has not landed yet is polled for (its CTA is still running). ----
+    if (!waited) grid.barrier_wait(std::move(arrived));
     __syncthreads();
     if (tid == 0) {
-        if (!early) draw_raw = atomicAdd(P.draw_ticket, 1ull);
-        s_ticket[0] = logical(draw_raw);
+        s_ticket[0] = early ? my_draw : logical(atomicAdd(P.draw_ticket, 1ull));
         s_first_n = first_n;
         s_first_u = first_u;
         next_raw = atomicAdd(P.draw_ticket, 1ull);
@@ -884,8 +917,8 @@ __global__ void __launch_bounds__(kThreads) shard_draw_kernel(const __grid_const
 
 size_t resample_workspace_layout(int B, int V, ResampleParams *P, char *base)
 {
-    // all of it is filled with 0xFF before the launch: counters then read "logical 0" (raw + 1)
-    // and the chunk sums read "not yet"
+    // the kernel sets all of it to 0xFF before use: counters then read "logical 0" (raw + 1) and
+    // the chunk sums read "not yet"
     size_t off = 0;
     auto take = [&](size_t bytes) {
         size_t o = off;
@@ -942,18 +975,21 @@ cudaError_t resample_launch(ResampleParams &P, void *workspace, cudaStream_t str
     }
     resample_workspace_layout(P.B, P.V, &P, static_cast<char *>(workspace));
     P.spin_limit = 1u << 20;
-    if ((err = cudaMemsetAsync(workspace, 0xFF, P.fill_bytes, stream)) != cudaSuccess) return err;
     const unsigned long long resident = (unsigned long long)sms * (unsigned long long)occ;
     const unsigned grid = (unsigned)(P.total_tickets < resident ? P.total_tickets : resident);
+    // a cooperative launch: all CTAs are resident at once (grid <= resident), which the kernel's
+    // grid-wide barrier after the clearing of the scratch relies on
+    const void *fn;
     if (P.logits) {
-        if (P.logits_dtype == DSSD_BF16) resample_kernel<RowLogits<DSSD_BF16>><<<grid, kThreads, 0, stream>>>(P);
-        else resample_kernel<RowLogits<DSSD_F32>><<<grid, kThreads, 0, stream>>>(P);
+        fn = P.logits_dtype == DSSD_BF16 ? reinterpret_cast<const void *>(resample_kernel<RowLogits<DSSD_BF16>>)
+                                         : reinterpret_cast<const void *>(resample_kernel<RowLogits<DSSD_F32>>);
     } else if (P.p_half) {
-        resample_kernel<RowF16><<<grid, kThreads, 0, stream>>>(P);
+        fn = reinterpret_cast<const void *>(resample_kernel<RowF16>);
     } else {
-        resample_kernel<RowF32><<<grid, kThreads, 0, stream>>>(P);
+        fn = reinterpret_cast<const void *>(resample_kernel<RowF32>);
     }
-    return cudaGetLastError();
+    void *args[] = {&P};
+    return cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kThreads), args, 0, stream);
 }
 
 size_t shard_resample_workspace_bytes(int B, int V)

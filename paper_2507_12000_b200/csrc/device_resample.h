@@ -39,6 +39,10 @@ struct ResampleParams {
     double *chunk_sum;   // [B, n_sub]
     size_t fill_bytes;
     unsigned spin_limit;
+    // test hook (0: off): the chunk sums of sequence test_drop_seq_plus1 - 1 are never stored, and its
+    // draw polls at most test_poll_limit times for a chunk sum
+    int test_drop_seq_plus1;
+    unsigned test_poll_limit;
 };
 
 // Carves the scratch (its size does not depend on P->subs, which the caller sets before: 1 or 2).

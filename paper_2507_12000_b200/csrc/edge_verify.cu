@@ -427,28 +427,35 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
         int x = -1;
         float zx = 0.f, qx = 0.f, ux = 0.f;
         bool owned = false;
-        if (live && i < P.gamma) {
-            const size_t di = (size_t)b * P.gamma + i;
-            x = P.draft_tokens[di];
-            if (P.uniforms) ux = P.uniforms[di];
-            if (P.shard_sum) {
-                // partial sums only: no test here
-            } else if (P.draft_q_rows) {
-                // a token id outside the vocabulary has no q: NaN (the id itself gets the position rejected and flagged)
-                qx = (x >= 0 && x < P.V) ? __ldg(P.draft_q_rows + di * (size_t)P.V + (size_t)x) : __int_as_float(0x7fc00000);
-            } else {
-                qx = P.draft_q_tok[di];
-            }
-            // (a shard of the vocabulary holds entries v_begin .. v_begin + V - 1; v_begin is 0 otherwise)
-            const long long xl = (long long)x - (long long)P.v_begin;
-            owned = xl >= 0 && xl < (long long)P.V;
-            if (owned) zx = E::load(row_ptr<DT>(P, row), xl);
+        unsigned long long tz = 0ull, tq = 0ull;
+        const bool tested = live && i < P.gamma;
+        if (tested) {
+            // the drafted token's logit, q_i(x_i) and u_i were looked up by the scout that drew the row's
+            // first ticket and wait in the row's two slots: nothing here goes to DRAM or depends on another load
+            tz = ld_relaxed_u64(P.tokz + row);
+            tq = ld_relaxed_u64(P.tokq + row);
         }
         // The sequence's arrival counter says every ticket has been counted; a partial whose
         // store has not landed yet still shows the fill pattern and is polled for.
         float Rr = DSSD_NEG_INF;
         double S = 0.0;
         bool bad = false, timeout = false;
+        if (tested) {
+            for (unsigned it = 0; (unsigned)(tz >> 32) == kFull && it < P.spin_limit; ++it) {
+                __nanosleep(32);
+                tz = ld_relaxed_u64(P.tokz + row);
+            }
+            for (unsigned it = 0; (unsigned)(tq >> 32) == kFull && it < P.spin_limit; ++it) {
+                __nanosleep(32);
+                tq = ld_relaxed_u64(P.tokq + row);
+            }
+            if ((unsigned)(tz >> 32) == kFull || (unsigned)(tq >> 32) == kFull) timeout = true;
+            owned = (unsigned)(tz >> 32) == 1u;  // the token lies in this row (this shard's slice of it)
+            x = owned ? 0 : -1;                  // all that the test needs to know of the id
+            zx = __uint_as_float((unsigned)tz);
+            qx = __uint_as_float((unsigned)tq);
+            ux = __uint_as_float((unsigned)(tq >> 32));
+        }
         if (live) {
             for (int k = 0; k < P.n_lse_runs; ++k) {
                 unsigned long long w = 0;
@@ -459,7 +466,8 @@ __device__ __noinline__ void fold_sequence(const EdgeParams &P, long long b)
                 } else {
                     w = ld_relaxed_u64(part + k);
                 }
-                for (unsigned it = 0; (unsigned)w == kFull && it < P.spin_limit; ++it) {
+                const unsigned polls = row + 1 == P.test_drop_row_plus1 ? P.test_poll_limit : P.spin_limit;
+                for (unsigned it = 0; (unsigned)w == kFull && it < polls; ++it) {
                     __nanosleep(32);
                     w = ld_relaxed_u64(part + k);
                 }
@@ -572,8 +580,9 @@ __device__ __forceinline__ void fold_warp(const EdgeParams &P, Shared *sh)
                 __threadfence_block();
                 *valid = 0;
                 ++*(volatile unsigned *)&sh->meet_gen[meet];  // the area may be used again
-                st_relaxed_u64(&P.part[(size_t)row * P.n_lse_runs + run],
-                               (unsigned long long)__float_as_uint(ref2) | ((unsigned long long)__float_as_uint(sum) << 32));
+                if (row + 1 != P.test_drop_row_plus1)  // (the test hook withholds this one store)
+                    st_relaxed_u64(&P.part[(size_t)row * P.n_lse_runs + run],
+                                   (unsigned long long)__float_as_uint(ref2) | ((unsigned long long)__float_as_uint(sum) << 32));
                 raw = atomicAdd(&P.seq_cnt[b], 1u);
             }
             if (npend == 0) {
@@ -1032,6 +1041,7 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
 template <int DT>
 __device__ __forceinline__ void scout_thread(const EdgeParams &P, Shared *sh)
 {
+    using E = Elem<DT>;
     Claim c;
     c.state = kWatch;
     c.exhausted = false;
@@ -1049,8 +1059,54 @@ __device__ __forceinline__ void scout_thread(const EdgeParams &P, Shared *sh)
                       *abort = &sh->abort;
     EmitWork w;
     bool have = false;  // a claimed, ready EMIT ticket waiting for room in the queue
+    // Whoever draws the first ticket of a row also looks up the row's drafted token and that token's
+    // logit (and, when the draft rows are given, its probability) and leaves them in the row's slots,
+    // long before the sequence is folded.  One look-up at a time: 0 idle, 1 the token id has been
+    // asked for, 2 the values have been asked for.
+    int pf = 0, pf_x = 0;
+    long long pf_row = 0;
+    size_t pf_di = 0;
+    float pf_z = 0.f, pf_q = 0.f, pf_u = 0.f;
+    bool pf_owned = false;
+    auto pf_advance = [&]() {
+        if (pf == 1) {
+            // (a shard of the vocabulary holds entries v_begin .. v_begin + V - 1; v_begin is 0 otherwise)
+            const long long xl = (long long)pf_x - (long long)P.v_begin;
+            pf_owned = xl >= 0 && xl < (long long)P.V;
+            pf_z = pf_owned ? E::load(row_ptr<DT>(P, pf_row), xl) : 0.f;
+            // a token id outside the vocabulary has no q: NaN (the id itself gets the position rejected and flagged)
+            if (P.draft_q_rows)
+                pf_q = (pf_x >= 0 && pf_x < P.V) ? __ldg(P.draft_q_rows + pf_di * (size_t)P.V + (size_t)pf_x) : __int_as_float(0x7fc00000);
+            pf = 2;
+        } else if (pf == 2) {
+            st_relaxed_u64(P.tokz + pf_row, (unsigned long long)__float_as_uint(pf_z) | ((unsigned long long)(pf_owned ? 1u : 0u) << 32));
+            // (q_i(x_i), u_i): a NaN is stored as the canonical one, so that the pair never equals the all-ones pattern
+            const float qs = pf_q != pf_q ? __int_as_float(0x7fc00000) : pf_q, us = pf_u != pf_u ? __int_as_float(0x7fc00000) : pf_u;
+            st_relaxed_u64(P.tokq + pf_row, (unsigned long long)__float_as_uint(qs) | ((unsigned long long)__float_as_uint(us) << 32));
+            pf = 0;
+        }
+    };
+    auto pf_start = [&](unsigned long long no) {
+        unsigned long long row;
+        int run;
+        split_ticket(no, P.n_lse_runs, P.lse_magic, row, run);
+        const unsigned i = (unsigned)(row % (unsigned)(P.gamma + 1));
+        if (run != 0 || (int)i >= P.gamma) return;
+        while (pf) pf_advance();
+        pf_row = (long long)row;
+        pf_di = (size_t)(row / (unsigned)(P.gamma + 1)) * (size_t)P.gamma + i;
+        pf_x = P.draft_tokens[pf_di];
+        pf_u = P.uniforms ? P.uniforms[pf_di] : 0.f;
+        if (P.draft_q_tok) pf_q = P.draft_q_tok[pf_di];
+        pf = 1;
+    };
+    if (more_lse) pf_start(blockIdx.x);
     for (;;) {
-        if (*abort) return;
+        if (*abort) {
+            while (pf) pf_advance();
+            return;
+        }
+        pf_advance();
         // the next LSE ticket: drawn as soon as the producer has taken the one before
         if (more_lse && !lse_pending && lse_pushed == *lse_popped) {
             lse_raw = atomicAdd(P.lse_ticket, 1ull);
@@ -1080,6 +1136,7 @@ __device__ __forceinline__ void scout_thread(const EdgeParams &P, Shared *sh)
             lse_pending = false;
             endgame = no + P.endgame_tickets >= P.total_lse;
             if (no >= P.total_lse) more_lse = false;
+            else pf_start(no);
             sh->lse_q[lse_pushed & (kLseQ - 1)] = no;  // a number beyond the last ticket tells the producer that none is left
             __threadfence_block();
             *(volatile unsigned *)&sh->lse_pushed = ++lse_pushed;
@@ -1087,12 +1144,13 @@ __device__ __forceinline__ void scout_thread(const EdgeParams &P, Shared *sh)
         }
         // done once no LSE ticket is left anywhere, no claim is under way, nothing waits here and every
         // EMIT ticket has been claimed by someone
-        if (!more_lse && !have && c.state == kWatch && (c.exhausted || logical(c.head_raw) >= P.total_emit)) {
+        if (!more_lse && !have && pf == 0 && c.state == kWatch && (c.exhausted || logical(c.head_raw) >= P.total_emit)) {
             __threadfence_block();
             *(volatile unsigned *)&sh->scout_done = 1u;
             return;
         }
         if (++idle > P.spin_limit) {
+            while (pf) pf_advance();
             *P.error = 1u;  // waited too long (for a sequence to become ready, or for the producer)
             *(volatile unsigned *)&sh->scout_done = 1u;
             return;
@@ -1413,7 +1471,11 @@ size_t edge_workspace_layout(int B, int gamma, int runs_per_row, EdgeParams *P, 
     const size_t o_seqcnt = take((size_t)B * 4);
     const size_t o_ready = take((size_t)B * sizeof(ReadySlot));
     const size_t o_part = take(R * (size_t)runs_per_row * 8);
+    const size_t o_tokz = take(R * 8);
+    const size_t o_tokq = take(R * 8);
     if (P) {
+        P->tokz = reinterpret_cast<unsigned long long *>(base + o_tokz);
+        P->tokq = reinterpret_cast<unsigned long long *>(base + o_tokq);
         P->lse_ticket = reinterpret_cast<unsigned long long *>(base + o_ctr);
         P->emit_head = reinterpret_cast<unsigned long long *>(base + o_ctr + 128);
         P->ready_count = reinterpret_cast<unsigned *>(base + o_ctr + 256);
@@ -1459,7 +1521,7 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
     // EMIT tickets, and what the draw needs about row n stays in the workspace (`ready`).
     const bool no_emit = !P.p_row && !P.p_row16;
     // small launches: a cluster of 1..8 CTAs per sequence, no workspace, one launch
-    if (!no_emit && !P.skip_bonus_row && !P.draft_q_rows && !P.shard_sum) {
+    if (!no_emit && !P.skip_bonus_row && !P.draft_q_rows && !P.shard_sum && !P.test_drop_row_plus1) {
         const long long seq_bytes = (long long)(P.gamma + 1) * P.V * esz;
         int csize = 1;
         while (csize < kSmallMaxCluster && seq_bytes / csize > kSmallCtaBytes) csize *= 2;

@@ -90,6 +90,10 @@ struct EdgeParams {
     unsigned long long endgame_tickets;  // EMIT claims are held back once so few LSE tickets are left
     unsigned long long lse_magic, emit_magic;  // ceil(2^64 / n_*_runs) when multiply-high division is exact, else 0
     unsigned spin_limit;
+    // test hook (0: off): the partial sums of row test_drop_row_plus1 - 1 are counted but never stored,
+    // and the fold polls at most test_poll_limit times for that row's partial sums
+    long long test_drop_row_plus1;
+    unsigned test_poll_limit;
     // workspace, set to 0xFF by the kernel before use: counters then read "logical 0" (raw + 1)
     // and 8-byte slots read "not yet" until their one store has landed
     unsigned long long *lse_ticket;  // next LSE ticket
@@ -98,6 +102,8 @@ struct EdgeParams {
     unsigned *error;                 // all ones = no error
     unsigned *seq_cnt;               // [B] LSE tickets of the sequence that have arrived
     unsigned long long *part;        // [rows, n_lse_runs] (ref2, sum) of one ticket
+    unsigned long long *tokz;        // [rows] (logit of the row's drafted token, 1 if the token lies in the row else 0)
+    unsigned long long *tokq;        // [rows] (q_i(x_i), u_i) of the row's position, NaNs canonical
     ReadySlot *ready;                // [B] indexed by sequence
     size_t fill_bytes;
 };

@@ -20,9 +20,14 @@ def B():
 
 
 def _declared():
-    src = open(os.path.join(ROOT, "include", "dssd.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(dssd_[a-z_0-9]+)\s*\(", src)))
+    """Every function that a header under include/ declares."""
+    import glob
+
+    names = set()
+    for path in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        src = re.sub(r"/\*.*?\*/", "", open(path).read(), flags=re.S)
+        names.update(re.findall(r"\b(dssd_[a-z_0-9]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(B):

@@ -103,3 +103,21 @@ def test_two_ranks_shard_by_vocabulary(tmp_path, oracle_mod):
     mp.spawn(_vocab_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     ok = np.load(tmp_path / "ok.npy")
     assert ok.tolist() == [1, 1, 1, 1]
+
+
+def test_bench_starts_its_own_ranks(oracle_mod):
+    """`bench.py --gpus 2` started by hand (no launcher, no WORLD_SIZE) re-executes itself under
+    torch.distributed.run with two ranks; with the reference arm rank 0 alone works and prints the one
+    JSON line, the other rank leaves with status 0."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload",
+                          "c1", "--steps", "1", "--warmup", "0"], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE,
+                         text=True, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["metric"] == "verified_rows_per_s"
