@@ -41,15 +41,21 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 451.6 MB read + 96.4 MB written
-    "c4": {"bytes": 548060928, "kernel_hash": "42fad7757195ce25"},
+    # profiles/edge_verify_kernel_c4.md: 456.2 MB read (389.0 MB of logits + 86 % of the second read of row n)
+    # and 96.9 MB written inside the kernel; the other 58.7 MB of p_row were still in L2 when the kernel ended
+    # and reach DRAM after it.  "bytes" counts all of p_row.
+    "c4": {"bytes": 456184320 + 155582464, "kernel_hash": "3a25cc07efade786",
+           "note": "dram__bytes_read.sum 456.2 MB + all 155.6 MB of p_row (96.9 MB of it written inside the "
+                   "kernel, the rest still in L2 at its end); reads are 1.17x the logits: the second read of "
+                   "row n misses L2 for 86 % of its bytes",
+           "counted_inside_kernel": 456184320 + 96895744},
 }
 
 
 # the same for topk_verify_kernel (k = 10)
 NCU_TRAFFIC_TOPK = {
-    # profiles/topk_verify_kernel_c4.md: 389.3 MB read + 5.9 MB written
-    "c4": {"bytes": 395289856, "kernel_hash": "d5288d706b12c071"},
+    # profiles/topk_verify_kernel_c4.md: 389.5 MB read + 7.5 MB written
+    "c4": {"bytes": 389480960 + 7505152, "kernel_hash": "ebb49caf8f4fc5d4"},
 }
 
 
@@ -63,7 +69,7 @@ def _kernel_hash_topk() -> str:
 
 def _kernel_hash() -> str:
     h = hashlib.sha256()
-    for f in ("edge_verify.cu", "edge_verify.h", "dssd_device.cuh"):
+    for f in ("edge_verify.cu", "edge_verify.h", "edge_judge.cuh", "dssd_device.cuh"):
         with open(os.path.join(ROOT, "paper_2507_12000_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -216,11 +222,13 @@ def _config(w: di.Workload, args):
 MIN_TIMED_MS = 300.0  # device time the timed loops add up to at least
 
 
-def timed_loops(one_loop, min_ms: float = MIN_TIMED_MS, max_loops: int = 400):
+def timed_loops(one_loop, min_ms: float = None, max_loops: int = 400):
     """one_loop() times exactly K steps on the device and returns a dict with "total_ms" (already the
     maximum over ranks).  It is repeated until the loops add up to min_ms of device time, so that the
     clock samples and the average rest on more than a few milliseconds; the reported loop is the
     median one.  Returns (median loop, all loops)."""
+    if min_ms is None:
+        min_ms = MIN_TIMED_MS
     first = one_loop()
     n = int(min(max_loops, max(1, math.ceil(min_ms / max(first["total_ms"], 1e-3)))))
     loops = [first] + [one_loop() for _ in range(n - 1)]
@@ -464,7 +472,8 @@ def run_ours(args, w: di.Workload, light: bool = False):
                      "algorithmic_bytes_per_launch": edge_bytes, "avg_launch_ms": edge_avg_ms,
                      "min_launch_ms": min(edge_ms),
                      "traffic": None if traffic is None else traffic["bytes"],
-                     "traffic_note": None if traffic is None else traffic.get("note")},
+                     "traffic_note": None if traffic is None else traffic.get("note"),
+                     "traffic_counted_inside_kernel": None if traffic is None else traffic.get("counted_inside_kernel")},
         "resample": {"avg_launch_ms": rs_avg_ms, "algorithmic_bytes_per_launch": rs_bytes,
                      "achieved_gbs": rs_bytes / (rs_avg_ms * 1e-3) / 1e9,
                      "frac": rs_bytes / (rs_avg_ms * 1e-3) / 1e9 / peak,
@@ -1013,11 +1022,15 @@ def main():
                          "(dssd_edge_verify), or the edge itself with no row emitted (dssd_edge_verify_bonus)")
     ap.add_argument("--k", type=int, default=10)
     ap.add_argument("--payload", default="f32", choices=["f32", "f16"], help="width of the emitted row P_n (full sampler only)")
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="the timed loop of --steps steps is repeated until this much device time has passed (0: once)")
+    ap.add_argument("--sweep", action="store_true", help="the 60 points of the V = 50272 float32 sweep, one record each")
     ap.add_argument("--shards", type=int, default=0,
                     help="time one shard of the vocabulary-sharded round (the vocabulary cut into this many slices)")
     ap.add_argument("--also", default="c5max,c3",
                     help="workloads measured after the default one and reported as sub-records (empty: none)")
     args = ap.parse_args()
+    globals()["MIN_TIMED_MS"] = args.min_timed_ms
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # started by hand rather than by a launcher: become the launcher, one rank per GPU of this node
         import socket
@@ -1039,6 +1052,19 @@ def main():
         (run_reference_topk if args.impl == "reference" else run_ours_topk)(args, w)
     elif args.impl == "reference":
         run_reference(args, w)
+    elif args.sweep:
+        # every point of the V = 50272 float32 sweep, one compact record each, in one JSON line
+        recs = []
+        for pt in di.sweep_points():
+            r = run_ours(args, pt, light=True)
+            if r is not None:
+                recs.append({"workload": pt.name, "B": pt.B, "gamma": pt.gamma, "sigma_d": pt.sigma_d,
+                             "edge_call_us": r["roofline"]["avg_launch_ms"] * 1e3, "frac": r["roofline"]["frac"],
+                             "achieved_gbs": r["roofline"]["achieved"], "resample_call_us": r["resample"]["avg_launch_ms"] * 1e3,
+                             "step_us": r["ms_per_step"] * 1e3, "rows_per_s": r["value"], "parity": r["parity"],
+                             "sm_mhz": r["clocks"]["sm_mhz"], "reasons": r["clocks"]["reasons"]})
+        if recs:
+            print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "sweep": recs}))
     else:
         line = run_ours(args, w)
         if line is not None and args.also and args.workload == "c4" and args.gpus == 1 and args.payload == "f32" \

@@ -24,14 +24,14 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > os.path.getmtime(LIB) for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, out: str = LIB, defines=()) -> str:
-    """Compile the library; `defines` are extra -D macros (tuning constants), `out` the .so path."""
-    if out == LIB and not defines and not force and not _stale():
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the library in-tree (nvcc cross-compiles sm_100a without a GPU)."""
+    if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", out] + [f"-D{d}" for d in defines] + sources()
+           "-o", LIB] + sources()
     if verbose:
         cmd += ["-Xptxas", "-v"]
     res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
@@ -39,7 +39,7 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, defines=()
         sys.stderr.write(res.stdout)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed building libdssd.so")
-    return out
+    return LIB
 
 
 if __name__ == "__main__":

@@ -30,12 +30,8 @@ namespace dssd {
 
 namespace {
 
-#ifndef DSSD_RS_WIDE
-#define DSSD_RS_WIDE 1  // whole tickets request all their loads at once (ticket_mass2)
-#endif
-#ifndef DSSD_RS_CTAS
-#define DSSD_RS_CTAS 4
-#endif
+constexpr bool kWideTickets = true;  // whole tickets request all their loads at once (ticket_mass2)
+constexpr int kResampleCtas = 4;      // resident CTAs per SM aimed at
 constexpr int kSub = kResampleSub;         // entries per chunk sum: a ticket covers P.subs of them
 constexpr int kRun = kSub / kThreads;      // contiguous entries per thread in pass B
 static_assert(kRun == 16, "pass B fetches a run as one group of 16 entries");
@@ -539,7 +535,7 @@ __device__ void draw(const ResampleParams &P, int64_t b, const RV &row, const fl
 }
 
 template <typename RV>
-__global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const __grid_constant__ ResampleParams P)
+__global__ void __launch_bounds__(kThreads, kResampleCtas) resample_kernel(const __grid_constant__ ResampleParams P)
 {
     __shared__ double s_w[2][kWarps][2];
     __shared__ double s_scan[kWarps];
@@ -600,7 +596,7 @@ __global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) resample_kernel(const 
             const float *q = n < P.gamma ? P.draft_q + ((size_t)b * P.gamma + n) * (size_t)P.V : nullptr;
             const int e0 = c * P.subs * kSub, e1 = min(P.V, e0 + kSub), e2 = min(P.V, e0 + P.subs * kSub);
             static_assert(kSub == 4 * 4 * kThreads, "a thread's four quads per chunk sum");
-            if (DSSD_RS_WIDE && e2 - e0 == 2 * kSub && row.aligned(e0) && (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0)) {
+            if (kWideTickets && e2 - e0 == 2 * kSub && row.aligned(e0) && (!q || (reinterpret_cast<uintptr_t>(q + e0) & 15u) == 0)) {
                 ticket_mass2(row, q, e0, acc0, acc1);
             } else {
                 acc0 = chunk_mass(row, q, e0, e1);
@@ -740,7 +736,7 @@ __device__ __forceinline__ RowF32 shard_row(const ShardResampleParams &P, int64_
     return r;
 }
 
-__global__ void __launch_bounds__(kThreads, DSSD_RS_CTAS) shard_mass_kernel(const __grid_constant__ ShardResampleParams P)
+__global__ void __launch_bounds__(kThreads, kResampleCtas) shard_mass_kernel(const __grid_constant__ ShardResampleParams P)
 {
     __shared__ double s_w[kWarps][2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1007,7 +1003,7 @@ cudaError_t shard_mass_launch(ShardResampleParams &P, void *workspace, cudaStrea
     P.n_sub = (P.V + kResampleSub - 1) / kResampleSub;
     P.chunk_sum = static_cast<double *>(workspace);
     const long long total = (long long)P.B * P.n_sub;
-    const long long resident = (long long)(sms < 1 ? 1 : sms) * DSSD_RS_CTAS;
+    const long long resident = (long long)(sms < 1 ? 1 : sms) * kResampleCtas;
     shard_mass_kernel<<<(unsigned)(total < resident ? total : resident), kThreads, 0, stream>>>(P);
     if ((err = cudaGetLastError()) != cudaSuccess) return err;
     shard_total_kernel<<<(unsigned)((P.B + kWarps - 1) / kWarps), kThreads, 0, stream>>>(P);

@@ -1,11 +1,13 @@
 // Edge half of the verification round as one persistent, warp-specialised streaming kernel.
 //
-// One CTA per SM.  Warp 0 is the producer: its lane 0 draws tickets from global counters and
-// streams the logits global -> shared memory with bulk asynchronous copies (TMA, untiled) into a
-// ring of kEdgeStages stages, each guarded by a "full" mbarrier (armed with the copy's bytes) and
-// an "empty" mbarrier (one arrival per consumer warp).  Warps 1..kEdgeConsumers are consumers:
-// every consumer takes a fixed 1/kEdgeConsumers share of each stage.  The last warp is the fold
-// warp, which serves a mailbox in shared memory.
+// One CTA per SM, launched cooperatively.  Lane 0 of warp 0 is the producer: it streams the logits
+// global -> shared memory with bulk asynchronous copies (TMA, untiled) into a ring of kEdgeStages
+// stages, each guarded by a "full" mbarrier (armed with the copy's bytes) and an "empty" mbarrier
+// (one arrival per consumer warp).  Warps 1..kEdgeConsumers are consumers: every consumer takes a
+// fixed 1/kEdgeConsumers share of each stage.  Then come the fold warp, which serves a mailbox in
+// shared memory, and the scout warp, one thread of which does every round trip to global memory
+// that scheduling needs (ticket draws, claims on EMIT work, look-ups of the drafted tokens) and
+// hands the results to the producer through two small queues in shared memory.
 //   LSE(row, run)    a run of consecutive stages of one target row (the whole row when it is
 //                    short enough): every consumer keeps, per lane, an online maximum and sum of
 //                    2^(l * c1 - ref2) in float32 over its shares.  At the run's last stage the
@@ -19,20 +21,18 @@
 // warp that brings a sequence's last partial folds the sequence: one lane per position adds up
 // the row's partials in float64 and evaluates the acceptance test, a ballot + find-first-set
 // over the lanes gives the accepted length n, and the sequence's `ready` entry (n and row n's
-// reference and 1/S) is written.  Producers claim EMIT tickets with one atomic add when ready
-// sequences have unclaimed tickets (or eagerly once they have no LSE work left); an EMIT ticket
-// goes before the next LSE stage, so the second read of row n follows the first as closely as
-// the fold allows.
+// reference and 1/S) is written.  Scouts claim EMIT tickets with one atomic add when ready
+// sequences have unclaimed tickets (or eagerly once their CTA has no LSE work left); an EMIT
+// ticket goes before the next LSE stage, so the second read of row n follows the first as closely
+// as the fold allows.
 // Nothing on the global path waits on a fence: results travel through 8-byte slots that carry
 // their own validity (the kernel itself sets the whole workspace to all ones before any CTA uses
-// it: one grid-wide barrier at the start of a cooperative launch, overlapped with the first
-// copies); a reader that sees the fill pattern asks again (bounded) for a store that a running
-// warp has already issued.  Values that
-// a thread will need later (ticket numbers, counters, `ready` entries) are requested one step
-// ahead and looked at one step later, so no round trip is waited for while streaming.
-// A producer only ever waits for work held by running CTAs, and never while its own CTA holds
-// unprocessed stages, so the kernel needs no co-residency guarantee.  Every wait is bounded;
-// when one runs out the error word is set and the warps wind down.
+// it: one grid-wide barrier at the start of the launch, overlapped with the first copies); a
+// reader that sees the fill pattern asks again (bounded) for a store that a running warp has
+// already issued.  The producer never touches global memory except to issue copies, so a freed
+// stage of the ring is re-armed at once.  Apart from that start-up barrier, which the
+// cooperative launch guarantees to complete, every wait is bounded; when one runs out the error
+// word is set and the warps wind down.
 #include "edge_verify.h"
 
 #include <math.h>
@@ -1174,11 +1174,8 @@ constexpr int kSmallThreads = 1024;
 constexpr int kSmallWarps = kSmallThreads / 32;
 constexpr int kSmallMaxRows = 64;                 // gamma + 1 at most
 constexpr int kSmallMaxCluster = 8;               // CTAs per sequence at most (the portable cluster size)
-#ifndef DSSD_EDGE_SMALL_CTA_BYTES
-#define DSSD_EDGE_SMALL_CTA_BYTES (128 << 10)
-#endif
 constexpr long long kSmallCtaBytes = 32 << 10;                        // share of a sequence aimed at per CTA
-constexpr long long kSmallMaxCtaBytes = DSSD_EDGE_SMALL_CTA_BYTES;   // ... and the most a CTA takes
+constexpr long long kSmallMaxCtaBytes = 128 << 10;   // ... and the most a CTA takes
 
 template <int DT>
 __global__ void __launch_bounds__(kSmallThreads, 1) edge_small_kernel(const __grid_constant__ EdgeParams P)

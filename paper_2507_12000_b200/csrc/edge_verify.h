@@ -7,45 +7,17 @@
 
 namespace dssd {
 
-#ifndef DSSD_EDGE_CONSUMERS
-#define DSSD_EDGE_CONSUMERS 16
-#endif
-#ifndef DSSD_EDGE_STAGE_BYTES
-#define DSSD_EDGE_STAGE_BYTES 32768
-#endif
-#ifndef DSSD_EDGE_STAGES
-#define DSSD_EDGE_STAGES 6
-#endif
-#ifndef DSSD_EDGE_MAX_RUN
-#define DSSD_EDGE_MAX_RUN 32
-#endif
-#ifndef DSSD_EDGE_EMIT_RUN
-#define DSSD_EDGE_EMIT_RUN 2
-#endif
-#ifndef DSSD_EDGE_TICKETS_PER_CTA
-#define DSSD_EDGE_TICKETS_PER_CTA 2
-#endif
-
-#ifndef DSSD_EDGE_ENDGAME_WAVES
-#define DSSD_EDGE_ENDGAME_WAVES 3
-#endif
-#ifndef DSSD_EDGE_ENDGAME_LONG_WAVES
-#define DSSD_EDGE_ENDGAME_LONG_WAVES 32
-#endif
-#ifndef DSSD_EDGE_ENDGAME_LONG_EIGHTHS
-#define DSSD_EDGE_ENDGAME_LONG_EIGHTHS 7
-#endif
-constexpr int kEdgeEndgameWaves = DSSD_EDGE_ENDGAME_WAVES;  // EMIT claims are held back during the last so many waves of LSE tickets
+constexpr int kEdgeEndgameWaves = 3;  // EMIT claims are held back during the last so many waves of LSE tickets
 constexpr int kEdgeEndgameLongRows = 8;                                  // ... with at least so many positions per sequence ...
-constexpr int kEdgeEndgameLongWaves = DSSD_EDGE_ENDGAME_LONG_WAVES;      // launches of at least so many waves ...
-constexpr int kEdgeEndgameLongEighths = DSSD_EDGE_ENDGAME_LONG_EIGHTHS;  // ... hold them back during the last so many eighths of the waves
-constexpr int kEdgeConsumers = DSSD_EDGE_CONSUMERS;      // consumer warps per CTA
+constexpr int kEdgeEndgameLongWaves = 32;      // launches of at least so many waves ...
+constexpr int kEdgeEndgameLongEighths = 7;  // ... hold them back during the last so many eighths of the waves
+constexpr int kEdgeConsumers = 16;      // consumer warps per CTA
 constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 3);  // + the producer warp, the fold warp and the scout warp
-constexpr int kEdgeStageBytes = DSSD_EDGE_STAGE_BYTES;   // logits bytes per ring stage (one bulk copy)
-constexpr int kEdgeStages = DSSD_EDGE_STAGES;            // ring stages per CTA
-constexpr int kEdgeMaxRun = DSSD_EDGE_MAX_RUN;           // most consecutive stages of a row in one ticket
-constexpr int kEdgeEmitRun = DSSD_EDGE_EMIT_RUN;        // most stages of row n in one EMIT ticket
-constexpr int kEdgeTicketsPerCta = DSSD_EDGE_TICKETS_PER_CTA;  // tickets aimed at per resident CTA
+constexpr int kEdgeStageBytes = 32768;   // logits bytes per ring stage (one bulk copy)
+constexpr int kEdgeStages = 6;            // ring stages per CTA
+constexpr int kEdgeMaxRun = 32;           // most consecutive stages of a row in one ticket
+constexpr int kEdgeEmitRun = 2;        // most stages of row n in one EMIT ticket
+constexpr int kEdgeTicketsPerCta = 2;  // tickets aimed at per resident CTA
 
 // What the emission of row P_n needs to know about a folded sequence: two 8-byte slots, each
 // valid once it differs from the all-ones pattern the kernel clears the workspace to.

@@ -46,6 +46,9 @@
 // Device kernel: one warp per sequence, everything in registers and shuffles, sums strictly
 // sequential in float64 so that the draw is reproducible bit for bit.
 #include <atomic>
+#include <utility>
+
+#include <cooperative_groups.h>
 #include "topk_verify.h"
 
 #include <math.h>
@@ -55,31 +58,16 @@
 namespace dssd {
 namespace {
 
-#ifndef DSSD_TOPK_CONS_WARPS
-#define DSSD_TOPK_CONS_WARPS 4
-#endif
-#ifndef DSSD_TOPK_STAGE_BYTES
-#define DSSD_TOPK_STAGE_BYTES 16384
-#endif
-#ifndef DSSD_TOPK_STAGES
-#define DSSD_TOPK_STAGES 3
-#endif
-#ifndef DSSD_TOPK_MIN_CTAS
-#define DSSD_TOPK_MIN_CTAS 4
-#endif
-constexpr int kConsWarps = DSSD_TOPK_CONS_WARPS;      // consumer warps per CTA (a power of two, 4..16)
+constexpr int kConsWarps = 4;      // consumer warps per CTA (a power of two, 4..16)
 constexpr int kConsThreads = 32 * kConsWarps;
 constexpr int kTkThreads = kConsThreads + 64;        // + the producer warp and the selection warp
-constexpr int kStages = DSSD_TOPK_STAGES;            // ring stages per CTA
-constexpr int kStageBytes = DSSD_TOPK_STAGE_BYTES;   // logits bytes per stage (one bulk copy)
+constexpr int kStages = 3;            // ring stages per CTA
+constexpr int kStageBytes = 16384;   // logits bytes per stage (one bulk copy)
 constexpr int kStageVecs = kStageBytes / 16;         // 16-byte vectors per stage
 constexpr int kU = kStageVecs / kConsThreads;        // vectors per consumer thread per stage
 constexpr int kGroup = kConsThreads / 32;            // threads per group of the first threshold
 static_assert(kU >= 1 && kU * kConsThreads == kStageVecs && kGroup >= 4 && kGroup <= 16, "stage / consumer shape");
-#ifndef DSSD_TOPK_QUEUE
-#define DSSD_TOPK_QUEUE 32
-#endif
-constexpr int kCap = DSSD_TOPK_QUEUE;                // candidate keys per consumer warp and channel (32: one batch of the selection warp)
+constexpr int kCap = 32;                // candidate keys per consumer warp and channel (32: one batch of the selection warp)
 constexpr unsigned kSpinLimit = 1u << 16;            // tries of a bounded wait (about 4 us each)
 constexpr unsigned kSpinLimitAborted = 8u;           // after a wait has run out
 constexpr unsigned long long kBadList = ~0ull;  // first key of a piece that held a NaN or +inf
@@ -366,21 +354,31 @@ __device__ __forceinline__ void ring_wait(const TopkParams &P, Smem &S, unsigned
 }
 
 // The producer thread: streams the CTA's span, stage by stage, in the order the consumers read it.
+// It can stop after a given number of stages and be resumed (the first stages go out before the
+// grid-wide barrier at the start of the kernel, the rest after it).
+struct ProducerPos {
+    unsigned long long blk;  // first block of the piece in progress
+    int s;                   // next stage of that piece
+    unsigned q;              // stages issued so far
+};
+
 template <int DT>
-__device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, unsigned long long blk, unsigned long long blk_end)
+__device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, ProducerPos &pos, unsigned long long blk_end,
+                         unsigned q_stop)
 {
-    unsigned q = 0;  // stages issued so far
-    while (blk < blk_end) {
-        const Piece pc = piece_at<DT>(P, blk, blk_end);
-        for (int s = 0; s < pc.stages; ++s, ++q) {
-            const unsigned slot = q % kStages, pass = q / kStages;
+    while (pos.blk < blk_end) {
+        const Piece pc = piece_at<DT>(P, pos.blk, blk_end);
+        for (; pos.s < pc.stages; ++pos.s, ++pos.q) {
+            if (pos.q == q_stop) return;
+            const unsigned slot = pos.q % kStages, pass = pos.q / kStages;
             if (pass > 0) ring_wait(P, S, &S.empty[slot], (pass - 1u) & 1u);
-            const uint32_t bytes = (uint32_t)min(kStageVecs, pc.nvec - s * kStageVecs) * 16u;
+            const uint32_t bytes = (uint32_t)min(kStageVecs, pc.nvec - pos.s * kStageVecs) * 16u;
             const uint32_t bar = smem_addr(&S.full[slot]);
             mbar_arrive_expect_tx(bar, bytes);
-            bulk_g2s(ring + slot * (uint32_t)kStageBytes, pc.vp + (size_t)s * kStageVecs, bytes, bar);
+            bulk_g2s(ring + slot * (uint32_t)kStageBytes, pc.vp + (size_t)pos.s * kStageVecs, bytes, bar);
         }
-        blk += (unsigned long long)(pc.lb - pc.fb);
+        pos.s = 0;
+        pos.blk += (unsigned long long)(pc.lb - pc.fb);
     }
 }
 
@@ -736,7 +734,7 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_kernel(const __grid_constant__ TopkParams P)
+__global__ void __launch_bounds__(kTkThreads, 4) topk_verify_kernel(const __grid_constant__ TopkParams P)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem &S = *reinterpret_cast<Smem *>(smem_raw + (size_t)kStages * kStageBytes);
@@ -759,16 +757,32 @@ __global__ void __launch_bounds__(kTkThreads, DSSD_TOPK_MIN_CTAS) topk_verify_ke
         S.abort = 0;
         mbar_init_fence();
     }
-    __syncthreads();
+    // The error word and the sequences' block counters are zeroed here, by the kernel itself: one
+    // grid-wide barrier (a cooperative launch: all CTAs are resident) separates that from their first
+    // use, and it is split around the producer's first copies, which need nothing of the workspace.
+    namespace cg = cooperative_groups;
+    cg::grid_group grid = cg::this_grid();
+    {
+        unsigned long long *z = reinterpret_cast<unsigned long long *>(P.error);
+        const size_t nz = P.zero_bytes / 8;
+        for (size_t i = (size_t)blockIdx.x * kTkThreads + tid; i < nz; i += (size_t)gridDim.x * kTkThreads) z[i] = 0ull;
+    }
+    auto arrived = grid.barrier_arrive();  // (a CTA-wide barrier is part of it)
     const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
     const unsigned long long blk_end = (c + 1ull) * TB / G;
     unsigned long long blk = c * TB / G;
+    ProducerPos pos;
+    pos.blk = blk;
+    pos.s = 0;
+    pos.q = 0;
+    if (tid == kConsThreads) producer<DT>(P, S, ring, pos, blk_end, (unsigned)kStages);  // the ring is empty: nothing is waited for
+    grid.barrier_wait(std::move(arrived));
     if (tid >= kConsThreads + 32) {
         selection_warp<DT>(P, S, blk, blk_end);
         return;
     }
     if (tid >= kConsThreads) {
-        if (tid == kConsThreads) producer<DT>(P, S, ring, blk, blk_end);
+        if (tid == kConsThreads) producer<DT>(P, S, ring, pos, blk_end, ~0u);
         return;
     }
     unsigned q = 0;
@@ -920,12 +934,12 @@ cudaError_t topk_verify_launch(TopkParams &P, int dtype, void *workspace, cudaSt
     if (grid > (unsigned long long)ctas) grid = (unsigned long long)ctas;
     if (grid < 1) grid = 1;
     P.grid = (int)grid;
-    if ((err = cudaMemsetAsync(P.error, 0, P.zero_bytes, stream)) != cudaSuccess) return err;
-    if (dtype == DSSD_BF16)
-        topk_verify_kernel<DSSD_BF16><<<P.grid, kTkThreads, kTopkSmemBytes, stream>>>(P);
-    else
-        topk_verify_kernel<DSSD_F32><<<P.grid, kTkThreads, kTopkSmemBytes, stream>>>(P);
-    return cudaGetLastError();
+    // a cooperative launch: all CTAs are resident at once (grid <= ctas), which the kernel's grid-wide
+    // barrier after the zeroing of the counters relies on
+    void *args[] = {&P};
+    const void *fn = dtype == DSSD_BF16 ? reinterpret_cast<const void *>(topk_verify_kernel<DSSD_BF16>)
+                                        : reinterpret_cast<const void *>(topk_verify_kernel<DSSD_F32>);
+    return cudaLaunchCooperativeKernel(fn, dim3((unsigned)P.grid), dim3(kTkThreads), args, kTopkSmemBytes, stream);
 }
 
 cudaError_t topk_resample_launch(const TopkResampleParams &P, cudaStream_t stream)

@@ -32,8 +32,8 @@ struct TopkParams {
     unsigned long long total_blocks;  // rows * nb
     int grid;
     // workspace
-    unsigned *error;                  // nonzero once a bounded wait has run out (zeroed before the launch)
-    unsigned long long *seq_done;     // [B] blocks of the sequence that have been scanned (zeroed before the launch)
+    unsigned *error;                  // nonzero once a bounded wait has run out (zeroed by the kernel before use)
+    unsigned long long *seq_done;     // [B] blocks of the sequence that have been scanned (zeroed by the kernel before use)
     unsigned long long *lists;        // [rows, max_pieces, k] candidate keys of each piece of a row
     size_t zero_bytes;
 };

@@ -456,3 +456,22 @@ def test_p7_sixteen_bit_payload(oracle_mod):
                                        d["uniforms_rs"], w.gamma)
     assert (again["token"] == half["token"]).all()
     assert (half["token"] == full["token"]).mean() > 0.7  # most draws do not sit within 2^-11 of a CDF step
+
+
+def test_batch_acceptance_rate_on_hand_made_rows():
+    """alpha = sum_v min(p_v, q_v) (Section 3.1) for rows worked out by hand, and its link to the
+    closed forms: a draft token is accepted with probability alpha."""
+    ln = np.log
+    # gamma = 2: p_0 = (1/2, 1/2) against q_0 = (3/4, 1/4): alpha = 3/4; p_1 = q_1 = (1/8, 7/8): alpha = 1
+    logits = np.array([[[ln(0.5), ln(0.5)], [ln(0.125), ln(0.875)], [0.0, 0.0]]], np.float32)
+    q = np.array([[[0.75, 0.25], [0.125, 0.875]]], np.float32)
+    assert abs(cf.batch_acceptance_rate(logits, q, 1.0) - 0.875) < 1e-7
+    # equal logits give the uniform row at any temperature
+    same = np.zeros((3, 2, 5), np.float32)
+    assert abs(cf.batch_acceptance_rate(same, np.full((3, 1, 5), 0.2, np.float32), 0.7) - 1.0) < 1e-12
+    # bfloat16 bit patterns are widened exactly: 0x3f80 = 1.0, 0x0000 = 0.0 -> p = (e, 1) / (e + 1)
+    bits = np.array([[[0x3F80, 0x0000], [0, 0]]], np.uint16)
+    p0 = np.e / (np.e + 1.0)
+    qq = np.array([[[0.5, 0.5]]], np.float32)
+    assert abs(cf.batch_acceptance_rate(bits, qq, 1.0) - (0.5 + (1.0 - p0))) < 1e-12
+    assert np.isnan(cf.batch_acceptance_rate(np.zeros((1, 1, 4), np.float32), np.zeros((1, 0, 4), np.float32), 1.0))
