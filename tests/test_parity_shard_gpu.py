@@ -242,3 +242,38 @@ def test_host_side_refusals(B):
         B.dssd_resample_shard_draw(m, 2, 0, p, q, n, u, 1, ws)  # shard index outside [0, G)
     assert e.value.status == B.DSSD_ERR_INVALID_ARG
     torch.cuda.synchronize()
+
+
+def test_the_rank_plumbing_on_a_group_of_one(B, oracle_mod):
+    """paper_2507_12000_b200/sharded.py on a process group with a single rank (all that one GPU allows):
+    the five calls, the two all-gathers and the final max run through NCCL on CUDA tensors, and the round
+    equals the dense oracle's."""
+    import os
+    import socket
+
+    import torch.distributed as dist
+
+    from paper_2507_12000_b200.sharded import verify_round_vocab_sharded
+
+    w = di.custom(B=40, gamma=3, V=20011, dtype="bf16", temperature=0.8, sigma_d=0.7, seed=77)
+    d = di.generate(w, threads=4)
+    ref = oracle_mod.verify_round(d, w.temperature, threads=4)
+    g = to_device(d)
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        out = verify_round_vocab_sharded(g["target_logits"], g["draft_tokens"], g["draft_q_tok"], g["uniforms"],
+                                         g["draft_q"], g["uniforms_rs"], w.temperature, 0, w.V)
+        torch.cuda.synchronize()
+    finally:
+        dist.destroy_process_group()
+    n = out["accept_len"].cpu().numpy()
+    assert ((n == ref["accept_len"]) | (ref["margin_acc"] < NEAR)).all()
+    same = n == ref["accept_len"]
+    slack = np.maximum(NEAR, 2 * RTOL / np.maximum(ref["Z"], 1e-30))
+    ok = (out["token"].cpu().numpy() == ref["token"]) | ~same | (ref["margin_cdf"] < slack)
+    assert ok.all()
+    assert prob_close(out["p_row_shard"].cpu().numpy()[same], ref["p_row"][same]).all()

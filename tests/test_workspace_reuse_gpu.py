@@ -39,6 +39,31 @@ def _round_fused(B, g, w, ws):
     return {"n": out["accept_len"], "tok": out["token"], "fl": out["edge_flags"], "rfl": out["rs_flags"]}
 
 
+def _round_sharded(B, g, w, ws_e, ws_r, G=3):
+    """All G shards in turn on this GPU, every call on the caller's (garbage-filled) workspaces."""
+    tl, dq = g["target_logits"], g["draft_q"]
+    base, extra = divmod(w.V, G)
+    bounds, v = [], 0
+    for i in range(G):
+        bounds.append((v, v + base + (1 if i < extra else 0)))
+        v = bounds[-1][1]
+    parts = [B.dssd_edge_partial(tl[:, :, a:b], g["draft_tokens"], a, w.temperature, workspace=ws_e) for a, b in bounds]
+    ev = B.dssd_edge_combine(torch.stack([p["part_ref"] for p in parts]), torch.stack([p["part_sum"] for p in parts]),
+                             torch.stack([p["tok_logit"] for p in parts]), g["draft_tokens"], g["draft_q_tok"],
+                             g["uniforms"], w.temperature, w.V)
+    p_row = torch.empty(w.B, w.V, dtype=torch.float32, device="cuda")
+    for a, b in bounds:
+        B.dssd_edge_emit_shard(tl[:, :, a:b], ev["accept_len"], ev["row_scale"], w.temperature, out=p_row[:, a:b])
+    need = B.dssd_resample_shard_workspace_bytes(w.B, w.gamma, bounds[0][1] - bounds[0][0])
+    chunks = [ws_r[i * ((need + 255) // 256 * 256):][:need] for i in range(G)]  # one piece of the scratch per shard
+    masses = torch.stack([B.dssd_resample_shard_mass(p_row[:, a:b], dq[:, :, a:b], ev["accept_len"], w.gamma,
+                                                     workspace=chunks[i])[0] for i, (a, b) in enumerate(bounds)])
+    toks = torch.stack([B.dssd_resample_shard_draw(masses, i, a, p_row[:, a:b], dq[:, :, a:b], ev["accept_len"],
+                                                   g["uniforms_rs"], w.gamma, chunks[i])["token"]
+                        for i, (a, b) in enumerate(bounds)])
+    return {"n": ev["accept_len"], "p": p_row, "tok": toks.max(dim=0).values, "fl": ev["flags"]}
+
+
 def _same(a, b):
     for k in a:
         x, y = a[k], b[k]
@@ -66,7 +91,8 @@ def test_garbage_and_stale_workspaces(B, shape):
     for fill in (0, 0xFF, 0x5A, None):
         ws1, ws2 = spaces(fill)
         cur = {"dense": _round_dense(B, g, w, ws1, ws2), "p16": _round_dense(B, g, w, ws1, ws2, payload="f16"),
-               "topk": _round_topk(B, gk, w, ws1), "fused": _round_fused(B, g, w, ws1)}
+               "topk": _round_topk(B, gk, w, ws1), "fused": _round_fused(B, g, w, ws1),
+               "sharded": _round_sharded(B, g, w, ws1, ws2)}
         torch.cuda.synchronize()
         if ref is None:
             ref = cur
