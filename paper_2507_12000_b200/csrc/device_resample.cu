@@ -2,8 +2,9 @@
 //
 // Pass A, ticket (b, c): stream chunk c of p_row[b] and of Q_n[b], form r = max(0, p - q) (or
 // r = p for the bonus draw) and add it up in float64 -> one or two chunk sums, 8-byte slots that are
-// valid once they differ from the all-ones pattern the workspace is filled with.  A ticket costs
-// one barrier and waits for no round trip.
+// valid once they differ from the all-ones pattern that the kernel itself clears its scratch to
+// (a cooperative launch; one grid-wide barrier, split around the first ticket's loads, separates
+// the clearing from the first use).  A ticket costs one barrier and waits for no round trip.
 // Pass B, ticket b, taken by a CTA once no chunk is left for it: a block-wide float64 prefix over
 // the sequence's chunk sums gives Z and the chunk holding u' * Z; every thread fetches its run of
 // that chunk (from L2 or HBM), a second prefix finds the thread, and the thread walks its run.
