@@ -41,21 +41,21 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum,
 # bytes per launch), valid only for the kernel source whose hash is recorded with it.
 NCU_TRAFFIC = {
-    # profiles/edge_verify_kernel_c4.md: 456.2 MB read (389.0 MB of logits + 86 % of the second read of row n)
-    # and 96.9 MB written inside the kernel; the other 58.7 MB of p_row were still in L2 when the kernel ended
+    # profiles/edge_verify_kernel_c4.md: 428.4 MB read (389.0 MB of logits + 51 % of the second read of row n)
+    # and 96.6 MB written inside the kernel; the other 59.0 MB of p_row were still in L2 when the kernel ended
     # and reach DRAM after it.  "bytes" counts all of p_row.
-    "c4": {"bytes": 456184320 + 155582464, "kernel_hash": "3a25cc07efade786",
-           "note": "dram__bytes_read.sum 456.2 MB + all 155.6 MB of p_row (96.9 MB of it written inside the "
-                   "kernel, the rest still in L2 at its end); reads are 1.17x the logits: the second read of "
-                   "row n misses L2 for 86 % of its bytes",
-           "counted_inside_kernel": 456184320 + 96895744},
+    "c4": {"bytes": 428413440 + 155582464, "kernel_hash": "174f9e8708fc9d97",
+           "note": "dram__bytes_read.sum 428.4 MB + all 155.6 MB of p_row (96.6 MB of it written inside the "
+                   "kernel, the rest still in L2 at its end); reads are 1.10x the logits: the second read of "
+                   "row n misses L2 for 51 % of its bytes",
+           "counted_inside_kernel": 428413440 + 96619264},
 }
 
 
 # the same for topk_verify_kernel (k = 10)
 NCU_TRAFFIC_TOPK = {
-    # profiles/topk_verify_kernel_c4.md: 389.5 MB read + 7.5 MB written
-    "c4": {"bytes": 389480960 + 7505152, "kernel_hash": "ebb49caf8f4fc5d4"},
+    # profiles/topk_verify_kernel_c4.md: 389.3 MB read + 4.3 MB written
+    "c4": {"bytes": 389315840 + 4342272, "kernel_hash": "881668b8c70d52bb"},
 }
 
 

@@ -763,6 +763,7 @@ struct Run {
     const char *src;   // source of stage k's copy
     long long remain;  // bytes of the row's body from stage k on (may be <= 0)
     int head;
+    bool evict_first;  // the copies carry the L2 evict_first hint
 };
 
 // The producer's claim on EMIT work advances one step per stage issued, and no step waits for
@@ -868,6 +869,7 @@ __device__ __forceinline__ void start_run(const EdgeParams &P, Shared *sh, Run &
         ++lse_tickets;
     }
     r.kind = kind;
+    r.evict_first = kind == kEmit;  // an emitted row is never read again
     r.slot = tickets++ & (kComb - 1);
     // The record's previous ticket was started kComb tickets ago; every consumer read it at that
     // ticket's first stage, which has been released since (more than kEdgeStages stages ago).
@@ -904,11 +906,18 @@ __device__ __forceinline__ void start_lse_ticket(const EdgeParams &P, Shared *sh
     const int k_begin = t.run * P.lse_run;
     const int k_end = min(P.n_slices, k_begin + P.lse_run);
     start_run<DT>(P, sh, lr, kLse, t, k_begin, k_end, tickets, lse_tickets);
+    // First reads leave L2 early too, so that the stream does not push the workspace's lines (the
+    // counters and slots that every hand-off goes through) out of it.  The exception is the last
+    // row of a short sequence, the likeliest one to be read again (with probability alpha^gamma).
+    if (P.first_read_hint) {
+        const unsigned pos = (unsigned)(row - (unsigned long long)t.seq * (unsigned)(P.gamma + 1));
+        lr.evict_first = !(pos == (unsigned)P.gamma && P.gamma <= kEdgeKeepLastRowGamma);
+    }
 }
 
 // Arms ring stage `st` with the next stage of run r and issues its copy.  The stage must be free.
 __device__ __forceinline__ void issue_stage(Shared *sh, uint32_t ring, Run &r, unsigned &st, unsigned &par,
-                                            unsigned &issued, uint64_t pol_emit)
+                                            unsigned &issued)
 {
     const unsigned len = r.remain <= 0 ? 0u : (r.remain >= kS ? (unsigned)kS : (unsigned)r.remain);
     const unsigned bulk = len & ~15u;
@@ -919,7 +928,7 @@ __device__ __forceinline__ void issue_stage(Shared *sh, uint32_t ring, Run &r, u
     const uint32_t bar = smem_addr(&sh->full[st]);
     if (bulk) {
         mbar_arrive_expect_tx(bar, bulk);
-        if (r.kind == kEmit) bulk_g2s_hint(ring + st * (uint32_t)kS, r.src, bulk, bar, pol_emit);
+        if (r.evict_first) bulk_g2s_hint(ring + st * (uint32_t)kS, r.src, bulk, bar, l2_policy_evict_first());
         else bulk_g2s(ring + st * (uint32_t)kS, r.src, bulk, bar);
     } else {
         mbar_arrive(bar);
@@ -952,7 +961,7 @@ __device__ __forceinline__ void producer_prologue(const EdgeParams &P, Shared *s
         return;
     }
     start_lse_ticket<DT>(P, sh, s.lr, no, s.tickets, s.lse_tickets);
-    for (int j = 0; j < kEdgeStages && s.lr.kind != kEnd; ++j) issue_stage(sh, ring, s.lr, s.st, s.par, s.issued, 0ull);
+    for (int j = 0; j < kEdgeStages && s.lr.kind != kEnd; ++j) issue_stage(sh, ring, s.lr, s.st, s.par, s.issued);
 }
 
 // The producer issues stages and nothing else: which ticket comes next it learns from two small
@@ -961,7 +970,6 @@ __device__ __forceinline__ void producer_prologue(const EdgeParams &P, Shared *s
 template <int DT>
 __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh, uint32_t ring, ProducerState &s)
 {
-    const uint64_t pol_emit = l2_policy_evict_first();
     bool lse_left = s.lse_left;
     Run lr = s.lr, er;  // the LSE and the EMIT run in progress; an EMIT run goes first
     er.kind = kEnd;
@@ -1008,7 +1016,7 @@ __device__ __forceinline__ void producer_thread(const EdgeParams &P, Shared *sh,
             failed = true;  // the consumers went silent
             break;
         }
-        issue_stage(sh, ring, r, st, par, issued, pol_emit);
+        issue_stage(sh, ring, r, st, par, issued);
     }
     if (!failed && mbar_wait(smem_addr(&sh->empty[st]), par, P.spin_limit)) {
         // tell the consumers that nothing follows
@@ -1567,6 +1575,9 @@ cudaError_t edge_verify_launch(EdgeParams &P, int dtype, void *workspace, cudaSt
         if (waves >= (unsigned long long)kEdgeEndgameLongWaves && P.gamma + 1 >= kEdgeEndgameLongRows)
             hold = waves * (unsigned long long)kEdgeEndgameLongEighths / 8;
         P.endgame_tickets = hold * resident_ctas;
+        // (a launch that holds its EMIT tickets back almost throughout streams reads alone: there
+        // the hint gains nothing and was measured to cost 2 %)
+        P.first_read_hint = hold == (unsigned long long)kEdgeEndgameWaves ? 1 : 0;
     }
     P.total_emit = no_emit ? 0ull : (unsigned long long)P.B * (unsigned long long)P.n_emit_runs;
     // t / d == mulhi64(t, ceil(2^64 / d)) for every t with t * d * d < 2^64

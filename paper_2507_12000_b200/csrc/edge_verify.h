@@ -11,6 +11,7 @@ constexpr int kEdgeEndgameWaves = 3;  // EMIT claims are held back during the la
 constexpr int kEdgeEndgameLongRows = 8;                                  // ... with at least so many positions per sequence ...
 constexpr int kEdgeEndgameLongWaves = 32;      // launches of at least so many waves ...
 constexpr int kEdgeEndgameLongEighths = 7;  // ... hold them back during the last so many eighths of the waves
+constexpr int kEdgeKeepLastRowGamma = 4;  // up to so many drafted positions the last row's first read carries no evict_first hint
 constexpr int kEdgeConsumers = 16;      // consumer warps per CTA
 constexpr int kEdgeThreads = 32 * (kEdgeConsumers + 3);  // + the producer warp, the fold warp and the scout warp
 constexpr int kEdgeStageBytes = 32768;   // logits bytes per ring stage (one bulk copy)
@@ -59,6 +60,7 @@ struct EdgeParams {
     int n_lse_runs, n_emit_runs;   // tickets per row
     unsigned long long total_lse;  // rows * n_lse_runs
     unsigned long long total_emit; // B * n_emit_runs
+    int first_read_hint;  // 1: the first reads of the rows carry the L2 evict_first hint
     unsigned long long endgame_tickets;  // EMIT claims are held back once so few LSE tickets are left
     unsigned long long lse_magic, emit_magic;  // ceil(2^64 / n_*_runs) when multiply-high division is exact, else 0
     unsigned spin_limit;

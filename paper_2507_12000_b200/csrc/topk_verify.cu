@@ -375,7 +375,10 @@ __device__ void producer(const TopkParams &P, Smem &S, uint32_t ring, ProducerPo
             const uint32_t bytes = (uint32_t)min(kStageVecs, pc.nvec - pos.s * kStageVecs) * 16u;
             const uint32_t bar = smem_addr(&S.full[slot]);
             mbar_arrive_expect_tx(bar, bytes);
-            bulk_g2s(ring + slot * (uint32_t)kStageBytes, pc.vp + (size_t)pos.s * kStageVecs, bytes, bar);
+            // no logit is read twice: the evict_first hint keeps the stream from pushing the
+            // workspace's lines (partial results, counters) out of L2
+            bulk_g2s_hint(ring + slot * (uint32_t)kStageBytes, pc.vp + (size_t)pos.s * kStageVecs, bytes, bar,
+                          l2_policy_evict_first());
         }
         pos.s = 0;
         pos.blk += (unsigned long long)(pc.lb - pc.fb);
