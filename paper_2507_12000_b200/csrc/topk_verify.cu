@@ -33,12 +33,16 @@
 //     goes through the rings: slow, never wrong; a full ring makes its warp wait.
 //   * Pieces alternate between two channels (rings, threshold, counters), so the consumers
 //     scan a piece while the selection warp still finishes the one before.  At the end of a
-//     piece the selection warp frees its channel and only then writes the list to the
-//     workspace and counts the piece's blocks; the CTA that
-//     completes a sequence folds it in the same warp: the rows' pieces are merged by rank
-//     counting, the k logits become probabilities in float64, the acceptance test runs, row n's
-//     k pairs are written.  The counter's answer is looked at one piece later, so nobody waits
-//     for the round trip.
+//     piece the selection warp frees its channel and then settles the row: a row that was one
+//     piece is judged on the spot, from the registers (its k logits become probabilities in
+//     float64, the acceptance test runs, the k pairs and a verdict word go to the workspace);
+//     a piece of a shared row is published and counted on the row, and the CTA that completes
+//     the row merges the pieces by rank counting and judges it.  Judged rows are counted on
+//     their sequence; the CTA that completes a sequence finds the first rejection among the
+//     verdict words and copies row n's pairs out: two small batches of loads.  So the float64
+//     work of a sequence is spread over the CTAs that scanned its rows and overlaps the stream,
+//     instead of following it in one warp.  No counter's answer is waited for: it is looked at
+//     one piece later.
 //   * Every wait (mbarrier, ring, channel hand-off) is bounded; a wait that runs out raises an
 //     error word in the workspace, the kernel runs to its end without faulting and every
 //     sequence folded after that carries DSSD_EDGE_FLAG_TIMEOUT.
@@ -554,66 +558,82 @@ __device__ __forceinline__ bool judge(const TopkParams &P, const RowDist &d, int
     return (ratio == ratio) && (u < (ratio < 1.0 ? ratio : 1.0));
 }
 
-// The selection warp of the CTA that scanned a sequence's last block: acceptance tests, first
-// rejection, row n's pairs.  Rows are taken eight at a time: their lists and their drafts are
-// all requested before the first is used, so that a group costs one trip to the L2, not eight.
-__device__ __noinline__ void fold_sequence(const TopkParams &P, int b, Smem &S)
+// A position's draft (token, uniform, q of the token), requested when its row's piece starts
+struct Draft {
+    int x;
+    float u, q;
+};
+
+__device__ __forceinline__ Draft load_draft(const TopkParams &P, int64_t row)
 {
-    constexpr int kBatch = 8;
+    Draft d;
+    d.x = 0;
+    d.u = d.q = 0.f;
+    const int b = (int)(row / (P.gamma + 1)), j = (int)(row - (int64_t)b * (P.gamma + 1));
+    if (j < P.gamma) {
+        const size_t o = (size_t)b * P.gamma + j;
+        d.x = __ldg(P.draft_tokens + o);
+        d.u = __ldg(P.uniforms + o);
+        d.q = __ldg(P.draft_q_tok + o);
+    }
+    return d;
+}
+
+// verdict word of a row: bit 0 = the position was accepted (always set for the bonus row), the
+// row's flag bits above it
+constexpr unsigned kVerdictAccept = 1u;
+constexpr int kVerdictFlagShift = 8;
+
+// One warp, lane r < k holding key r of `row`'s support: the row's k pairs (index, probability)
+// go to the first list slot of the row, its verdict word to `verdict`; counts the row on its
+// sequence and returns the count including this row (lane 0; the caller decides when to look).
+__device__ __forceinline__ unsigned judge_row(const TopkParams &P, int64_t row, unsigned long long key, const Draft &dr)
+{
+    const int lane = threadIdx.x & 31, k = P.k;
+    const int b = (int)(row / (P.gamma + 1)), j = (int)(row - (int64_t)b * (P.gamma + 1));
+    const RowDist d = dist_from_keys(P, key);
+    unsigned fl = d.bad ? DSSD_EDGE_FLAG_NONFINITE : 0u;
+    bool accept = true;
+    if (j < P.gamma) {
+        double p;
+        accept = judge(P, d, dr.x, (double)dr.u, (double)dr.q, fl, p);
+        if (lane == 0 && P.p_tok) P.p_tok[(size_t)b * P.gamma + j] = (float)p;
+    }
+    if (lane < k) {
+        const unsigned long long pair = (unsigned long long)(uint32_t)(d.bad ? -1 : d.idx) |
+                                        ((unsigned long long)__float_as_uint(d.bad ? NAN : (float)d.prob) << 32);
+        __stcg(P.lists + (size_t)row * P.max_pieces * k + lane, pair);
+    }
+    if (lane == 0) __stcg(P.verdict + row, (accept ? kVerdictAccept : 0u) | (fl << kVerdictFlagShift));
+    fence_gpu();
+    __syncwarp();
+    unsigned cnt = 0;
+    if (lane == 0) cnt = atomicAdd(P.seq_done + b, 1u) + 1u;
+    return cnt;
+}
+
+// The selection warp of the CTA that judged a sequence's last row: first rejection over the
+// rows' verdict words (one batch of loads), then row n's pairs (a second one).
+__device__ __noinline__ void fold_sequence(const TopkParams &P, int b)
+{
     const int lane = threadIdx.x & 31;
     const int gamma = P.gamma, k = P.k;
     unsigned fl = ld_relaxed_u32(P.error) ? DSSD_EDGE_FLAG_TIMEOUT : 0u;
-    int n = gamma;
-    unsigned long long key_n = 0ull;   // row n's keys: the first rejected row's, else the bonus row's
     const int64_t row0 = (int64_t)b * (gamma + 1);
-    for (int base = 0; base <= gamma; base += kBatch) {
-        const int nrow = min(kBatch, gamma + 1 - base);
-        // lane r looks after row base + r: its number of pieces and its draft
-        int my_pieces = 1, my_x = 0;
-        float my_u = 0.f, my_q = 0.f;
-        if (lane < nrow) {
-            my_pieces = pieces_of(P, row0 + base + lane);
-            if (base + lane < gamma) {
-                const size_t o = (size_t)b * gamma + base + lane;
-                my_x = __ldg(P.draft_tokens + o);
-                my_u = __ldg(P.uniforms + o);
-                my_q = __ldg(P.draft_q_tok + o);
-            }
-        }
-        unsigned long long kk[kBatch];
-#pragma unroll
-        for (int r = 0; r < kBatch; ++r) {
-            const int pcs = __shfl_sync(kFullMask, my_pieces, r);
-            kk[r] = 0ull;
-            if (r < nrow && pcs == 1 && lane < k) kk[r] = __ldcg(P.lists + (size_t)(row0 + base + r) * P.max_pieces * k + lane);
-        }
-#pragma unroll
-        for (int r = 0; r < kBatch; ++r) {
-            if (r >= nrow) break;
-            const int j = base + r;
-            const int pcs = __shfl_sync(kFullMask, my_pieces, r);
-            const unsigned long long key = pcs == 1 ? kk[r] : merged_keys(P, row0 + j, pcs, S.fold_keys, S.fold_top);
-            const RowDist d = dist_from_keys(P, key);
-            if (d.bad) fl |= DSSD_EDGE_FLAG_NONFINITE;
-            if (j == gamma) {
-                if (n == gamma) key_n = key;
-                break;
-            }
-            const int x = __shfl_sync(kFullMask, my_x, r);
-            const double u = (double)__shfl_sync(kFullMask, my_u, r), q = (double)__shfl_sync(kFullMask, my_q, r);
-            double p;
-            const bool accept = judge(P, d, x, u, q, fl, p);
-            if (lane == 0 && P.p_tok) P.p_tok[(size_t)b * gamma + j] = (float)p;
-            if (!accept && j < n) {
-                n = j;
-                key_n = key;
-            }
-        }
+    int n = gamma;
+    for (int base = 0; base <= gamma; base += 32) {
+        const int j = base + lane;
+        const unsigned v = j <= gamma ? __ldcg(P.verdict + row0 + j) : kVerdictAccept;
+        fl |= v >> kVerdictFlagShift;
+        const unsigned rej = __ballot_sync(kFullMask, !(v & kVerdictAccept));
+        if (rej && n == gamma) n = base + __ffs(rej) - 1;
     }
-    const RowDist d = dist_from_keys(P, key_n);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) fl |= __shfl_xor_sync(kFullMask, fl, o);
     if (lane < k) {
-        P.p_idx[(size_t)b * k + lane] = d.bad ? -1 : d.idx;
-        P.p_val[(size_t)b * k + lane] = d.bad ? NAN : (float)d.prob;
+        const unsigned long long pair = __ldcg(P.lists + (size_t)(row0 + n) * P.max_pieces * k + lane);
+        P.p_idx[(size_t)b * k + lane] = (int)(uint32_t)pair;
+        P.p_val[(size_t)b * k + lane] = __uint_as_float((uint32_t)(pair >> 32));
     }
     if (lane == 0) {
         P.accept_len[b] = n;
@@ -632,16 +652,46 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
 {
     const int lane = threadIdx.x & 31, k = P.k;
     const unsigned long long G = (unsigned long long)P.grid, TB = P.total_blocks, c = blockIdx.x;
-    const unsigned long long per_seq = (unsigned long long)(P.gamma + 1) * (unsigned long long)P.nb;
+    const unsigned per_seq = (unsigned)(P.gamma + 1);
     unsigned tails[2] = {0u, 0u};  // lane w < kConsWarps: keys taken from warp w's ring, per channel
-    // the sequence counter's answer is not waited for: it is looked at one piece later
-    unsigned long long prev_sum = 0ull;
-    int prev_b = -1;
+    // No counter's answer is waited for: it is looked at one piece later (or after the last piece).
+    //   seq_b[i], seq_cnt[i]   a sequence and (lane 0) its count of judged rows after a row of it
+    //                          was judged here: i = 0 a row that was one piece, i = 1 a merged row
+    //   def_row, def_cnt, ...  a row of several pieces and (lane 0) its count of published pieces
+    int seq_b[2] = {-1, -1};
+    unsigned seq_cnt[2] = {0u, 0u};
+    int64_t def_row = -1;
+    unsigned def_cnt = 0u;
+    int def_pcs = 0;
+    Draft def_draft = {0, 0.f, 0.f};
+    auto settle = [&]() {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            if (seq_b[i] < 0) continue;
+            const bool last = __shfl_sync(kFullMask, (int)(seq_cnt[i] == per_seq), 0);
+            if (last) {
+                fence_gpu();
+                fold_sequence(P, seq_b[i]);
+            }
+            seq_b[i] = -1;
+        }
+        if (def_row >= 0) {
+            const bool last = __shfl_sync(kFullMask, (int)(def_cnt == (unsigned)def_pcs), 0);
+            if (last) {
+                fence_gpu();
+                const unsigned long long key = merged_keys(P, def_row, def_pcs, S.fold_keys, S.fold_top);
+                seq_cnt[1] = judge_row(P, def_row, key, def_draft);
+                seq_b[1] = (int)(def_row / (P.gamma + 1));
+            }
+            def_row = -1;
+        }
+    };
     boundary_arrive(0);  // both channels start free
     boundary_arrive(1);
     int parity = 0;
     while (blk < blk_end) {
         const Piece pc = piece_at<DT>(P, blk, blk_end);
+        const Draft draft = load_draft(P, pc.row);  // used when the piece ends
         Channel &C = S.ch[parity];
         unsigned tl = parity ? tails[1] : tails[0];
         // empty slots hold distinct small keys (k - r in slot r), below every real key
@@ -703,37 +753,30 @@ __device__ void selection_warp(const TopkParams &P, Smem &S, unsigned long long 
         }
         __syncwarp();
         boundary_arrive(parity);
-        // publish the list, then count the piece's blocks
-        const int slot = (int)(c - owner_of((unsigned long long)pc.row * P.nb, G, TB));
-        if (lane < k) {
-            unsigned long long out = key;
-            if (bad) out = lane == 0 ? kBadList : 0ull;
-            __stcg(P.lists + ((size_t)pc.row * P.max_pieces + slot) * k + lane, out);
-        }
-        fence_gpu();
-        __syncwarp();
-        const int b = (int)(pc.row / (P.gamma + 1));
-        int fold_b = -1;
-        if (lane == 0) {
-            fold_b = (prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
-            const unsigned long long done = (unsigned long long)(pc.lb - pc.fb);
-            prev_sum = atomicAdd(P.seq_done + b, done) + done;
-            prev_b = b;
-        }
-        fold_b = __shfl_sync(kFullMask, fold_b, 0);
-        if (fold_b >= 0) {
+        settle();  // what the piece before this one asked for
+        const int pcs = pieces_of(P, pc.row);
+        unsigned long long out = key;
+        if (bad) out = lane == 0 ? kBadList : 0ull;
+        if (pcs == 1) {
+            // the whole row: judged from the registers
+            seq_cnt[0] = judge_row(P, pc.row, lane < k ? out : 0ull, draft);
+            seq_b[0] = (int)(pc.row / (P.gamma + 1));
+        } else {
+            // publish the list, then count the piece on its row
+            const int slot = (int)(c - owner_of((unsigned long long)pc.row * P.nb, G, TB));
+            if (lane < k) __stcg(P.lists + ((size_t)pc.row * P.max_pieces + slot) * k + lane, out);
             fence_gpu();
-            fold_sequence(P, fold_b, S);
+            __syncwarp();
+            if (lane == 0) def_cnt = atomicAdd(P.row_done + pc.row, 1u) + 1u;
+            def_row = pc.row;
+            def_pcs = pcs;
+            def_draft = draft;
         }
         blk += (unsigned long long)(pc.lb - pc.fb);
         parity ^= 1;
     }
-    int fold_b = (lane == 0 && prev_b >= 0 && prev_sum == per_seq) ? prev_b : -1;
-    fold_b = __shfl_sync(kFullMask, fold_b, 0);
-    if (fold_b >= 0) {
-        fence_gpu();
-        fold_sequence(P, fold_b, S);
-    }
+    settle();  // the last piece's row or sequence ...
+    settle();  // ... and the sequence of a row merged just now
 }
 
 template <int DT>
@@ -890,13 +933,16 @@ int topk_max_pieces(int k)
 size_t topk_workspace_layout(int B, int gamma, int k, TopkParams *P, char *base)
 {
     const size_t rows = (size_t)B * (size_t)(gamma + 1);
-    const size_t cnt = (8 + (size_t)B * 8 + 255) & ~(size_t)255;
+    const size_t zero = (8 + ((size_t)B + rows) * 4 + 7) & ~(size_t)7;  // error word, seq_done, row_done
+    const size_t cnt = (zero + rows * 4 + 255) & ~(size_t)255;          // ... and verdict
     const size_t lists = rows * (size_t)topk_max_pieces(k) * (size_t)k * 8;
     if (P) {
         P->error = reinterpret_cast<unsigned *>(base);
-        P->seq_done = reinterpret_cast<unsigned long long *>(base + 8);
+        P->seq_done = reinterpret_cast<unsigned *>(base + 8);
+        P->row_done = P->seq_done + B;
+        P->verdict = reinterpret_cast<unsigned *>(base + zero);
         P->lists = reinterpret_cast<unsigned long long *>(base + cnt);
-        P->zero_bytes = 8 + (size_t)B * 8;
+        P->zero_bytes = zero;
         P->max_pieces = topk_max_pieces(k);
     }
     return cnt + ((lists + 255) & ~(size_t)255);

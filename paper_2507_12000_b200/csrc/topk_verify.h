@@ -33,8 +33,11 @@ struct TopkParams {
     int grid;
     // workspace
     unsigned *error;                  // nonzero once a bounded wait has run out (zeroed by the kernel before use)
-    unsigned long long *seq_done;     // [B] blocks of the sequence that have been scanned (zeroed by the kernel before use)
-    unsigned long long *lists;        // [rows, max_pieces, k] candidate keys of each piece of a row
+    unsigned *seq_done;               // [B] rows of the sequence that have been judged (zeroed by the kernel before use)
+    unsigned *row_done;               // [rows] pieces of the row whose lists have been published (zeroed likewise)
+    unsigned *verdict;                // [rows] accepted / rejected and the row's flag bits, written when the row is judged
+    unsigned long long *lists;        // [rows, max_pieces, k] candidate keys of each piece of a row; once the row has
+                                      // been judged its first slot holds the row's k (index, probability) pairs
     size_t zero_bytes;
 };
 
