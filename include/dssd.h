@@ -34,6 +34,10 @@
  *     dssd_device_resample_static.
  *   - The streaming kernels are launched cooperatively (every CTA resident at once): two calls
  *     issued to different streams run one after the other on the GPU, not side by side.
+ *   - Every call with device pointers only can be recorded in a CUDA graph by stream capture
+ *     (it enqueues kernels and nothing else), provided one call of the same entry point was made
+ *     on that device before the capture began (the first call looks the launch constants up).
+ *     dssd_round_host synchronises the stream in the middle and cannot be captured.
  *   - Buffers need only their natural alignment; 16-byte aligned rows take the fast path.
  *   - A status other than DSSD_OK means nothing was enqueued (except DSSD_ERR_CUDA, after
  *     which the outputs are undefined).  Data-dependent anomalies never fault or trap: they
