@@ -588,8 +588,11 @@ __global__ void __launch_bounds__(kThreads, kResampleCtas) resample_kernel(const
     unsigned long long t = blockIdx.x;
     for (int it = 0; t < P.total_tickets; ++it) {
         const int buf = it & 1;
-        const int64_t b = (int64_t)(t / (unsigned)P.n_chunks);
-        const int c = (int)(t - (unsigned long long)b * (unsigned)P.n_chunks);
+        // tickets run from the last sequence's last chunk backwards: when the rows were written by a
+        // kernel just before this one, the end of the array is the part most likely still in L2
+        const unsigned long long tr = P.total_tickets - 1ull - t;
+        const int64_t b = (int64_t)(tr / (unsigned)P.n_chunks);
+        const int c = (int)(tr - (unsigned long long)b * (unsigned)P.n_chunks);
         const int n = __ldg(P.accept_len + b);
         double acc0 = 0.0, acc1 = 0.0;  // the ticket's chunk sums
         if (n >= 0 && n <= P.gamma && selected(P, n)) {
@@ -618,8 +621,8 @@ __global__ void __launch_bounds__(kThreads, kResampleCtas) resample_kernel(const
             s_ticket[buf] = it == 0 ? t + gridDim.x : logical(next_raw);
             next_raw = atomicAdd(P.ticket, 1ull);
             if (it == 0 && early && my_draw < (unsigned long long)P.B) {
-                first_n = __ldg(P.accept_len + my_draw);
-                first_u = __ldg(P.uniforms + my_draw);
+                first_n = __ldg(P.accept_len + ((unsigned long long)P.B - 1ull - my_draw));
+                first_u = __ldg(P.uniforms + ((unsigned long long)P.B - 1ull - my_draw));
             }
         }
         __syncthreads();
@@ -659,7 +662,7 @@ __global__ void __launch_bounds__(kThreads, kResampleCtas) resample_kernel(const
             s_ticket[buf] = logical(next_raw);
             next_raw = atomicAdd(P.draw_ticket, 1ull);
         }
-        const int64_t b = (int64_t)d;
+        const int64_t b = (int64_t)P.B - 1 - (int64_t)d;  // in the order in which pass A completes the sequences
         const int n = (it == 1 && prefetched) ? s_first_n : __ldg(P.accept_len + b);
         const float u = (it == 1 && prefetched) ? s_first_u : __ldg(P.uniforms + b);
         if (n < 0 || n > P.gamma) {
