@@ -1087,7 +1087,9 @@ def main():
                 recs.append({"workload": pt.name, "B": pt.B, "gamma": pt.gamma, "sigma_d": pt.sigma_d,
                              "edge_call_us": r["roofline"]["avg_launch_ms"] * 1e3, "frac": r["roofline"]["frac"],
                              "achieved_gbs": r["roofline"]["achieved"], "resample_call_us": r["resample"]["avg_launch_ms"] * 1e3,
-                             "step_us": r["ms_per_step"] * 1e3, "rows_per_s": r["value"], "parity": r["parity"],
+                             "step_us": r["ms_per_step"] * 1e3, "rows_per_s": r["value"],
+                             "graph_step_us": None if r["graph"] is None else r["graph"]["ms_per_step"] * 1e3,
+                             "parity": r["parity"],
                              "sm_mhz": r["clocks"]["sm_mhz"], "reasons": r["clocks"]["reasons"]})
         if recs:
             print(json.dumps({"metric": METRIC, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "sweep": recs}))
