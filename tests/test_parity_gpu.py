@@ -173,6 +173,27 @@ def test_anomalies_are_flagged_not_faulted(B, oracle_mod):
     assert list(rr["flags"]) == [2, 4, 4, 5] and list(rr["token"]) == [V // 2, -1, -1, -1]
 
 
+@pytest.mark.parametrize("Bn,V", [(6, 9000), (200, 4500)])
+def test_first_rejection_beyond_32_positions(B, oracle_mod, Bn, V):
+    """Long runs of accepted positions: first rejection exactly at 31, 32, 33, at the last position, at 0,
+    and no rejection at all (u = 0 accepts whatever has p > 0; u close to 1 with q = 1 rejects), through
+    the small-launch kernel (few sequences) and the streaming kernel (many)."""
+    gamma = 45
+    rejects = [31, 32, 33, 44, None, 0]
+    w = di.custom(B=Bn, gamma=gamma, V=V, dtype="bf16", temperature=0.9, sigma_d=0.4, seed=43)
+    d = di.generate(w, threads=4)
+    d["uniforms"][:] = 0.0
+    for b in range(Bn):
+        j = rejects[b % len(rejects)]
+        if j is not None:
+            d["uniforms"][b, j] = 0.99999
+            d["draft_q_tok"][b, j] = 1.0
+    ref = oracle_mod.edge_verify(d["target_logits"], d["draft_tokens"], d["draft_q_tok"], d["uniforms"], w.temperature)
+    want = [gamma if rejects[b % len(rejects)] is None else rejects[b % len(rejects)] for b in range(Bn)]
+    assert list(ref["accept_len"]) == want
+    compare_round(B, oracle_mod, d, w.temperature)
+
+
 def test_outputs_stay_inside_their_buffers(B):
     """Canary words either side of every output survive the call."""
     w = di.custom(B=5, gamma=3, V=12345, dtype="bf16", seed=3)

@@ -159,6 +159,25 @@ def test_anomalies_are_flagged_not_faulted(B, oracle_mod):
     compare_topk(B, oracle_mod, d, 1.0, k)
 
 
+def test_first_rejection_beyond_32_positions(B, oracle_mod):
+    """The sequence fold looks at 32 verdicts at a time: runs of accepted positions that cross that
+    boundary, a first rejection exactly at 31, 32, 33 and at the last position, and no rejection at all."""
+    V, gamma, k = 9000, 45, 10
+    rejects = [31, 32, 33, 44, None, 0]
+    w = di.custom(B=len(rejects), gamma=gamma, V=V, dtype="bf16", temperature=0.9, sigma_d=0.4, seed=41)
+    d = di.generate_topk(w, k)
+    d["uniforms"][:] = 0.0          # u = 0 accepts every token with p > 0 ...
+    top = np.argmax(di.bf16_bits_to_f32(d["target_logits"][:, :gamma]), axis=-1)
+    d["draft_tokens"][:] = top.astype(np.int32)   # ... and the row's best token is in its support
+    for b, j in enumerate(rejects):
+        if j is not None:
+            d["uniforms"][b, j] = 0.99999         # ... except here: q = 1 and p < 1 reject
+            d["draft_q_tok"][b, j] = 1.0
+    ref = oracle_mod.edge_verify_topk(d["target_logits"], d["draft_tokens"], d["draft_q_tok"], d["uniforms"], w.temperature, k)
+    assert list(ref["accept_len"]) == [gamma if j is None else j for j in rejects]
+    compare_topk(B, oracle_mod, d, w.temperature, k)
+
+
 def test_run_to_run_determinism(B):
     w = di.custom(B=300, gamma=4, V=50000, dtype="bf16", seed=77)
     g = to_device(di.generate_topk(w, 10, threads=4))
