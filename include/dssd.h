@@ -10,7 +10,7 @@
  *                         bonus draw x_{gamma+1} ~ P_{gamma+1} that Algorithm 2 performs when
  *                         every draft token was accepted;
  *   dssd_round_host       both halves on host buffers, with the copies to and from the GPU;
- *   dssd_edge_verify_topk, dssd_device_resample_topk
+ *   dssd_edge_verify_topk, dssd_device_resample_topk, dssd_round_host_topk
  *                         the same round on distributions truncated to their k most likely
  *                         tokens, the sampler of the paper's experiments (Section 4);
  *   dssd_edge_verify_p16, dssd_device_resample_p16
@@ -301,6 +301,32 @@ dssd_status dssd_device_resample_topk(const int32_t *p_idx, const float *p_val,
                                       const int32_t *accept_len, const float *uniforms, int B,
                                       int gamma, int k, int32_t *token, uint32_t *flags,
                                       void *cuda_stream);
+
+/* Bytes of device memory that dssd_round_host_topk needs as its arena (0 if the sizes are invalid). */
+size_t dssd_round_host_topk_arena_bytes(int B, int gamma, int V, int k, dssd_dtype dtype);
+
+/*
+ * Both halves of the truncated-support round on HOST buffers: copies the inputs to the GPU, runs
+ * dssd_edge_verify_topk and dssd_device_resample_topk, and copies the results back, all enqueued
+ * on `cuda_stream` (the draft side's lists are k pairs per position, so all of them are
+ * uploaded and nothing is waited for: unlike dssd_round_host the call returns without
+ * synchronising and can be captured).  The host buffers must stay valid until the stream has
+ * finished; use pinned memory for the copies to be asynchronous.
+ *
+ * host inputs:  target_logits [B, gamma+1, V] contiguous, draft_tokens, draft_q_tok, uniforms
+ *               [B, gamma], q_idx, q_val [B, gamma, k], uniforms_rs [B]
+ * host outputs: accept_len [B], token [B], edge_flags [B] (NULL ok), rs_flags [B] (NULL ok),
+ *               p_idx, p_val [B, k] (NULL ok: the downlink pairs then stay on the GPU)
+ * device_arena  device memory, >= dssd_round_host_topk_arena_bytes(...) bytes, 256-byte aligned
+ * Errors as for dssd_edge_verify_topk; DSSD_ERR_WORKSPACE for a missing, misaligned or short arena.
+ */
+dssd_status dssd_round_host_topk(const void *target_logits, dssd_dtype dtype,
+                                 const int32_t *draft_tokens, const float *draft_q_tok,
+                                 const float *uniforms, const int32_t *q_idx, const float *q_val,
+                                 const float *uniforms_rs, float temperature, int B, int gamma, int V,
+                                 int k, int32_t *accept_len, int32_t *token, uint32_t *edge_flags,
+                                 uint32_t *rs_flags, int32_t *p_idx, float *p_val, void *device_arena,
+                                 size_t arena_bytes, void *cuda_stream);
 
 /*
  * ---------------------------------------------------------------------------------------------

@@ -129,6 +129,13 @@ def _load(path: Optional[str] = None) -> ctypes.CDLL:
         c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
         c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
         c.c_void_p, c.c_size_t, c.c_void_p]
+    L.dssd_round_host_topk_arena_bytes.restype = c.c_size_t
+    L.dssd_round_host_topk_arena_bytes.argtypes = [c.c_int, c.c_int, c.c_int, c.c_int, c.c_int]
+    L.dssd_round_host_topk.restype = c.c_int
+    L.dssd_round_host_topk.argtypes = [
+        c.c_void_p, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_float,
+        c.c_int, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+        c.c_void_p, c.c_size_t, c.c_void_p]
     return L
 
 
@@ -438,6 +445,36 @@ def dssd_round_host(host: Dict[str, torch.Tensor], temperature: float, arena: to
         arena.data_ptr(), arena.numel(), _stream(stream))
     if st != DSSD_OK:
         raise DssdError(st, "dssd_round_host")
+    return out
+
+
+def dssd_round_host_topk_arena_bytes(B: int, gamma: int, V: int, k: int, dtype: int) -> int:
+    return int(lib.dssd_round_host_topk_arena_bytes(B, gamma, V, k, dtype))
+
+
+def dssd_round_host_topk(host: Dict[str, torch.Tensor], temperature: float, k: int, arena: torch.Tensor, *,
+                         out: Optional[Dict[str, torch.Tensor]] = None, want_pairs: bool = False,
+                         stream=None) -> Dict[str, torch.Tensor]:
+    """The truncated-support round on HOST tensors (pinned for asynchronous copies); `arena` is CUDA
+    scratch of dssd_round_host_topk_arena_bytes(...) bytes.  Results land in host tensors once the stream is done."""
+    tl = host["target_logits"]
+    assert not tl.is_cuda and tl.is_contiguous() and tl.dim() == 3
+    B, g1, V = tl.shape
+    gamma = g1 - 1
+    if out is None:
+        pin = torch.cuda.is_available()
+        out = {n: torch.empty(B, dtype=torch.int32, pin_memory=pin)
+               for n in ("accept_len", "token", "edge_flags", "rs_flags")}
+        out["p_idx"] = torch.empty(B, k, dtype=torch.int32, pin_memory=pin) if want_pairs else None
+        out["p_val"] = torch.empty(B, k, dtype=torch.float32, pin_memory=pin) if want_pairs else None
+    st = lib.dssd_round_host_topk(
+        tl.data_ptr(), _dtype_code(tl), _ptr(host.get("draft_tokens")), _ptr(host.get("draft_q_tok")),
+        _ptr(host.get("uniforms")), _ptr(host.get("q_idx")), _ptr(host.get("q_val")), host["uniforms_rs"].data_ptr(),
+        ctypes.c_float(temperature), B, gamma, V, k, out["accept_len"].data_ptr(), out["token"].data_ptr(),
+        _ptr(out.get("edge_flags")), _ptr(out.get("rs_flags")), _ptr(out.get("p_idx")), _ptr(out.get("p_val")),
+        arena.data_ptr(), arena.numel(), _stream(stream))
+    if st != DSSD_OK:
+        raise DssdError(st, "dssd_round_host_topk")
     return out
 
 

@@ -734,4 +734,97 @@ dssd_status dssd_round_host(const void *target_logits, dssd_dtype dtype,
     return DSSD_OK;
 }
 
+size_t dssd_round_host_topk_arena_bytes(int B, int gamma, int V, int k, dssd_dtype dtype)
+{
+    if (check_sizes(B, gamma, V) != DSSD_OK) return 0;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return 0;
+    if (k < 1 || k > V || k > DSSD_TOPK_MAX) return 0;
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    const size_t Bz = (size_t)B, g = (size_t)gamma, Vz = (size_t)V, kz = (size_t)k;
+    size_t n = 0;
+    n += align256(Bz * (g + 1) * Vz * esz);  // target_logits
+    n += 3 * align256(Bz * g * 4);           // draft_tokens, draft_q_tok, uniforms
+    n += 2 * align256(Bz * g * kz * 4);      // q_idx, q_val
+    n += align256(Bz * 4);                   // uniforms_rs
+    n += 2 * align256(Bz * kz * 4);          // p_idx, p_val
+    n += 4 * align256(Bz * 4);               // accept_len, token, edge flags, resample flags
+    n += align256(dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k));
+    return n;
+}
+
+dssd_status dssd_round_host_topk(const void *target_logits, dssd_dtype dtype,
+                                 const int32_t *draft_tokens, const float *draft_q_tok,
+                                 const float *uniforms, const int32_t *q_idx, const float *q_val,
+                                 const float *uniforms_rs, float temperature, int B, int gamma, int V,
+                                 int k, int32_t *accept_len, int32_t *token, uint32_t *edge_flags,
+                                 uint32_t *rs_flags, int32_t *p_idx, float *p_val, void *device_arena,
+                                 size_t arena_bytes, void *cuda_stream)
+{
+    t_last_cuda_error = 0;
+    dssd_status st = check_sizes(B, gamma, V);
+    if (st != DSSD_OK) return st;
+    if (dtype != DSSD_F32 && dtype != DSSD_BF16) return DSSD_ERR_UNSUPPORTED;
+    if (k < 1 || k > V) return DSSD_ERR_INVALID_ARG;
+    if (k > DSSD_TOPK_MAX) return DSSD_ERR_UNSUPPORTED;
+    if (!target_logits || !uniforms_rs || !accept_len || !token) return DSSD_ERR_INVALID_ARG;
+    if (gamma > 0 && (!draft_tokens || !draft_q_tok || !uniforms || !q_idx || !q_val)) return DSSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !isfinite(temperature)) return DSSD_ERR_INVALID_ARG;
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255u) ||
+        arena_bytes < dssd_round_host_topk_arena_bytes(B, gamma, V, k, dtype))
+        return DSSD_ERR_WORKSPACE;
+
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t esz = dtype == DSSD_BF16 ? 2 : 4;
+    const size_t Bz = (size_t)B, g = (size_t)gamma, Vz = (size_t)V, kz = (size_t)k;
+    char *cur = static_cast<char *>(device_arena);
+    auto take = [&](size_t bytes) {
+        char *p = cur;
+        cur += align256(bytes);
+        return p;
+    };
+    void *d_logits = take(Bz * (g + 1) * Vz * esz);
+    int32_t *d_tok_in = reinterpret_cast<int32_t *>(take(Bz * g * 4));
+    float *d_qtok = reinterpret_cast<float *>(take(Bz * g * 4));
+    float *d_u = reinterpret_cast<float *>(take(Bz * g * 4));
+    int32_t *d_qidx = reinterpret_cast<int32_t *>(take(Bz * g * kz * 4));
+    float *d_qval = reinterpret_cast<float *>(take(Bz * g * kz * 4));
+    float *d_urs = reinterpret_cast<float *>(take(Bz * 4));
+    int32_t *d_pidx = reinterpret_cast<int32_t *>(take(Bz * kz * 4));
+    float *d_pval = reinterpret_cast<float *>(take(Bz * kz * 4));
+    int32_t *d_n = reinterpret_cast<int32_t *>(take(Bz * 4));
+    int32_t *d_token = reinterpret_cast<int32_t *>(take(Bz * 4));
+    uint32_t *d_ef = reinterpret_cast<uint32_t *>(take(Bz * 4));
+    uint32_t *d_rf = reinterpret_cast<uint32_t *>(take(Bz * 4));
+    const size_t ws = dssd_edge_verify_topk_workspace_bytes(B, gamma, V, k);
+    void *d_ws = take(ws);
+
+    cudaError_t e;
+#define DSSD_TRY(call) \
+    if ((e = (call)) != cudaSuccess) return cuda_fail(e)
+    DSSD_TRY(cudaMemcpyAsync(d_logits, target_logits, Bz * (g + 1) * Vz * esz, cudaMemcpyHostToDevice, s));
+    if (gamma > 0) {
+        DSSD_TRY(cudaMemcpyAsync(d_tok_in, draft_tokens, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_qtok, draft_q_tok, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_u, uniforms, Bz * g * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_qidx, q_idx, Bz * g * kz * 4, cudaMemcpyHostToDevice, s));
+        DSSD_TRY(cudaMemcpyAsync(d_qval, q_val, Bz * g * kz * 4, cudaMemcpyHostToDevice, s));
+    }
+    DSSD_TRY(cudaMemcpyAsync(d_urs, uniforms_rs, Bz * 4, cudaMemcpyHostToDevice, s));
+    st = dssd_edge_verify_topk(d_logits, dtype, (int64_t)V, gamma ? d_tok_in : nullptr, gamma ? d_qtok : nullptr,
+                               gamma ? d_u : nullptr, temperature, B, gamma, V, k, d_n, d_pidx, d_pval, nullptr,
+                               d_ef, d_ws, ws, cuda_stream);
+    if (st != DSSD_OK) return st;
+    st = dssd_device_resample_topk(d_pidx, d_pval, gamma ? d_qidx : nullptr, gamma ? d_qval : nullptr, d_n, d_urs, B,
+                                   gamma, k, d_token, d_rf, cuda_stream);
+    if (st != DSSD_OK) return st;
+    DSSD_TRY(cudaMemcpyAsync(accept_len, d_n, Bz * 4, cudaMemcpyDeviceToHost, s));
+    DSSD_TRY(cudaMemcpyAsync(token, d_token, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (edge_flags) DSSD_TRY(cudaMemcpyAsync(edge_flags, d_ef, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (rs_flags) DSSD_TRY(cudaMemcpyAsync(rs_flags, d_rf, Bz * 4, cudaMemcpyDeviceToHost, s));
+    if (p_idx) DSSD_TRY(cudaMemcpyAsync(p_idx, d_pidx, Bz * kz * 4, cudaMemcpyDeviceToHost, s));
+    if (p_val) DSSD_TRY(cudaMemcpyAsync(p_val, d_pval, Bz * kz * 4, cudaMemcpyDeviceToHost, s));
+#undef DSSD_TRY
+    return DSSD_OK;
+}
+
 }  // extern "C"

@@ -178,6 +178,41 @@ def test_first_rejection_beyond_32_positions(B, oracle_mod):
     compare_topk(B, oracle_mod, d, w.temperature, k)
 
 
+@pytest.mark.parametrize("name,k", [("c2", 10), ("c1", 1)])
+def test_round_on_host_buffers(B, oracle_mod, name, k):
+    """dssd_round_host_topk on pinned host tensors and a garbage-filled arena, against the oracle's round;
+    a second call on the same arena (captured-style reuse) gives the same results."""
+    w = di.get_workload(name)
+    d = di.generate_topk(w, k)
+    ref = oracle_mod.verify_round_topk(d, w.temperature, k, threads=4)
+    host = {}
+    for key, v in d.items():
+        t = torch.from_numpy(v.view(np.int16)).view(torch.bfloat16) if v.dtype == np.uint16 else torch.from_numpy(v)
+        host[key] = t.pin_memory()
+    code = B.DSSD_BF16 if w.dtype == "bf16" else B.DSSD_F32
+    arena = torch.randint(0, 256, (B.dssd_round_host_topk_arena_bytes(w.B, w.gamma, w.V, k, code),), dtype=torch.uint8,
+                          device="cuda")
+    for _ in range(2):
+        out = B.dssd_round_host_topk(host, w.temperature, k, arena, want_pairs=True)
+        torch.cuda.synchronize()
+        edge = ref["margin_acc"] < EDGE
+        n = out["accept_len"].numpy()
+        assert ((n == ref["accept_len"]) | edge).all()
+        same = n == ref["accept_len"]
+        assert (out["edge_flags"].numpy().astype(np.uint32) == ref["flags"]).all()
+        assert (out["p_idx"].numpy()[same] == ref["p_idx"][same]).all()
+        assert _val_close(out["p_val"].numpy()[same], ref["p_val"][same]).all()
+        slack = np.maximum(1e-6, 4 * RTOL_VAL / np.maximum(ref["Z"], 1e-30))
+        bad = (out["token"].numpy() != ref["token"]) & same & ~(ref["margin_cdf"] < slack)
+        assert not bad.any()
+    # host-side refusals: nothing is enqueued
+    with pytest.raises(B.DssdError):
+        B.dssd_round_host_topk(host, w.temperature, k, arena[: arena.numel() // 2])
+    with pytest.raises(B.DssdError):
+        B.dssd_round_host_topk(host, w.temperature, 33, arena)
+    assert B.dssd_round_host_topk_arena_bytes(w.B, w.gamma, w.V, 0, code) == 0
+
+
 def test_run_to_run_determinism(B):
     w = di.custom(B=300, gamma=4, V=50000, dtype="bf16", seed=77)
     g = to_device(di.generate_topk(w, 10, threads=4))
