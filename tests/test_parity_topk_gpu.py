@@ -205,6 +205,18 @@ def test_round_on_host_buffers(B, oracle_mod, name, k):
         slack = np.maximum(1e-6, 4 * RTOL_VAL / np.maximum(ref["Z"], 1e-30))
         bad = (out["token"].numpy() != ref["token"]) & same & ~(ref["margin_cdf"] < slack)
         assert not bad.any()
+    # the call waits for nothing on the host, so it can be recorded in a CUDA graph and replayed
+    want_n, want_tok = out["accept_len"].clone(), out["token"].clone()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            B.dssd_round_host_topk(host, w.temperature, k, arena, out=out)
+    out["accept_len"].fill_(-7)
+    out["token"].fill_(-7)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert (out["accept_len"] == want_n).all() and (out["token"] == want_tok).all()
     # host-side refusals: nothing is enqueued
     with pytest.raises(B.DssdError):
         B.dssd_round_host_topk(host, w.temperature, k, arena[: arena.numel() // 2])
