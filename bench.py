@@ -988,6 +988,39 @@ def run_ours_sharded(args, w: di.Workload):
     clocks = sampler.summary(t_host0, t_host1)
     ms_per_step = loop["total_ms"] / K
     per_call = dict(zip(names, loop["per_call_ms"]))
+    # the same steps (flush included) replayed from a CUDA graph: the four small calls are launch- and
+    # latency-bound, so this is what a rank pays once the host's launch work is off the path
+    KG = min(K, 32)
+    side = torch.cuda.Stream()
+    cg = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(cg, stream=side):
+            for i in range(KG):
+                if flush is not None:
+                    flush.fill_(i & 1)
+                for _ in calls():
+                    pass
+    torch.cuda.synchronize()
+    cg.replay()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for _ in range(5):
+        cg.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    graph_ms = g0.elapsed_time(g1) / (5 * KG)
+    flush_ms = 0.0
+    if flush is not None:
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(20):
+            flush.fill_(i & 1)
+        f1.record()
+        torch.cuda.synchronize()
+        flush_ms = f0.elapsed_time(f1) / 20
+    graph_rec = {"ms_per_step_with_flush": graph_ms, "flush_ms": flush_ms, "ms_per_step": graph_ms - flush_ms,
+                 "steps_per_graph": KG, "replays": 5}
     peak, peak_kind = _peaks()
     part_bytes = w.rows * Vs * w.logit_bytes  # every logit of the slice once
     achieved = part_bytes / (per_call["partial"] * 1e-3) / 1e9
@@ -1026,6 +1059,7 @@ def run_ours_sharded(args, w: di.Workload):
         "per_call_ms": per_call, "step_algorithmic_bytes": step_bytes,
         "step_gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
         "timed": {"loops": len(loops), "device_ms": sum(lp["total_ms"] for lp in loops), "reported": "median loop"},
+        "graph": graph_rec,
         "cpu_baseline": cpu, "parity": parity, "e2e": None, "gpu_launches": 7 * K * len(loops), "clocks": clocks,
     }))
 
